@@ -1,0 +1,215 @@
+/*
+ * Bounded-cache attention oracle: TEST INFRASTRUCTURE, not a product path.
+ *
+ * A plain, slow, double-precision CPU statement of what one Bounded-Cache
+ * Transformer attention layer computes per token and per (sequence, kv-head)
+ * unit.  It shares no code with the CUDA library and is only ever called from
+ * the tests, the smoke check and the CPU-baseline leg of the benchmark.
+ *
+ * Notation follows the paper's Method section:
+ *   M   (here C, "capacity")  number of cache slots
+ *   MK  [C][d]                key vector sequence; never assigned by Algorithm 1
+ *   MV  [C][d]                key-value vector sequence; the state the rule rewrites
+ *   wq_t (here k_t)           write query of token t
+ *   wv_t (here v_t)           write key-value vector of token t
+ *   score_t = wq_t . MK^T     (Algorithm 1, "Calculate similarity scores")
+ *   ww_t    = softmax(score_t) (Algorithm 1, "Normalize scores to weights")
+ *   MV_t    = MV_{t-1} + ww_t^T . wv_t   (Method step 4; Illustration step 3)
+ *
+ * The paper does not print the read path; the layer is an attention layer
+ * (Method, "Model Structure"), so the read is ordinary softmax attention of the
+ * token's G read queries over the resident (MK, MV).
+ *
+ * Readings taken where the paper is silent (each is also a switch here):
+ *   - no scale factor is printed on score_t: write_scale is an explicit argument
+ *     (1.0 = literal); read_scale likewise.
+ *   - order inside a token: read MV_{t-1}, then write (default), or write then
+ *     read (BCT_ORACLE_WRITE_THEN_READ).
+ *   - Algorithm 1's "if t = 1" branch keeps MV_0 for the first token, while the
+ *     exception-free formula of Method step 4 updates on every token.  Default:
+ *     every token writes.  BCT_ORACLE_SKIP_FIRST_WRITE takes the branch literally.
+ *   - fill phase (not in the paper, whose MV_0 is full-size): while len < C the
+ *     token's (k_t, v_t) is appended at slot len, the read then covers the
+ *     len+1 resident slots (so the token sees itself), and no soft write happens.
+ *
+ * No blocking, fusion or reordering: every loop below is the definition.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define BCT_ORACLE_SKIP_FIRST_WRITE 1u
+#define BCT_ORACLE_WRITE_THEN_READ 2u
+
+/* p[j] = exp(s[j] - max s) / sum_j exp(s[j] - max s), j < n  (softmax, Algorithm 1). */
+static void softmax(const double *s, int64_t n, double *p) {
+    double m = s[0];
+    for (int64_t j = 1; j < n; ++j)
+        if (s[j] > m) m = s[j];
+    double sum = 0.0;
+    for (int64_t j = 0; j < n; ++j) {
+        p[j] = exp(s[j] - m);
+        sum += p[j];
+    }
+    for (int64_t j = 0; j < n; ++j) p[j] /= sum;
+}
+
+/* Read path for one query head: o = softmax(read_scale * q . MK[0:n]^T) . MV[0:n]. */
+static void read_head(const double *q, const double *MK, const double *MV, int64_t n, int d,
+                      double read_scale, double *s, double *p, double *o) {
+    for (int64_t j = 0; j < n; ++j) {
+        double dot = 0.0;
+        for (int e = 0; e < d; ++e) dot += q[e] * MK[j * d + e];
+        s[j] = read_scale * dot;
+    }
+    softmax(s, n, p);
+    for (int e = 0; e < d; ++e) o[e] = 0.0;
+    for (int64_t j = 0; j < n; ++j)
+        for (int e = 0; e < d; ++e) o[e] += p[j] * MV[j * d + e];
+}
+
+/* Write path: score = write_scale * wq . MK^T; ww = softmax(score); MV += ww^T . wv.
+ * ww (length C) is left in `ww` for the caller. */
+static void write_update(const double *wq, const double *wv, const double *MK, double *MV,
+                         int64_t C, int d, double write_scale, double *s, double *ww) {
+    for (int64_t j = 0; j < C; ++j) {
+        double dot = 0.0;
+        for (int e = 0; e < d; ++e) dot += wq[e] * MK[j * d + e];
+        s[j] = write_scale * dot;
+    }
+    softmax(s, C, ww);
+    for (int64_t j = 0; j < C; ++j)
+        for (int e = 0; e < d; ++e) MV[j * d + e] += ww[j] * wv[e];
+}
+
+/*
+ * One token for one unit.  `len` is the number of resident slots before the
+ * token; the return value is the number after it.  `do_write` is 0 only for
+ * the literal first-token branch of Algorithm 1.  `out` may be NULL
+ * (state-only, as UpdateKV returns only MV_N).
+ */
+static int64_t unit_token(int G, int d, int64_t C, int64_t len, double *MK, double *MV,
+                          const double *q, const double *k, const double *v, double *out,
+                          double read_scale, double write_scale, unsigned flags, int do_write,
+                          double *s, double *p) {
+    if (len < C) { /* fill phase: append, then read over len+1 slots, no soft write */
+        memcpy(MK + len * d, k, sizeof(double) * (size_t)d);
+        memcpy(MV + len * d, v, sizeof(double) * (size_t)d);
+        len += 1;
+        if (out)
+            for (int g = 0; g < G; ++g)
+                read_head(q + (int64_t)g * d, MK, MV, len, d, read_scale, s, p, out + (int64_t)g * d);
+        return len;
+    }
+    if ((flags & BCT_ORACLE_WRITE_THEN_READ) && do_write)
+        write_update(k, v, MK, MV, C, d, write_scale, s, p);
+    if (out)
+        for (int g = 0; g < G; ++g)
+            read_head(q + (int64_t)g * d, MK, MV, C, d, read_scale, s, p, out + (int64_t)g * d);
+    if (!(flags & BCT_ORACLE_WRITE_THEN_READ) && do_write)
+        write_update(k, v, MK, MV, C, d, write_scale, s, p);
+    return len;
+}
+
+/*
+ * T tokens through U independent units.
+ *
+ * Layouts (all row-major, double):
+ *   MK, MV  [U][C][d]      in/out (MK rows >= len are ignored until filled)
+ *   q       [U][T][G][d]
+ *   k, v    [U][T][d]
+ *   out     [U][T][G][d]   or NULL
+ * len_io        resident slots, the same for every unit (in/out)
+ * n_written_io  soft writes applied so far per unit history (in/out); only its
+ *               being zero matters (BCT_ORACLE_SKIP_FIRST_WRITE)
+ * nthreads      OpenMP threads over units (<= 0: library default)
+ * Returns the number of threads used, or -1 on bad arguments / allocation failure.
+ */
+int bct_oracle_stream(int64_t U, int64_t T, int G, int d, int64_t C, int64_t *len_io,
+                      int64_t *n_written_io, double *MK, double *MV, const double *q,
+                      const double *k, const double *v, double *out, double read_scale,
+                      double write_scale, unsigned flags, int nthreads) {
+    if (U < 0 || T < 0 || G < 1 || d < 1 || C < 1 || !len_io || !n_written_io) return -1;
+    if (*len_io < 0 || *len_io > C) return -1;
+    int used = 1;
+#ifdef _OPENMP
+    if (nthreads > 0) omp_set_num_threads(nthreads);
+    used = omp_get_max_threads();
+    if (used > U && U > 0) used = (int)U;
+#endif
+    int failed = 0;
+    const int64_t len0 = *len_io;
+    const int64_t w0 = *n_written_io;
+#ifdef _OPENMP
+#pragma omp parallel for schedule(dynamic, 1)
+#endif
+    for (int64_t u = 0; u < U; ++u) {
+        double *s = (double *)malloc(sizeof(double) * (size_t)C);
+        double *p = (double *)malloc(sizeof(double) * (size_t)C);
+        if (!s || !p) {
+            failed = 1;
+        } else {
+            int64_t len = len0, nw = w0;
+            double *mk = MK + u * C * d, *mv = MV + u * C * d;
+            for (int64_t t = 0; t < T; ++t) {
+                const double *qt = q + ((u * T + t) * G) * d;
+                const double *kt = k + (u * T + t) * d;
+                const double *vt = v + (u * T + t) * d;
+                double *ot = out ? out + ((u * T + t) * G) * d : NULL;
+                int full = (len == C);
+                int do_write = !((flags & BCT_ORACLE_SKIP_FIRST_WRITE) && nw == 0);
+                len = unit_token(G, d, C, len, mk, mv, qt, kt, vt, ot, read_scale, write_scale,
+                                 flags, do_write, s, p);
+                if (full) nw += 1; /* counts full-phase tokens seen, written or skipped */
+            }
+        }
+        free(s);
+        free(p);
+    }
+    if (failed) return -1;
+    /* every unit advances identically */
+    int64_t len = len0, nw = w0;
+    for (int64_t t = 0; t < T; ++t) {
+        if (len < C) len += 1; else nw += 1;
+    }
+    *len_io = len;
+    *n_written_io = nw;
+    return used;
+}
+
+/* The write weights ww = softmax(write_scale * wq . MK^T) of one unit, for tests
+ * of the row-sum and hard-addressing properties.  MK [C][d], wq [d], ww [C]. */
+int bct_oracle_write_weights(int64_t C, int d, const double *MK, const double *wq,
+                             double write_scale, double *ww) {
+    if (C < 1 || d < 1) return -1;
+    double *s = (double *)malloc(sizeof(double) * (size_t)C);
+    if (!s) return -1;
+    for (int64_t j = 0; j < C; ++j) {
+        double dot = 0.0;
+        for (int e = 0; e < d; ++e) dot += wq[e] * MK[j * d + e];
+        s[j] = write_scale * dot;
+    }
+    softmax(s, C, ww);
+    free(s);
+    return 0;
+}
+
+/* The read weights p = softmax(read_scale * q . MK[0:n]^T) of one head. */
+int bct_oracle_read_weights(int64_t n, int d, const double *MK, const double *q,
+                            double read_scale, double *p) {
+    if (n < 1 || d < 1) return -1;
+    double *s = (double *)malloc(sizeof(double) * (size_t)n);
+    if (!s) return -1;
+    for (int64_t j = 0; j < n; ++j) {
+        double dot = 0.0;
+        for (int e = 0; e < d; ++e) dot += q[e] * MK[j * d + e];
+        s[j] = read_scale * dot;
+    }
+    softmax(s, n, p);
+    free(s);
+    return 0;
+}

@@ -1,0 +1,187 @@
+"""ctypes front end of the double-precision CPU oracle (TEST INFRASTRUCTURE).
+
+Only the tests, the smoke check and the benchmark's CPU-baseline leg may import
+this module; nothing in the CUDA product path does.  All arithmetic lives in
+``bct_oracle.c``; this file builds it with gcc, marshals numpy arrays and moves
+the caller's ``[B, T, H, d]`` layouts to the oracle's unit-major layout.
+
+Semantics per (sequence, kv-head) unit and token (Method steps 2-5, Algorithm 1,
+Illustration step 3 of the paper; read path = softmax attention over the
+resident slots):
+
+    read :  o_g  = softmax(read_scale * q_g . MK^T) . MV_{t-1}
+    write:  MV_t = MV_{t-1} + softmax(write_scale * k_t . MK^T)^T . v_t
+
+with a hard-append fill phase while fewer than ``capacity`` slots are resident.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+SKIP_FIRST_WRITE = 1
+WRITE_THEN_READ = 2
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "bct_oracle.c")
+_LIB = os.path.join(_HERE, "libbct_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile ``bct_oracle.c`` into ``libbct_oracle.so`` next to it (gcc, OpenMP)."""
+    with _lock:
+        stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+        if force or stale:
+            tmp = _LIB + ".tmp%d" % os.getpid()
+            cmd = ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp",
+                   "-ffp-contract=off", "-o", tmp, _SRC, "-lm"]
+            subprocess.run(cmd, check=True)
+            os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        try:
+            lib = ctypes.CDLL(_LIB)
+        except OSError:
+            build(force=True)
+            lib = ctypes.CDLL(_LIB)
+        dp = ctypes.POINTER(ctypes.c_double)
+        lib.bct_oracle_stream.restype = ctypes.c_int
+        lib.bct_oracle_stream.argtypes = [
+            ctypes.c_int64, ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.c_int64,
+            ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64),
+            dp, dp, dp, dp, dp, dp, ctypes.c_double, ctypes.c_double, ctypes.c_uint, ctypes.c_int]
+        lib.bct_oracle_write_weights.restype = ctypes.c_int
+        lib.bct_oracle_write_weights.argtypes = [ctypes.c_int64, ctypes.c_int, dp, dp,
+                                                 ctypes.c_double, dp]
+        lib.bct_oracle_read_weights.restype = ctypes.c_int
+        lib.bct_oracle_read_weights.argtypes = [ctypes.c_int64, ctypes.c_int, dp, dp,
+                                                ctypes.c_double, dp]
+        _lib = lib
+    return _lib
+
+
+def _dptr(a: np.ndarray):
+    return a.ctypes.data_as(ctypes.POINTER(ctypes.c_double))
+
+
+def _f64(a) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(a, dtype=np.float64))
+
+
+def write_weights(MK, wq, write_scale: float = 1.0) -> np.ndarray:
+    """ww = softmax(write_scale * wq . MK^T) for one unit (Algorithm 1)."""
+    MK = _f64(MK)
+    wq = _f64(wq)
+    C, d = MK.shape
+    ww = np.empty(C, dtype=np.float64)
+    rc = _load().bct_oracle_write_weights(C, d, _dptr(MK), _dptr(wq), float(write_scale), _dptr(ww))
+    if rc != 0:
+        raise RuntimeError("bct_oracle_write_weights failed")
+    return ww
+
+
+def read_weights(MK, q, read_scale: float) -> np.ndarray:
+    """p = softmax(read_scale * q . MK^T) for one head over the rows of MK given."""
+    MK = _f64(MK)
+    q = _f64(q)
+    n, d = MK.shape
+    p = np.empty(n, dtype=np.float64)
+    rc = _load().bct_oracle_read_weights(n, d, _dptr(MK), _dptr(q), float(read_scale), _dptr(p))
+    if rc != 0:
+        raise RuntimeError("bct_oracle_read_weights failed")
+    return p
+
+
+class OracleCache:
+    """Bounded cache of ``capacity`` slots for ``batch * n_kv_heads`` independent units.
+
+    ``mk_init`` / ``mv_init``: ``[batch, n_kv_heads, init_len, head_dim]`` (the paper's
+    MK and MV_0; ``mv_init=None`` with ``init_len > 0`` means zeros, one of the two
+    initialisations the Method section allows).  ``read_scale=None`` means
+    ``1/sqrt(head_dim)``; ``write_scale=None`` means 1.0 (Algorithm 1 prints no scale).
+    """
+
+    def __init__(self, batch, n_q_heads, n_kv_heads, head_dim, capacity, *, read_scale=None,
+                 write_scale=None, init_len=0, mk_init=None, mv_init=None, flags=0,
+                 nthreads=0):
+        if n_q_heads % n_kv_heads:
+            raise ValueError("n_q_heads must be a multiple of n_kv_heads")
+        if not (0 <= init_len <= capacity):
+            raise ValueError("init_len out of range")
+        self.B, self.Hq, self.Hkv, self.d, self.C = batch, n_q_heads, n_kv_heads, head_dim, capacity
+        self.G = n_q_heads // n_kv_heads
+        self.U = batch * n_kv_heads
+        self.read_scale = float(1.0 / np.sqrt(head_dim) if read_scale is None else read_scale)
+        self.write_scale = float(1.0 if write_scale is None else write_scale)
+        self.flags = int(flags)
+        self.nthreads = int(nthreads)
+        self.threads_used = 0
+        self.len = int(init_len)
+        self.n_written = 0
+        self.MK = np.zeros((self.U, capacity, head_dim), dtype=np.float64)
+        self.MV = np.zeros((self.U, capacity, head_dim), dtype=np.float64)
+        if init_len > 0:
+            if mk_init is None:
+                raise ValueError("mk_init required when init_len > 0")
+            self.MK[:, :init_len] = _f64(mk_init).reshape(self.U, init_len, head_dim)
+            if mv_init is not None:
+                self.MV[:, :init_len] = _f64(mv_init).reshape(self.U, init_len, head_dim)
+
+    # -- state in the caller's layout ------------------------------------------------
+    def keys(self) -> np.ndarray:
+        return self.MK.reshape(self.B, self.Hkv, self.C, self.d)
+
+    def values(self) -> np.ndarray:
+        return self.MV.reshape(self.B, self.Hkv, self.C, self.d)
+
+    # -- steps -------------------------------------------------------------------
+    def prefill_stream(self, q, k, v, want_out: bool = True):
+        """q ``[B, T, Hq, d]``, k, v ``[B, T, Hkv, d]`` -> out ``[B, T, Hq, d]`` (float64)."""
+        q = _f64(q)
+        k = _f64(k)
+        v = _f64(v)
+        B, T = q.shape[0], q.shape[1]
+        assert q.shape == (self.B, T, self.Hq, self.d), q.shape
+        assert k.shape == (self.B, T, self.Hkv, self.d), k.shape
+        assert v.shape == (self.B, T, self.Hkv, self.d), v.shape
+        # unit-major: unit u = b * Hkv + h ; query heads of kv-head h are h*G .. h*G+G-1
+        qu = np.ascontiguousarray(
+            q.reshape(B, T, self.Hkv, self.G, self.d).transpose(0, 2, 1, 3, 4)
+        ).reshape(self.U, T, self.G, self.d)
+        ku = np.ascontiguousarray(k.transpose(0, 2, 1, 3)).reshape(self.U, T, self.d)
+        vu = np.ascontiguousarray(v.transpose(0, 2, 1, 3)).reshape(self.U, T, self.d)
+        ou = np.empty((self.U, T, self.G, self.d), dtype=np.float64) if want_out else None
+        ln = ctypes.c_int64(self.len)
+        nw = ctypes.c_int64(self.n_written)
+        rc = _load().bct_oracle_stream(
+            self.U, T, self.G, self.d, self.C, ctypes.byref(ln), ctypes.byref(nw),
+            _dptr(self.MK), _dptr(self.MV), _dptr(qu), _dptr(ku), _dptr(vu),
+            _dptr(ou) if want_out else None, self.read_scale, self.write_scale,
+            self.flags, self.nthreads)
+        if rc < 0:
+            raise RuntimeError("bct_oracle_stream failed")
+        self.threads_used = rc
+        self.len, self.n_written = ln.value, nw.value
+        if not want_out:
+            return None
+        return np.ascontiguousarray(
+            ou.reshape(B, self.Hkv, T, self.G, self.d).transpose(0, 2, 1, 3, 4)
+        ).reshape(B, T, self.Hq, self.d)
+
+    def decode_step(self, q, k, v):
+        """q ``[B, Hq, d]``, k, v ``[B, Hkv, d]`` -> out ``[B, Hq, d]``."""
+        q = _f64(q)[:, None]
+        k = _f64(k)[:, None]
+        v = _f64(v)[:, None]
+        return self.prefill_stream(q, k, v)[:, 0]

@@ -1,0 +1,151 @@
+"""Seeded synthetic inputs for the bounded-cache attention path.
+
+This module holds the input recipes only: shapes, distributions, seeds and the
+rounding of every drawn value to the io dtype.  It contains none of the
+method's arithmetic, so that both the CUDA path and the CPU checker can be fed
+from it.  The paper evaluates on web-text corpora with a trained 1B-parameter
+model (Experimental Setup); the cost and the numerics of the attention step
+depend only on shapes and value scales, so i.i.d. Gaussians of the stated
+variances stand in for those activations.
+
+Every tensor is a pure function of (workload, index, device type): a step's
+q/k/v can be regenerated without drawing the steps before it, and a sequence's
+initial cache without drawing the other sequences.  CPU and CUDA generators
+give different streams; a comparison always draws once and hands the same
+rounded values to both sides.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, replace
+from typing import Dict, Tuple
+
+import torch
+
+_DTYPES = {"f32": torch.float32, "bf16": torch.bfloat16}
+STREAM_BLOCK = 1024  # tokens per independently seeded block of a long stream
+
+
+@dataclass(frozen=True)
+class Workload:
+    name: str
+    batch: int
+    n_q_heads: int
+    n_kv_heads: int
+    head_dim: int
+    capacity: int
+    dtype: str          # "f32" | "bf16": cache and step-vector storage type
+    init_len: int       # resident slots at create (capacity = paper-literal full MV_0)
+    steps: int          # tokens pushed through the cache
+    seed: int
+    q_std: float        # read query std
+    kv_std: float       # write query (k) / write value (v) std
+    init_std: float     # std of the pre-filled MK / MV_0
+    api: str            # "decode" (one call per token) | "stream" (prefill_stream)
+    read_scale: float = 1.0
+    write_scale: float = 1.0
+
+    @property
+    def group(self) -> int:
+        return self.n_q_heads // self.n_kv_heads
+
+    @property
+    def units(self) -> int:
+        return self.batch * self.n_kv_heads
+
+    @property
+    def torch_dtype(self) -> torch.dtype:
+        return _DTYPES[self.dtype]
+
+    @property
+    def elem_bytes(self) -> int:
+        return 4 if self.dtype == "f32" else 2
+
+    def scaled(self, **kw) -> "Workload":
+        return replace(self, **kw)
+
+
+def _w(name, B, Hq, Hkv, d, C, dtype, init_len, steps, seed, q_std, kv_std, api="decode"):
+    return Workload(name, B, Hq, Hkv, d, C, dtype, init_len, steps, seed, q_std, kv_std, 1.0, api)
+
+
+# The five configurations of the benchmark contract.  q already carries the
+# 1/sqrt(d) factor (q ~ N(0, 1/d) against N(0,1) keys gives unit-variance read
+# scores), hence read_scale = 1.  write_scale = 1 is the literal Algorithm 1.
+CONFIGS: Dict[str, Workload] = {
+    "single_fp32_c128": _w("single_fp32_c128", 1, 1, 1, 64, 128, "f32", 0, 512, 0,
+                           64 ** -0.5, 64 ** -0.5),
+    "mha7b_b64_c2048": _w("mha7b_b64_c2048", 64, 32, 32, 128, 2048, "bf16", 2048, 1024, 1,
+                          128 ** -0.5, 1.0),
+    "gqa8b_b128_c4096": _w("gqa8b_b128_c4096", 128, 32, 8, 128, 4096, "bf16", 4096, 512, 2,
+                           128 ** -0.5, 1.0),
+    "stream_b8_c1024": _w("stream_b8_c1024", 8, 32, 32, 128, 1024, "bf16", 0, 131072, 3,
+                          128 ** -0.5, 1.0, api="stream"),
+}
+for _C in (256, 1024, 4096, 16384):
+    CONFIGS["sweep_b256_c%d" % _C] = _w("sweep_b256_c%d" % _C, 256, 32, 8, 128, _C, "bf16", _C,
+                                        256, 4, 128 ** -0.5, 1.0)
+
+
+def _gen(device, *key: int) -> torch.Generator:
+    g = torch.Generator(device=device)
+    s = 0x9E3779B97F4A7C15
+    for x in key:
+        s = (s * 6364136223846793005 + int(x) + 1442695040888963407) % (1 << 63)
+    g.manual_seed(s)
+    return g
+
+
+def _draw(shape, std, dtype, gen, device) -> torch.Tensor:
+    x = torch.randn(shape, generator=gen, device=device, dtype=torch.float32)
+    return (x * std).to(dtype)
+
+
+def initial_cache_seq(w: Workload, b: int, device="cpu") -> Tuple[torch.Tensor, torch.Tensor]:
+    """(mk_init, mv_init) of sequence ``b``: ``[n_kv_heads, init_len, head_dim]`` each."""
+    shape = (w.n_kv_heads, w.init_len, w.head_dim)
+    mk = _draw(shape, w.init_std, w.torch_dtype, _gen(device, w.seed, 1, b), device)
+    mv = _draw(shape, w.init_std, w.torch_dtype, _gen(device, w.seed, 2, b), device)
+    return mk, mv
+
+
+def initial_cache(w: Workload, device="cpu") -> Tuple[torch.Tensor, torch.Tensor]:
+    """(mk_init, mv_init): ``[batch, n_kv_heads, init_len, head_dim]`` in the io dtype."""
+    shape = (w.batch, w.n_kv_heads, w.init_len, w.head_dim)
+    mk = torch.empty(shape, dtype=w.torch_dtype, device=device)
+    mv = torch.empty(shape, dtype=w.torch_dtype, device=device)
+    if w.init_len:
+        for b in range(w.batch):
+            mk[b], mv[b] = initial_cache_seq(w, b, device)
+    return mk, mv
+
+
+def step_inputs(w: Workload, t: int, device="cpu"):
+    """Token ``t`` of every sequence: q ``[B, Hq, d]``, k, v ``[B, Hkv, d]`` in the io dtype."""
+    dt = w.torch_dtype
+    q = _draw((w.batch, w.n_q_heads, w.head_dim), w.q_std, dt, _gen(device, w.seed, 3, t), device)
+    k = _draw((w.batch, w.n_kv_heads, w.head_dim), w.kv_std, dt, _gen(device, w.seed, 4, t), device)
+    v = _draw((w.batch, w.n_kv_heads, w.head_dim), w.kv_std, dt, _gen(device, w.seed, 5, t), device)
+    return q, k, v
+
+
+def stream_block(w: Workload, blk: int, device="cpu"):
+    """Tokens ``[blk*STREAM_BLOCK, (blk+1)*STREAM_BLOCK)`` of the stream:
+    q ``[B, STREAM_BLOCK, Hq, d]``, k, v ``[B, STREAM_BLOCK, Hkv, d]``."""
+    dt = w.torch_dtype
+    n = STREAM_BLOCK
+    q = _draw((w.batch, n, w.n_q_heads, w.head_dim), w.q_std, dt, _gen(device, w.seed, 6, blk), device)
+    k = _draw((w.batch, n, w.n_kv_heads, w.head_dim), w.kv_std, dt, _gen(device, w.seed, 7, blk), device)
+    v = _draw((w.batch, n, w.n_kv_heads, w.head_dim), w.kv_std, dt, _gen(device, w.seed, 8, blk), device)
+    return q, k, v
+
+
+def stream_inputs(w: Workload, t0: int, T: int, device="cpu"):
+    """Tokens ``[t0, t0+T)`` of the stream, assembled from whole seeded blocks."""
+    b0, b1 = t0 // STREAM_BLOCK, (t0 + T - 1) // STREAM_BLOCK
+    parts = [stream_block(w, b, device) for b in range(b0, b1 + 1)]
+    lo = t0 - b0 * STREAM_BLOCK
+    out = []
+    for i in range(3):
+        x = parts[0][i] if len(parts) == 1 else torch.cat([p[i] for p in parts], dim=1)
+        out.append(x[:, lo:lo + T].contiguous())
+    return tuple(out)

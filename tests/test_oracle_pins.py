@@ -1,0 +1,369 @@
+"""Pins for the CPU oracle: what the paper and the mathematics fix, independent of the oracle.
+
+Each test states which passage or identity it uses.  None of them re-types the
+oracle's loops: they use textbook routines (causal softmax attention), closed
+forms that follow from the update rule, invariances, hand-worked fixtures and a
+long-hand brute force on tiny inputs.
+"""
+import math
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import bct_oracle as O
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+RNG = np.random.default_rng(20241016)
+
+
+def _rand(*shape, scale=1.0):
+    return RNG.normal(size=shape) * scale
+
+
+def _np_softmax(x, axis=-1):
+    x = x - x.max(axis=axis, keepdims=True)
+    e = np.exp(x)
+    return e / e.sum(axis=axis, keepdims=True)
+
+
+# ---------------------------------------------------------------------------------------
+# Hand-worked fixtures (tests/golden): Algorithm 1 + Method step 4 evaluated by hand
+# ---------------------------------------------------------------------------------------
+def _parse_golden(name):
+    vals = {}
+    with open(os.path.join(GOLDEN, name)) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            key, rest = line.split(None, 1)
+            rows = []
+            for row in rest.split(";"):
+                r = []
+                for tok in row.split():
+                    if tok == "L3":
+                        r.append(math.log(3.0))
+                    else:
+                        r.append(float(Fraction(tok)))
+                rows.append(r)
+            vals[key] = np.array(rows if len(rows) > 1 else rows[0], dtype=np.float64)
+    return vals
+
+
+def test_golden_full_phase_hand_worked():
+    g = _parse_golden("hand_worked_full_c2_d2.txt")
+    c = O.OracleCache(1, 1, 1, 2, 2, read_scale=1.0, write_scale=1.0, init_len=2,
+                      mk_init=g["MK"][None, None], mv_init=g["MV0"][None, None])
+    o1 = c.decode_step(g["q1"][None, None], g["k1"][None, None], g["v1"][None, None])
+    np.testing.assert_allclose(o1[0, 0], g["o1"], rtol=0, atol=1e-14)
+    np.testing.assert_allclose(c.values()[0, 0], g["MV1"], rtol=0, atol=1e-14)
+    o2 = c.decode_step(g["q2"][None, None], g["k2"][None, None], g["v2"][None, None])
+    np.testing.assert_allclose(o2[0, 0], g["o2"], rtol=0, atol=1e-14)
+    np.testing.assert_allclose(c.values()[0, 0], g["MV2"], rtol=0, atol=1e-13)
+    np.testing.assert_array_equal(c.keys()[0, 0], g["MK"])  # MK is never assigned by Algorithm 1
+
+
+def test_golden_fill_phase_hand_worked():
+    g = _parse_golden("hand_worked_fill_c2_d2.txt")
+    c = O.OracleCache(1, 1, 1, 2, 2, read_scale=1.0, write_scale=1.0)
+    for t in (1, 2, 3):
+        o = c.decode_step(g["q%d" % t][None, None], g["k%d" % t][None, None], g["v%d" % t][None, None])
+        np.testing.assert_allclose(o[0, 0], g["o%d" % t], rtol=0, atol=1e-14)
+        assert c.len == min(t, 2)
+    np.testing.assert_allclose(c.keys()[0, 0], g["MK3"], rtol=0, atol=0)
+    np.testing.assert_allclose(c.values()[0, 0], g["MV3"], rtol=0, atol=1e-14)
+
+
+# ---------------------------------------------------------------------------------------
+# Capacity >= sequence length, cache starting empty  ==>  full causal softmax attention
+# ---------------------------------------------------------------------------------------
+@pytest.mark.parametrize("B,Hq,Hkv,d,T,C", [(2, 4, 2, 8, 13, 13), (1, 3, 1, 5, 9, 32), (2, 2, 2, 16, 20, 21)])
+def test_capacity_ge_length_is_full_causal_attention(B, Hq, Hkv, d, T, C):
+    q, k, v = _rand(B, T, Hq, d), _rand(B, T, Hkv, d), _rand(B, T, Hkv, d)
+    scale = 0.37
+    c = O.OracleCache(B, Hq, Hkv, d, C, read_scale=scale)
+    out = c.prefill_stream(q, k, v)
+    assert c.len == T and c.n_written == 0
+    G = Hq // Hkv
+    tq = torch.from_numpy(q).permute(0, 2, 1, 3)                                   # [B,Hq,T,d]
+    tk = torch.from_numpy(k).permute(0, 2, 1, 3).repeat_interleave(G, dim=1)       # kv head h serves q heads h*G..
+    tv = torch.from_numpy(v).permute(0, 2, 1, 3).repeat_interleave(G, dim=1)
+    ref = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, is_causal=True, scale=scale)
+    ref = ref.permute(0, 2, 1, 3).numpy()
+    np.testing.assert_allclose(out, ref, rtol=0, atol=1e-12)
+    # and with a plain numpy causal attention, head by head
+    for b in range(B):
+        for h in range(Hq):
+            s = scale * q[b, :, h] @ k[b, :, h // G].T
+            s[np.triu_indices(T, 1)] = -np.inf
+            np.testing.assert_allclose(out[b, :, h], _np_softmax(s) @ v[b, :, h // G], rtol=0, atol=1e-12)
+
+
+def test_len_never_exceeds_capacity_and_keys_freeze():
+    B, H, d, C, T = 1, 2, 4, 5, 17
+    q, k, v = _rand(B, T, H, d), _rand(B, T, H, d), _rand(B, T, H, d)
+    c = O.OracleCache(B, H, H, d, C)
+    lens = []
+    for t in range(T):
+        c.decode_step(q[:, t], k[:, t], v[:, t])
+        lens.append(c.len)
+        assert c.MK.shape == (B * H, C, d) and c.MV.shape == (B * H, C, d)  # allocation fixed
+    assert lens == [min(t + 1, C) for t in range(T)]
+    # keys resident after the fill are exactly the first C write queries, untouched afterwards
+    np.testing.assert_array_equal(c.keys()[0], np.transpose(k[0, :C], (1, 0, 2)))
+    assert c.n_written == T - C
+
+
+# ---------------------------------------------------------------------------------------
+# Softmax rows sum to one
+# ---------------------------------------------------------------------------------------
+def test_weight_rows_sum_to_one():
+    C, d = 257, 16
+    MK = _rand(C, d)
+    for scale in (1.0, 0.05, 7.0):
+        ww = O.write_weights(MK, _rand(d), scale)
+        assert abs(ww.sum() - 1.0) < 1e-14 and (ww >= 0).all()
+        p = O.read_weights(MK[:100], _rand(d), scale)
+        assert abs(p.sum() - 1.0) < 1e-14 and (p >= 0).all()
+    big = O.write_weights(MK * 100.0, _rand(d) * 100.0, 1.0)  # scores ~1e4: max-subtraction needed
+    assert np.isfinite(big).all() and abs(big.sum() - 1.0) < 1e-14
+
+
+# ---------------------------------------------------------------------------------------
+# Mass conservation: sum_j MV_t[j] - sum_j MV_{t-1}[j] = wv_t   (ww sums to one)
+# ---------------------------------------------------------------------------------------
+def test_mass_conservation_per_step_and_total():
+    B, Hq, Hkv, d, C, T = 2, 4, 2, 8, 11, 9
+    mk, mv = _rand(B, Hkv, C, d), _rand(B, Hkv, C, d)
+    q, k, v = _rand(B, T, Hq, d), _rand(B, T, Hkv, d), _rand(B, T, Hkv, d)
+    c = O.OracleCache(B, Hq, Hkv, d, C, init_len=C, mk_init=mk, mv_init=mv, write_scale=0.8)
+    prev = c.values().sum(axis=2).copy()
+    for t in range(T):
+        c.decode_step(q[:, t], k[:, t], v[:, t])
+        cur = c.values().sum(axis=2)
+        np.testing.assert_allclose(cur - prev, v[:, t], rtol=0, atol=1e-12)
+        prev = cur.copy()
+    np.testing.assert_allclose(c.values().sum(axis=2), mv.sum(axis=2) + v.sum(axis=1), rtol=0, atol=1e-11)
+    np.testing.assert_array_equal(c.keys(), mk)
+
+
+# ---------------------------------------------------------------------------------------
+# Dense restatement (token-level parallelism, "Optimized for Parallelism"): with MK frozen
+#   MV_N = MV_0 + softmax(Kc MK^T)^T Vc ,  O = Pr MV_0 + strict_tril(Pr WW^T) Vc
+# ---------------------------------------------------------------------------------------
+@pytest.mark.parametrize("G", [1, 3])
+def test_dense_two_matmul_restatement(G):
+    d, C, T = 8, 10, 14
+    rs, ws = 0.3, 0.9
+    mk, mv0 = _rand(1, 1, C, d), _rand(1, 1, C, d)
+    q, k, v = _rand(1, T, G, d), _rand(1, T, 1, d), _rand(1, T, 1, d)
+    c = O.OracleCache(1, G, 1, d, C, init_len=C, mk_init=mk, mv_init=mv0, read_scale=rs, write_scale=ws)
+    out = c.prefill_stream(q, k, v)
+    MK, MV0, Kc, Vc = mk[0, 0], mv0[0, 0], k[0, :, 0], v[0, :, 0]
+    WW = _np_softmax(ws * Kc @ MK.T)                      # [T, C]
+    np.testing.assert_allclose(c.values()[0, 0], MV0 + WW.T @ Vc, rtol=0, atol=1e-12)
+    for g in range(G):
+        Pr = _np_softmax(rs * q[0, :, g] @ MK.T)          # [T, C]
+        A = np.tril(Pr @ WW.T, -1)                        # token t sees writes of tokens < t
+        np.testing.assert_allclose(out[0, :, g], Pr @ MV0 + A @ Vc, rtol=0, atol=1e-12)
+
+
+def test_write_then_read_differs_by_closed_form_term():
+    d, C, T = 6, 7, 5
+    mk, mv0 = _rand(1, 1, C, d), _rand(1, 1, C, d)
+    q, k, v = _rand(1, T, 1, d), _rand(1, T, 1, d), _rand(1, T, 1, d)
+    a = O.OracleCache(1, 1, 1, d, C, init_len=C, mk_init=mk, mv_init=mv0, read_scale=0.5)
+    b = O.OracleCache(1, 1, 1, d, C, init_len=C, mk_init=mk, mv_init=mv0, read_scale=0.5,
+                      flags=O.WRITE_THEN_READ)
+    oa, ob = a.prefill_stream(q, k, v), b.prefill_stream(q, k, v)
+    np.testing.assert_allclose(a.values(), b.values(), rtol=0, atol=1e-13)
+    for t in range(T):
+        p = O.read_weights(mk[0, 0], q[0, t, 0], 0.5)
+        ww = O.write_weights(mk[0, 0], k[0, t, 0], 1.0)
+        np.testing.assert_allclose(ob[0, t, 0] - oa[0, t, 0], (p @ ww) * v[0, t, 0], rtol=0, atol=1e-12)
+
+
+def test_skip_first_write_is_algorithm_1_literal():
+    d, C, T = 4, 6, 5
+    mk, mv0 = _rand(1, 1, C, d), _rand(1, 1, C, d)
+    q, k, v = _rand(1, T, 1, d), _rand(1, T, 1, d), _rand(1, T, 1, d)
+    lit = O.OracleCache(1, 1, 1, d, C, init_len=C, mk_init=mk, mv_init=mv0, flags=O.SKIP_FIRST_WRITE)
+    lit.prefill_stream(q, k, v)
+    WW = _np_softmax(k[0, :, 0] @ mk[0, 0].T)
+    # Algorithm 1: MV_1 = MV_0, then MV_t = MV_{t-1} + ww_t^T wv_t for t = 2..N
+    np.testing.assert_allclose(lit.values()[0, 0], mv0[0, 0] + WW[1:].T @ v[0, 1:, 0], rtol=0, atol=1e-12)
+
+
+# ---------------------------------------------------------------------------------------
+# Closed forms of special cases
+# ---------------------------------------------------------------------------------------
+def test_zero_write_query_gives_uniform_write():
+    d, C, T = 5, 8, 6
+    mk, mv0 = _rand(1, 1, C, d), _rand(1, 1, C, d)
+    q, v = _rand(1, T, 1, d), _rand(1, T, 1, d)
+    k = np.zeros((1, T, 1, d))
+    c = O.OracleCache(1, 1, 1, d, C, init_len=C, mk_init=mk, mv_init=mv0)
+    c.prefill_stream(q, k, v)
+    expect = mv0[0, 0] + np.ones((C, 1)) / C * v[0, :, 0].sum(axis=0)[None, :]
+    np.testing.assert_allclose(c.values()[0, 0], expect, rtol=0, atol=1e-13)
+    # identical keys give the same uniform weights whatever the write query
+    mk_same = np.repeat(_rand(1, 1, 1, d), C, axis=2)
+    c2 = O.OracleCache(1, 1, 1, d, C, init_len=C, mk_init=mk_same, mv_init=mv0)
+    c2.prefill_stream(q, _rand(1, T, 1, d), v)
+    np.testing.assert_allclose(c2.values()[0, 0], expect, rtol=0, atol=1e-12)
+
+
+def test_capacity_one_is_running_sum():
+    d, T = 4, 7
+    mk, mv0 = _rand(1, 1, 1, d), _rand(1, 1, 1, d)
+    q, k, v = _rand(1, T, 2, d), _rand(1, T, 1, d), _rand(1, T, 1, d)
+    c = O.OracleCache(1, 2, 1, d, 1, init_len=1, mk_init=mk, mv_init=mv0)
+    out = c.prefill_stream(q, k, v)
+    run = mv0[0, 0, 0] + np.concatenate([np.zeros((1, d)), np.cumsum(v[0, :, 0], axis=0)])
+    for t in range(T):  # o_t = MV_{t-1}: the fixed-size-state (RNN-like) corner of Table 1
+        np.testing.assert_allclose(out[0, t, 0], run[t], rtol=0, atol=1e-13)
+        np.testing.assert_allclose(out[0, t, 1], run[t], rtol=0, atol=1e-13)
+    np.testing.assert_allclose(c.values()[0, 0, 0], run[T], rtol=0, atol=1e-13)
+
+
+def test_hard_addressing_limit():
+    d, C = 8, 8
+    mk = np.eye(C, d)[None, None] * 1.0
+    mv0 = _rand(1, 1, C, d)
+    i, beta = 5, 200.0
+    k = (beta * mk[0, 0, i])[None, None, None]
+    v = _rand(1, 1, 1, d)
+    c = O.OracleCache(1, 1, 1, d, C, init_len=C, mk_init=mk, mv_init=mv0)
+    c.prefill_stream(_rand(1, 1, 1, d), k, v, want_out=False)
+    expect = mv0[0, 0].copy()
+    expect[i] += v[0, 0, 0]
+    np.testing.assert_allclose(c.values()[0, 0], expect, rtol=0, atol=1e-13)
+
+
+# ---------------------------------------------------------------------------------------
+# Invariances
+# ---------------------------------------------------------------------------------------
+def test_slot_permutation_equivariance():
+    B, Hq, Hkv, d, C, T = 1, 2, 1, 6, 9, 7
+    mk, mv0 = _rand(B, Hkv, C, d), _rand(B, Hkv, C, d)
+    q, k, v = _rand(B, T, Hq, d), _rand(B, T, Hkv, d), _rand(B, T, Hkv, d)
+    perm = RNG.permutation(C)
+    a = O.OracleCache(B, Hq, Hkv, d, C, init_len=C, mk_init=mk, mv_init=mv0)
+    b = O.OracleCache(B, Hq, Hkv, d, C, init_len=C, mk_init=mk[:, :, perm], mv_init=mv0[:, :, perm])
+    oa, ob = a.prefill_stream(q, k, v), b.prefill_stream(q, k, v)
+    np.testing.assert_allclose(oa, ob, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(a.values()[:, :, perm], b.values(), rtol=0, atol=1e-12)
+
+
+def test_score_shift_invariance_and_value_linearity():
+    d, C, T = 6, 8, 5
+    mk, q, k, v = _rand(1, 1, C, d), _rand(1, T, 1, d), _rand(1, T, 1, d), _rand(1, T, 1, d)
+    # make every q_t and k_t orthogonal to u up to a fixed component, so MK + c*u shifts all
+    # scores of a token by the same constant
+    u = np.zeros(d)
+    u[0] = 1.0
+    q[..., 0] = 0.7
+    k[..., 0] = -1.3
+    a = O.OracleCache(1, 1, 1, d, C, init_len=C, mk_init=mk)  # MV_0 = 0
+    b = O.OracleCache(1, 1, 1, d, C, init_len=C, mk_init=mk + 50.0 * u)
+    oa, ob = a.prefill_stream(q, k, v), b.prefill_stream(q, k, v)
+    np.testing.assert_allclose(oa, ob, rtol=0, atol=1e-11)
+    np.testing.assert_allclose(a.values(), b.values(), rtol=0, atol=1e-11)
+    s = O.OracleCache(1, 1, 1, d, C, init_len=C, mk_init=mk)
+    os_ = s.prefill_stream(q, k, -2.5 * v)
+    np.testing.assert_allclose(os_, -2.5 * oa, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(s.values(), -2.5 * a.values(), rtol=0, atol=1e-12)
+
+
+def test_units_are_independent_and_gqa_head_mapping():
+    B, Hq, Hkv, d, C, T = 2, 6, 3, 4, 5, 8
+    q, k, v = _rand(B, T, Hq, d), _rand(B, T, Hkv, d), _rand(B, T, Hkv, d)
+    full = O.OracleCache(B, Hq, Hkv, d, C)
+    out = full.prefill_stream(q, k, v)
+    G = Hq // Hkv
+    for b in range(B):
+        for h in range(Hkv):
+            one = O.OracleCache(1, G, 1, d, C)
+            o1 = one.prefill_stream(q[b:b + 1, :, h * G:(h + 1) * G], k[b:b + 1, :, h:h + 1], v[b:b + 1, :, h:h + 1])
+            np.testing.assert_array_equal(o1[0], out[b, :, h * G:(h + 1) * G])
+            np.testing.assert_array_equal(one.values()[0, 0], full.values()[b, h])
+
+
+# ---------------------------------------------------------------------------------------
+# Consistency: chunked streams concatenate; stream == repeated decode steps
+# ---------------------------------------------------------------------------------------
+def test_split_stream_equals_one_stream_and_decode_steps():
+    B, Hq, Hkv, d, C, T = 2, 2, 1, 4, 6, 15
+    q, k, v = _rand(B, T, Hq, d), _rand(B, T, Hkv, d), _rand(B, T, Hkv, d)
+    a = O.OracleCache(B, Hq, Hkv, d, C)
+    oa = a.prefill_stream(q, k, v)
+    b = O.OracleCache(B, Hq, Hkv, d, C)
+    ob = np.concatenate([b.prefill_stream(q[:, :4], k[:, :4], v[:, :4]),
+                         b.prefill_stream(q[:, 4:9], k[:, 4:9], v[:, 4:9]),
+                         b.prefill_stream(q[:, 9:], k[:, 9:], v[:, 9:])], axis=1)
+    np.testing.assert_array_equal(oa, ob)
+    np.testing.assert_array_equal(a.values(), b.values())
+    c = O.OracleCache(B, Hq, Hkv, d, C)
+    oc = np.stack([c.decode_step(q[:, t], k[:, t], v[:, t]) for t in range(T)], axis=1)
+    np.testing.assert_array_equal(oa, oc)
+    # resume from an exported state
+    r = O.OracleCache(B, Hq, Hkv, d, C, init_len=b.len, mk_init=b.keys(), mv_init=b.values())
+    x = _rand(B, 3, Hq, d), _rand(B, 3, Hkv, d), _rand(B, 3, Hkv, d)
+    np.testing.assert_array_equal(r.prefill_stream(*x), b.prefill_stream(*x))
+
+
+# ---------------------------------------------------------------------------------------
+# Brute force on tiny inputs, long-hand in pure Python (no numpy, no oracle code)
+# ---------------------------------------------------------------------------------------
+def _longhand(C, d, G, T, MK0, MV0, init_len, q, k, v, rs, ws):
+    """Evaluate the method token by token with Python scalars and math.exp only."""
+    MK = [[MK0[j][e] for e in range(d)] for j in range(init_len)]
+    MV = [[MV0[j][e] for e in range(d)] for j in range(init_len)]
+    outs = []
+    for t in range(T):
+        full = len(MK) == C
+        if not full:
+            MK.append(list(k[t]))
+            MV.append(list(v[t]))
+        n = len(MK)
+        row = []
+        for g in range(G):
+            sc = [rs * sum(q[t][g][e] * MK[j][e] for e in range(d)) for j in range(n)]
+            z = sum(math.exp(x) for x in sc)              # no max-subtraction: tiny scores
+            row.append([sum(math.exp(sc[j]) / z * MV[j][e] for j in range(n)) for e in range(d)])
+        outs.append(row)
+        if full:
+            sc = [ws * sum(k[t][e] * MK[j][e] for e in range(d)) for j in range(C)]
+            z = sum(math.exp(x) for x in sc)
+            MV = [[MV[j][e] + math.exp(sc[j]) / z * v[t][e] for e in range(d)] for j in range(C)]
+    return outs, MV
+
+
+@pytest.mark.parametrize("C,d,G,T,init_len", [(1, 1, 1, 3, 0), (2, 2, 1, 4, 0), (3, 2, 2, 4, 3), (3, 1, 1, 4, 1),
+                                              (2, 2, 2, 3, 2)])
+def test_brute_force_tiny(C, d, G, T, init_len):
+    MK0, MV0 = _rand(C, d), _rand(C, d)
+    q, k, v = _rand(T, G, d), _rand(T, d), _rand(T, d)
+    rs, ws = 0.6, 1.1
+    outs, MV = _longhand(C, d, G, T, MK0.tolist(), MV0.tolist(), init_len, q.tolist(), k.tolist(), v.tolist(), rs, ws)
+    c = O.OracleCache(1, G, 1, d, C, read_scale=rs, write_scale=ws, init_len=init_len,
+                      mk_init=MK0[None, None, :init_len] if init_len else None,
+                      mv_init=MV0[None, None, :init_len] if init_len else None)
+    out = c.prefill_stream(q[None], k[None, :, None], v[None, :, None])
+    np.testing.assert_allclose(out[0], np.array(outs), rtol=0, atol=1e-12)
+    np.testing.assert_allclose(c.values()[0, 0, :len(MV)], np.array(MV), rtol=0, atol=1e-12)
+
+
+def test_default_scales():
+    d, C = 16, 4
+    mk, mv0 = _rand(1, 1, C, d), _rand(1, 1, C, d)
+    q, k, v = _rand(1, 1, 1, d), _rand(1, 1, 1, d), _rand(1, 1, 1, d)
+    c = O.OracleCache(1, 1, 1, d, C, init_len=C, mk_init=mk, mv_init=mv0)
+    o = c.prefill_stream(q, k, v)
+    p = _np_softmax((q[0, 0, 0] @ mk[0, 0].T) / math.sqrt(d))  # textbook 1/sqrt(d) read scale
+    ww = _np_softmax(k[0, 0, 0] @ mk[0, 0].T)                  # Algorithm 1 prints no write scale
+    np.testing.assert_allclose(o[0, 0, 0], p @ mv0[0, 0], rtol=0, atol=1e-13)
+    np.testing.assert_allclose(c.values()[0, 0], mv0[0, 0] + np.outer(ww, v[0, 0, 0]), rtol=0, atol=1e-13)
