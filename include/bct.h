@@ -1,0 +1,193 @@
+/*
+ * bct.h: C ABI of the bounded-cache attention library for NVIDIA B200 (sm_100a).
+ *
+ * One attention layer of a Bounded-Cache Transformer keeps, per (sequence, kv-head)
+ * "unit", a key vector sequence MK and a key-value vector sequence MV of a predefined
+ * number of slots M (Method, "Model Structure"); here M is called `capacity` (C).
+ * Per token, every query head of the unit reads the resident slots with softmax
+ * attention, and the update rule of the paper then rewrites MV in place
+ * (Method step 4, Algorithm 1, Illustration step 3):
+ *
+ *     read :  o_g  = softmax(read_scale  * q_g . MK^T) . MV_{t-1}       g = 0..G-1
+ *     write:  MV_t = MV_{t-1} + softmax(write_scale * k_t . MK^T)^T . v_t
+ *
+ * q_g are the token's read queries (G = n_q_heads / n_kv_heads per unit), k_t is the
+ * paper's write query wq_t and v_t its write key-value vector wv_t; the projections
+ * that produce them (Algorithm 1, first two statements of the loop) are upstream of
+ * this library.  MK is never assigned by Algorithm 1 and is frozen once resident.
+ * While fewer than `capacity` slots are resident (a cache created with
+ * init_len < capacity), a token's (k_t, v_t) is appended at slot `len`, the read covers
+ * the len+1 resident slots, and no soft write happens.
+ *
+ * General conventions
+ *  - Every pointer marked DEVICE is a device address on the current CUDA device,
+ *    16-byte aligned, in memory the caller owns.  Pointers marked HOST are host
+ *    addresses (pinned memory makes the copies asynchronous).
+ *  - The library never allocates or frees device memory: all device storage is the
+ *    caller's workspace given to bct_cache_create.
+ *  - Every call validates its arguments on the host before enqueuing anything and
+ *    returns a bct_status_t; a failed call enqueues nothing and leaves the cache as
+ *    it was.  bct_last_error() gives a thread-local message for the last failure.
+ *  - Work is enqueued on the `cuda_stream` argument (a cudaStream_t passed as void*;
+ *    NULL is the default stream) and the call returns without synchronising, except
+ *    where stated.
+ *  - A handle is not thread-safe; different handles are independent.
+ *  - `len` (resident slots) is the same for every sequence of the batch.
+ */
+#ifndef BCT_H_
+#define BCT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum bct_status {
+    BCT_OK = 0,
+    BCT_ERR_INVALID_ARG = 1, /* NULL / misaligned pointer, out-of-range size */
+    BCT_ERR_UNSUPPORTED = 2, /* a shape or flag this build has no kernel for */
+    BCT_ERR_STATE = 3,       /* destroyed or corrupted handle */
+    BCT_ERR_CUDA = 4,        /* a CUDA runtime call failed; see bct_last_error() */
+    BCT_ERR_TIMEOUT = 5      /* a bounded device-side wait gave up (bct_cache_status) */
+} bct_status_t;
+
+typedef enum bct_dtype {
+    BCT_F32 = 0, /* cache planes and step vectors in float */
+    BCT_BF16 = 1 /* cache planes and step vectors in bfloat16, fp32 accumulation;
+                    MV additionally carries a bfloat16 residual plane so that the
+                    accumulated state keeps about 16 significand bits */
+} bct_dtype_t;
+
+/* flags */
+#define BCT_FLAG_SKIP_FIRST_WRITE 1u /* Algorithm 1's literal "if t = 1": the first
+                                        full-phase token leaves MV unchanged */
+#define BCT_FLAG_WRITE_THEN_READ 2u  /* the token's read sees its own write */
+#define BCT_FLAG_DENSE_WRITE 4u      /* rewrite every slot, whatever its write weight */
+
+typedef struct bct_params {
+    int32_t batch;      /* B  >= 1 sequences */
+    int32_t n_q_heads;  /* Hq >= 1, a multiple of n_kv_heads; G = Hq / Hkv <= 8 */
+    int32_t n_kv_heads; /* Hkv >= 1; one (MK, MV) memory per (sequence, kv-head) */
+    int32_t head_dim;   /* d in {64, 128} */
+    int32_t capacity;   /* C >= 1: the paper's predefined number of slots M */
+    int32_t dtype;      /* bct_dtype_t */
+    float read_scale;   /* <= 0 selects 1/sqrt(head_dim) */
+    float write_scale;  /* <= 0 selects 1.0 (Algorithm 1 prints no scale) */
+    int32_t init_len;   /* resident slots at create, 0..C; C is the paper's full-size MV_0 */
+    uint32_t flags;     /* BCT_FLAG_* */
+    float write_eps;    /* a slot whose write weight ww_j is below this is not rewritten
+                           (its increment ww_j * v_t is dropped); <= 0 selects 2^-24.
+                           Ignored with BCT_FLAG_DENSE_WRITE. */
+    int32_t max_stream; /* largest T a later bct_prefill_stream_host call may pass;
+                           sizes the staging area of the host-buffer entry points.
+                           <= 0 selects 1. */
+} bct_params_t;
+
+typedef struct bct_cache bct_cache_t; /* opaque, host-side */
+
+/* Library version as major*10000 + minor*100 + patch. */
+int32_t bct_version(void);
+
+/* Message of the calling thread's last failed call ("" if none).  Never NULL. */
+const char *bct_last_error(void);
+
+/*
+ * Size and alignment of the device workspace a cache with these parameters needs
+ * (Method, "Model Structure": MK and MV of M slots each, per unit; plus the bfloat16
+ * residual plane, the status words and the staging area of the *_host entry points).
+ * The size depends on the parameters only and never grows afterwards, which is the
+ * bounded-memory property of the method ("Fixed-Length Cache").
+ */
+bct_status_t bct_cache_bytes(const bct_params_t *params, size_t *bytes, size_t *align);
+
+/*
+ * Build a cache over caller-owned device memory and import its initial state.
+ *   workspace  DEVICE, `bytes` >= bct_cache_bytes, aligned as bct_cache_bytes says;
+ *              owned by the caller, must outlive the handle; the library writes to it.
+ *   mk_init    DEVICE [B][Hkv][init_len][d] in `dtype`: the paper's MK (rows beyond
+ *              init_len do not exist yet).  NULL allowed iff init_len == 0.
+ *   mv_init    DEVICE, same shape: the paper's MV_0.  NULL with init_len > 0 means
+ *              zeros ("initialized to zero or random values").
+ * The import is enqueued on cuda_stream.  On success *out receives the handle.
+ */
+bct_status_t bct_cache_create(const bct_params_t *params, void *workspace, size_t bytes,
+                              const void *mk_init, const void *mv_init, void *cuda_stream,
+                              bct_cache_t **out);
+
+/*
+ * One token per sequence (Method steps 2-5 for the write, softmax attention for the read).
+ *   q    DEVICE [B][Hq][d]   read queries; heads h*G .. h*G+G-1 belong to kv-head h
+ *   k    DEVICE [B][Hkv][d]  write queries wq_t (appended as keys during the fill phase)
+ *   v    DEVICE [B][Hkv][d]  write key-value vectors wv_t
+ *   out  DEVICE [B][Hq][d]   attention outputs, written by the call
+ * all contiguous, in the cache's dtype.  The cache advances by one token.
+ */
+bct_status_t bct_decode_step(bct_cache_t *cache, const void *q, const void *k, const void *v,
+                             void *out, void *cuda_stream);
+
+/*
+ * T tokens per sequence, equivalent to T successive bct_decode_step calls within
+ * rounding (Algorithm 1's loop over t = 1..N; with out == NULL it is UpdateKV itself,
+ * which returns only the final MV_N).
+ *   q    DEVICE [B][T][Hq][d]
+ *   k,v  DEVICE [B][T][Hkv][d]
+ *   out  DEVICE [B][T][Hq][d] or NULL
+ * May be called repeatedly; successive calls concatenate.  T >= 1.
+ */
+bct_status_t bct_prefill_stream(bct_cache_t *cache, const void *q, const void *k, const void *v,
+                                void *out, int64_t T, void *cuda_stream);
+
+/*
+ * Host-buffer forms of the two calls above: the same shapes, but q, k, v and out are
+ * HOST pointers.  The inputs are copied into the workspace's staging area, the step
+ * runs, and out is copied back, all on cuda_stream; the call returns without
+ * synchronising, so out is valid once the stream has drained, and q, k, v must stay
+ * unchanged until then.  T must not exceed the max_stream given at create.
+ */
+bct_status_t bct_decode_step_host(bct_cache_t *cache, const void *q, const void *k, const void *v,
+                                  void *out, void *cuda_stream);
+bct_status_t bct_prefill_stream_host(bct_cache_t *cache, const void *q, const void *k,
+                                     const void *v, void *out, int64_t T, void *cuda_stream);
+
+/* Resident slots (0..C) after the work enqueued so far. Host bookkeeping; no sync. */
+bct_status_t bct_cache_len(const bct_cache_t *cache, int32_t *len);
+
+/*
+ * Copy the state out in the canonical layout (Method step 5, "stored back into the
+ * cache", made visible): k_out DEVICE [B][Hkv][C][d] in the cache dtype, v_out DEVICE
+ * [B][Hkv][C][d] in v_dtype (BCT_F32 gives the bfloat16 value plus its residual,
+ * exactly; BCT_BF16 the rounded value).  Rows >= len are written as zeros.  Either
+ * pointer may be NULL to skip that plane.
+ */
+bct_status_t bct_cache_export(bct_cache_t *cache, void *k_out, void *v_out, int32_t v_dtype,
+                              void *cuda_stream);
+
+/*
+ * Replace the state: k_in DEVICE [B][Hkv][len][d] in the cache dtype, v_in DEVICE
+ * [B][Hkv][len][d] in v_dtype (NULL = zeros), 0 <= len <= C.  Counters of tokens seen
+ * are kept.  export followed by import into a fresh cache resumes bit-exactly when
+ * v_dtype is BCT_F32.
+ */
+bct_status_t bct_cache_import(bct_cache_t *cache, const void *k_in, const void *v_in,
+                              int32_t v_dtype, int32_t len, void *cuda_stream);
+
+/*
+ * Synchronise cuda_stream and report the device-side status word: BCT_OK, or
+ * BCT_ERR_TIMEOUT if a bounded wait inside a kernel gave up (the affected step's
+ * results are then undefined; the context stays usable).  The only call that blocks.
+ */
+bct_status_t bct_cache_status(bct_cache_t *cache, void *cuda_stream);
+
+/* Number of kernels this handle has launched so far (host counter). */
+bct_status_t bct_cache_launches(const bct_cache_t *cache, int64_t *launches);
+
+/* Free the host-side handle (NULL is accepted).  Never touches the workspace, never
+ * synchronises: the caller drains the stream before reusing the workspace. */
+bct_status_t bct_cache_destroy(bct_cache_t *cache);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BCT_H_ */
