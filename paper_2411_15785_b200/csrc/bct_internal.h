@@ -1,0 +1,69 @@
+// Host-side internals of the bounded-cache attention library (not part of the ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/bct.h"
+
+namespace bct {
+
+constexpr uint64_t kMagic = 0x4243545f43414348ull;  // "BCT_CACH"
+constexpr size_t kAlign = 256;                      // alignment of every workspace section
+constexpr int kMaxGroup = 8;
+
+// Where the step vectors of one launch live and how to walk them.
+struct StepIO {
+    const void* q;   // read queries
+    const void* k;   // write queries
+    const void* v;   // write key-value vectors
+    void* out;       // may be NULL in state-only streams
+    int64_t q_batch_stride;   // elements between sequences in q / out
+    int64_t kv_batch_stride;  // elements between sequences in k / v
+};
+
+}  // namespace bct
+
+struct bct_cache {
+    uint64_t magic;
+    bct_params_t p;  // scales, eps and max_stream resolved to their effective values
+    int G;           // query heads per kv-head
+    int U;           // units = batch * n_kv_heads
+    int elem_bytes;
+    size_t row_bytes;    // head_dim * elem_bytes
+    size_t plane_bytes;  // U * capacity * row_bytes
+    char* ws;
+    size_t ws_bytes;
+    char* kplane;   // MK  [U][C][d]
+    char* vhi;      // MV  [U][C][d] (value, or its bfloat16 head)
+    char* vlo;      // MV residual plane (bfloat16 only), else NULL
+    int* status;    // device status words
+    char* stage_q;  // staging of the host-buffer entry points
+    char* stage_k;
+    char* stage_v;
+    char* stage_out;
+    int len;                // resident slots after the work enqueued so far
+    int64_t n_full_tokens;  // full-phase tokens enqueued so far
+    int64_t launches;
+    int device;
+    int sm_count;
+    int smem_optin;  // max dynamic shared memory per block (opt-in)
+};
+
+namespace bct {
+
+// One token for every unit: fill-phase append + read, or read + soft write.
+// `len` is the number of resident slots before the token; do_write = 0 suppresses the
+// soft write (literal first-token branch of Algorithm 1).  Returns the number of
+// kernels launched (>= 1) or a negative value with *err set.
+int launch_decode(const bct_cache* c, const StepIO& io, int len, int do_write, cudaStream_t stream,
+                  cudaError_t* err);
+
+// Whether launch_decode has a kernel for these parameters (shape limits of this build).
+bool decode_supported(const bct_params_t& p, int smem_optin, const char** why);
+
+// State import / export.
+cudaError_t launch_import(const bct_cache* c, const void* k_in, const void* v_in, int v_dtype, int len,
+                          cudaStream_t stream);
+cudaError_t launch_export(const bct_cache* c, void* k_out, void* v_out, int v_dtype, cudaStream_t stream);
+
+}  // namespace bct
