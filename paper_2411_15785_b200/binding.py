@@ -1,0 +1,210 @@
+"""Thin ctypes binding of ``libbct_b200.so`` with the names of ``include/bct.h``.
+
+Argument marshalling only: every step of the path runs in the library's CUDA kernels.
+PyTorch supplies device memory (the workspace and the step tensors) and the stream.
+There is no CPU fallback: ``load()`` raises when the library has not been built.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+import torch
+
+BCT_OK, BCT_ERR_INVALID_ARG, BCT_ERR_UNSUPPORTED, BCT_ERR_STATE, BCT_ERR_CUDA, BCT_ERR_TIMEOUT = range(6)
+BCT_F32, BCT_BF16 = 0, 1
+FLAG_SKIP_FIRST_WRITE, FLAG_WRITE_THEN_READ, FLAG_DENSE_WRITE = 1, 2, 4
+
+LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libbct_b200.so")
+
+EXPORTS = (
+    "bct_version", "bct_last_error", "bct_cache_bytes", "bct_cache_create", "bct_decode_step",
+    "bct_prefill_stream", "bct_decode_step_host", "bct_prefill_stream_host", "bct_cache_len",
+    "bct_cache_export", "bct_cache_import", "bct_cache_status", "bct_cache_launches", "bct_cache_destroy",
+)
+
+
+class BctParams(ctypes.Structure):
+    _fields_ = [
+        ("batch", ctypes.c_int32), ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
+        ("head_dim", ctypes.c_int32), ("capacity", ctypes.c_int32), ("dtype", ctypes.c_int32),
+        ("read_scale", ctypes.c_float), ("write_scale", ctypes.c_float), ("init_len", ctypes.c_int32),
+        ("flags", ctypes.c_uint32), ("write_eps", ctypes.c_float), ("max_stream", ctypes.c_int32),
+    ]
+
+
+class BctError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__("bct status %d: %s" % (status, message))
+        self.status = status
+
+
+_lib = None
+
+
+def load() -> ctypes.CDLL:
+    """Open the C-ABI library; raise if it is missing (build it with ``python -m paper_2411_15785_b200.build``)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError("%s not found: run `python -m paper_2411_15785_b200.build` (no CPU fallback exists)" % LIB_PATH)
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+    pp = ctypes.POINTER(BctParams)
+    lib.bct_version.restype = i32
+    lib.bct_version.argtypes = []
+    lib.bct_last_error.restype = ctypes.c_char_p
+    lib.bct_last_error.argtypes = []
+    lib.bct_cache_bytes.argtypes = [pp, ctypes.POINTER(ctypes.c_size_t), ctypes.POINTER(ctypes.c_size_t)]
+    lib.bct_cache_create.argtypes = [pp, vp, ctypes.c_size_t, vp, vp, vp, ctypes.POINTER(vp)]
+    lib.bct_decode_step.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.bct_prefill_stream.argtypes = [vp, vp, vp, vp, vp, i64, vp]
+    lib.bct_decode_step_host.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.bct_prefill_stream_host.argtypes = [vp, vp, vp, vp, vp, i64, vp]
+    lib.bct_cache_len.argtypes = [vp, ctypes.POINTER(i32)]
+    lib.bct_cache_export.argtypes = [vp, vp, vp, i32, vp]
+    lib.bct_cache_import.argtypes = [vp, vp, vp, i32, i32, vp]
+    lib.bct_cache_status.argtypes = [vp, vp]
+    lib.bct_cache_launches.argtypes = [vp, ctypes.POINTER(i64)]
+    lib.bct_cache_destroy.argtypes = [vp]
+    for name in EXPORTS[2:]:
+        getattr(lib, name).restype = ctypes.c_int
+    _lib = lib
+    return lib
+
+
+def last_error() -> str:
+    return load().bct_last_error().decode()
+
+
+def _check(status: int) -> None:
+    if status != BCT_OK:
+        raise BctError(status, last_error())
+
+
+def _dtype_code(dt: torch.dtype) -> int:
+    if dt == torch.float32:
+        return BCT_F32
+    if dt == torch.bfloat16:
+        return BCT_BF16
+    raise ValueError("dtype must be torch.float32 or torch.bfloat16")
+
+
+def make_params(batch, n_q_heads, n_kv_heads, head_dim, capacity, dtype, *, read_scale=0.0, write_scale=0.0,
+                init_len=0, flags=0, write_eps=0.0, max_stream=1) -> BctParams:
+    return BctParams(batch, n_q_heads, n_kv_heads, head_dim, capacity, _dtype_code(dtype), read_scale,
+                     write_scale, init_len, flags, write_eps, max_stream)
+
+
+def cache_bytes(params: BctParams) -> Tuple[int, int]:
+    b, a = ctypes.c_size_t(0), ctypes.c_size_t(0)
+    _check(load().bct_cache_bytes(ctypes.byref(params), ctypes.byref(b), ctypes.byref(a)))
+    return b.value, a.value
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return s.cuda_stream
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else t.data_ptr()
+
+
+class Cache:
+    """A bounded cache over a torch-allocated workspace.  Methods map 1:1 to the C calls."""
+
+    def __init__(self, batch, n_q_heads, n_kv_heads, head_dim, capacity, dtype=torch.bfloat16, *,
+                 read_scale=0.0, write_scale=0.0, init_len=0, flags=0, write_eps=0.0, max_stream=1,
+                 mk_init: Optional[torch.Tensor] = None, mv_init: Optional[torch.Tensor] = None,
+                 device="cuda", stream=None):
+        self.lib = load()
+        self.params = make_params(batch, n_q_heads, n_kv_heads, head_dim, capacity, dtype,
+                                  read_scale=read_scale, write_scale=write_scale, init_len=init_len,
+                                  flags=flags, write_eps=write_eps, max_stream=max_stream)
+        self.dtype = dtype
+        self.device = torch.device(device)
+        self.B, self.Hq, self.Hkv, self.d, self.C = batch, n_q_heads, n_kv_heads, head_dim, capacity
+        nbytes, align = cache_bytes(self.params)
+        self.workspace = torch.empty(nbytes + align, dtype=torch.uint8, device=self.device)
+        base = self.workspace.data_ptr()
+        self._ws_ptr = (base + align - 1) // align * align
+        self.workspace_bytes = nbytes
+        for t, name in ((mk_init, "mk_init"), (mv_init, "mv_init")):
+            if t is not None:
+                assert t.is_cuda and t.is_contiguous() and t.dtype == dtype, name
+                assert tuple(t.shape) == (batch, n_kv_heads, init_len, head_dim), (name, t.shape)
+        self._h = ctypes.c_void_p(None)
+        with torch.cuda.device(self.device):
+            _check(self.lib.bct_cache_create(ctypes.byref(self.params), self._ws_ptr, nbytes, _ptr(mk_init),
+                                             _ptr(mv_init), _stream_ptr(stream), ctypes.byref(self._h)))
+
+    # ---- steps ----------------------------------------------------------------------
+    def decode_step(self, q, k, v, out=None, stream=None):
+        if out is None:
+            out = torch.empty_like(q)
+        _check(self.lib.bct_decode_step(self._h, q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
+                                        _stream_ptr(stream)))
+        return out
+
+    def prefill_stream(self, q, k, v, out=None, want_out=True, stream=None):
+        T = q.shape[1]
+        if out is None and want_out:
+            out = torch.empty_like(q)
+        _check(self.lib.bct_prefill_stream(self._h, q.data_ptr(), k.data_ptr(), v.data_ptr(), _ptr(out), T,
+                                           _stream_ptr(stream)))
+        return out
+
+    def decode_step_host(self, q, k, v, out, stream=None):
+        """q, k, v, out: CPU tensors (pinned for asynchronous copies)."""
+        _check(self.lib.bct_decode_step_host(self._h, q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
+                                             _stream_ptr(stream)))
+        return out
+
+    def prefill_stream_host(self, q, k, v, out, stream=None):
+        _check(self.lib.bct_prefill_stream_host(self._h, q.data_ptr(), k.data_ptr(), v.data_ptr(), _ptr(out),
+                                                q.shape[1], _stream_ptr(stream)))
+        return out
+
+    # ---- state ----------------------------------------------------------------------
+    @property
+    def len(self) -> int:
+        n = ctypes.c_int32(0)
+        _check(self.lib.bct_cache_len(self._h, ctypes.byref(n)))
+        return n.value
+
+    @property
+    def launches(self) -> int:
+        n = ctypes.c_int64(0)
+        _check(self.lib.bct_cache_launches(self._h, ctypes.byref(n)))
+        return n.value
+
+    def export(self, v_dtype=torch.float32, stream=None):
+        shape = (self.B, self.Hkv, self.C, self.d)
+        k = torch.empty(shape, dtype=self.dtype, device=self.device)
+        v = torch.empty(shape, dtype=v_dtype, device=self.device)
+        _check(self.lib.bct_cache_export(self._h, k.data_ptr(), v.data_ptr(), _dtype_code(v_dtype), _stream_ptr(stream)))
+        return k, v
+
+    def import_state(self, k, v, length, stream=None):
+        vd = _dtype_code(v.dtype) if v is not None else _dtype_code(self.dtype)
+        _check(self.lib.bct_cache_import(self._h, _ptr(k), _ptr(v), vd, length, _stream_ptr(stream)))
+
+    def status(self, stream=None) -> int:
+        return self.lib.bct_cache_status(self._h, _stream_ptr(stream))
+
+    def check_status(self, stream=None) -> None:
+        _check(self.status(stream))
+
+    def destroy(self) -> None:
+        if self._h:
+            self.lib.bct_cache_destroy(self._h)
+            self._h = ctypes.c_void_p(None)
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass

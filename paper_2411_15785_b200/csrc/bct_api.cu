@@ -1,0 +1,337 @@
+// The C ABI of the bounded-cache attention library: argument validation, the opaque
+// handle, workspace carve-up and the launch sequence of each entry point.  No device
+// memory is allocated here; everything lives in the caller's workspace.
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "bct_internal.h"
+
+namespace {
+
+thread_local char g_err[512] = "";
+
+bct_status_t fail(bct_status_t st, const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return st;
+}
+
+bct_status_t fail_cuda(const char* what, cudaError_t e) {
+    return fail(BCT_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Offsets of the workspace sections.
+struct Carve {
+    size_t kplane, vhi, vlo, status, stage_q, stage_k, stage_v, stage_out, total;
+    size_t plane_bytes, q_bytes, kv_bytes;  // q_bytes / kv_bytes: staging for max_stream tokens
+};
+
+bct_status_t resolve_params(const bct_params_t* in, bct_params_t* p) {
+    if (in == nullptr) return fail(BCT_ERR_INVALID_ARG, "params is NULL");
+    *p = *in;
+    if (p->batch < 1 || p->n_q_heads < 1 || p->n_kv_heads < 1 || p->capacity < 1)
+        return fail(BCT_ERR_INVALID_ARG, "batch, n_q_heads, n_kv_heads and capacity must be >= 1");
+    if (p->n_q_heads % p->n_kv_heads != 0)
+        return fail(BCT_ERR_INVALID_ARG, "n_q_heads (%d) is not a multiple of n_kv_heads (%d)", p->n_q_heads,
+                    p->n_kv_heads);
+    if (p->dtype != BCT_F32 && p->dtype != BCT_BF16) return fail(BCT_ERR_INVALID_ARG, "unknown dtype %d", p->dtype);
+    if (p->head_dim < 1) return fail(BCT_ERR_INVALID_ARG, "head_dim must be >= 1");
+    if (p->init_len < 0 || p->init_len > p->capacity)
+        return fail(BCT_ERR_INVALID_ARG, "init_len %d outside 0..capacity (%d)", p->init_len, p->capacity);
+    if (p->flags & ~(BCT_FLAG_SKIP_FIRST_WRITE | BCT_FLAG_WRITE_THEN_READ | BCT_FLAG_DENSE_WRITE))
+        return fail(BCT_ERR_INVALID_ARG, "unknown flag bits 0x%x", p->flags);
+    if (!(p->read_scale > 0.f)) p->read_scale = 1.0f / std::sqrt((float)p->head_dim);
+    if (!(p->write_scale > 0.f)) p->write_scale = 1.0f;
+    if (!(p->write_eps > 0.f)) p->write_eps = 5.9604644775390625e-08f;  // 2^-24
+    if (p->max_stream <= 0) p->max_stream = 1;
+    if ((long long)p->batch * p->n_kv_heads > (1LL << 24))
+        return fail(BCT_ERR_INVALID_ARG, "batch * n_kv_heads too large");
+    if (p->head_dim != 64 && p->head_dim != 128)
+        return fail(BCT_ERR_UNSUPPORTED, "head_dim %d: this build has kernels for 64 and 128", p->head_dim);
+    if (p->n_q_heads / p->n_kv_heads > bct::kMaxGroup)
+        return fail(BCT_ERR_UNSUPPORTED, "group size %d > %d", p->n_q_heads / p->n_kv_heads, bct::kMaxGroup);
+    return BCT_OK;
+}
+
+Carve carve(const bct_params_t& p) {
+    Carve c;
+    const size_t eb = p.dtype == BCT_F32 ? 4 : 2;
+    const size_t U = (size_t)p.batch * p.n_kv_heads;
+    c.plane_bytes = U * (size_t)p.capacity * p.head_dim * eb;
+    c.q_bytes = (size_t)p.batch * p.max_stream * p.n_q_heads * p.head_dim * eb;
+    c.kv_bytes = (size_t)p.batch * p.max_stream * p.n_kv_heads * p.head_dim * eb;
+    size_t off = 0;
+    c.kplane = off;
+    off += round_up(c.plane_bytes, bct::kAlign);
+    c.vhi = off;
+    off += round_up(c.plane_bytes, bct::kAlign);
+    c.vlo = off;
+    off += (p.dtype == BCT_BF16) ? round_up(c.plane_bytes, bct::kAlign) : 0;
+    c.status = off;
+    off += bct::kAlign;
+    c.stage_q = off;
+    off += round_up(c.q_bytes, bct::kAlign);
+    c.stage_k = off;
+    off += round_up(c.kv_bytes, bct::kAlign);
+    c.stage_v = off;
+    off += round_up(c.kv_bytes, bct::kAlign);
+    c.stage_out = off;
+    off += round_up(c.q_bytes, bct::kAlign);
+    c.total = off;
+    return c;
+}
+
+bct_status_t check_handle(const bct_cache_t* c) {
+    if (c == nullptr) return fail(BCT_ERR_INVALID_ARG, "cache handle is NULL");
+    if (c->magic != bct::kMagic) return fail(BCT_ERR_STATE, "cache handle is destroyed or corrupted");
+    return BCT_OK;
+}
+
+bct_status_t check_step_ptrs(const void* q, const void* k, const void* v, const void* out, bool out_optional) {
+    if (q == nullptr || k == nullptr || v == nullptr) return fail(BCT_ERR_INVALID_ARG, "q, k and v must not be NULL");
+    if (out == nullptr && !out_optional) return fail(BCT_ERR_INVALID_ARG, "out must not be NULL");
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out))
+        return fail(BCT_ERR_INVALID_ARG, "q, k, v and out must be 16-byte aligned");
+    return BCT_OK;
+}
+
+// T tokens, one decode launch each.  Pointers are device pointers in [B][T][H][d].
+bct_status_t run_tokens(bct_cache_t* c, const void* q, const void* k, const void* v, void* out, int64_t T,
+                        cudaStream_t stream) {
+    const bct_params_t& p = c->p;
+    const size_t eb = (size_t)c->elem_bytes;
+    const size_t q_tok = (size_t)p.n_q_heads * p.head_dim;   // elements per token per sequence
+    const size_t kv_tok = (size_t)p.n_kv_heads * p.head_dim;
+    for (int64_t t = 0; t < T; ++t) {
+        bct::StepIO io;
+        io.q = static_cast<const char*>(q) + (size_t)t * q_tok * eb;
+        io.k = static_cast<const char*>(k) + (size_t)t * kv_tok * eb;
+        io.v = static_cast<const char*>(v) + (size_t)t * kv_tok * eb;
+        io.out = out ? static_cast<char*>(out) + (size_t)t * q_tok * eb : nullptr;
+        io.q_batch_stride = (int64_t)(T * q_tok);
+        io.kv_batch_stride = (int64_t)(T * kv_tok);
+        const bool full = (c->len == p.capacity);
+        const int do_write = !((p.flags & BCT_FLAG_SKIP_FIRST_WRITE) && c->n_full_tokens == 0);
+        cudaError_t e = cudaSuccess;
+        const int n = bct::launch_decode(c, io, c->len, do_write, stream, &e);
+        if (n < 0) return fail_cuda("decode launch", e);
+        c->launches += n;
+        if (full)
+            c->n_full_tokens += 1;
+        else
+            c->len += 1;
+    }
+    return BCT_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int32_t bct_version(void) { return 100; }
+
+const char* bct_last_error(void) { return g_err; }
+
+bct_status_t bct_cache_bytes(const bct_params_t* params, size_t* bytes, size_t* align) {
+    bct_params_t p;
+    bct_status_t st = resolve_params(params, &p);
+    if (st != BCT_OK) return st;
+    if (bytes == nullptr) return fail(BCT_ERR_INVALID_ARG, "bytes is NULL");
+    *bytes = carve(p).total;
+    if (align) *align = bct::kAlign;
+    return BCT_OK;
+}
+
+bct_status_t bct_cache_create(const bct_params_t* params, void* workspace, size_t bytes, const void* mk_init,
+                              const void* mv_init, void* cuda_stream, bct_cache_t** out) {
+    bct_params_t p;
+    bct_status_t st = resolve_params(params, &p);
+    if (st != BCT_OK) return st;
+    if (out == nullptr) return fail(BCT_ERR_INVALID_ARG, "out is NULL");
+    *out = nullptr;
+    if (workspace == nullptr) return fail(BCT_ERR_INVALID_ARG, "workspace is NULL");
+    if (reinterpret_cast<uintptr_t>(workspace) % bct::kAlign)
+        return fail(BCT_ERR_INVALID_ARG, "workspace must be %zu-byte aligned", bct::kAlign);
+    const Carve cv = carve(p);
+    if (bytes < cv.total) return fail(BCT_ERR_INVALID_ARG, "workspace of %zu bytes, %zu needed", bytes, cv.total);
+    if (p.init_len > 0 && mk_init == nullptr) return fail(BCT_ERR_INVALID_ARG, "mk_init is NULL with init_len > 0");
+    if (!aligned16(mk_init) || !aligned16(mv_init)) return fail(BCT_ERR_INVALID_ARG, "mk_init / mv_init misaligned");
+
+    int dev = 0, sms = 0, optin = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    if (e != cudaSuccess) return fail_cuda("device query", e);
+    const char* why = "";
+    if (!bct::decode_supported(p, optin, &why)) return fail(BCT_ERR_UNSUPPORTED, "%s", why);
+
+    bct_cache_t* c = new (std::nothrow) bct_cache_t();
+    if (c == nullptr) return fail(BCT_ERR_STATE, "out of host memory");
+    c->magic = bct::kMagic;
+    c->p = p;
+    c->G = p.n_q_heads / p.n_kv_heads;
+    c->U = p.batch * p.n_kv_heads;
+    c->elem_bytes = p.dtype == BCT_F32 ? 4 : 2;
+    c->row_bytes = (size_t)p.head_dim * c->elem_bytes;
+    c->plane_bytes = cv.plane_bytes;
+    c->ws = static_cast<char*>(workspace);
+    c->ws_bytes = bytes;
+    c->kplane = c->ws + cv.kplane;
+    c->vhi = c->ws + cv.vhi;
+    c->vlo = p.dtype == BCT_BF16 ? c->ws + cv.vlo : nullptr;
+    c->status = reinterpret_cast<int*>(c->ws + cv.status);
+    c->stage_q = c->ws + cv.stage_q;
+    c->stage_k = c->ws + cv.stage_k;
+    c->stage_v = c->ws + cv.stage_v;
+    c->stage_out = c->ws + cv.stage_out;
+    c->len = p.init_len;
+    c->n_full_tokens = 0;
+    c->launches = 0;
+    c->device = dev;
+    c->sm_count = sms;
+    c->smem_optin = optin;
+
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    e = cudaMemsetAsync(c->status, 0, bct::kAlign, stream);
+    if (e == cudaSuccess) e = bct::launch_import(c, mk_init, mv_init, p.dtype, p.init_len, stream);
+    if (e != cudaSuccess) {
+        c->magic = 0;
+        delete c;
+        return fail_cuda("state import", e);
+    }
+    c->launches += 1;
+    *out = c;
+    return BCT_OK;
+}
+
+bct_status_t bct_decode_step(bct_cache_t* c, const void* q, const void* k, const void* v, void* out,
+                             void* cuda_stream) {
+    bct_status_t st = check_handle(c);
+    if (st != BCT_OK) return st;
+    st = check_step_ptrs(q, k, v, out, false);
+    if (st != BCT_OK) return st;
+    return run_tokens(c, q, k, v, out, 1, static_cast<cudaStream_t>(cuda_stream));
+}
+
+bct_status_t bct_prefill_stream(bct_cache_t* c, const void* q, const void* k, const void* v, void* out, int64_t T,
+                                void* cuda_stream) {
+    bct_status_t st = check_handle(c);
+    if (st != BCT_OK) return st;
+    if (T < 1) return fail(BCT_ERR_INVALID_ARG, "T must be >= 1 (got %lld)", (long long)T);
+    st = check_step_ptrs(q, k, v, out, true);
+    if (st != BCT_OK) return st;
+    return run_tokens(c, q, k, v, out, T, static_cast<cudaStream_t>(cuda_stream));
+}
+
+bct_status_t bct_prefill_stream_host(bct_cache_t* c, const void* q, const void* k, const void* v, void* out,
+                                     int64_t T, void* cuda_stream) {
+    bct_status_t st = check_handle(c);
+    if (st != BCT_OK) return st;
+    if (T < 1) return fail(BCT_ERR_INVALID_ARG, "T must be >= 1 (got %lld)", (long long)T);
+    if (T > c->p.max_stream)
+        return fail(BCT_ERR_INVALID_ARG, "T = %lld exceeds max_stream = %d given at create", (long long)T,
+                    c->p.max_stream);
+    if (q == nullptr || k == nullptr || v == nullptr) return fail(BCT_ERR_INVALID_ARG, "q, k and v must not be NULL");
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const size_t eb = (size_t)c->elem_bytes;
+    const size_t qb = (size_t)c->p.batch * T * c->p.n_q_heads * c->p.head_dim * eb;
+    const size_t kb = (size_t)c->p.batch * T * c->p.n_kv_heads * c->p.head_dim * eb;
+    cudaError_t e = cudaMemcpyAsync(c->stage_q, q, qb, cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(c->stage_k, k, kb, cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(c->stage_v, v, kb, cudaMemcpyHostToDevice, stream);
+    if (e != cudaSuccess) return fail_cuda("host-to-device copy", e);
+    st = run_tokens(c, c->stage_q, c->stage_k, c->stage_v, out ? c->stage_out : nullptr, T, stream);
+    if (st != BCT_OK) return st;
+    if (out != nullptr) {
+        e = cudaMemcpyAsync(out, c->stage_out, qb, cudaMemcpyDeviceToHost, stream);
+        if (e != cudaSuccess) return fail_cuda("device-to-host copy", e);
+    }
+    return BCT_OK;
+}
+
+bct_status_t bct_decode_step_host(bct_cache_t* c, const void* q, const void* k, const void* v, void* out,
+                                  void* cuda_stream) {
+    if (out == nullptr) return fail(BCT_ERR_INVALID_ARG, "out must not be NULL");
+    return bct_prefill_stream_host(c, q, k, v, out, 1, cuda_stream);
+}
+
+bct_status_t bct_cache_len(const bct_cache_t* c, int32_t* len) {
+    bct_status_t st = check_handle(c);
+    if (st != BCT_OK) return st;
+    if (len == nullptr) return fail(BCT_ERR_INVALID_ARG, "len is NULL");
+    *len = c->len;
+    return BCT_OK;
+}
+
+bct_status_t bct_cache_export(bct_cache_t* c, void* k_out, void* v_out, int32_t v_dtype, void* cuda_stream) {
+    bct_status_t st = check_handle(c);
+    if (st != BCT_OK) return st;
+    if (v_dtype != BCT_F32 && v_dtype != BCT_BF16) return fail(BCT_ERR_INVALID_ARG, "unknown v_dtype %d", v_dtype);
+    if (c->p.dtype == BCT_F32 && v_dtype != BCT_F32)
+        return fail(BCT_ERR_UNSUPPORTED, "a float cache exports its values as float");
+    if (!aligned16(k_out) || !aligned16(v_out)) return fail(BCT_ERR_INVALID_ARG, "k_out / v_out misaligned");
+    if (k_out == nullptr && v_out == nullptr) return BCT_OK;
+    cudaError_t e = bct::launch_export(c, k_out, v_out, v_dtype, static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return fail_cuda("state export", e);
+    c->launches += 1;
+    return BCT_OK;
+}
+
+bct_status_t bct_cache_import(bct_cache_t* c, const void* k_in, const void* v_in, int32_t v_dtype, int32_t len,
+                              void* cuda_stream) {
+    bct_status_t st = check_handle(c);
+    if (st != BCT_OK) return st;
+    if (len < 0 || len > c->p.capacity) return fail(BCT_ERR_INVALID_ARG, "len %d outside 0..capacity", len);
+    if (v_dtype != BCT_F32 && v_dtype != BCT_BF16) return fail(BCT_ERR_INVALID_ARG, "unknown v_dtype %d", v_dtype);
+    if (c->p.dtype == BCT_F32 && v_dtype != BCT_F32)
+        return fail(BCT_ERR_UNSUPPORTED, "a float cache imports its values as float");
+    if (len > 0 && k_in == nullptr) return fail(BCT_ERR_INVALID_ARG, "k_in is NULL with len > 0");
+    if (!aligned16(k_in) || !aligned16(v_in)) return fail(BCT_ERR_INVALID_ARG, "k_in / v_in misaligned");
+    cudaError_t e = bct::launch_import(c, k_in, v_in, v_dtype, len, static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return fail_cuda("state import", e);
+    c->len = len;
+    c->launches += 1;
+    return BCT_OK;
+}
+
+bct_status_t bct_cache_status(bct_cache_t* c, void* cuda_stream) {
+    bct_status_t st = check_handle(c);
+    if (st != BCT_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    int host[2] = {0, 0};
+    cudaError_t e = cudaMemcpyAsync(host, c->status, sizeof(host), cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+    if (e != cudaSuccess) return fail_cuda("status read", e);
+    if (host[0] == BCT_ERR_TIMEOUT)
+        return fail(BCT_ERR_TIMEOUT, "a bounded wait inside a kernel gave up (site %d)", host[1]);
+    if (host[0] != 0) return fail(BCT_ERR_STATE, "device status word holds %d", host[0]);
+    return BCT_OK;
+}
+
+bct_status_t bct_cache_launches(const bct_cache_t* c, int64_t* launches) {
+    bct_status_t st = check_handle(c);
+    if (st != BCT_OK) return st;
+    if (launches == nullptr) return fail(BCT_ERR_INVALID_ARG, "launches is NULL");
+    *launches = c->launches;
+    return BCT_OK;
+}
+
+bct_status_t bct_cache_destroy(bct_cache_t* c) {
+    if (c == nullptr) return BCT_OK;
+    if (c->magic != bct::kMagic) return fail(BCT_ERR_STATE, "cache handle is destroyed or corrupted");
+    c->magic = 0;
+    delete c;
+    return BCT_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,158 @@
+"""GPU parity of bct_decode_step / bct_prefill_stream against the CPU oracle (through the C ABI)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import bct_oracle as O
+from paper_2411_15785_b200 import binding as B
+from paper_2411_15785_b200 import build as bld
+from paper_2411_15785_b200 import workloads as W
+
+from _parity import TOL, compare_out, compare_state, make_pair, pick_units, run_decode_parity, _unit_slices
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    bld.build()
+    B.load()
+
+
+def _small(name, **kw):
+    return W.CONFIGS[name].scaled(**kw)
+
+
+# ---- small shapes spanning several tiles, ragged tails, every dtype / head_dim / group -------------
+@pytest.mark.parametrize("dtype,d,G,C,init_len,steps", [
+    ("f32", 64, 1, 128, 0, 160),        # fills, then updates
+    ("f32", 64, 2, 197, 197, 6),        # ragged: not a multiple of the 64-row tile
+    ("f32", 128, 1, 75, 70, 12),        # fill finishes mid-run, 32-row tiles
+    ("f32", 128, 3, 300, 300, 4),
+    ("bf16", 128, 1, 333, 333, 8),
+    ("bf16", 128, 4, 520, 500, 30),
+    ("bf16", 64, 2, 1000, 1000, 5),     # 128-row tiles
+    ("bf16", 64, 8, 130, 0, 140),
+    ("bf16", 128, 8, 257, 257, 5),
+    ("bf16", 128, 5, 64, 64, 5),
+    ("f32", 64, 7, 3, 0, 9),            # tiny capacity
+    ("bf16", 128, 1, 1, 1, 4),          # C = 1: running sum
+])
+def test_small_shapes_match_oracle(dtype, d, G, C, init_len, steps):
+    w = W.Workload("t", 2, 2 * G, 2, d, C, dtype, init_len, steps, 11, d ** -0.5, 1.0, 1.0, "decode")
+    units = pick_units(w, 4)
+    out_err, state_err = run_decode_parity(w, units)
+    assert out_err <= TOL[dtype], out_err
+    assert state_err <= TOL[dtype], state_err
+
+
+def test_diffuse_writes_rewrite_every_row():
+    d = 128
+    w = W.Workload("t", 2, 4, 2, d, 700, "bf16", 700, 12, 5, d ** -0.5, 1.0, 1.0, "decode", 1.0, d ** -0.5)
+    out_err, state_err = run_decode_parity(w, pick_units(w, 4))
+    assert out_err <= TOL["bf16"] and state_err <= 1e-3, (out_err, state_err)
+
+
+def test_cluster_split_path_small_batch_large_capacity():
+    # one unit, C = 8192: the planner spreads the slots over an 8-CTA cluster
+    d = 128
+    w = W.Workload("t", 1, 4, 1, d, 8192, "bf16", 8192, 6, 6, d ** -0.5, 1.0, 1.0, "decode")
+    out_err, state_err = run_decode_parity(w, pick_units(w, 1))
+    assert out_err <= TOL["bf16"] and state_err <= TOL["bf16"], (out_err, state_err)
+    w2 = W.Workload("t", 1, 1, 1, 64, 5000, "f32", 4990, 20, 7, 0.125, 1.0, 1.0, "decode")
+    out_err, state_err = run_decode_parity(w2, pick_units(w2, 1))
+    assert out_err <= TOL["f32"] and state_err <= TOL["f32"], (out_err, state_err)
+
+
+@pytest.mark.parametrize("flag,oflag", [(B.FLAG_WRITE_THEN_READ, O.WRITE_THEN_READ),
+                                        (B.FLAG_SKIP_FIRST_WRITE, O.SKIP_FIRST_WRITE),
+                                        (B.FLAG_DENSE_WRITE, 0)])
+def test_flags_match_oracle(flag, oflag):
+    w = W.Workload("t", 2, 4, 2, 64, 150, "f32", 150, 5, 8, 0.125, 0.5, 1.0, "decode")
+    out_err, state_err = run_decode_parity(w, pick_units(w, 4), flags=flag, oracle_flags=oflag)
+    assert out_err <= TOL["f32"] and state_err <= TOL["f32"], (out_err, state_err)
+
+
+def test_prefill_stream_equals_decode_steps_and_state_only_mode():
+    w = W.CONFIGS["stream_b8_c1024"].scaled(batch=2, n_q_heads=4, n_kv_heads=4, capacity=96, steps=160)
+    units = pick_units(w, 8)
+    q, k, v = W.stream_inputs(w, 0, w.steps, "cuda")
+    gpu, ora = make_pair(w, units)
+    out = gpu.prefill_stream(q[:, :100].contiguous(), k[:, :100].contiguous(), v[:, :100].contiguous())
+    out2 = gpu.prefill_stream(q[:, 100:].contiguous(), k[:, 100:].contiguous(), v[:, 100:].contiguous())
+    ref = ora.prefill_stream(*_unit_slices(w, units, q, k, v))
+    err = compare_out(w, units, torch.cat([out, out2], dim=1), ref)
+    assert err <= TOL["bf16"], err
+    assert compare_state(w, units, gpu, ora) <= TOL["bf16"]
+    # the same tokens one decode step at a time give the same bits
+    gpu2, _ = make_pair(w, units)
+    outs = [gpu2.decode_step(q[:, t].contiguous(), k[:, t].contiguous(), v[:, t].contiguous()) for t in range(w.steps)]
+    assert torch.equal(torch.stack(outs, dim=1), torch.cat([out, out2], dim=1))
+    # state-only (UpdateKV): out = NULL
+    gpu3, _ = make_pair(w, units)
+    assert gpu3.prefill_stream(q, k, v, want_out=False) is None
+    k1, v1 = gpu.export()
+    k3, v3 = gpu3.export()
+    assert torch.equal(k1, k3) and torch.equal(v1, v3)
+
+
+def test_export_import_resume_is_bitwise():
+    w = W.Workload("t", 2, 4, 2, 128, 200, "bf16", 200, 10, 9, 128 ** -0.5, 1.0, 1.0, "decode")
+    units = pick_units(w, 4)
+    a, _ = make_pair(w, units)
+    b, _ = make_pair(w, units)
+    for t in range(5):
+        x = W.step_inputs(w, t, "cuda")
+        a.decode_step(*x)
+        b.decode_step(*x)
+    k, v = b.export(torch.float32)
+    c = B.Cache(w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.capacity, w.torch_dtype,
+                read_scale=w.read_scale, write_scale=w.write_scale)
+    c.import_state(k, v, b.len)
+    for t in range(5, 10):
+        x = W.step_inputs(w, t, "cuda")
+        oa, oc = a.decode_step(*x), c.decode_step(*x)
+        assert torch.equal(oa, oc)
+    ka, va = a.export()
+    kc, vc = c.export()
+    assert torch.equal(ka, kc) and torch.equal(va, vc)
+
+
+def test_run_twice_is_deterministic_and_host_entry_matches_device_entry():
+    w = W.Workload("t", 3, 8, 2, 128, 600, "bf16", 590, 24, 10, 128 ** -0.5, 1.0, 1.0, "decode")
+    units = pick_units(w, 6)
+    a, _ = make_pair(w, units)
+    b, _ = make_pair(w, units)
+    for t in range(w.steps):
+        q, k, v = W.step_inputs(w, t, "cuda")
+        oa = a.decode_step(q, k, v)
+        hq, hk, hv = q.cpu().pin_memory(), k.cpu().pin_memory(), v.cpu().pin_memory()
+        ho = torch.empty_like(hq).pin_memory()
+        b.decode_step_host(hq, hk, hv, ho)
+        torch.cuda.synchronize()
+        assert torch.equal(oa.cpu(), ho)
+    assert all(torch.equal(x, y) for x, y in zip(a.export(), b.export()))
+
+
+def test_create_rejects_bad_arguments_on_device_and_launches_nothing():
+    c = B.Cache(1, 1, 1, 64, 16, torch.float32)
+    n0 = c.launches
+    q = torch.zeros(1, 1, 64, device="cuda")
+    with pytest.raises(B.BctError) as e:
+        c.lib.bct_decode_step(c._h, q.data_ptr() + 4, q.data_ptr(), q.data_ptr(), q.data_ptr(), None) and B._check(1)
+    assert c.lib.bct_decode_step(c._h, q.data_ptr() + 4, q.data_ptr(), q.data_ptr(), q.data_ptr(), None) == B.BCT_ERR_INVALID_ARG
+    assert c.lib.bct_prefill_stream(c._h, q.data_ptr(), q.data_ptr(), q.data_ptr(), None, 0, None) == B.BCT_ERR_INVALID_ARG
+    assert c.lib.bct_prefill_stream_host(c._h, 4096, 4096, 4096, 4096, 5, None) == B.BCT_ERR_INVALID_ARG  # > max_stream
+    assert c.launches == n0 and c.len == 0
+    assert c.status() == B.BCT_OK
+    with pytest.raises(B.BctError):
+        B.Cache(1, 1, 1, 64, 16, torch.float32, init_len=4)  # mk_init missing
+    # capacity too large for the score array of an 8-CTA cluster
+    with pytest.raises(B.BctError) as e:
+        B.make_params  # noqa
+        p = B.make_params(1, 8, 1, 128, 1 << 20, torch.bfloat16)
+        import ctypes
+        h = ctypes.c_void_p(None)
+        ws = torch.empty(1024, dtype=torch.uint8, device="cuda")
+        B._check(c.lib.bct_cache_create(ctypes.byref(p), ws.data_ptr(), 1 << 62, None, None, None, ctypes.byref(h)))
+    assert e.value.status == B.BCT_ERR_UNSUPPORTED
