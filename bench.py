@@ -1,0 +1,289 @@
+#!/usr/bin/env python
+"""Benchmark of the bounded-cache decode step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+A "step" is one pass of the whole hot path over one batch: one bct_decode_step (one token
+per sequence: K stream, softmax statistics, V stream with the in-place update rule).
+The default workload is the batched 7B-MHA-shaped configuration (batch 64, 32 heads,
+head_dim 128, capacity 2048, bfloat16 cache) with seeded Gaussian inputs.  Prints ONE
+JSON line.  With N > 1 (torchrun) every rank runs the same per-GPU batch on its own GPU
+(units are independent: no collective on the data path) and the value is the aggregate.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2411_15785_b200 import workloads as W  # noqa: E402
+
+METRIC = "bounded-cache decode tokens/s"
+UNIT = "tokens/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            return float(json.load(open(path))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        mhz, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                mhz.append(float(parts[0]))
+                mx = float(parts[1])
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        mhz.sort()
+        return {"sm_mhz": mhz[len(mhz) // 2] if mhz else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(mhz)}
+
+
+def algorithmic_bytes_per_step(w: W.Workload) -> int:
+    """Bytes the method must move per step: MK once + MV once per unit, plus the step vectors.
+    The write-back of the few rows the update rule changes is left out (a conservative count)."""
+    s = w.elem_bytes
+    per_unit = 2 * w.capacity * w.head_dim * s + (2 * w.group + 2) * w.head_dim * s
+    return w.units * per_unit
+
+
+def cpu_oracle_sample(w: W.Workload, budget_s: float = 15.0):
+    """Time the CPU oracle, as it stands, on a bounded sample of the workload."""
+    from oracle import bct_oracle as O
+    import numpy as np
+    cores = os.cpu_count() or 1
+    n_units = max(cores, 8)
+    n_units = min(n_units, w.units)
+    rng = np.random.default_rng(w.seed)
+    mk = rng.standard_normal((n_units, 1, w.init_len, w.head_dim)) * w.init_std if w.init_len else None
+    mv = rng.standard_normal((n_units, 1, w.init_len, w.head_dim)) * w.init_std if w.init_len else None
+    ora = O.OracleCache(n_units, w.group, 1, w.head_dim, w.capacity, read_scale=w.read_scale,
+                        write_scale=w.write_scale, init_len=w.init_len, mk_init=mk, mv_init=mv)
+
+    def draw(T):
+        return (rng.standard_normal((n_units, T, w.group, w.head_dim)) * w.q_std,
+                rng.standard_normal((n_units, T, 1, w.head_dim)) * w.kv_std,
+                rng.standard_normal((n_units, T, 1, w.head_dim)) * w.kv_std)
+
+    t0 = time.perf_counter()
+    ora.prefill_stream(*draw(1))
+    one = max(time.perf_counter() - t0, 1e-4)
+    T = int(max(2, min(w.steps, budget_s / one)))
+    x = draw(T)
+    t0 = time.perf_counter()
+    ora.prefill_stream(*x)
+    dt = time.perf_counter() - t0
+    unit_tokens_per_s = n_units * T / dt
+    return {"value": unit_tokens_per_s / w.n_kv_heads, "unit": UNIT, "cores": int(ora.threads_used), "kind": "oracle",
+            "sample": "%d of %d (sequence, kv-head) units x %d tokens in %.1f s, scaled by units per sequence"
+                      % (n_units, w.units, T, dt), "seconds": dt, "tokens": T}
+
+
+def run_reference(args, w):
+    """The reference arm: the double-precision CPU oracle on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    per_step = []
+    total = args.steps + args.warmup
+    budget = min(20.0, 120.0 / max(total, 1))
+    res = None
+    for i in range(total):
+        res = cpu_oracle_sample(w, budget_s=budget)
+        if i >= args.warmup:
+            per_step.append(res)
+    val = sum(r["value"] for r in per_step) / len(per_step)
+    ms = 1e3 * w.batch / val
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "batch": w.batch, "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads,
+                       "head_dim": w.head_dim, "capacity": w.capacity},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": res["cores"], "kind": "oracle", "sample": res["sample"]},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--workload", default="mha7b_b64_c2048", choices=sorted(W.CONFIGS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--write-scale", type=float, default=None, help="override the write score scale")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    w = W.CONFIGS[args.workload]
+    if args.write_scale is not None:
+        w = w.scaled(write_scale=args.write_scale)
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+    if args.warmup < 3:
+        args.warmup = 3
+
+    from paper_2411_15785_b200 import binding as B
+    from paper_2411_15785_b200 import build as bld
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        bld.build()
+    if world > 1:
+        dist.barrier()
+    B.load()
+
+    # per-rank workload: the same per-GPU batch on every rank (weak scaling), a different seed per rank
+    wr = w.scaled(seed=w.seed + 1000 * rank)
+    mk, mv = W.initial_cache(wr, dev)
+    cache = B.Cache(w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.capacity, w.torch_dtype,
+                    read_scale=w.read_scale, write_scale=w.write_scale, init_len=w.init_len, mk_init=mk, mv_init=mv,
+                    device=dev)
+    torch.cuda.synchronize()
+    del mk, mv
+    pool = [W.step_inputs(wr, t, dev) for t in range(min(args.steps + args.warmup, 64))]
+    outs = [torch.empty_like(pool[0][0]) for _ in range(2)]
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    # ---------- device-resident timing ----------
+    for i in range(args.warmup):
+        cache.decode_step(*pool[i % len(pool)], out=outs[i & 1])
+    sync_all()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    launches0 = cache.launches
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        cache.decode_step(*pool[(args.warmup + i) % len(pool)], out=outs[i & 1])
+    e1.record()
+    sync_all()
+    ms_total = e0.elapsed_time(e1)
+    launches = cache.launches - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    cache.check_status()
+
+    # ---------- end to end through the host-buffer entry point ----------
+    hpool = [tuple(x.cpu().pin_memory() for x in pool[i]) for i in range(min(len(pool), 16))]
+    hout = [torch.empty_like(hpool[0][0]).pin_memory() for _ in range(2)]
+    for i in range(3):
+        cache.decode_step_host(*hpool[i % len(hpool)], hout[i & 1])
+    sync_all()
+    e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e2.record()
+    for i in range(args.steps):
+        cache.decode_step_host(*hpool[i % len(hpool)], hout[i & 1])
+    e3.record()
+    sync_all()
+    ms_e2e = e2.elapsed_time(e3)
+    cache.check_status()
+    h2d = sum(x.numel() * x.element_size() for x in hpool[0])
+    d2h = hout[0].numel() * hout[0].element_size()
+
+    if world > 1:
+        t = torch.tensor([ms_total, ms_e2e], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total, ms_e2e = t.tolist()
+
+    if rank == 0:
+        peak, peak_kind = _peaks()
+        ms_step = ms_total / args.steps
+        tokens = w.batch * world * args.steps
+        alg = algorithmic_bytes_per_step(w)
+        achieved = alg / (ms_step * 1e-3) / 1e9
+        line = {
+            "metric": METRIC, "value": tokens / (ms_total * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32" if w.dtype == "f32" else "bf16 cache, f32 accumulate",
+            "data": "synthetic",
+            "config": {"workload": w.name, "batch_per_gpu": w.batch, "n_q_heads": w.n_q_heads,
+                       "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim, "capacity": w.capacity,
+                       "write_scale": w.write_scale, "read_scale": w.read_scale,
+                       "l2": "cache planes streamed per step (%.2f GB) exceed L2" % (alg / 1e9),
+                       "parallelism": "independent units; replicas per GPU" if world > 1 else "1 GPU"},
+            "clocks": clocks,
+            "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.steps},
+            "gpu_launches": launches,
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": None, "peak_kind": "of " + peak_kind, "kernel": "decode_kernel",
+                         "algorithmic_bytes_per_launch": alg, "frac_of_8TBps_nominal": achieved / 8000.0},
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            cb = cpu_oracle_sample(w)
+            line["cpu_baseline"] = {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")}
+        print(json.dumps(line))
+    cache.destroy()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -58,6 +58,10 @@ typedef enum bct_dtype {
     BCT_BF16 = 1 /* cache planes and step vectors in bfloat16, fp32 accumulation;
                     MV additionally carries a bfloat16 residual plane so that the
                     accumulated state keeps about 16 significand bits */
+    ,
+    BCT_BF16_PAIR = 2 /* checkpoint format of a bfloat16 cache's MV only (export / import):
+                         one 32-bit word per element, value plane bits in the high half,
+                         residual plane bits in the low half; lossless */
 } bct_dtype_t;
 
 /* flags */
@@ -158,8 +162,8 @@ bct_status_t bct_cache_len(const bct_cache_t *cache, int32_t *len);
  * Copy the state out in the canonical layout (Method step 5, "stored back into the
  * cache", made visible): k_out DEVICE [B][Hkv][C][d] in the cache dtype, v_out DEVICE
  * [B][Hkv][C][d] in v_dtype (BCT_F32 gives the bfloat16 value plus its residual,
- * exactly; BCT_BF16 the rounded value).  Rows >= len are written as zeros.  Either
- * pointer may be NULL to skip that plane.
+ * exactly; BCT_BF16 the rounded value; BCT_BF16_PAIR both planes bit for bit).  Rows
+ * >= len are written as zeros.  Either pointer may be NULL to skip that plane.
  */
 bct_status_t bct_cache_export(bct_cache_t *cache, void *k_out, void *v_out, int32_t v_dtype,
                               void *cuda_stream);
@@ -167,8 +171,10 @@ bct_status_t bct_cache_export(bct_cache_t *cache, void *k_out, void *v_out, int3
 /*
  * Replace the state: k_in DEVICE [B][Hkv][len][d] in the cache dtype, v_in DEVICE
  * [B][Hkv][len][d] in v_dtype (NULL = zeros), 0 <= len <= C.  Counters of tokens seen
- * are kept.  export followed by import into a fresh cache resumes bit-exactly when
- * v_dtype is BCT_F32.
+ * are kept.  export followed by import into a fresh cache resumes bit-exactly with
+ * v_dtype BCT_BF16_PAIR (bfloat16 cache) or BCT_F32 (float cache); a bfloat16 cache
+ * re-imported from BCT_F32 holds the same values but may split a few of them
+ * differently between the value and residual planes.
  */
 bct_status_t bct_cache_import(bct_cache_t *cache, const void *k_in, const void *v_in,
                               int32_t v_dtype, int32_t len, void *cuda_stream);

@@ -13,7 +13,7 @@ from typing import Optional, Tuple
 import torch
 
 BCT_OK, BCT_ERR_INVALID_ARG, BCT_ERR_UNSUPPORTED, BCT_ERR_STATE, BCT_ERR_CUDA, BCT_ERR_TIMEOUT = range(6)
-BCT_F32, BCT_BF16 = 0, 1
+BCT_F32, BCT_BF16, BCT_BF16_PAIR = 0, 1, 2
 FLAG_SKIP_FIRST_WRITE, FLAG_WRITE_THEN_READ, FLAG_DENSE_WRITE = 1, 2, 4
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libbct_b200.so")
@@ -85,6 +85,8 @@ def _check(status: int) -> None:
 
 
 def _dtype_code(dt: torch.dtype) -> int:
+    if dt == torch.int32:  # checkpoint words: value-plane bits << 16 | residual-plane bits
+        return BCT_BF16_PAIR
     if dt == torch.float32:
         return BCT_F32
     if dt == torch.bfloat16:

@@ -276,7 +276,8 @@ bct_status_t bct_cache_len(const bct_cache_t* c, int32_t* len) {
 bct_status_t bct_cache_export(bct_cache_t* c, void* k_out, void* v_out, int32_t v_dtype, void* cuda_stream) {
     bct_status_t st = check_handle(c);
     if (st != BCT_OK) return st;
-    if (v_dtype != BCT_F32 && v_dtype != BCT_BF16) return fail(BCT_ERR_INVALID_ARG, "unknown v_dtype %d", v_dtype);
+    if (v_dtype != BCT_F32 && v_dtype != BCT_BF16 && v_dtype != BCT_BF16_PAIR)
+        return fail(BCT_ERR_INVALID_ARG, "unknown v_dtype %d", v_dtype);
     if (c->p.dtype == BCT_F32 && v_dtype != BCT_F32)
         return fail(BCT_ERR_UNSUPPORTED, "a float cache exports its values as float");
     if (!aligned16(k_out) || !aligned16(v_out)) return fail(BCT_ERR_INVALID_ARG, "k_out / v_out misaligned");
@@ -292,7 +293,8 @@ bct_status_t bct_cache_import(bct_cache_t* c, const void* k_in, const void* v_in
     bct_status_t st = check_handle(c);
     if (st != BCT_OK) return st;
     if (len < 0 || len > c->p.capacity) return fail(BCT_ERR_INVALID_ARG, "len %d outside 0..capacity", len);
-    if (v_dtype != BCT_F32 && v_dtype != BCT_BF16) return fail(BCT_ERR_INVALID_ARG, "unknown v_dtype %d", v_dtype);
+    if (v_dtype != BCT_F32 && v_dtype != BCT_BF16 && v_dtype != BCT_BF16_PAIR)
+        return fail(BCT_ERR_INVALID_ARG, "unknown v_dtype %d", v_dtype);
     if (c->p.dtype == BCT_F32 && v_dtype != BCT_F32)
         return fail(BCT_ERR_UNSUPPORTED, "a float cache imports its values as float");
     if (len > 0 && k_in == nullptr) return fail(BCT_ERR_INVALID_ARG, "k_in is NULL with len > 0");

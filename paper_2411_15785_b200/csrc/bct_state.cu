@@ -17,7 +17,7 @@ __device__ __forceinline__ float load_as_float(const void* p, size_t i) {
 // One thread per element of the [U][C][d] planes.
 template <typename CacheT>
 __global__ void import_kernel(CacheT* kplane, CacheT* vhi, __nv_bfloat16* vlo, const CacheT* k_in,
-                              const void* v_in, int v_is_f32, size_t U, int C, int d, int len) {
+                              const void* v_in, int v_mode, size_t U, int C, int d, int len) {
     const size_t n = U * (size_t)C * d;
     for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
         const size_t e = i % d;
@@ -25,27 +25,45 @@ __global__ void import_kernel(CacheT* kplane, CacheT* vhi, __nv_bfloat16* vlo, c
         const size_t u = i / ((size_t)C * d);
         CacheT kk = (CacheT)0.f;
         float vv = 0.f;
+        uint32_t pair = 0;
         if ((int)j < len) {
             const size_t src = (u * len + j) * d + e;
             kk = k_in[src];
-            if (v_in != nullptr) vv = v_is_f32 ? load_as_float<float>(v_in, src) : load_as_float<CacheT>(v_in, src);
+            if (v_in != nullptr) {
+                if (v_mode == 2)
+                    pair = reinterpret_cast<const uint32_t*>(v_in)[src];
+                else
+                    vv = v_mode == 1 ? load_as_float<float>(v_in, src) : load_as_float<CacheT>(v_in, src);
+            }
         }
         kplane[i] = kk;
-        const CacheT hi = (CacheT)vv;
-        vhi[i] = hi;
-        if (vlo != nullptr) vlo[i] = __float2bfloat16_rn(vv - (float)hi);
+        if (v_mode == 2) {  // bfloat16 cache only: both planes bit for bit
+            reinterpret_cast<uint16_t*>(vhi)[i] = (uint16_t)(pair >> 16);
+            reinterpret_cast<uint16_t*>(vlo)[i] = (uint16_t)(pair & 0xffffu);
+        } else {
+            const CacheT hi = (CacheT)vv;
+            vhi[i] = hi;
+            if (vlo != nullptr) vlo[i] = __float2bfloat16_rn(vv - (float)hi);
+        }
     }
 }
 
 template <typename CacheT>
 __global__ void export_kernel(const CacheT* kplane, const CacheT* vhi, const __nv_bfloat16* vlo, CacheT* k_out,
-                              void* v_out, int v_is_f32, size_t U, int C, int d, int len) {
+                              void* v_out, int v_mode, size_t U, int C, int d, int len) {
     const size_t n = U * (size_t)C * d;
     for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
         const size_t j = (i / d) % C;
         const bool live = (int)j < len;
         if (k_out != nullptr) k_out[i] = live ? kplane[i] : (CacheT)0.f;
-        if (v_out != nullptr) {
+        if (v_out != nullptr && v_mode == 2) {
+            uint32_t pair = 0;
+            if (live)
+                pair = ((uint32_t) reinterpret_cast<const uint16_t*>(vhi)[i] << 16) |
+                       reinterpret_cast<const uint16_t*>(vlo)[i];
+            reinterpret_cast<uint32_t*>(v_out)[i] = pair;
+        } else if (v_out != nullptr) {
+            const bool v_is_f32 = (v_mode == 1);
             float vv = 0.f;
             if (live) {
                 vv = (float)vhi[i];
@@ -71,7 +89,7 @@ cudaError_t launch_import(const bct_cache* c, const void* k_in, const void* v_in
                           cudaStream_t stream) {
     const size_t n = (size_t)c->U * c->p.capacity * c->p.head_dim;
     const unsigned grid = grid_for(n, c->sm_count);
-    const int v_is_f32 = (v_dtype == BCT_F32);
+    const int v_mode = (v_dtype == BCT_F32) ? 1 : (v_dtype == BCT_BF16_PAIR ? 2 : 0);
     if (c->p.dtype == BCT_F32) {
         import_kernel<float><<<grid, 256, 0, stream>>>(reinterpret_cast<float*>(c->kplane), reinterpret_cast<float*>(c->vhi),
                                                        nullptr, static_cast<const float*>(k_in), v_in, 1, (size_t)c->U,
@@ -79,7 +97,7 @@ cudaError_t launch_import(const bct_cache* c, const void* k_in, const void* v_in
     } else {
         import_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>(
             reinterpret_cast<__nv_bfloat16*>(c->kplane), reinterpret_cast<__nv_bfloat16*>(c->vhi),
-            reinterpret_cast<__nv_bfloat16*>(c->vlo), static_cast<const __nv_bfloat16*>(k_in), v_in, v_is_f32,
+            reinterpret_cast<__nv_bfloat16*>(c->vlo), static_cast<const __nv_bfloat16*>(k_in), v_in, v_mode,
             (size_t)c->U, c->p.capacity, c->p.head_dim, len);
     }
     return cudaGetLastError();
@@ -88,7 +106,7 @@ cudaError_t launch_import(const bct_cache* c, const void* k_in, const void* v_in
 cudaError_t launch_export(const bct_cache* c, void* k_out, void* v_out, int v_dtype, cudaStream_t stream) {
     const size_t n = (size_t)c->U * c->p.capacity * c->p.head_dim;
     const unsigned grid = grid_for(n, c->sm_count);
-    const int v_is_f32 = (v_dtype == BCT_F32);
+    const int v_mode = (v_dtype == BCT_F32) ? 1 : (v_dtype == BCT_BF16_PAIR ? 2 : 0);
     if (c->p.dtype == BCT_F32) {
         export_kernel<float><<<grid, 256, 0, stream>>>(reinterpret_cast<const float*>(c->kplane),
                                                        reinterpret_cast<const float*>(c->vhi), nullptr,
@@ -97,7 +115,7 @@ cudaError_t launch_export(const bct_cache* c, void* k_out, void* v_out, int v_dt
     } else {
         export_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>(
             reinterpret_cast<const __nv_bfloat16*>(c->kplane), reinterpret_cast<const __nv_bfloat16*>(c->vhi),
-            reinterpret_cast<const __nv_bfloat16*>(c->vlo), static_cast<__nv_bfloat16*>(k_out), v_out, v_is_f32,
+            reinterpret_cast<const __nv_bfloat16*>(c->vlo), static_cast<__nv_bfloat16*>(k_out), v_out, v_mode,
             (size_t)c->U, c->p.capacity, c->p.head_dim, c->len);
     }
     return cudaGetLastError();
