@@ -101,12 +101,53 @@ def algorithmic_bytes_per_step(w: W.Workload) -> int:
 
 
 def cpu_oracle_sample(w: W.Workload, budget_s: float = 15.0):
-    """Time the CPU oracle, as it stands, on a bounded sample of the workload."""
+    """Time the CPU oracle, as it stands, on a bounded sample of the workload: a few
+    (sequence, kv-head) units per core, for as many tokens as fit the time budget."""
     from oracle import bct_oracle as O
     import numpy as np
     cores = os.cpu_count() or 1
-    n_units = max(cores, 8)
-    n_units = min(n_units, w.units)
+    n_units = min(w.units, 2 * cores)
+    rng = np.random.default_rng(w.seed)
+
+    def fresh():
+        mk = rng.standard_normal((n_units, 1, w.init_len, w.head_dim)) * w.init_std if w.init_len else None
+        mv = rng.standard_normal((n_units, 1, w.init_len, w.head_dim)) * w.init_std if w.init_len else None
+        return O.OracleCache(n_units, w.group, 1, w.head_dim, w.capacity, read_scale=w.read_scale,
+                             write_scale=w.write_scale, init_len=w.init_len, mk_init=mk, mv_init=mv)
+
+    def draw(T):
+        return (rng.standard_normal((n_units, T, w.group, w.head_dim)) * w.q_std,
+                rng.standard_normal((n_units, T, 1, w.head_dim)) * w.kv_std,
+                rng.standard_normal((n_units, T, 1, w.head_dim)) * w.kv_std)
+
+    ora = fresh()
+    ora.prefill_stream(*draw(2))                      # loads the library, warms the caches
+    x = draw(8)
+    t0 = time.perf_counter()
+    ora.prefill_stream(*x)
+    per_token = max((time.perf_counter() - t0) / 8, 1e-6)
+    T = int(max(8, min(20000, budget_s / per_token)))
+    x = draw(T)
+    t0 = time.perf_counter()
+    ora.prefill_stream(*x)
+    dt = time.perf_counter() - t0
+    unit_tokens_per_s = n_units * T / dt
+    return {"value": unit_tokens_per_s / w.n_kv_heads, "unit": UNIT, "cores": int(ora.threads_used), "kind": "oracle",
+            "sample": "%d of %d (sequence, kv-head) units x %d tokens in %.1f s of wall time, scaled by %d units per sequence"
+                      % (n_units, w.units, T, dt, w.n_kv_heads), "seconds": dt, "tokens": T}
+
+
+def run_reference(args, w):
+    """The reference arm: the double-precision CPU oracle, as it stands, on the host cores.
+    Each step is a bounded sample of the workload (a few units per core for a few tokens),
+    sized so that the whole run ends within about two minutes."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import bct_oracle as O
+    import numpy as np
+    cores = os.cpu_count() or 1
+    n_units = min(w.units, 2 * cores)
     rng = np.random.default_rng(w.seed)
     mk = rng.standard_normal((n_units, 1, w.init_len, w.head_dim)) * w.init_std if w.init_len else None
     mv = rng.standard_normal((n_units, 1, w.init_len, w.head_dim)) * w.init_std if w.init_len else None
@@ -118,41 +159,30 @@ def cpu_oracle_sample(w: W.Workload, budget_s: float = 15.0):
                 rng.standard_normal((n_units, T, 1, w.head_dim)) * w.kv_std,
                 rng.standard_normal((n_units, T, 1, w.head_dim)) * w.kv_std)
 
-    t0 = time.perf_counter()
-    ora.prefill_stream(*draw(1))
-    one = max(time.perf_counter() - t0, 1e-4)
-    T = int(max(2, min(w.steps, budget_s / one)))
-    x = draw(T)
+    ora.prefill_stream(*draw(2))
+    x = draw(8)
     t0 = time.perf_counter()
     ora.prefill_stream(*x)
-    dt = time.perf_counter() - t0
-    unit_tokens_per_s = n_units * T / dt
-    return {"value": unit_tokens_per_s / w.n_kv_heads, "unit": UNIT, "cores": int(ora.threads_used), "kind": "oracle",
-            "sample": "%d of %d (sequence, kv-head) units x %d tokens in %.1f s, scaled by units per sequence"
-                      % (n_units, w.units, T, dt), "seconds": dt, "tokens": T}
-
-
-def run_reference(args, w):
-    """The reference arm: the double-precision CPU oracle on the host cores."""
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
-        return
-    per_step = []
+    per_token = max((time.perf_counter() - t0) / 8, 1e-6)
     total = args.steps + args.warmup
-    budget = min(20.0, 120.0 / max(total, 1))
-    res = None
+    T = int(max(1, min(4096, (100.0 / total) / per_token)))
+    elapsed = 0.0
     for i in range(total):
-        res = cpu_oracle_sample(w, budget_s=budget)
+        x = draw(T)
+        t0 = time.perf_counter()
+        ora.prefill_stream(*x)
         if i >= args.warmup:
-            per_step.append(res)
-    val = sum(r["value"] for r in per_step) / len(per_step)
-    ms = 1e3 * w.batch / val
+            elapsed += time.perf_counter() - t0
+    val = n_units * T * args.steps / elapsed / w.n_kv_heads
+    sample = ("each step: %d of %d (sequence, kv-head) units x %d tokens; value scaled by %d units per sequence"
+              % (n_units, w.units, T, w.n_kv_heads))
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * w.batch / val, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": w.name, "batch": w.batch, "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads,
-                       "head_dim": w.head_dim, "capacity": w.capacity},
-            "cpu_baseline": {"value": val, "unit": UNIT, "cores": res["cores"], "kind": "oracle", "sample": res["sample"]},
+            "config": {"workload": w.name, "batch_per_gpu": w.batch, "n_q_heads": w.n_q_heads,
+                       "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim, "capacity": w.capacity,
+                       "write_scale": w.write_scale, "read_scale": w.read_scale},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": int(ora.threads_used), "kind": "oracle", "sample": sample},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
@@ -161,7 +191,7 @@ def run_reference(args, w):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default="mha7b_b64_c2048", choices=sorted(W.CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])

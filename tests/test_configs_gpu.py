@@ -1,0 +1,79 @@
+"""Parity at the benchmark contract's full sizes and step counts, in the launch configuration
+bench.py times: every configuration runs on the device in full, and the CPU oracle follows a
+sample of (sequence, kv-head) units for ALL steps (exact for those units, since units never
+interact).  Checked per step and on the exported state after the last step."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2411_15785_b200 import binding as B
+from paper_2411_15785_b200 import build as bld
+from paper_2411_15785_b200 import workloads as W
+
+from _parity import TOL, compare_out, compare_state, make_pair, pick_units, run_decode_parity, _unit_slices
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    bld.build()
+    B.load()
+
+
+def _n_units():
+    return max(8, min(32, 2 * (os.cpu_count() or 4)))
+
+
+def test_config1_single_sequence_fp32_fill_then_update():
+    w = W.CONFIGS["single_fp32_c128"]
+    out_err, state_err = run_decode_parity(w, pick_units(w, 1))
+    assert out_err <= TOL["f32"] and state_err <= TOL["f32"], (out_err, state_err)
+
+
+def test_config2_mha_batch64_c2048_bf16():
+    w = W.CONFIGS["mha7b_b64_c2048"]
+    out_err, state_err = run_decode_parity(w, pick_units(w, _n_units(), seed=1))
+    assert out_err <= TOL["bf16"] and state_err <= TOL["bf16"], (out_err, state_err)
+
+
+def test_config3_gqa_batch128_c4096_bf16():
+    w = W.CONFIGS["gqa8b_b128_c4096"]
+    out_err, state_err = run_decode_parity(w, pick_units(w, _n_units(), seed=2))
+    assert out_err <= TOL["bf16"] and state_err <= TOL["bf16"], (out_err, state_err)
+
+
+@pytest.mark.parametrize("C", [256, 1024, 4096, 16384])
+def test_config5_capacity_sweep(C):
+    w = W.CONFIGS["sweep_b256_c%d" % C]
+    n = _n_units() if C <= 4096 else 8
+    out_err, state_err = run_decode_parity(w, pick_units(w, n, seed=4))
+    assert out_err <= TOL["bf16"] and state_err <= TOL["bf16"], (out_err, state_err)
+    torch.cuda.empty_cache()
+
+
+def test_config2_diffuse_write_regime():
+    # secondary regime: write_scale = 1/sqrt(d) makes every slot's weight matter (all rows rewritten)
+    w = W.CONFIGS["mha7b_b64_c2048"].scaled(write_scale=128 ** -0.5, steps=256)
+    out_err, state_err = run_decode_parity(w, pick_units(w, 8, seed=1))
+    assert out_err <= TOL["bf16"] and state_err <= TOL["bf16"], (out_err, state_err)
+
+
+def test_config4_long_stream_through_prefill_stream():
+    w = W.CONFIGS["stream_b8_c1024"]
+    units = pick_units(w, 8, seed=3)
+    gpu, ora = make_pair(w, units)
+    chunk = W.STREAM_BLOCK
+    worst = 0.0
+    for blk in range(w.steps // chunk):
+        q, k, v = W.stream_block(w, blk, "cuda")
+        out = gpu.prefill_stream(q, k, v)
+        ref = ora.prefill_stream(*_unit_slices(w, units, q, k, v))
+        worst = max(worst, compare_out(w, units, out, ref))
+        assert gpu.len == min((blk + 1) * chunk, w.capacity)   # never exceeds the capacity
+    gpu.check_status()
+    assert ora.n_written == w.steps - w.capacity
+    state = compare_state(w, units, gpu, ora)
+    assert worst <= TOL["bf16"] and state <= TOL["bf16"], (worst, state)
