@@ -69,6 +69,11 @@ typedef enum bct_dtype {
                                         full-phase token leaves MV unchanged */
 #define BCT_FLAG_WRITE_THEN_READ 2u  /* the token's read sees its own write */
 #define BCT_FLAG_DENSE_WRITE 4u      /* rewrite every slot, whatever its write weight */
+#define BCT_FLAG_PRECISE_READ 16u     /* bfloat16 cache: the read uses MV's value plus its
+                                        residual (one more plane streamed per token); for
+                                        states whose magnitude makes a bfloat16 ulp matter */
+#define BCT_FLAG_OUT_F32 8u          /* `out` is float (the fp32 accumulator, unrounded)
+                                        whatever the cache dtype */
 
 typedef struct bct_params {
     int32_t batch;      /* B  >= 1 sequences */
@@ -126,7 +131,7 @@ bct_status_t bct_cache_create(const bct_params_t *params, void *workspace, size_
  *   k    DEVICE [B][Hkv][d]  write queries wq_t (appended as keys during the fill phase)
  *   v    DEVICE [B][Hkv][d]  write key-value vectors wv_t
  *   out  DEVICE [B][Hq][d]   attention outputs, written by the call
- * all contiguous, in the cache's dtype.  The cache advances by one token.
+ * all contiguous, in the cache's dtype (out in float with BCT_FLAG_OUT_F32).  The cache advances by one token.
  */
 bct_status_t bct_decode_step(bct_cache_t *cache, const void *q, const void *k, const void *v,
                              void *out, void *cuda_stream);

@@ -14,7 +14,7 @@ import torch
 
 BCT_OK, BCT_ERR_INVALID_ARG, BCT_ERR_UNSUPPORTED, BCT_ERR_STATE, BCT_ERR_CUDA, BCT_ERR_TIMEOUT = range(6)
 BCT_F32, BCT_BF16, BCT_BF16_PAIR = 0, 1, 2
-FLAG_SKIP_FIRST_WRITE, FLAG_WRITE_THEN_READ, FLAG_DENSE_WRITE = 1, 2, 4
+FLAG_SKIP_FIRST_WRITE, FLAG_WRITE_THEN_READ, FLAG_DENSE_WRITE, FLAG_OUT_F32, FLAG_PRECISE_READ = 1, 2, 4, 8, 16
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libbct_b200.so")
 
@@ -127,6 +127,7 @@ class Cache:
                                   read_scale=read_scale, write_scale=write_scale, init_len=init_len,
                                   flags=flags, write_eps=write_eps, max_stream=max_stream)
         self.dtype = dtype
+        self.out_dtype = torch.float32 if (flags & FLAG_OUT_F32) else dtype
         self.device = torch.device(device)
         self.B, self.Hq, self.Hkv, self.d, self.C = batch, n_q_heads, n_kv_heads, head_dim, capacity
         nbytes, align = cache_bytes(self.params)
@@ -146,7 +147,7 @@ class Cache:
     # ---- steps ----------------------------------------------------------------------
     def decode_step(self, q, k, v, out=None, stream=None):
         if out is None:
-            out = torch.empty_like(q)
+            out = torch.empty_like(q, dtype=self.out_dtype)
         _check(self.lib.bct_decode_step(self._h, q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
                                         _stream_ptr(stream)))
         return out
@@ -154,7 +155,7 @@ class Cache:
     def prefill_stream(self, q, k, v, out=None, want_out=True, stream=None):
         T = q.shape[1]
         if out is None and want_out:
-            out = torch.empty_like(q)
+            out = torch.empty_like(q, dtype=self.out_dtype)
         _check(self.lib.bct_prefill_stream(self._h, q.data_ptr(), k.data_ptr(), v.data_ptr(), _ptr(out), T,
                                            _stream_ptr(stream)))
         return out

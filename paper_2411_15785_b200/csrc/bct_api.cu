@@ -33,7 +33,7 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 // Offsets of the workspace sections.
 struct Carve {
     size_t kplane, vhi, vlo, status, stage_q, stage_k, stage_v, stage_out, total;
-    size_t plane_bytes, q_bytes, kv_bytes;  // q_bytes / kv_bytes: staging for max_stream tokens
+    size_t plane_bytes, q_bytes, kv_bytes, out_bytes;  // staging for max_stream tokens
 };
 
 bct_status_t resolve_params(const bct_params_t* in, bct_params_t* p) {
@@ -48,7 +48,8 @@ bct_status_t resolve_params(const bct_params_t* in, bct_params_t* p) {
     if (p->head_dim < 1) return fail(BCT_ERR_INVALID_ARG, "head_dim must be >= 1");
     if (p->init_len < 0 || p->init_len > p->capacity)
         return fail(BCT_ERR_INVALID_ARG, "init_len %d outside 0..capacity (%d)", p->init_len, p->capacity);
-    if (p->flags & ~(BCT_FLAG_SKIP_FIRST_WRITE | BCT_FLAG_WRITE_THEN_READ | BCT_FLAG_DENSE_WRITE))
+    if (p->flags & ~(BCT_FLAG_SKIP_FIRST_WRITE | BCT_FLAG_WRITE_THEN_READ | BCT_FLAG_DENSE_WRITE | BCT_FLAG_OUT_F32 |
+                     BCT_FLAG_PRECISE_READ))
         return fail(BCT_ERR_INVALID_ARG, "unknown flag bits 0x%x", p->flags);
     if (!(p->read_scale > 0.f)) p->read_scale = 1.0f / std::sqrt((float)p->head_dim);
     if (!(p->write_scale > 0.f)) p->write_scale = 1.0f;
@@ -70,6 +71,7 @@ Carve carve(const bct_params_t& p) {
     c.plane_bytes = U * (size_t)p.capacity * p.head_dim * eb;
     c.q_bytes = (size_t)p.batch * p.max_stream * p.n_q_heads * p.head_dim * eb;
     c.kv_bytes = (size_t)p.batch * p.max_stream * p.n_kv_heads * p.head_dim * eb;
+    c.out_bytes = (p.flags & BCT_FLAG_OUT_F32) ? c.q_bytes / eb * 4 : c.q_bytes;
     size_t off = 0;
     c.kplane = off;
     off += round_up(c.plane_bytes, bct::kAlign);
@@ -86,7 +88,7 @@ Carve carve(const bct_params_t& p) {
     c.stage_v = off;
     off += round_up(c.kv_bytes, bct::kAlign);
     c.stage_out = off;
-    off += round_up(c.q_bytes, bct::kAlign);
+    off += round_up(c.out_bytes, bct::kAlign);
     c.total = off;
     return c;
 }
@@ -117,7 +119,8 @@ bct_status_t run_tokens(bct_cache_t* c, const void* q, const void* k, const void
         io.q = static_cast<const char*>(q) + (size_t)t * q_tok * eb;
         io.k = static_cast<const char*>(k) + (size_t)t * kv_tok * eb;
         io.v = static_cast<const char*>(v) + (size_t)t * kv_tok * eb;
-        io.out = out ? static_cast<char*>(out) + (size_t)t * q_tok * eb : nullptr;
+        const size_t ob = (p.flags & BCT_FLAG_OUT_F32) ? 4 : eb;
+        io.out = out ? static_cast<char*>(out) + (size_t)t * q_tok * ob : nullptr;
         io.q_batch_stride = (int64_t)(T * q_tok);
         io.kv_batch_stride = (int64_t)(T * kv_tok);
         const bool full = (c->len == p.capacity);
@@ -253,7 +256,8 @@ bct_status_t bct_prefill_stream_host(bct_cache_t* c, const void* q, const void* 
     st = run_tokens(c, c->stage_q, c->stage_k, c->stage_v, out ? c->stage_out : nullptr, T, stream);
     if (st != BCT_OK) return st;
     if (out != nullptr) {
-        e = cudaMemcpyAsync(out, c->stage_out, qb, cudaMemcpyDeviceToHost, stream);
+        const size_t ob = (c->p.flags & BCT_FLAG_OUT_F32) ? qb / eb * 4 : qb;
+        e = cudaMemcpyAsync(out, c->stage_out, ob, cudaMemcpyDeviceToHost, stream);
         if (e != cudaSuccess) return fail_cuda("device-to-host copy", e);
     }
     return BCT_OK;

@@ -51,6 +51,8 @@ struct DecodeArgs {
     int do_write;  // the soft write happens this token
     int wtr;       // the read sees the token's own write
     int dense;     // rewrite every slot
+    int out_f32;   // out is float whatever the cache dtype
+    int precise;   // bfloat16 cache: the read uses value + residual (streams the residual plane too)
     float read_scale;
     float write_scale;
     float write_eps;
@@ -84,6 +86,15 @@ __host__ __device__ inline SmemLayout smem_layout(int G, int D, int score_stride
 
 __device__ __forceinline__ void consumer_sync() {
     asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory");
+}
+
+// out has the layout of q; q_off is the unit's byte offset in q's element size.
+template <typename T>
+__device__ __forceinline__ void store_out(const DecodeArgs& a, size_t q_off, int idx, float val) {
+    if (a.out_f32)
+        reinterpret_cast<float*>(a.out + q_off / sizeof(T) * sizeof(float))[idx] = val;
+    else
+        reinterpret_cast<T*>(a.out + q_off)[idx] = (T)val;
 }
 
 template <typename T, int D, int G>
@@ -133,6 +144,7 @@ __global__ void __launch_bounds__(kThreads, (G <= 4 ? 2 : 1)) decode_kernel(cons
     const size_t unit_off = (size_t)u * a.C * ROW_BYTES;
     const char* kslice = a.kplane + unit_off + (size_t)slice_start * ROW_BYTES;
     char* vslice = a.vhi + unit_off + (size_t)slice_start * ROW_BYTES;
+    const bool precise = (sizeof(T) == 2) && a.precise;
     const size_t q_off = ((size_t)b * a.q_bs + (size_t)h_kv * G * D) * sizeof(T);
     const size_t kv_off = ((size_t)b * a.kv_bs + (size_t)h_kv * D) * sizeof(T);
 
@@ -154,7 +166,9 @@ __global__ void __launch_bounds__(kThreads, (G <= 4 ? 2 : 1)) decode_kernel(cons
     if (warp == kConsumerWarps) {
         // ---------------- producer warp: K tiles, then V tiles, through the ring ----------------
         if (lane == 0) {
-            for (int item = 0; item < 2 * nt; ++item) {
+            const char* loslice = precise ? a.vlo + unit_off + (size_t)slice_start * ROW_BYTES : nullptr;
+            const int n_items = precise ? 3 * nt : 2 * nt;  // K tiles, then V tiles (value, residual interleaved)
+            for (int item = 0; item < n_items; ++item) {
                 const int stage = item % kStages;
                 if (item >= kStages) {
                     const uint32_t parity = ((item / kStages) - 1) & 1;
@@ -164,9 +178,15 @@ __global__ void __launch_bounds__(kThreads, (G <= 4 ? 2 : 1)) decode_kernel(cons
                         break;
                     }
                 }
-                const int t = (item < nt) ? item : item - nt;
+                int t = item;
+                const char* base = kslice;
+                if (item >= nt) {
+                    const int j = item - nt;
+                    t = precise ? (j >> 1) : j;
+                    base = (precise && (j & 1)) ? loslice : (const char*)vslice;
+                }
                 const int rows = min(TILE_ROWS, n_stream - t * TILE_ROWS);
-                const char* src = ((item < nt) ? kslice : (const char*)vslice) + (size_t)t * kTileBytes;
+                const char* src = base + (size_t)t * kTileBytes;
                 const uint32_t bytes = (uint32_t)rows * ROW_BYTES;
                 mbar_arrive_expect_tx(&full[stage], bytes);
                 bulk_load(ring + stage * kTileBytes, src, bytes, &full[stage]);
@@ -345,14 +365,20 @@ __global__ void __launch_bounds__(kThreads, (G <= 4 ? 2 : 1)) decode_kernel(cons
         float vt[EPL];
         Ck::unpack(v_raw, vt);
         for (int i = 0; i < nt; ++i) {
-            const int item = nt + i;
+            const int item = precise ? nt + 2 * i : nt + i;
             const int stage = item % kStages;
             if (!mbar_wait(&full[stage], (item / kStages) & 1, *abort_flag ? 1024u : kWaitLimit)) {
                 report_timeout(a.status, 4);
                 *abort_flag = 1;
             }
+            const int stage_lo = (item + 1) % kStages;
+            if (precise && !mbar_wait(&full[stage_lo], ((item + 1) / kStages) & 1, *abort_flag ? 1024u : kWaitLimit)) {
+                report_timeout(a.status, 5);
+                *abort_flag = 1;
+            }
             const int rows = min(TILE_ROWS, n_stream - i * TILE_ROWS);
             const unsigned char* tile = ring + stage * kTileBytes;
+            const unsigned char* tile_lo = ring + stage_lo * kTileBytes;
             uint4 w[PASSES];
 #pragma unroll
             for (int ps = 0; ps < PASSES; ++ps) {
@@ -367,6 +393,14 @@ __global__ void __launch_bounds__(kThreads, (G <= 4 ? 2 : 1)) decode_kernel(cons
                     const int row = i * TILE_ROWS + r;
                     float x[EPL];
                     Ck::unpack(w[ps], x);
+                    float lo[EPL];
+                    if constexpr (sizeof(T) == 2) {
+                        if (precise) {
+                            Ck::unpack(*reinterpret_cast<const uint4*>(tile_lo + r * ROW_BYTES + chunk * 16), lo);
+#pragma unroll
+                            for (int e = 0; e < EPL; ++e) x[e] += lo[e];  // exact: <= 17 significant bits
+                        }
+                    }
                     float p[G];
 #pragma unroll
                     for (int g = 0; g < G; ++g) {
@@ -383,10 +417,13 @@ __global__ void __launch_bounds__(kThreads, (G <= 4 ? 2 : 1)) decode_kernel(cons
                             float nv[EPL];
                             if constexpr (sizeof(T) == 2) {
                                 char* lo_ptr = a.vlo + unit_off + (size_t)slice_start * ROW_BYTES + off;
-                                float lo[EPL];
-                                Ck::unpack(*reinterpret_cast<const uint4*>(lo_ptr), lo);
+                                if (!precise) {
+                                    Ck::unpack(*reinterpret_cast<const uint4*>(lo_ptr), lo);
 #pragma unroll
-                                for (int e = 0; e < EPL; ++e) nv[e] = fmaf(ww, vt[e], x[e] + lo[e]);
+                                    for (int e = 0; e < EPL; ++e) x[e] += lo[e];
+                                }
+#pragma unroll
+                                for (int e = 0; e < EPL; ++e) nv[e] = fmaf(ww, vt[e], x[e]);
                                 const uint4 hi_new = Ck::pack(nv);
                                 float hf[EPL];
                                 Ck::unpack(hi_new, hf);
@@ -404,7 +441,10 @@ __global__ void __launch_bounds__(kThreads, (G <= 4 ? 2 : 1)) decode_kernel(cons
                 }
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(&empty[stage]);
+            if (lane == 0) {
+                mbar_arrive(&empty[stage]);
+                if (precise) mbar_arrive(&empty[stage_lo]);
+            }
         }
         if (has_virtual && warp == 0 && sub == 0) {  // the appended slot's own value row
 #pragma unroll
@@ -448,14 +488,13 @@ __global__ void __launch_bounds__(kThreads, (G <= 4 ? 2 : 1)) decode_kernel(cons
         const bool add_own = a.wtr && a.do_write;
         if (S == 1) {
             if (a.out != nullptr && !*abort_flag) {
-                T* outp = reinterpret_cast<T*>(a.out + q_off);
                 const T* vin = reinterpret_cast<const T*>(a.v + kv_off);
                 for (int idx = tid; idx < G * D; idx += kConsumerThreads) {
                     const int g = idx / D, e = idx - g * D;
                     const float inv = 1.f / stat[(G + 1) + g];
                     float val = ofin[g * (D + 1) + e] * inv;
                     if (add_own) val = fmaf(ofin[g * (D + 1) + D] * inv, (float)vin[e], val);
-                    outp[idx] = (T)val;
+                    store_out<T>(a, q_off, idx, val);
                 }
             }
         } else if (rank != 0) {
@@ -475,7 +514,6 @@ __global__ void __launch_bounds__(kThreads, (G <= 4 ? 2 : 1)) decode_kernel(cons
         cluster_wait();
         if (rank == 0 && warp < kConsumerWarps && a.out != nullptr && !*abort_flag) {
             const float* ofin = reinterpret_cast<float*>(ring) + kConsumerWarps * G * (D + 1);
-            T* outp = reinterpret_cast<T*>(a.out + q_off);
             const T* vin = reinterpret_cast<const T*>(a.v + kv_off);
             const bool add_own = a.wtr && a.do_write;
             for (int idx = tid; idx < G * D; idx += kConsumerThreads) {
@@ -495,7 +533,7 @@ __global__ void __launch_bounds__(kThreads, (G <= 4 ? 2 : 1)) decode_kernel(cons
                 }
                 float val = num / den;
                 if (add_own) val = fmaf(own / den, (float)vin[e], val);
-                outp[idx] = (T)val;
+                store_out<T>(a, q_off, idx, val);
             }
         }
     }
@@ -609,6 +647,8 @@ int launch_decode(const bct_cache* c, const StepIO& io, int len, int do_write, c
     a.do_write = (len == p.capacity) && do_write;
     a.wtr = (p.flags & BCT_FLAG_WRITE_THEN_READ) ? 1 : 0;
     a.dense = (p.flags & BCT_FLAG_DENSE_WRITE) ? 1 : 0;
+    a.out_f32 = (p.flags & BCT_FLAG_OUT_F32) ? 1 : 0;
+    a.precise = (p.flags & BCT_FLAG_PRECISE_READ) ? 1 : 0;
     a.read_scale = p.read_scale;
     a.write_scale = p.write_scale;
     a.write_eps = p.write_eps;

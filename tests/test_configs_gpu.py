@@ -64,7 +64,9 @@ def test_config2_diffuse_write_regime():
 def test_config4_long_stream_through_prefill_stream():
     w = W.CONFIGS["stream_b8_c1024"]
     units = pick_units(w, 8, seed=3)
-    gpu, ora = make_pair(w, units)
+    # after ~1e5 tokens |MV| reaches ~75 and |out| ~10, where one bfloat16 ulp (0.25 resp. 0.06) exceeds
+    # the 2e-2 bar by itself: the read uses value + residual and out is the fp32 accumulator
+    gpu, ora = make_pair(w, units, flags=B.FLAG_PRECISE_READ | B.FLAG_OUT_F32)
     chunk = W.STREAM_BLOCK
     worst = 0.0
     for blk in range(w.steps // chunk):

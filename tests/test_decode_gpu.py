@@ -73,6 +73,33 @@ def test_flags_match_oracle(flag, oflag):
     assert out_err <= TOL["f32"] and state_err <= TOL["f32"], (out_err, state_err)
 
 
+@pytest.mark.parametrize("C,G,init_len", [(333, 1, 333), (520, 4, 500), (8192, 2, 8192)])
+def test_precise_read_and_float_out_on_large_magnitude_state(C, G, init_len):
+    # MV_0 ~ N(0, 100^2): a bfloat16 ulp of the state is ~0.5, so the default value-plane-only read
+    # cannot meet an absolute 2e-2; value + residual with float out does.
+    d = 128
+    B_ = 1 if C > 4096 else 2
+    w = W.Workload("t", B_, 2 * G, 2, d, C, "bf16", init_len, 25, 21, d ** -0.5, 1.0, 1.0, "decode")
+    units = pick_units(w, 4)
+    gpu, ora = make_pair(w, units, flags=B.FLAG_PRECISE_READ | B.FLAG_OUT_F32)
+    scale = torch.tensor(100.0, device="cuda")
+    k0, v0 = gpu.export(torch.float32)
+    v0 = (v0 * scale).to(torch.bfloat16).float() + 0.001953125 * torch.sign(v0)  # value + a residual part
+    gpu.import_state(k0[:, :, :init_len].contiguous(), v0[:, :, :init_len].contiguous(), init_len)
+    for i, (b, h) in enumerate(units):
+        ora.MV[i, :init_len] = v0[b, h, :init_len].double().cpu().numpy()
+    worst = 0.0
+    for t in range(w.steps):
+        q, k, v = W.step_inputs(w, t, "cuda")
+        out = gpu.decode_step(q, k, v)
+        assert out.dtype == torch.float32
+        ref = ora.prefill_stream(*_unit_slices(w, units, q, k, v))
+        worst = max(worst, compare_out(w, units, out, ref))
+    gpu.check_status()
+    state = compare_state(w, units, gpu, ora)
+    assert worst <= 2e-3 and state <= TOL["bf16"], (worst, state)
+
+
 def test_prefill_stream_equals_decode_steps_and_state_only_mode():
     w = W.CONFIGS["stream_b8_c1024"].scaled(batch=2, n_q_heads=4, n_kv_heads=4, capacity=96, steps=160)
     units = pick_units(w, 8)
