@@ -196,11 +196,14 @@ def main():
     ap.add_argument("--workload", default="mha7b_b64_c2048", choices=sorted(W.CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--write-scale", type=float, default=None, help="override the write score scale")
+    ap.add_argument("--batch", type=int, default=None, help="override the batch (profiling on a smaller case)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     w = W.CONFIGS[args.workload]
     if args.write_scale is not None:
         w = w.scaled(write_scale=args.write_scale)
+    if args.batch is not None:
+        w = w.scaled(batch=args.batch, name="%s@batch%d" % (w.name, args.batch))
     if args.impl == "reference":
         run_reference(args, w)
         return
