@@ -14,7 +14,7 @@ import torch
 
 BCT_OK, BCT_ERR_INVALID_ARG, BCT_ERR_UNSUPPORTED, BCT_ERR_STATE, BCT_ERR_CUDA, BCT_ERR_TIMEOUT = range(6)
 BCT_F32, BCT_BF16, BCT_BF16_PAIR = 0, 1, 2
-FLAG_SKIP_FIRST_WRITE, FLAG_WRITE_THEN_READ, FLAG_DENSE_WRITE, FLAG_OUT_F32, FLAG_PRECISE_READ = 1, 2, 4, 8, 16
+FLAG_SKIP_FIRST_WRITE, FLAG_WRITE_THEN_READ, FLAG_DENSE_WRITE, FLAG_OUT_F32, FLAG_PRECISE_READ, FLAG_CUDA_CORES = 1, 2, 4, 8, 16, 32
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libbct_b200.so")
 
@@ -22,6 +22,7 @@ EXPORTS = (
     "bct_version", "bct_last_error", "bct_cache_bytes", "bct_cache_create", "bct_decode_step",
     "bct_prefill_stream", "bct_decode_step_host", "bct_prefill_stream_host", "bct_cache_len",
     "bct_cache_export", "bct_cache_import", "bct_cache_status", "bct_cache_launches", "bct_cache_destroy",
+    "bct_cache_tensor_path",
 )
 
 
@@ -69,6 +70,7 @@ def load() -> ctypes.CDLL:
     lib.bct_cache_status.argtypes = [vp, vp]
     lib.bct_cache_launches.argtypes = [vp, ctypes.POINTER(i64)]
     lib.bct_cache_destroy.argtypes = [vp]
+    lib.bct_cache_tensor_path.argtypes = [vp, ctypes.POINTER(i32)]
     for name in EXPORTS[2:]:
         getattr(lib, name).restype = ctypes.c_int
     _lib = lib
@@ -177,6 +179,12 @@ class Cache:
         n = ctypes.c_int32(0)
         _check(self.lib.bct_cache_len(self._h, ctypes.byref(n)))
         return n.value
+
+    @property
+    def tensor_path(self) -> bool:
+        n = ctypes.c_int32(0)
+        _check(self.lib.bct_cache_tensor_path(self._h, ctypes.byref(n)))
+        return bool(n.value)
 
     @property
     def launches(self) -> int:

@@ -49,7 +49,7 @@ bct_status_t resolve_params(const bct_params_t* in, bct_params_t* p) {
     if (p->init_len < 0 || p->init_len > p->capacity)
         return fail(BCT_ERR_INVALID_ARG, "init_len %d outside 0..capacity (%d)", p->init_len, p->capacity);
     if (p->flags & ~(BCT_FLAG_SKIP_FIRST_WRITE | BCT_FLAG_WRITE_THEN_READ | BCT_FLAG_DENSE_WRITE | BCT_FLAG_OUT_F32 |
-                     BCT_FLAG_PRECISE_READ))
+                     BCT_FLAG_PRECISE_READ | BCT_FLAG_CUDA_CORES))
         return fail(BCT_ERR_INVALID_ARG, "unknown flag bits 0x%x", p->flags);
     if (!(p->read_scale > 0.f)) p->read_scale = 1.0f / std::sqrt((float)p->head_dim);
     if (!(p->write_scale > 0.f)) p->write_scale = 1.0f;
@@ -204,6 +204,8 @@ bct_status_t bct_cache_create(const bct_params_t* params, void* workspace, size_
     c->sm_count = sms;
     c->smem_optin = optin;
 
+    bct::tc_prepare(c);  // tensor maps of the planes; without them the CUDA-core kernel serves every shape
+
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     e = cudaMemsetAsync(c->status, 0, bct::kAlign, stream);
     if (e == cudaSuccess) e = bct::launch_import(c, mk_init, mv_init, p.dtype, p.init_len, stream);
@@ -321,6 +323,14 @@ bct_status_t bct_cache_status(bct_cache_t* c, void* cuda_stream) {
     if (host[0] == BCT_ERR_TIMEOUT)
         return fail(BCT_ERR_TIMEOUT, "a bounded wait inside a kernel gave up (site %d)", host[1]);
     if (host[0] != 0) return fail(BCT_ERR_STATE, "device status word holds %d", host[0]);
+    return BCT_OK;
+}
+
+bct_status_t bct_cache_tensor_path(const bct_cache_t* c, int32_t* yes) {
+    bct_status_t st = check_handle(c);
+    if (st != BCT_OK) return st;
+    if (yes == nullptr) return fail(BCT_ERR_INVALID_ARG, "yes is NULL");
+    *yes = (!(c->p.flags & BCT_FLAG_CUDA_CORES) && bct::tc_eligible(c)) ? 1 : 0;
     return BCT_OK;
 }
 

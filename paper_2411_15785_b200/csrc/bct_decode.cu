@@ -621,6 +621,7 @@ bool decode_supported(const bct_params_t& p, int smem_optin, const char** why) {
 int launch_decode(const bct_cache* c, const StepIO& io, int len, int do_write, cudaStream_t stream,
                   cudaError_t* err) {
     const bct_params_t& p = c->p;
+    if (!(p.flags & BCT_FLAG_CUDA_CORES) && tc_eligible(c)) return launch_decode_tc(c, io, len, do_write, stream, err);
     KernelFn fn = pick_kernel(p.dtype, p.head_dim, c->G);
     Plan pl = make_plan(c->G, p.head_dim, c->elem_bytes, p.capacity, c->U, c->sm_count, c->smem_optin);
     if (fn == nullptr || !pl.ok) {

@@ -1,0 +1,800 @@
+// Decode step of the bounded-cache attention layer on the sm_100a tensor path
+// (bfloat16 cache, head_dim 128, up to 7 query heads per kv-head).
+//
+// The two contractions of a token are small-N GEMMs against the resident tiles:
+//   scores   S[slot, h]  = sum_d MK[slot, d] * Q[h, d]      h = G read queries + the write query
+//                                                           (score_t = wq_t . MK^T, Algorithm 1)
+//   outputs  O[d, g]     = sum_slot MV[slot, d] * P[g, slot] (softmax numerators P; read path)
+// Both run as tcgen05.mma (M = 128, N = 16, K = 16) straight out of the shared-memory tiles that
+// TMA tensor copies deliver (128-byte swizzle), with the accumulators in tensor memory, so the
+// SM's issue slots carry only the softmax and the update rule
+//   MV_t = MV_{t-1} + ww_t^T . wv_t   (Method step 4)
+// on the few rows whose weight reaches write_eps.
+//
+// One persistent CTA per SM (or a cluster of S CTAs per unit when C > 2048 slots), three roles:
+//   warp 4  producer : TMA loads of K tiles then V tiles into a ring, running ahead across units
+//   warp 5  MMA      : issues the tensor-core work as tiles land, commits to mbarriers
+//   warps 0-3        : softmax statistics from tensor memory, P operand, update rule, epilogue
+// Every wait is bounded; a timeout sets the status word and the kernel runs to its end.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "bct_device.cuh"
+#include "bct_internal.h"
+
+namespace bct {
+namespace {
+
+constexpr int kTcThreads = 192;
+constexpr int kSThreads = 128;
+constexpr int kTileRows = 128;
+constexpr int kHalfBytes = 128 * 128;          // 64 columns (128 bytes) x 128 rows
+constexpr int kTcTileBytes = 2 * kHalfBytes;   // one 128 x 128 bfloat16 tile
+constexpr int kMaxTiles = 16;                  // a CTA's slice holds at most 2048 slots
+constexpr int kPTileBytes = 2048;              // P operand of one tile: 2 halves x (8 rows x 128 B)
+constexpr int kQBufBytes = 3072;               // Q operand (2 halves x 8 rows x 128 B) + 1 KiB of zeros
+constexpr int kScoreCols = 16;                 // tensor-memory columns per score tile (N = 16)
+constexpr int kOCol = kMaxTiles * kScoreCols;  // output accumulator behind the score tiles
+constexpr int kTmemCols = 512;
+constexpr int kMaxClusterTc = 8;
+constexpr int kLoCap = 64;                     // residual rows prefetched per unit; further rows take the slow path
+constexpr float kNegBigTc = -3.0e38f;
+
+struct TcArgs {
+    char* vhi;
+    char* vlo;
+    char* kplane;
+    const char* q;
+    const char* k;
+    const char* v;
+    char* out;
+    int* status;
+    long long q_bs;
+    long long kv_bs;
+    int C, len, slice_rows, S, Hkv, U, stages;
+    int do_write, wtr, dense, out_f32;
+    float read_scale, write_scale, write_eps;
+};
+
+struct TcSmem {
+    int ring, pbuf, qbuf, wsm, idx, lostage, red, stat, wstat, merge, bars, total;
+};
+__host__ __device__ inline TcSmem tc_smem(int stages, int G, int S) {
+    TcSmem L;
+    int off = 0;
+    L.ring = off;
+    off += stages * kTcTileBytes;
+    L.pbuf = off;
+    off += kMaxTiles * kPTileBytes + 1024;
+    L.qbuf = off;
+    off += 2 * kQBufBytes;
+    L.wsm = off;
+    off += kMaxTiles * kTileRows * 4;
+    L.idx = off;  // per slot: staging row of its residual, -1 untouched, -2 not staged
+    off += kMaxTiles * kTileRows * 2;
+    L.lostage = off;
+    off += kLoCap * 256;
+    L.red = off;
+    off += 4 * 16 * 4;
+    L.stat = off;  // m[8], l[8], wd[8], ev[8], abort, tmem address
+    off += 4 * 8 * 4 + 16;
+    L.wstat = off;
+    off += 2 * kMaxClusterTc * 2 * 4;
+    L.merge = off;
+    off += (S > 1) ? 2 * (S - 1) * G * (128 + 3) * 4 : 0;
+    off = (off + 15) & ~15;
+    L.bars = off;
+    off += (3 * stages + 2 + 1 + 1 + 2 + 2 + 1) * 8;
+    L.total = ((off + 127) & ~127) + 1024;  // + slack to align the ring to 1024 bytes
+    return L;
+}
+
+// ---- PTX wrappers of the tensor path ---------------------------------------------------
+__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, int x, int y, int z, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar))
+        : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tmem_alloc(uint32_t* slot, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(slot)), "r"(cols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, bool accum) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"((uint32_t)accum)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+// 8 consecutive columns of this thread's tensor-memory lane.
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, float* x) {
+    uint32_t r[8];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 8; ++i) x[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle (layout type 2), descriptor version 1.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = (uint64_t)((saddr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+// Instruction descriptor: bf16 x bf16 -> f32, M = 128, N = 16; A K-major or MN-major, B K-major.
+__host__ __device__ constexpr uint32_t instr_desc(bool a_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn_major ? 1u : 0u) << 15) | ((16u >> 3) << 17) |
+           ((128u >> 4) << 24);
+}
+
+__device__ __forceinline__ void s_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kSThreads) : "memory"); }
+
+template <int G>
+__global__ void __launch_bounds__(kTcThreads, 1)
+decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const TcArgs a) {
+    constexpr int D = 128;
+    constexpr int ROW_BYTES = 256;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int S = a.S;
+    const int NST = a.stages;
+    const TcSmem L = tc_smem(NST, G, S);
+    unsigned char* ring = smem + L.ring;
+    unsigned char* pbuf = smem + L.pbuf;
+    unsigned char* qbuf = smem + L.qbuf;
+    float* wsm = reinterpret_cast<float*>(smem + L.wsm);
+    short* idx = reinterpret_cast<short*>(smem + L.idx);
+    unsigned char* lostage = smem + L.lostage;
+    float* red = reinterpret_cast<float*>(smem + L.red);
+    float* st_m = reinterpret_cast<float*>(smem + L.stat);
+    float* st_l = st_m + 8;
+    float* st_wd = st_m + 16;
+    float* st_ev = st_m + 24;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(st_m + 32);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(st_m + 33);
+    int* lo_count = reinterpret_cast<int*>(st_m + 34);
+    float* wstat = reinterpret_cast<float*>(smem + L.wstat);
+    float* merge = reinterpret_cast<float*>(smem + L.merge);
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + L.bars);
+    uint64_t* empty = full + NST;
+    uint64_t* sready = empty + NST;
+    uint64_t* qready = sready + NST;  // [2]
+    uint64_t* pready = qready + 2;
+    uint64_t* oready = pready + 1;
+    uint64_t* xbar = oready + 1;      // [2]
+    uint64_t* mbar = xbar + 2;        // [2]
+    uint64_t* lobar = mbar + 2;
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5;
+    const int lane = tid & 31;
+    const int rank = (S > 1) ? (int)cluster_ctarank() : 0;
+    const int cid = blockIdx.x / S;
+    const int ncl = gridDim.x / S;
+
+    const int slice_start = rank * a.slice_rows;
+    const int n_slice = max(0, min(a.slice_rows, a.C - slice_start));
+    const int n_stream = max(0, min(a.len - slice_start, n_slice));
+    const bool has_virtual = (a.len < a.C) && (a.len >= slice_start) && (a.len < slice_start + n_slice);
+    const int nt = (n_stream + kTileRows - 1) / kTileRows;
+
+    if (tid == 0) {
+        for (int i = 0; i < NST; ++i) {
+            mbar_init(&full[i], 1);
+            mbar_init(&empty[i], 5);  // the MMA commit + one lane of each softmax warp
+            mbar_init(&sready[i], 1);
+        }
+        mbar_init(&qready[0], kSThreads);
+        mbar_init(&qready[1], kSThreads);
+        mbar_init(pready, kSThreads);
+        mbar_init(oready, 1);
+        mbar_init(&xbar[0], S);
+        mbar_init(&xbar[1], S);
+        mbar_init(&mbar[0], kSThreads * (S > 1 ? S - 1 : 1));
+        mbar_init(&mbar[1], kSThreads * (S > 1 ? S - 1 : 1));
+        mbar_init(lobar, kSThreads);
+        *abort_flag = 0;
+        *lo_count = 0;
+        fence_mbar_init_cluster();
+    }
+    // zero the operand padding: Q rows above the write query, the dummy rows behind Q and P
+    for (int i = tid; i < 2 * kQBufBytes / 16; i += kTcThreads) reinterpret_cast<uint4*>(qbuf)[i] = make_uint4(0, 0, 0, 0);
+    for (int i = tid; i < 1024 / 16; i += kTcThreads)
+        reinterpret_cast<uint4*>(pbuf + kMaxTiles * kPTileBytes)[i] = make_uint4(0, 0, 0, 0);
+    if (warp == 5) tmem_alloc(tmem_slot, kTmemCols);
+    fence_proxy_async_smem();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    if (S > 1) {
+        cluster_arrive();
+        cluster_wait();
+    }
+
+    if (warp == 4) {
+        // =========================== producer ===========================
+        if (lane == 0) {
+            uint32_t kc = 0;
+            bool ok = true;
+            for (int u = cid; u < a.U && ok; u += ncl) {
+                for (int ph = 0; ph < 2 && ok; ++ph) {
+                    const CUtensorMap* map = ph == 0 ? &tmK : &tmV;
+                    for (int t = 0; t < nt; ++t, ++kc) {
+                        const int stage = kc % NST;
+                        if (kc >= (uint32_t)NST &&
+                            !mbar_wait(&empty[stage], ((kc / NST) - 1) & 1, *abort_flag ? 1024u : kWaitLimit)) {
+                            report_timeout(a.status, 11);
+                            *abort_flag = 1;
+                            ok = false;
+                            break;
+                        }
+                        unsigned char* dst = ring + (size_t)stage * kTcTileBytes;
+                        mbar_arrive_expect_tx(&full[stage], kTcTileBytes);
+                        tma_load_3d(dst, map, 0, slice_start + t * kTileRows, u, &full[stage]);
+                        tma_load_3d(dst + kHalfBytes, map, 64, slice_start + t * kTileRows, u, &full[stage]);
+                    }
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 5) {
+        // =========================== MMA issuer ===========================
+        if (lane == 0) {
+            constexpr uint32_t idesc_s = instr_desc(false);
+            constexpr uint32_t idesc_o = instr_desc(true);
+            uint32_t kc = 0;
+            int it = 0;
+            for (int u = cid; u < a.U; u += ncl, ++it) {
+                if (!mbar_wait(&qready[it & 1], (it >> 1) & 1, *abort_flag ? 1024u : kWaitLimit)) {
+                    report_timeout(a.status, 12);
+                    *abort_flag = 1;
+                }
+                tc_fence_after();
+                const uint32_t qaddr = smem_u32(qbuf + (it & 1) * kQBufBytes);
+                for (int t = 0; t < nt; ++t, ++kc) {  // scores: A = K tile (K-major), B = Q (K-major)
+                    const int stage = kc % NST;
+                    if (!mbar_wait(&full[stage], (kc / NST) & 1, *abort_flag ? 1024u : kWaitLimit)) {
+                        report_timeout(a.status, 13);
+                        *abort_flag = 1;
+                    }
+                    tc_fence_after();
+                    const uint32_t taddr = smem_u32(ring + (size_t)stage * kTcTileBytes);
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk) {
+                        const uint64_t ad = smem_desc(taddr + (kk >> 2) * kHalfBytes + (kk & 3) * 32, 16, 1024);
+                        const uint64_t bd = smem_desc(qaddr + (kk >> 2) * 1024 + (kk & 3) * 32, 16, 1024);
+                        umma_bf16(tmem_base + t * kScoreCols, ad, bd, idesc_s, kk > 0);
+                    }
+                    umma_commit(&sready[stage]);
+                    umma_commit(&empty[stage]);
+                }
+                if (!mbar_wait(pready, it & 1, *abort_flag ? 1024u : kWaitLimit)) {
+                    report_timeout(a.status, 14);
+                    *abort_flag = 1;
+                }
+                tc_fence_after();
+                for (int t = 0; t < nt; ++t, ++kc) {  // outputs: A = V tile (MN-major), B = P (K-major)
+                    const int stage = kc % NST;
+                    if (!mbar_wait(&full[stage], (kc / NST) & 1, *abort_flag ? 1024u : kWaitLimit)) {
+                        report_timeout(a.status, 15);
+                        *abort_flag = 1;
+                    }
+                    tc_fence_after();
+                    const uint32_t taddr = smem_u32(ring + (size_t)stage * kTcTileBytes);
+                    const uint32_t paddr = smem_u32(pbuf + t * kPTileBytes);
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk) {  // 16 slots per step
+                        const uint64_t ad = smem_desc(taddr + kk * 2048, kHalfBytes, 1024);
+                        const uint64_t bd = smem_desc(paddr + (kk >> 2) * 1024 + (kk & 3) * 32, 16, 1024);
+                        umma_bf16(tmem_base + kOCol, ad, bd, idesc_o, (t > 0) || (kk > 0));
+                    }
+                    umma_commit(&sready[stage]);  // keeps this barrier's phase in step with the ring
+                    umma_commit(&empty[stage]);
+                }
+                umma_commit(oready);
+            }
+        }
+        __syncwarp();
+    } else {
+        // =========================== softmax / update / epilogue warps ===========================
+        const int r = tid;  // tensor-memory lane: slot row of a score tile, d of the output
+        const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
+        uint32_t kc = 0;
+        int it = 0;
+        for (int u = cid; u < a.U; u += ncl, ++it) {
+            const int b = u / a.Hkv;
+            const int h_kv = u - b * a.Hkv;
+            const size_t q_off = ((size_t)b * a.q_bs + (size_t)h_kv * G * D) * 2;
+            const size_t kv_off = ((size_t)b * a.kv_bs + (size_t)h_kv * D) * 2;
+            const size_t unit_off = (size_t)u * a.C * ROW_BYTES;
+
+            // ---- Q operand: rows 0..G-1 read queries, row G the write query (128-byte swizzle) ----
+            {
+                const int h = tid >> 4, c = tid & 15;
+                if (h <= G) {
+                    const char* src = (h < G) ? a.q + q_off + (size_t)h * ROW_BYTES : a.k + kv_off;
+                    const uint4 w = *reinterpret_cast<const uint4*>(src + c * 16);
+                    unsigned char* dst = qbuf + (it & 1) * kQBufBytes + (c >> 3) * 1024 + h * 128 + (((c & 7) ^ h) * 16);
+                    *reinterpret_cast<uint4*>(dst) = w;
+                }
+            }
+            fence_proxy_async_smem();
+            tc_fence_before();
+            mbar_arrive(&qready[it & 1]);
+
+            // ---- pass 1: row maxima of the raw scores, as the score tiles complete ----
+            float mx[8];
+#pragma unroll
+            for (int h = 0; h < 8; ++h) mx[h] = kNegBigTc;
+            for (int t = 0; t < nt; ++t, ++kc) {
+                const int stage = kc % NST;
+                if (!mbar_wait(&sready[stage], (kc / NST) & 1, *abort_flag ? 1024u : kWaitLimit)) {
+                    report_timeout(a.status, 16);
+                    *abort_flag = 1;
+                }
+                tc_fence_after();
+                float s[8];
+                tmem_ld8(lane_base + t * kScoreCols, s);
+                if (t * kTileRows + r < n_stream) {
+#pragma unroll
+                    for (int h = 0; h < 8; ++h) mx[h] = fmaxf(mx[h], s[h]);
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&empty[stage]);
+            }
+            // the appended slot (fill phase) is scored from the step vectors
+            float vq[G > 0 ? G : 1];
+            const float kd = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(a.k + kv_off)[r]);
+            const float vd = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(a.v + kv_off)[r]);
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                vq[g] = 0.f;
+                if (has_virtual) {
+                    const float qd = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(a.q + q_off)[g * D + r]);
+                    vq[g] = warp_sum(qd * kd);
+                }
+            }
+#pragma unroll
+            for (int h = 0; h < 8; ++h) {
+                mx[h] = warp_max(mx[h]);
+                if (lane == 0) red[warp * 16 + h] = mx[h];
+                if (lane == 0 && h < G) red[warp * 16 + 8 + h] = vq[h];
+            }
+            s_sync();
+            if (tid < 8) {
+                const float scale = (tid < G) ? a.read_scale : a.write_scale;
+                float m = fmaxf(fmaxf(red[tid], red[16 + tid]), fmaxf(red[32 + tid], red[48 + tid]));
+                m = (m <= kNegBigTc) ? kNegBigTc : m * scale;
+                if (has_virtual && tid < G) {
+                    const float vs = (red[8 + tid] + red[24 + tid] + red[40 + tid] + red[56 + tid]) * a.read_scale;
+                    st_ev[tid] = vs;  // scaled score of the appended slot, turned into a numerator below
+                    m = fmaxf(m, vs);
+                }
+                st_m[tid] = m;
+            }
+            s_sync();
+
+            // ---- pass 2: numerators, row sums, P operand (bfloat16, swizzled), write numerators ----
+            float sum[8];
+            float wdacc[G > 0 ? G : 1];
+#pragma unroll
+            for (int h = 0; h < 8; ++h) sum[h] = 0.f;
+#pragma unroll
+            for (int g = 0; g < G; ++g) wdacc[g] = 0.f;
+            for (int t = 0; t < nt; ++t) {
+                float s[8];
+                tmem_ld8(lane_base + t * kScoreCols, s);
+                const bool valid = t * kTileRows + r < n_stream;
+                float e[8];
+#pragma unroll
+                for (int h = 0; h < 8; ++h) {
+                    const float scale = (h < G) ? a.read_scale : a.write_scale;
+                    e[h] = (valid && h <= G) ? __expf(s[h] * scale - st_m[h]) : 0.f;
+                    sum[h] += e[h];
+                }
+                unsigned char* prow = pbuf + t * kPTileBytes + (r >> 6) * 1024 + (r & 7) * 2;
+                const int c8 = (r & 63) >> 3;
+#pragma unroll
+                for (int h = 0; h < 8; ++h) {
+                    const __nv_bfloat16 pv = __float2bfloat16_rn(h < G ? e[h] : 0.f);
+                    *reinterpret_cast<__nv_bfloat16*>(prow + h * 128 + ((c8 ^ h) * 16)) = pv;
+                }
+                wsm[t * kTileRows + r] = e[G];
+#pragma unroll
+                for (int g = 0; g < G; ++g) wdacc[g] = fmaf(e[g], e[G], wdacc[g]);
+            }
+            fence_proxy_async_smem();
+            mbar_arrive(pready);
+#pragma unroll
+            for (int h = 0; h < 8; ++h) {
+                sum[h] = warp_sum(sum[h]);
+                if (lane == 0) red[warp * 16 + h] = sum[h];
+            }
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                wdacc[g] = warp_sum(wdacc[g]);
+                if (lane == 0) red[warp * 16 + 8 + g] = wdacc[g];
+            }
+            s_sync();
+            if (tid < 8) {
+                float l = red[tid] + red[16 + tid] + red[32 + tid] + red[48 + tid];
+                if (has_virtual && tid < G) {
+                    const float ev = __expf(st_ev[tid] - st_m[tid]);
+                    st_ev[tid] = ev;
+                    l += ev;
+                }
+                st_l[tid] = l;
+                st_wd[tid] = red[8 + tid] + red[24 + tid] + red[40 + tid] + red[56 + tid];
+            }
+            s_sync();
+
+            // ---- write weights are normalised over ALL C slots: exchange across the cluster ----
+            float wfac = 0.f;
+            if (a.do_write) {
+                if (S > 1) {
+                    float* ws = wstat + (it & 1) * kMaxClusterTc * 2;
+                    if (tid == 0) {
+                        for (int rr = 0; rr < S; ++rr) {
+                            const uint32_t dst = map_to_rank(ws + 2 * rank, rr);
+                            st_cluster_f32(dst, st_m[G]);
+                            st_cluster_f32(dst + 4, st_l[G]);
+                            mbar_arrive_remote(map_to_rank(&xbar[it & 1], rr));
+                        }
+                    }
+                    if (!mbar_wait<true>(&xbar[it & 1], (it >> 1) & 1, *abort_flag ? 1024u : kWaitLimit)) {
+                        report_timeout(a.status, 17);
+                        *abort_flag = 1;
+                    }
+                    float M = kNegBigTc;
+                    for (int rr = 0; rr < S; ++rr) M = fmaxf(M, ws[2 * rr]);
+                    float Ls = 0.f;
+                    for (int rr = 0; rr < S; ++rr) Ls += ws[2 * rr + 1] * __expf(ws[2 * rr] - M);
+                    wfac = __expf(st_m[G] - M) / Ls;
+                } else {
+                    wfac = 1.f / st_l[G];
+                }
+            }
+
+            // ---- stage the residual rows of the slots the rule will rewrite (bulk copies, no stall later) ----
+            if (a.do_write) {
+                uint32_t my_bytes = 0;
+                for (int t = 0; t < nt; ++t) {
+                    const int row = t * kTileRows + r;
+                    short slot = -1;
+                    if (row < n_stream && (a.dense || wsm[row] * wfac >= a.write_eps)) {
+                        const int sl = atomicAdd(lo_count, 1);
+                        slot = -2;
+                        if (sl < kLoCap) {
+                            slot = (short)sl;
+                            bulk_load(lostage + sl * ROW_BYTES, a.vlo + unit_off + (size_t)(slice_start + row) * ROW_BYTES,
+                                      ROW_BYTES, lobar);
+                            my_bytes += ROW_BYTES;
+                        }
+                    }
+                    idx[row] = slot;
+                }
+                mbar_arrive_expect_tx(lobar, my_bytes);
+                if (!mbar_wait(lobar, it & 1, *abort_flag ? 1024u : kWaitLimit)) {
+                    report_timeout(a.status, 21);
+                    *abort_flag = 1;
+                }
+            }
+
+            // ---- the update rule on the rows it changes, while the V tiles sit in the ring ----
+            float vt[8];  // this lane's 16-byte chunk of the write key-value vector
+            Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(a.v + kv_off + (lane & 15) * 16), vt);
+            for (int t = 0; t < nt; ++t, ++kc) {
+                const int stage = kc % NST;
+                if (!mbar_wait(&full[stage], (kc / NST) & 1, *abort_flag ? 1024u : kWaitLimit)) {
+                    report_timeout(a.status, 18);
+                    *abort_flag = 1;
+                }
+                const float ww = a.do_write ? wsm[t * kTileRows + r] * wfac : 0.f;
+                const int my_slot = a.do_write ? (int)idx[t * kTileRows + r] : -1;
+                uint32_t mask = __ballot_sync(0xffffffffu, my_slot != -1);
+                const unsigned char* tile = ring + (size_t)stage * kTcTileBytes;
+                while (mask) {
+                    const int r0 = __ffs(mask) - 1;
+                    mask &= mask - 1;
+                    int r1 = -1;
+                    if (mask) {
+                        r1 = __ffs(mask) - 1;
+                        mask &= mask - 1;
+                    }
+                    const float w0 = __shfl_sync(0xffffffffu, ww, r0);
+                    const float w1 = __shfl_sync(0xffffffffu, ww, r1 < 0 ? 0 : r1);
+                    const int s0 = __shfl_sync(0xffffffffu, my_slot, r0);
+                    const int s1 = __shfl_sync(0xffffffffu, my_slot, r1 < 0 ? 0 : r1);
+                    const int myr = (lane < 16) ? r0 : r1;
+                    if (myr >= 0) {
+                        const int slot = (lane < 16) ? s0 : s1;
+                        const float wr = (lane < 16) ? w0 : w1;
+                        const int R = warp * 32 + myr;  // row of the tile
+                        const int c = lane & 15;        // 16-byte chunk of the 256-byte row
+                        const uint4 hw = *reinterpret_cast<const uint4*>(tile + (c >> 3) * kHalfBytes + R * 128 +
+                                                                         (((c & 7) ^ (R & 7)) * 16));
+                        const size_t goff = unit_off + (size_t)(slice_start + t * kTileRows + R) * ROW_BYTES + c * 16;
+                        float x[8], lo[8], nv[8];
+                        Chunk<__nv_bfloat16>::unpack(hw, x);
+                        const uint4 lw = (slot >= 0) ? *reinterpret_cast<const uint4*>(lostage + slot * ROW_BYTES + c * 16)
+                                                     : *reinterpret_cast<const uint4*>(a.vlo + goff);
+                        Chunk<__nv_bfloat16>::unpack(lw, lo);
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) nv[e] = fmaf(wr, vt[e], x[e] + lo[e]);
+                        const uint4 hi_new = Chunk<__nv_bfloat16>::pack(nv);
+                        float hf[8];
+                        Chunk<__nv_bfloat16>::unpack(hi_new, hf);
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) nv[e] -= hf[e];
+                        *reinterpret_cast<uint4*>(a.vhi + goff) = hi_new;
+                        *reinterpret_cast<uint4*>(a.vlo + goff) = Chunk<__nv_bfloat16>::pack(nv);
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&empty[stage]);
+            }
+            if (has_virtual && tid < 16) {  // store the appended slot
+                const size_t off = unit_off + (size_t)a.len * ROW_BYTES + tid * 16;
+                *reinterpret_cast<uint4*>(a.kplane + off) = *reinterpret_cast<const uint4*>(a.k + kv_off + tid * 16);
+                *reinterpret_cast<uint4*>(a.vhi + off) = *reinterpret_cast<const uint4*>(a.v + kv_off + tid * 16);
+                *reinterpret_cast<uint4*>(a.vlo + off) = make_uint4(0, 0, 0, 0);
+            }
+
+            // ---- epilogue: O[d][g] from tensor memory, normalise, store ----
+            if (!mbar_wait(oready, it & 1, *abort_flag ? 1024u : kWaitLimit)) {
+                report_timeout(a.status, 19);
+                *abort_flag = 1;
+            }
+            tc_fence_after();
+            float o[8];
+            if (nt > 0) {
+                tmem_ld8(lane_base + kOCol, o);
+            } else {
+#pragma unroll
+                for (int h = 0; h < 8; ++h) o[h] = 0.f;
+            }
+            if (has_virtual) {
+#pragma unroll
+                for (int g = 0; g < G; ++g) o[g] = fmaf(st_ev[g], vd, o[g]);
+            }
+            const bool add_own = a.wtr && a.do_write;
+            if (S == 1) {
+                if (a.out != nullptr && !*abort_flag) {
+#pragma unroll
+                    for (int g = 0; g < G; ++g) {
+                        const float inv = 1.f / st_l[g];
+                        float val = o[g] * inv;
+                        if (add_own) val = fmaf(st_wd[g] * inv * wfac, vd, val);
+                        if (a.out_f32)
+                            reinterpret_cast<float*>(a.out + q_off * 2)[g * D + r] = val;
+                        else
+                            reinterpret_cast<__nv_bfloat16*>(a.out + q_off)[g * D + r] = __float2bfloat16_rn(val);
+                    }
+                }
+            } else {
+                float* mg = merge + (size_t)(it & 1) * (S - 1) * G * (D + 3);
+                if (rank != 0) {
+                    float* dst0 = mg + (size_t)(rank - 1) * G * (D + 3);
+#pragma unroll
+                    for (int g = 0; g < G; ++g) {
+                        st_cluster_f32(map_to_rank(dst0 + g * (D + 3) + r, 0), o[g]);
+                        if (r == 0) {
+                            st_cluster_f32(map_to_rank(dst0 + g * (D + 3) + D, 0), st_wd[g] * wfac);
+                            st_cluster_f32(map_to_rank(dst0 + g * (D + 3) + D + 1, 0), st_m[g]);
+                            st_cluster_f32(map_to_rank(dst0 + g * (D + 3) + D + 2, 0), st_l[g]);
+                        }
+                    }
+                    mbar_arrive_remote(map_to_rank(&mbar[it & 1], 0));
+                } else {
+                    if (!mbar_wait<true>(&mbar[it & 1], (it >> 1) & 1, *abort_flag ? 1024u : kWaitLimit)) {
+                        report_timeout(a.status, 20);
+                        *abort_flag = 1;
+                    }
+                    if (a.out != nullptr && !*abort_flag) {
+#pragma unroll
+                        for (int g = 0; g < G; ++g) {
+                            float M = st_m[g];
+                            for (int rr = 1; rr < S; ++rr) M = fmaxf(M, mg[((rr - 1) * G + g) * (D + 3) + D + 1]);
+                            const float f0 = __expf(st_m[g] - M);
+                            float num = o[g] * f0, own = st_wd[g] * wfac * f0, den = st_l[g] * f0;
+                            for (int rr = 1; rr < S; ++rr) {
+                                const float* mr = mg + ((rr - 1) * G + g) * (D + 3);
+                                const float f = __expf(mr[D + 1] - M);
+                                num = fmaf(mr[r], f, num);
+                                own = fmaf(mr[D], f, own);
+                                den = fmaf(mr[D + 2], f, den);
+                            }
+                            float val = num / den;
+                            if (add_own) val = fmaf(own / den, vd, val);
+                            if (a.out_f32)
+                                reinterpret_cast<float*>(a.out + q_off * 2)[g * D + r] = val;
+                            else
+                                reinterpret_cast<__nv_bfloat16*>(a.out + q_off)[g * D + r] = __float2bfloat16_rn(val);
+                        }
+                    }
+                }
+            }
+            if (tid == 0) *lo_count = 0;
+            s_sync();  // st_*, red and the staging rows are reused by the next unit
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (S > 1) {  // nobody leaves while a peer may still write its shared memory
+        cluster_arrive();
+        cluster_wait();
+    }
+    if (warp == 5) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+using TcKernelFn = void (*)(const CUtensorMap, const CUtensorMap, const TcArgs);
+
+TcKernelFn pick_tc(int G) {
+    switch (G) {
+        case 1: return decode_tc_kernel<1>;
+        case 2: return decode_tc_kernel<2>;
+        case 3: return decode_tc_kernel<3>;
+        case 4: return decode_tc_kernel<4>;
+        case 5: return decode_tc_kernel<5>;
+        case 6: return decode_tc_kernel<6>;
+        case 7: return decode_tc_kernel<7>;
+        default: return nullptr;
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// [U][C][128] bfloat16 plane as a 3-D tensor (d, slot, unit); boxes of 64 x 128 x 1 with the
+// 128-byte swizzle; rows past C read as zeros.
+bool make_plane_map(CUtensorMap* map, void* base, int U, int C) {
+    EncodeTiledFn fn = encode_fn();
+    if (fn == nullptr) return false;
+    const cuuint64_t dims[3] = {128, (cuuint64_t)C, (cuuint64_t)U};
+    const cuuint64_t strides[2] = {256, (cuuint64_t)C * 256};
+    const cuuint32_t box[3] = {64, (cuuint32_t)kTileRows, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+bool tc_eligible(const bct_cache* c) {
+    const bct_params_t& p = c->p;
+    if (p.dtype != BCT_BF16 || p.head_dim != 128 || c->G > 7) return false;
+    if (p.flags & BCT_FLAG_PRECISE_READ) return false;
+    if (p.capacity < kTileRows || p.capacity > kMaxClusterTc * kMaxTiles * kTileRows) return false;
+    if (c->plane_bytes < (size_t)1 << 18) return false;  // tiny planes stay on the CUDA-core kernel
+    return c->tc_ready != 0;
+}
+
+bool tc_prepare(bct_cache* c) {
+    c->tc_ready = 0;
+    static_assert(sizeof(CUtensorMap) <= sizeof(c->tmap_k), "tensor map storage too small");
+    if (c->p.dtype != BCT_BF16 || c->p.head_dim != 128) return false;
+    if (!make_plane_map(reinterpret_cast<CUtensorMap*>(c->tmap_k), c->kplane, c->U, c->p.capacity)) return false;
+    if (!make_plane_map(reinterpret_cast<CUtensorMap*>(c->tmap_v), c->vhi, c->U, c->p.capacity)) return false;
+    c->tc_ready = 1;
+    return true;
+}
+
+int launch_decode_tc(const bct_cache* c, const StepIO& io, int len, int do_write, cudaStream_t stream,
+                     cudaError_t* err) {
+    const bct_params_t& p = c->p;
+    TcKernelFn fn = pick_tc(c->G);
+    if (fn == nullptr) {
+        *err = cudaErrorInvalidConfiguration;
+        return -1;
+    }
+    const int max_slice = kMaxTiles * kTileRows;
+    int S = 1;
+    while (S < kMaxClusterTc && (p.capacity + S - 1) / S > max_slice) S *= 2;
+    while (S < kMaxClusterTc && (long long)c->U * S * 2 <= c->sm_count && (p.capacity + 2 * S - 1) / (2 * S) >= kTileRows)
+        S *= 2;  // few units: spread each over more SMs
+    int slice = (p.capacity + S - 1) / S;
+    slice = (slice + kTileRows - 1) / kTileRows * kTileRows;  // whole tiles per CTA
+    int stages = 4;
+    while (stages > 2 && tc_smem(stages, c->G, S).total > c->smem_optin) --stages;
+    const int smem = tc_smem(stages, c->G, S).total;
+
+    TcArgs a;
+    a.vhi = c->vhi;
+    a.vlo = c->vlo;
+    a.kplane = c->kplane;
+    a.q = static_cast<const char*>(io.q);
+    a.k = static_cast<const char*>(io.k);
+    a.v = static_cast<const char*>(io.v);
+    a.out = static_cast<char*>(io.out);
+    a.status = c->status;
+    a.q_bs = io.q_batch_stride;
+    a.kv_bs = io.kv_batch_stride;
+    a.C = p.capacity;
+    a.len = len;
+    a.slice_rows = slice;
+    a.S = S;
+    a.Hkv = p.n_kv_heads;
+    a.U = c->U;
+    a.stages = stages;
+    a.do_write = (len == p.capacity) && do_write;
+    a.wtr = (p.flags & BCT_FLAG_WRITE_THEN_READ) ? 1 : 0;
+    a.dense = (p.flags & BCT_FLAG_DENSE_WRITE) ? 1 : 0;
+    a.out_f32 = (p.flags & BCT_FLAG_OUT_F32) ? 1 : 0;
+    a.read_scale = p.read_scale;
+    a.write_scale = p.write_scale;
+    a.write_eps = p.write_eps;
+
+    *err = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (*err != cudaSuccess) return -1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.blockDim = dim3(kTcThreads, 1, 1);
+    cfg.dynamicSmemBytes = (size_t)smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)S;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n_clusters = c->sm_count / S;
+    if (S > 1) {
+        cfg.gridDim = dim3((unsigned)(S * (c->sm_count / S)), 1, 1);
+        int active = 0;
+        *err = cudaOccupancyMaxActiveClusters(&active, reinterpret_cast<const void*>(fn), &cfg);
+        if (*err != cudaSuccess) return -1;
+        if (active < 1) {
+            *err = cudaErrorInvalidConfiguration;
+            return -1;
+        }
+        n_clusters = active < n_clusters ? active : n_clusters;
+    }
+    if (n_clusters > c->U) n_clusters = c->U;
+    cfg.gridDim = dim3((unsigned)(n_clusters * S), 1, 1);
+    *err = cudaLaunchKernelEx(&cfg, fn, *reinterpret_cast<const CUtensorMap*>(c->tmap_k),
+                              *reinterpret_cast<const CUtensorMap*>(c->tmap_v), a);
+    if (*err != cudaSuccess) return -1;
+    return 1;
+}
+
+}  // namespace bct

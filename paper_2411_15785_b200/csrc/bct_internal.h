@@ -47,6 +47,9 @@ struct bct_cache {
     int device;
     int sm_count;
     int smem_optin;  // max dynamic shared memory per block (opt-in)
+    int tc_ready;    // tensor maps below are valid (bfloat16, head_dim 128)
+    alignas(64) unsigned char tmap_k[128];  // CUtensorMap of the MK plane
+    alignas(64) unsigned char tmap_v[128];  // CUtensorMap of the MV value plane
 };
 
 namespace bct {
@@ -60,6 +63,12 @@ int launch_decode(const bct_cache* c, const StepIO& io, int len, int do_write, c
 
 // Whether launch_decode has a kernel for these parameters (shape limits of this build).
 bool decode_supported(const bct_params_t& p, int smem_optin, const char** why);
+
+// Tensor-core (tcgen05 + TMA) decode path: bfloat16, head_dim 128, group <= 7.
+bool tc_prepare(bct_cache* c);          // encode the planes' tensor maps; false if unavailable
+bool tc_eligible(const bct_cache* c);   // this cache's decode steps run on the tensor path
+int launch_decode_tc(const bct_cache* c, const StepIO& io, int len, int do_write, cudaStream_t stream,
+                     cudaError_t* err);
 
 // State import / export.
 cudaError_t launch_import(const bct_cache* c, const void* k_in, const void* v_in, int v_dtype, int len,

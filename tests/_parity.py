@@ -82,10 +82,12 @@ def compare_state(w, units, gpu, ora):
     return err
 
 
-def run_decode_parity(w: W.Workload, units, steps=None, device="cuda", **kw):
+def run_decode_parity(w: W.Workload, units, steps=None, device="cuda", expect_tensor_path=None, **kw):
     """Step both sides token by token; return (max out error, state error)."""
     steps = w.steps if steps is None else steps
     gpu, ora = make_pair(w, units, device, **kw)
+    if expect_tensor_path is not None:
+        assert gpu.tensor_path == expect_tensor_path
     worst = 0.0
     for t in range(steps):
         q, k, v = W.step_inputs(w, t, device)

@@ -35,7 +35,13 @@ def test_config1_single_sequence_fp32_fill_then_update():
 
 def test_config2_mha_batch64_c2048_bf16():
     w = W.CONFIGS["mha7b_b64_c2048"]
-    out_err, state_err = run_decode_parity(w, pick_units(w, _n_units(), seed=1))
+    out_err, state_err = run_decode_parity(w, pick_units(w, _n_units(), seed=1), expect_tensor_path=True)
+    assert out_err <= TOL["bf16"] and state_err <= TOL["bf16"], (out_err, state_err)
+
+
+def test_config2_on_the_cuda_core_kernel():
+    w = W.CONFIGS["mha7b_b64_c2048"].scaled(steps=128)
+    out_err, state_err = run_decode_parity(w, pick_units(w, 8, seed=1), flags=B.FLAG_CUDA_CORES)
     assert out_err <= TOL["bf16"] and state_err <= TOL["bf16"], (out_err, state_err)
 
 

@@ -46,6 +46,39 @@ def test_small_shapes_match_oracle(dtype, d, G, C, init_len, steps):
     assert state_err <= TOL[dtype], state_err
 
 
+# ---- the tensor-core kernel (bfloat16, head_dim 128, G <= 7, C >= 128) and the CUDA-core kernel
+# ---- on the same shapes: both must match the oracle ----------------------------------------------------
+@pytest.mark.parametrize("cores", [False, True])
+@pytest.mark.parametrize("B_,G,C,init_len,steps", [
+    (2, 1, 333, 333, 8),       # ragged last tile
+    (2, 4, 520, 500, 30),      # fill finishes mid-run
+    (5, 7, 128, 0, 140),       # fills from empty, one tile
+    (5, 2, 2048, 2048, 6),     # 16 tiles: a full slice
+    (2, 3, 2500, 2500, 5),     # cluster of 2, ragged
+    (40, 4, 300, 290, 14),     # more units than one pass of the persistent grid
+    (1, 1, 16384, 16384, 3),   # cluster of 8, full slices
+])
+def test_tensor_core_and_cuda_core_kernels_match_oracle(cores, B_, G, C, init_len, steps):
+    d = 128
+    w = W.Workload("t", B_, 2 * G, 2, d, C, "bf16", init_len, steps, 13, d ** -0.5, 1.0, 1.0, "decode")
+    units = pick_units(w, 6)
+    out_err, state_err = run_decode_parity(w, units, flags=B.FLAG_CUDA_CORES if cores else 0,
+                                           expect_tensor_path=not cores)
+    assert out_err <= TOL["bf16"], out_err
+    assert state_err <= TOL["bf16"], state_err
+
+
+@pytest.mark.parametrize("flag,oflag", [(B.FLAG_WRITE_THEN_READ, O.WRITE_THEN_READ), (B.FLAG_DENSE_WRITE, 0),
+                                        (B.FLAG_OUT_F32, 0)])
+@pytest.mark.parametrize("C", [400, 5000])
+def test_tensor_core_kernel_flags(flag, oflag, C):
+    d = 128
+    w = W.Workload("t", 2, 6, 2, d, C, "bf16", C, 6, 17, d ** -0.5, 1.0, 1.0, "decode", 1.0, 0.3)
+    out_err, state_err = run_decode_parity(w, pick_units(w, 4), flags=flag, oracle_flags=oflag,
+                                           expect_tensor_path=True)
+    assert out_err <= TOL["bf16"] and state_err <= TOL["bf16"], (out_err, state_err)
+
+
 def test_diffuse_writes_rewrite_every_row():
     d = 128
     w = W.Workload("t", 2, 4, 2, d, 700, "bf16", 700, 12, 5, d ** -0.5, 1.0, 1.0, "decode", 1.0, d ** -0.5)
