@@ -196,6 +196,8 @@ def main():
     ap.add_argument("--workload", default="mha7b_b64_c2048", choices=sorted(W.CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--write-scale", type=float, default=None, help="override the write score scale")
+    ap.add_argument("--write-eps", type=float, default=0.0, help="override write_eps (0 = library default 2^-24)")
+    ap.add_argument("--flags", type=int, default=0, help="BCT_FLAG_* bits for the cache")
     ap.add_argument("--batch", type=int, default=None, help="override the batch (profiling on a smaller case)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -232,7 +234,7 @@ def main():
     mk, mv = W.initial_cache(wr, dev)
     cache = B.Cache(w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.capacity, w.torch_dtype,
                     read_scale=w.read_scale, write_scale=w.write_scale, init_len=w.init_len, mk_init=mk, mv_init=mv,
-                    device=dev)
+                    write_eps=args.write_eps, flags=args.flags, device=dev)
     torch.cuda.synchronize()
     del mk, mv
     pool = [W.step_inputs(wr, t, dev) for t in range(min(args.steps + args.warmup, 64))]

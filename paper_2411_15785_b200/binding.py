@@ -16,7 +16,8 @@ BCT_OK, BCT_ERR_INVALID_ARG, BCT_ERR_UNSUPPORTED, BCT_ERR_STATE, BCT_ERR_CUDA, B
 BCT_F32, BCT_BF16, BCT_BF16_PAIR = 0, 1, 2
 FLAG_SKIP_FIRST_WRITE, FLAG_WRITE_THEN_READ, FLAG_DENSE_WRITE, FLAG_OUT_F32, FLAG_PRECISE_READ, FLAG_CUDA_CORES = 1, 2, 4, 8, 16, 32
 
-LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libbct_b200.so")
+# BCT_LIBRARY selects another build of the same ABI (e.g. one compiled with different tuning constants).
+LIB_PATH = os.environ.get("BCT_LIBRARY") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "libbct_b200.so")
 
 EXPORTS = (
     "bct_version", "bct_last_error", "bct_cache_bytes", "bct_cache_create", "bct_decode_step",

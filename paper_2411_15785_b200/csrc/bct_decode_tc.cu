@@ -13,12 +13,16 @@
 //
 // One persistent CTA per SM (or a cluster of S CTAs per unit when C > 2048 slots), three roles:
 //   warp 4  producer : TMA loads of K tiles then V tiles into a ring, running ahead across units
-//   warp 5  MMA      : issues the tensor-core work as tiles land, commits to mbarriers
-//   warps 0-3        : softmax statistics from tensor memory, P operand, update rule, epilogue
+//   warp 5  MMA      : issues the tensor-core work as tiles land; its commits free the ring stages
+//   warps 0-3        : softmax statistics from tensor memory, P operand, epilogue, and the update
+//                      rule from staged copies of the rows to rewrite (applied once the unit's V
+//                      tiles have all been read, so the read sees MV_{t-1})
 // Every wait is bounded; a timeout sets the status word and the kernel runs to its end.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
+
+#include <cstdlib>
 
 #include "bct_device.cuh"
 #include "bct_internal.h"
@@ -38,7 +42,7 @@ constexpr int kScoreCols = 16;                 // tensor-memory columns per scor
 constexpr int kOCol = kMaxTiles * kScoreCols;  // output accumulator behind the score tiles
 constexpr int kTmemCols = 512;
 constexpr int kMaxClusterTc = 8;
-constexpr int kLoCap = 64;                     // residual rows prefetched per unit; further rows take the slow path
+constexpr int kLoCap = 80;                     // rewritten rows staged per unit slice; further rows take a slow path
 constexpr float kNegBigTc = -3.0e38f;
 
 struct TcArgs {
@@ -58,7 +62,7 @@ struct TcArgs {
 };
 
 struct TcSmem {
-    int ring, pbuf, qbuf, wsm, idx, lostage, red, stat, wstat, merge, bars, total;
+    int ring, pbuf, qbuf, wsm, idx, lostage, list, red, stat, wstat, merge, bars, total;
 };
 __host__ __device__ inline TcSmem tc_smem(int stages, int G, int S) {
     TcSmem L;
@@ -71,10 +75,12 @@ __host__ __device__ inline TcSmem tc_smem(int stages, int G, int S) {
     off += 2 * kQBufBytes;
     L.wsm = off;
     off += kMaxTiles * kTileRows * 4;
-    L.idx = off;  // per slot: staging row of its residual, -1 untouched, -2 not staged
+    L.idx = off;  // per slot: -1 untouched, >= 0 staging row, -2 rewritten but not staged
     off += kMaxTiles * kTileRows * 2;
-    L.lostage = off;
-    off += kLoCap * 256;
+    L.lostage = off;  // staged rows of the slots to rewrite: value plane rows, then residual rows
+    off += 2 * kLoCap * 256;
+    L.list = off;     // per staged row: slot index and write weight
+    off += kLoCap * 8;
     L.red = off;
     off += 4 * 16 * 4;
     L.stat = off;  // m[8], l[8], wd[8], ev[8], abort, tmem address
@@ -85,7 +91,7 @@ __host__ __device__ inline TcSmem tc_smem(int stages, int G, int S) {
     off += (S > 1) ? 2 * (S - 1) * G * (128 + 3) * 4 : 0;
     off = (off + 15) & ~15;
     L.bars = off;
-    off += (3 * stages + 2 + 1 + 1 + 2 + 2 + 1) * 8;
+    off += (2 * stages + 2 * kMaxTiles + 2 + 1 + 2 + 2) * 8;
     L.total = ((off + 127) & ~127) + 1024;  // + slack to align the ring to 1024 bytes
     return L;
 }
@@ -146,6 +152,12 @@ __host__ __device__ constexpr uint32_t instr_desc(bool a_mn_major) {
            ((128u >> 4) << 24);
 }
 
+__device__ __forceinline__ void cp_async16(void* dst_smem, const void* src_gmem) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst_smem)), "l"(src_gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+
 __device__ __forceinline__ void s_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kSThreads) : "memory"); }
 
 template <int G>
@@ -163,7 +175,10 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     unsigned char* qbuf = smem + L.qbuf;
     float* wsm = reinterpret_cast<float*>(smem + L.wsm);
     short* idx = reinterpret_cast<short*>(smem + L.idx);
-    unsigned char* lostage = smem + L.lostage;
+    unsigned char* histage = smem + L.lostage;
+    unsigned char* lostage = histage + kLoCap * ROW_BYTES;
+    int* list_row = reinterpret_cast<int*>(smem + L.list);
+    float* list_ww = reinterpret_cast<float*>(smem + L.list) + kLoCap;
     float* red = reinterpret_cast<float*>(smem + L.red);
     float* st_m = reinterpret_cast<float*>(smem + L.stat);
     float* st_l = st_m + 8;
@@ -176,13 +191,12 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     float* merge = reinterpret_cast<float*>(smem + L.merge);
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + L.bars);
     uint64_t* empty = full + NST;
-    uint64_t* sready = empty + NST;
-    uint64_t* qready = sready + NST;  // [2]
-    uint64_t* pready = qready + 2;
-    uint64_t* oready = pready + 1;
-    uint64_t* xbar = oready + 1;      // [2]
-    uint64_t* mbar = xbar + 2;        // [2]
-    uint64_t* lobar = mbar + 2;
+    uint64_t* sready = empty + NST;         // [kMaxTiles]: score tile t of the current unit is complete
+    uint64_t* pready = sready + kMaxTiles;  // [kMaxTiles]: P operand of tile t of the current unit is written
+    uint64_t* qready = pready + kMaxTiles;  // [2]
+    uint64_t* oready = qready + 2;
+    uint64_t* xbar = oready + 1;            // [2]
+    uint64_t* mbar = xbar + 2;              // [2]
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
@@ -200,26 +214,28 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     if (tid == 0) {
         for (int i = 0; i < NST; ++i) {
             mbar_init(&full[i], 1);
-            mbar_init(&empty[i], 5);  // the MMA commit + one lane of each softmax warp
+            mbar_init(&empty[i], 1);  // the MMA commit alone frees a stage
+        }
+        for (int i = 0; i < kMaxTiles; ++i) {
             mbar_init(&sready[i], 1);
+            mbar_init(&pready[i], kSThreads);
         }
         mbar_init(&qready[0], kSThreads);
         mbar_init(&qready[1], kSThreads);
-        mbar_init(pready, kSThreads);
         mbar_init(oready, 1);
         mbar_init(&xbar[0], S);
         mbar_init(&xbar[1], S);
         mbar_init(&mbar[0], kSThreads * (S > 1 ? S - 1 : 1));
         mbar_init(&mbar[1], kSThreads * (S > 1 ? S - 1 : 1));
-        mbar_init(lobar, kSThreads);
         *abort_flag = 0;
         *lo_count = 0;
         fence_mbar_init_cluster();
     }
-    // zero the operand padding: Q rows above the write query, the dummy rows behind Q and P
+    // zero the operands: rows G..7 of P and rows above the write query of Q stay zero for good,
+    // and so do the dummy rows behind them that the N = 16 instruction shape reads
     for (int i = tid; i < 2 * kQBufBytes / 16; i += kTcThreads) reinterpret_cast<uint4*>(qbuf)[i] = make_uint4(0, 0, 0, 0);
-    for (int i = tid; i < 1024 / 16; i += kTcThreads)
-        reinterpret_cast<uint4*>(pbuf + kMaxTiles * kPTileBytes)[i] = make_uint4(0, 0, 0, 0);
+    for (int i = tid; i < (kMaxTiles * kPTileBytes + 1024) / 16; i += kTcThreads)
+        reinterpret_cast<uint4*>(pbuf)[i] = make_uint4(0, 0, 0, 0);
     if (warp == 5) tmem_alloc(tmem_slot, kTmemCols);
     fence_proxy_async_smem();
     tc_fence_before();
@@ -285,16 +301,15 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         const uint64_t bd = smem_desc(qaddr + (kk >> 2) * 1024 + (kk & 3) * 32, 16, 1024);
                         umma_bf16(tmem_base + t * kScoreCols, ad, bd, idesc_s, kk > 0);
                     }
-                    umma_commit(&sready[stage]);
+                    umma_commit(&sready[t]);
                     umma_commit(&empty[stage]);
                 }
-                if (!mbar_wait(pready, it & 1, *abort_flag ? 1024u : kWaitLimit)) {
-                    report_timeout(a.status, 14);
-                    *abort_flag = 1;
-                }
-                tc_fence_after();
                 for (int t = 0; t < nt; ++t, ++kc) {  // outputs: A = V tile (MN-major), B = P (K-major)
                     const int stage = kc % NST;
+                    if (!mbar_wait(&pready[t], it & 1, *abort_flag ? 1024u : kWaitLimit)) {
+                        report_timeout(a.status, 14);
+                        *abort_flag = 1;
+                    }
                     if (!mbar_wait(&full[stage], (kc / NST) & 1, *abort_flag ? 1024u : kWaitLimit)) {
                         report_timeout(a.status, 15);
                         *abort_flag = 1;
@@ -308,18 +323,35 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         const uint64_t bd = smem_desc(paddr + (kk >> 2) * 1024 + (kk & 3) * 32, 16, 1024);
                         umma_bf16(tmem_base + kOCol, ad, bd, idesc_o, (t > 0) || (kk > 0));
                     }
-                    umma_commit(&sready[stage]);  // keeps this barrier's phase in step with the ring
                     umma_commit(&empty[stage]);
                 }
-                umma_commit(oready);
+                umma_commit(oready);  // every V tile of the unit has been read
             }
         }
         __syncwarp();
     } else {
-        // =========================== softmax / update / epilogue warps ===========================
+        // =========================== softmax / epilogue / update warps ===========================
         const int r = tid;  // tensor-memory lane: slot row of a score tile, d of the output
         const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
-        uint32_t kc = 0;
+
+        // Q operand of a unit: rows 0..G-1 its read queries, row G its write query (128-byte swizzle)
+        auto write_q = [&](int u, int buf) {
+            const int b = u / a.Hkv;
+            const int h_kv = u - b * a.Hkv;
+            const int h = tid >> 4, c = tid & 15;
+            if (h <= G) {
+                const char* src = (h < G) ? a.q + ((size_t)b * a.q_bs + (size_t)h_kv * G * D) * 2 + (size_t)h * ROW_BYTES
+                                          : a.k + ((size_t)b * a.kv_bs + (size_t)h_kv * D) * 2;
+                const uint4 w = *reinterpret_cast<const uint4*>(src + c * 16);
+                unsigned char* dst = qbuf + buf * kQBufBytes + (c >> 3) * 1024 + h * 128 + (((c & 7) ^ h) * 16);
+                *reinterpret_cast<uint4*>(dst) = w;
+            }
+            fence_proxy_async_smem();
+            tc_fence_before();
+            mbar_arrive(&qready[buf]);
+        };
+        if (cid < a.U) write_q(cid, 0);
+
         int it = 0;
         for (int u = cid; u < a.U; u += ncl, ++it) {
             const int b = u / a.Hkv;
@@ -328,27 +360,12 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             const size_t kv_off = ((size_t)b * a.kv_bs + (size_t)h_kv * D) * 2;
             const size_t unit_off = (size_t)u * a.C * ROW_BYTES;
 
-            // ---- Q operand: rows 0..G-1 read queries, row G the write query (128-byte swizzle) ----
-            {
-                const int h = tid >> 4, c = tid & 15;
-                if (h <= G) {
-                    const char* src = (h < G) ? a.q + q_off + (size_t)h * ROW_BYTES : a.k + kv_off;
-                    const uint4 w = *reinterpret_cast<const uint4*>(src + c * 16);
-                    unsigned char* dst = qbuf + (it & 1) * kQBufBytes + (c >> 3) * 1024 + h * 128 + (((c & 7) ^ h) * 16);
-                    *reinterpret_cast<uint4*>(dst) = w;
-                }
-            }
-            fence_proxy_async_smem();
-            tc_fence_before();
-            mbar_arrive(&qready[it & 1]);
-
             // ---- pass 1: row maxima of the raw scores, as the score tiles complete ----
             float mx[8];
 #pragma unroll
             for (int h = 0; h < 8; ++h) mx[h] = kNegBigTc;
-            for (int t = 0; t < nt; ++t, ++kc) {
-                const int stage = kc % NST;
-                if (!mbar_wait(&sready[stage], (kc / NST) & 1, *abort_flag ? 1024u : kWaitLimit)) {
+            for (int t = 0; t < nt; ++t) {
+                if (!mbar_wait(&sready[t], it & 1, *abort_flag ? 1024u : kWaitLimit)) {
                     report_timeout(a.status, 16);
                     *abort_flag = 1;
                 }
@@ -359,11 +376,9 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 #pragma unroll
                     for (int h = 0; h < 8; ++h) mx[h] = fmaxf(mx[h], s[h]);
                 }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&empty[stage]);
             }
             // the appended slot (fill phase) is scored from the step vectors
-            float vq[G > 0 ? G : 1];
+            float vq[G];
             const float kd = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(a.k + kv_off)[r]);
             const float vd = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(a.v + kv_off)[r]);
 #pragma unroll
@@ -396,7 +411,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 
             // ---- pass 2: numerators, row sums, P operand (bfloat16, swizzled), write numerators ----
             float sum[8];
-            float wdacc[G > 0 ? G : 1];
+            float wdacc[G];
 #pragma unroll
             for (int h = 0; h < 8; ++h) sum[h] = 0.f;
 #pragma unroll
@@ -415,16 +430,18 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 unsigned char* prow = pbuf + t * kPTileBytes + (r >> 6) * 1024 + (r & 7) * 2;
                 const int c8 = (r & 63) >> 3;
 #pragma unroll
-                for (int h = 0; h < 8; ++h) {
-                    const __nv_bfloat16 pv = __float2bfloat16_rn(h < G ? e[h] : 0.f);
-                    *reinterpret_cast<__nv_bfloat16*>(prow + h * 128 + ((c8 ^ h) * 16)) = pv;
-                }
+                for (int h = 0; h < G; ++h)  // rows G..7 of the operand stay zero
+                    *reinterpret_cast<__nv_bfloat16*>(prow + h * 128 + ((c8 ^ h) * 16)) = __float2bfloat16_rn(e[h]);
                 wsm[t * kTileRows + r] = e[G];
 #pragma unroll
                 for (int g = 0; g < G; ++g) wdacc[g] = fmaf(e[g], e[G], wdacc[g]);
+                fence_proxy_async_smem();
+                tc_fence_before();
+                mbar_arrive(&pready[t]);  // the V tile's MMAs may go as soon as its weights are in place
             }
-            fence_proxy_async_smem();
-            mbar_arrive(pready);
+            // the next unit's scores may start as soon as this unit's V tiles are through
+            if (u + ncl < a.U) write_q(u + ncl, (it + 1) & 1);
+
 #pragma unroll
             for (int h = 0; h < 8; ++h) {
                 sum[h] = warp_sum(sum[h]);
@@ -475,92 +492,36 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 }
             }
 
-            // ---- stage the residual rows of the slots the rule will rewrite (bulk copies, no stall later) ----
+            // ---- stage copies of the rows the rule will rewrite (value and residual rows) with 16-byte
+            // ---- asynchronous copies, so that no global-memory latency is left for the update itself ----
             if (a.do_write) {
-                uint32_t my_bytes = 0;
                 for (int t = 0; t < nt; ++t) {
                     const int row = t * kTileRows + r;
                     short slot = -1;
-                    if (row < n_stream && (a.dense || wsm[row] * wfac >= a.write_eps)) {
+                    const float ww = wsm[row] * wfac;
+                    if (row < n_stream && (a.dense || ww >= a.write_eps)) {
                         const int sl = atomicAdd(lo_count, 1);
                         slot = -2;
                         if (sl < kLoCap) {
                             slot = (short)sl;
-                            bulk_load(lostage + sl * ROW_BYTES, a.vlo + unit_off + (size_t)(slice_start + row) * ROW_BYTES,
-                                      ROW_BYTES, lobar);
-                            my_bytes += ROW_BYTES;
+                            list_row[sl] = row;
+                            list_ww[sl] = ww;
                         }
                     }
                     idx[row] = slot;
                 }
-                mbar_arrive_expect_tx(lobar, my_bytes);
-                if (!mbar_wait(lobar, it & 1, *abort_flag ? 1024u : kWaitLimit)) {
-                    report_timeout(a.status, 21);
-                    *abort_flag = 1;
+                s_sync();
+                const int n_staged = min(*lo_count, kLoCap);
+                const int c = tid & 15;
+                for (int sl = tid >> 4; sl < n_staged; sl += kSThreads / 16) {
+                    const size_t goff = unit_off + (size_t)(slice_start + list_row[sl]) * ROW_BYTES + c * 16;
+                    cp_async16(histage + sl * ROW_BYTES + c * 16, a.vhi + goff);
+                    cp_async16(lostage + sl * ROW_BYTES + c * 16, a.vlo + goff);
                 }
+                cp_async_commit();
             }
 
-            // ---- the update rule on the rows it changes, while the V tiles sit in the ring ----
-            float vt[8];  // this lane's 16-byte chunk of the write key-value vector
-            Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(a.v + kv_off + (lane & 15) * 16), vt);
-            for (int t = 0; t < nt; ++t, ++kc) {
-                const int stage = kc % NST;
-                if (!mbar_wait(&full[stage], (kc / NST) & 1, *abort_flag ? 1024u : kWaitLimit)) {
-                    report_timeout(a.status, 18);
-                    *abort_flag = 1;
-                }
-                const float ww = a.do_write ? wsm[t * kTileRows + r] * wfac : 0.f;
-                const int my_slot = a.do_write ? (int)idx[t * kTileRows + r] : -1;
-                uint32_t mask = __ballot_sync(0xffffffffu, my_slot != -1);
-                const unsigned char* tile = ring + (size_t)stage * kTcTileBytes;
-                while (mask) {
-                    const int r0 = __ffs(mask) - 1;
-                    mask &= mask - 1;
-                    int r1 = -1;
-                    if (mask) {
-                        r1 = __ffs(mask) - 1;
-                        mask &= mask - 1;
-                    }
-                    const float w0 = __shfl_sync(0xffffffffu, ww, r0);
-                    const float w1 = __shfl_sync(0xffffffffu, ww, r1 < 0 ? 0 : r1);
-                    const int s0 = __shfl_sync(0xffffffffu, my_slot, r0);
-                    const int s1 = __shfl_sync(0xffffffffu, my_slot, r1 < 0 ? 0 : r1);
-                    const int myr = (lane < 16) ? r0 : r1;
-                    if (myr >= 0) {
-                        const int slot = (lane < 16) ? s0 : s1;
-                        const float wr = (lane < 16) ? w0 : w1;
-                        const int R = warp * 32 + myr;  // row of the tile
-                        const int c = lane & 15;        // 16-byte chunk of the 256-byte row
-                        const uint4 hw = *reinterpret_cast<const uint4*>(tile + (c >> 3) * kHalfBytes + R * 128 +
-                                                                         (((c & 7) ^ (R & 7)) * 16));
-                        const size_t goff = unit_off + (size_t)(slice_start + t * kTileRows + R) * ROW_BYTES + c * 16;
-                        float x[8], lo[8], nv[8];
-                        Chunk<__nv_bfloat16>::unpack(hw, x);
-                        const uint4 lw = (slot >= 0) ? *reinterpret_cast<const uint4*>(lostage + slot * ROW_BYTES + c * 16)
-                                                     : *reinterpret_cast<const uint4*>(a.vlo + goff);
-                        Chunk<__nv_bfloat16>::unpack(lw, lo);
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) nv[e] = fmaf(wr, vt[e], x[e] + lo[e]);
-                        const uint4 hi_new = Chunk<__nv_bfloat16>::pack(nv);
-                        float hf[8];
-                        Chunk<__nv_bfloat16>::unpack(hi_new, hf);
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) nv[e] -= hf[e];
-                        *reinterpret_cast<uint4*>(a.vhi + goff) = hi_new;
-                        *reinterpret_cast<uint4*>(a.vlo + goff) = Chunk<__nv_bfloat16>::pack(nv);
-                    }
-                }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&empty[stage]);
-            }
-            if (has_virtual && tid < 16) {  // store the appended slot
-                const size_t off = unit_off + (size_t)a.len * ROW_BYTES + tid * 16;
-                *reinterpret_cast<uint4*>(a.kplane + off) = *reinterpret_cast<const uint4*>(a.k + kv_off + tid * 16);
-                *reinterpret_cast<uint4*>(a.vhi + off) = *reinterpret_cast<const uint4*>(a.v + kv_off + tid * 16);
-                *reinterpret_cast<uint4*>(a.vlo + off) = make_uint4(0, 0, 0, 0);
-            }
-
-            // ---- epilogue: O[d][g] from tensor memory, normalise, store ----
+            // ---- epilogue: O[d][g] from tensor memory once every V tile has been read ----
             if (!mbar_wait(oready, it & 1, *abort_flag ? 1024u : kWaitLimit)) {
                 report_timeout(a.status, 19);
                 *abort_flag = 1;
@@ -573,6 +534,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 #pragma unroll
                 for (int h = 0; h < 8; ++h) o[h] = 0.f;
             }
+            tc_fence_before();
             if (has_virtual) {
 #pragma unroll
                 for (int g = 0; g < G; ++g) o[g] = fmaf(st_ev[g], vd, o[g]);
@@ -634,8 +596,52 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     }
                 }
             }
+
+            // ---- the update rule MV_t = MV_{t-1} + ww_t^T . wv_t on the rows it changes ----
+            if (a.do_write) {
+                cp_async_wait_all();
+                s_sync();  // every thread's staged chunks have landed
+                const int n_touched = *lo_count;
+                const int n_staged = min(n_touched, kLoCap);
+                const int c = tid & 15;  // 16-byte chunk of the 256-byte row
+                float vt[8];
+                Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(a.v + kv_off + c * 16), vt);
+                auto rewrite = [&](const uint4 hw, const uint4 lw, float ww, size_t goff) {
+                    float x[8], lo[8], nv[8], hf[8];
+                    Chunk<__nv_bfloat16>::unpack(hw, x);
+                    Chunk<__nv_bfloat16>::unpack(lw, lo);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) nv[e] = fmaf(ww, vt[e], x[e] + lo[e]);
+                    const uint4 hi_new = Chunk<__nv_bfloat16>::pack(nv);
+                    Chunk<__nv_bfloat16>::unpack(hi_new, hf);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) nv[e] -= hf[e];
+                    *reinterpret_cast<uint4*>(a.vhi + goff) = hi_new;
+                    *reinterpret_cast<uint4*>(a.vlo + goff) = Chunk<__nv_bfloat16>::pack(nv);
+                };
+                for (int sl = tid >> 4; sl < n_staged; sl += kSThreads / 16) {
+                    const size_t goff = unit_off + (size_t)(slice_start + list_row[sl]) * ROW_BYTES + c * 16;
+                    rewrite(*reinterpret_cast<const uint4*>(histage + sl * ROW_BYTES + c * 16),
+                            *reinterpret_cast<const uint4*>(lostage + sl * ROW_BYTES + c * 16), list_ww[sl], goff);
+                }
+                if (n_touched > kLoCap) {  // rows beyond the staging area: straight from global memory
+                    for (int row = tid >> 4; row < n_stream; row += kSThreads / 16) {
+                        if (idx[row] == -2) {
+                            const size_t goff = unit_off + (size_t)(slice_start + row) * ROW_BYTES + c * 16;
+                            rewrite(*reinterpret_cast<const uint4*>(a.vhi + goff),
+                                    *reinterpret_cast<const uint4*>(a.vlo + goff), wsm[row] * wfac, goff);
+                        }
+                    }
+                }
+            }
+            if (has_virtual && tid < 16) {  // store the appended slot
+                const size_t off = unit_off + (size_t)a.len * ROW_BYTES + tid * 16;
+                *reinterpret_cast<uint4*>(a.kplane + off) = *reinterpret_cast<const uint4*>(a.k + kv_off + tid * 16);
+                *reinterpret_cast<uint4*>(a.vhi + off) = *reinterpret_cast<const uint4*>(a.v + kv_off + tid * 16);
+                *reinterpret_cast<uint4*>(a.vlo + off) = make_uint4(0, 0, 0, 0);
+            }
+            s_sync();  // st_*, red, wsm, idx and the staging rows are reused by the next unit
             if (tid == 0) *lo_count = 0;
-            s_sync();  // st_*, red and the staging rows are reused by the next unit
         }
     }
 
@@ -735,6 +741,10 @@ int launch_decode_tc(const bct_cache* c, const StepIO& io, int len, int do_write
     int slice = (p.capacity + S - 1) / S;
     slice = (slice + kTileRows - 1) / kTileRows * kTileRows;  // whole tiles per CTA
     int stages = 4;
+    if (const char* e = getenv("BCT_TC_STAGES")) {  // tuning knob: depth of the tile ring (2..5)
+        const int v = atoi(e);
+        if (v >= 2 && v <= 5) stages = v;
+    }
     while (stages > 2 && tc_smem(stages, c->G, S).total > c->smem_optin) --stages;
     const int smem = tc_smem(stages, c->G, S).total;
 
