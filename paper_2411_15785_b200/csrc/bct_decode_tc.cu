@@ -42,7 +42,7 @@ constexpr int kScoreCols = 16;                 // tensor-memory columns per scor
 constexpr int kOCol = kMaxTiles * kScoreCols;  // output accumulator behind the score tiles
 constexpr int kTmemCols = 512;
 constexpr int kMaxClusterTc = 8;
-constexpr int kLoCap = 80;                     // rewritten rows staged per unit slice; further rows take a slow path
+constexpr int kLoCap = 80;                     // rewritten rows staged per round (more rows: more rounds)
 constexpr float kNegBigTc = -3.0e38f;
 
 struct TcArgs {
@@ -62,7 +62,7 @@ struct TcArgs {
 };
 
 struct TcSmem {
-    int ring, pbuf, qbuf, wsm, idx, lostage, list, red, stat, wstat, merge, bars, total;
+    int ring, pbuf, qbuf, wsm, list, lostage, red, stat, wstat, merge, bars, total;
 };
 __host__ __device__ inline TcSmem tc_smem(int stages, int G, int S) {
     TcSmem L;
@@ -75,12 +75,10 @@ __host__ __device__ inline TcSmem tc_smem(int stages, int G, int S) {
     off += 2 * kQBufBytes;
     L.wsm = off;
     off += kMaxTiles * kTileRows * 4;
-    L.idx = off;  // per slot: -1 untouched, >= 0 staging row, -2 rewritten but not staged
+    L.list = off;     // slots the update rule rewrites this token, in no particular order
     off += kMaxTiles * kTileRows * 2;
-    L.lostage = off;  // staged rows of the slots to rewrite: value plane rows, then residual rows
+    L.lostage = off;  // staged copies of up to kLoCap of those rows: value plane rows, then residual rows
     off += 2 * kLoCap * 256;
-    L.list = off;     // per staged row: slot index and write weight
-    off += kLoCap * 8;
     L.red = off;
     off += 4 * 16 * 4;
     L.stat = off;  // m[8], l[8], wd[8], ev[8], abort, tmem address
@@ -174,11 +172,9 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     unsigned char* pbuf = smem + L.pbuf;
     unsigned char* qbuf = smem + L.qbuf;
     float* wsm = reinterpret_cast<float*>(smem + L.wsm);
-    short* idx = reinterpret_cast<short*>(smem + L.idx);
+    unsigned short* list = reinterpret_cast<unsigned short*>(smem + L.list);
     unsigned char* histage = smem + L.lostage;
     unsigned char* lostage = histage + kLoCap * ROW_BYTES;
-    int* list_row = reinterpret_cast<int*>(smem + L.list);
-    float* list_ww = reinterpret_cast<float*>(smem + L.list) + kLoCap;
     float* red = reinterpret_cast<float*>(smem + L.red);
     float* st_m = reinterpret_cast<float*>(smem + L.stat);
     float* st_l = st_m + 8;
@@ -492,33 +488,27 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 }
             }
 
-            // ---- stage copies of the rows the rule will rewrite (value and residual rows) with 16-byte
-            // ---- asynchronous copies, so that no global-memory latency is left for the update itself ----
+            // ---- list the slots the rule rewrites and stage copies of their value and residual rows with
+            // ---- 16-byte asynchronous copies, so that no global-memory latency is left for the update ----
+            const int c16 = tid & 15;  // 16-byte chunk of a 256-byte row
+            auto stage_rows = [&](int base, int n) {
+                for (int i = tid >> 4; i < n; i += kSThreads / 16) {
+                    const size_t goff = unit_off + (size_t)(slice_start + list[base + i]) * ROW_BYTES + c16 * 16;
+                    cp_async16(histage + i * ROW_BYTES + c16 * 16, a.vhi + goff);
+                    cp_async16(lostage + i * ROW_BYTES + c16 * 16, a.vlo + goff);
+                }
+                cp_async_commit();
+            };
+            int n_touched = 0;
             if (a.do_write) {
                 for (int t = 0; t < nt; ++t) {
                     const int row = t * kTileRows + r;
-                    short slot = -1;
-                    const float ww = wsm[row] * wfac;
-                    if (row < n_stream && (a.dense || ww >= a.write_eps)) {
-                        const int sl = atomicAdd(lo_count, 1);
-                        slot = -2;
-                        if (sl < kLoCap) {
-                            slot = (short)sl;
-                            list_row[sl] = row;
-                            list_ww[sl] = ww;
-                        }
-                    }
-                    idx[row] = slot;
+                    if (row < n_stream && (a.dense || wsm[row] * wfac >= a.write_eps))
+                        list[atomicAdd(lo_count, 1)] = (unsigned short)row;
                 }
                 s_sync();
-                const int n_staged = min(*lo_count, kLoCap);
-                const int c = tid & 15;
-                for (int sl = tid >> 4; sl < n_staged; sl += kSThreads / 16) {
-                    const size_t goff = unit_off + (size_t)(slice_start + list_row[sl]) * ROW_BYTES + c * 16;
-                    cp_async16(histage + sl * ROW_BYTES + c * 16, a.vhi + goff);
-                    cp_async16(lostage + sl * ROW_BYTES + c * 16, a.vlo + goff);
-                }
-                cp_async_commit();
+                n_touched = *lo_count;
+                stage_rows(0, min(n_touched, kLoCap));
             }
 
             // ---- epilogue: O[d][g] from tensor memory once every V tile has been read ----
@@ -599,38 +589,31 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 
             // ---- the update rule MV_t = MV_{t-1} + ww_t^T . wv_t on the rows it changes ----
             if (a.do_write) {
-                cp_async_wait_all();
-                s_sync();  // every thread's staged chunks have landed
-                const int n_touched = *lo_count;
-                const int n_staged = min(n_touched, kLoCap);
-                const int c = tid & 15;  // 16-byte chunk of the 256-byte row
                 float vt[8];
-                Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(a.v + kv_off + c * 16), vt);
-                auto rewrite = [&](const uint4 hw, const uint4 lw, float ww, size_t goff) {
-                    float x[8], lo[8], nv[8], hf[8];
-                    Chunk<__nv_bfloat16>::unpack(hw, x);
-                    Chunk<__nv_bfloat16>::unpack(lw, lo);
+                Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(a.v + kv_off + c16 * 16), vt);
+                for (int base = 0; base < n_touched; base += kLoCap) {
+                    const int n = min(n_touched - base, kLoCap);
+                    if (base > 0) {
+                        s_sync();  // the previous round's staged rows have been consumed
+                        stage_rows(base, n);
+                    }
+                    cp_async_wait_all();
+                    s_sync();  // every thread's staged chunks have landed
+                    for (int i = tid >> 4; i < n; i += kSThreads / 16) {
+                        const int row = list[base + i];
+                        const float ww = wsm[row] * wfac;
+                        const size_t goff = unit_off + (size_t)(slice_start + row) * ROW_BYTES + c16 * 16;
+                        float x[8], lo[8], nv[8], hf[8];
+                        Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(histage + i * ROW_BYTES + c16 * 16), x);
+                        Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(lostage + i * ROW_BYTES + c16 * 16), lo);
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) nv[e] = fmaf(ww, vt[e], x[e] + lo[e]);
-                    const uint4 hi_new = Chunk<__nv_bfloat16>::pack(nv);
-                    Chunk<__nv_bfloat16>::unpack(hi_new, hf);
+                        for (int e = 0; e < 8; ++e) nv[e] = fmaf(ww, vt[e], x[e] + lo[e]);
+                        const uint4 hi_new = Chunk<__nv_bfloat16>::pack(nv);
+                        Chunk<__nv_bfloat16>::unpack(hi_new, hf);
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) nv[e] -= hf[e];
-                    *reinterpret_cast<uint4*>(a.vhi + goff) = hi_new;
-                    *reinterpret_cast<uint4*>(a.vlo + goff) = Chunk<__nv_bfloat16>::pack(nv);
-                };
-                for (int sl = tid >> 4; sl < n_staged; sl += kSThreads / 16) {
-                    const size_t goff = unit_off + (size_t)(slice_start + list_row[sl]) * ROW_BYTES + c * 16;
-                    rewrite(*reinterpret_cast<const uint4*>(histage + sl * ROW_BYTES + c * 16),
-                            *reinterpret_cast<const uint4*>(lostage + sl * ROW_BYTES + c * 16), list_ww[sl], goff);
-                }
-                if (n_touched > kLoCap) {  // rows beyond the staging area: straight from global memory
-                    for (int row = tid >> 4; row < n_stream; row += kSThreads / 16) {
-                        if (idx[row] == -2) {
-                            const size_t goff = unit_off + (size_t)(slice_start + row) * ROW_BYTES + c * 16;
-                            rewrite(*reinterpret_cast<const uint4*>(a.vhi + goff),
-                                    *reinterpret_cast<const uint4*>(a.vlo + goff), wsm[row] * wfac, goff);
-                        }
+                        for (int e = 0; e < 8; ++e) nv[e] -= hf[e];
+                        *reinterpret_cast<uint4*>(a.vhi + goff) = hi_new;
+                        *reinterpret_cast<uint4*>(a.vlo + goff) = Chunk<__nv_bfloat16>::pack(nv);
                     }
                 }
             }
@@ -640,7 +623,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 *reinterpret_cast<uint4*>(a.vhi + off) = *reinterpret_cast<const uint4*>(a.v + kv_off + tid * 16);
                 *reinterpret_cast<uint4*>(a.vlo + off) = make_uint4(0, 0, 0, 0);
             }
-            s_sync();  // st_*, red, wsm, idx and the staging rows are reused by the next unit
+            s_sync();  // st_*, red, wsm, the list and the staging rows are reused by the next unit
             if (tid == 0) *lo_count = 0;
         }
     }
