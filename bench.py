@@ -100,7 +100,18 @@ def algorithmic_bytes_per_step(w: W.Workload) -> int:
     return w.units * per_unit
 
 
-def cpu_oracle_sample(w: W.Workload, budget_s: float = 15.0):
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the committed ncu capture of
+# decode_tc_kernel (profiles/decode_tc_kernel_ncu_full.txt), taken at batch 37 and scaled by units:
+# 1.0949 MB per (sequence, kv-head) unit of the mha7b shape.  None for any other kernel / shape.
+TRAFFIC_PER_UNIT = {("mha7b", True): 1.2964e9 / 1184}
+
+
+def measured_traffic(w, tensor_path):
+    per_unit = TRAFFIC_PER_UNIT.get((w.name.split("_")[0], bool(tensor_path)))
+    return None if per_unit is None else per_unit * w.units
+
+
+def cpu_oracle_sample(w: W.Workload, budget_s: float = 25.0):
     """Time the CPU oracle, as it stands, on a bounded sample of the workload: a few
     (sequence, kv-head) units per core, for as many tokens as fit the time budget."""
     from oracle import bct_oracle as O
@@ -308,7 +319,8 @@ def main():
                     "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.steps},
             "gpu_launches": launches,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": None, "peak_kind": "of " + peak_kind, "kernel": "decode_kernel",
+                         "traffic": measured_traffic(w, cache.tensor_path), "peak_kind": "of " + peak_kind,
+                         "kernel": "decode_tc_kernel" if cache.tensor_path else "decode_kernel",
                          "algorithmic_bytes_per_launch": alg, "frac_of_8TBps_nominal": achieved / 8000.0},
         }
         if world == 1 and not args.no_cpu_baseline:
