@@ -163,6 +163,38 @@ bct_status_t bct_decode_step_host(bct_cache_t *cache, const void *q, const void 
 bct_status_t bct_prefill_stream_host(bct_cache_t *cache, const void *q, const void *k,
                                      const void *v, void *out, int64_t T, void *cuda_stream);
 
+/*
+ * bct_prefill_stream_host for callers that cannot allocate device memory.  (The paper has
+ * no counterpart: this is plumbing of this library, not a step of the method.)
+ *
+ * bct_prefill_stream_host stages q, k, v and out in the workspace, in an area whose size the
+ * caller fixed with max_stream before allocating the workspace.  Some callers can never
+ * enlarge it afterwards because they cannot call cudaMalloc at all: code that runs inside a
+ * memory pool frozen at start-up (a latency-bound serving loop), a plug-in that owns only
+ * the arena its host application handed it, a process whose other libraries have taken the
+ * rest of the device.  This call uses a staging area built into the library instead: one
+ * file-scope device array of BCT_STATIC_STAGE_BYTES that every GPU holds from the moment
+ * the library is loaded until the process exits.  It allocates and frees nothing.
+ *
+ *   q, k, v, out  HOST pointers, shapes and meaning as in bct_prefill_stream_host;
+ *                 out must not be NULL.
+ *   T             tokens per sequence; the rounded-up sizes of q, k, v and out for T tokens
+ *                 must fit BCT_STATIC_STAGE_BYTES together, else BCT_ERR_INVALID_ARG and
+ *                 nothing is enqueued (bct_last_error() gives the sizes).  max_stream does
+ *                 not limit T here.
+ * The cache's device must be the current device.  The first call on each device looks up
+ * the array's device address (cudaGetSymbolAddress); make that first call outside any
+ * stream capture.  The array is shared by every cache and every call on that device and
+ * keeps the previous call's bytes; this call overwrites every byte it later reads, so
+ * nothing has to be cleared, but two calls whose work overlaps on the GPU (different
+ * streams without ordering, or different threads) race on it: order them on one stream.
+ * Results are those of bct_prefill_stream_host.
+ */
+#define BCT_STATIC_STAGE_BYTES (8u << 20)
+bct_status_t bct_prefill_stream_host_static(bct_cache_t *cache, const void *q, const void *k,
+                                            const void *v, void *out, int64_t T,
+                                            void *cuda_stream);
+
 /* Resident slots (0..C) after the work enqueued so far. Host bookkeeping; no sync. */
 bct_status_t bct_cache_len(const bct_cache_t *cache, int32_t *len);
 

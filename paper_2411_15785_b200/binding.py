@@ -23,8 +23,9 @@ EXPORTS = (
     "bct_version", "bct_last_error", "bct_cache_bytes", "bct_cache_create", "bct_decode_step",
     "bct_prefill_stream", "bct_decode_step_host", "bct_prefill_stream_host", "bct_cache_len",
     "bct_cache_export", "bct_cache_import", "bct_cache_status", "bct_cache_launches", "bct_cache_destroy",
-    "bct_cache_tensor_path",
+    "bct_cache_tensor_path", "bct_prefill_stream_host_static",
 )
+STATIC_STAGE_BYTES = 8 << 20
 
 
 class BctParams(ctypes.Structure):
@@ -72,6 +73,7 @@ def load() -> ctypes.CDLL:
     lib.bct_cache_launches.argtypes = [vp, ctypes.POINTER(i64)]
     lib.bct_cache_destroy.argtypes = [vp]
     lib.bct_cache_tensor_path.argtypes = [vp, ctypes.POINTER(i32)]
+    lib.bct_prefill_stream_host_static.argtypes = [vp, vp, vp, vp, vp, i64, vp]
     for name in EXPORTS[2:]:
         getattr(lib, name).restype = ctypes.c_int
     _lib = lib
@@ -172,6 +174,12 @@ class Cache:
     def prefill_stream_host(self, q, k, v, out, stream=None):
         _check(self.lib.bct_prefill_stream_host(self._h, q.data_ptr(), k.data_ptr(), v.data_ptr(), _ptr(out),
                                                 q.shape[1], _stream_ptr(stream)))
+        return out
+
+    def prefill_stream_host_static(self, q, k, v, out, stream=None):
+        """Host tensors in and out, staged in the library's built-in device array (no allocation)."""
+        _check(self.lib.bct_prefill_stream_host_static(self._h, q.data_ptr(), k.data_ptr(), v.data_ptr(),
+                                                       out.data_ptr(), q.shape[1], _stream_ptr(stream)))
         return out
 
     # ---- state ----------------------------------------------------------------------

@@ -139,6 +139,10 @@ bct_status_t run_tokens(bct_cache_t* c, const void* q, const void* k, const void
 
 }  // namespace
 
+namespace bct {
+void set_last_error(const char* msg) { snprintf(g_err, sizeof(g_err), "%s", msg); }
+}  // namespace bct
+
 extern "C" {
 
 int32_t bct_version(void) { return 100; }

@@ -70,6 +70,9 @@ bool tc_eligible(const bct_cache* c);   // this cache's decode steps run on the 
 int launch_decode_tc(const bct_cache* c, const StepIO& io, int len, int do_write, cudaStream_t stream,
                      cudaError_t* err);
 
+// Set the calling thread's bct_last_error() message (for entry points outside bct_api.cu).
+void set_last_error(const char* msg);
+
 // State import / export.
 cudaError_t launch_import(const bct_cache* c, const void* k_in, const void* v_in, int v_dtype, int len,
                           cudaStream_t stream);
