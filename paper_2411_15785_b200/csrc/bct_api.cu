@@ -114,7 +114,22 @@ bct_status_t run_tokens(bct_cache_t* c, const void* q, const void* k, const void
     const size_t eb = (size_t)c->elem_bytes;
     const size_t q_tok = (size_t)p.n_q_heads * p.head_dim;   // elements per token per sequence
     const size_t kv_tok = (size_t)p.n_kv_heads * p.head_dim;
-    for (int64_t t = 0; t < T; ++t) {
+    const int Tc = bct::stream_chunk_tokens(c);
+    int64_t t = 0;
+    while (t < T) {
+        const bool full = (c->len == p.capacity);
+        const int do_write = !((p.flags & BCT_FLAG_SKIP_FIRST_WRITE) && c->n_full_tokens == 0);
+        // whole chunks against a full cache go through the chunked tensor-core kernel
+        if (Tc > 0 && full && do_write && T - t >= Tc) {
+            const int64_t n_chunks = (T - t) / Tc;
+            cudaError_t e = cudaSuccess;
+            const int n = bct::launch_stream_tc(c, q, k, v, out, T, t, n_chunks, stream, &e);
+            if (n < 0) return fail_cuda("stream launch", e);
+            c->launches += n;
+            c->n_full_tokens += n_chunks * Tc;
+            t += n_chunks * Tc;
+            continue;
+        }
         bct::StepIO io;
         io.q = static_cast<const char*>(q) + (size_t)t * q_tok * eb;
         io.k = static_cast<const char*>(k) + (size_t)t * kv_tok * eb;
@@ -123,8 +138,6 @@ bct_status_t run_tokens(bct_cache_t* c, const void* q, const void* k, const void
         io.out = out ? static_cast<char*>(out) + (size_t)t * q_tok * ob : nullptr;
         io.q_batch_stride = (int64_t)(T * q_tok);
         io.kv_batch_stride = (int64_t)(T * kv_tok);
-        const bool full = (c->len == p.capacity);
-        const int do_write = !((p.flags & BCT_FLAG_SKIP_FIRST_WRITE) && c->n_full_tokens == 0);
         cudaError_t e = cudaSuccess;
         const int n = bct::launch_decode(c, io, c->len, do_write, stream, &e);
         if (n < 0) return fail_cuda("decode launch", e);
@@ -133,6 +146,7 @@ bct_status_t run_tokens(bct_cache_t* c, const void* q, const void* k, const void
             c->n_full_tokens += 1;
         else
             c->len += 1;
+        ++t;
     }
     return BCT_OK;
 }

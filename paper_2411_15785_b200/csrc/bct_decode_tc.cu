@@ -642,6 +642,7 @@ bool tc_prepare(bct_cache* c) {
     if (c->p.dtype != BCT_BF16 || c->p.head_dim != 128) return false;
     if (!make_plane_map(reinterpret_cast<CUtensorMap*>(c->tmap_k), c->kplane, c->U, c->p.capacity)) return false;
     if (!make_plane_map(reinterpret_cast<CUtensorMap*>(c->tmap_v), c->vhi, c->U, c->p.capacity)) return false;
+    if (!make_plane_map(reinterpret_cast<CUtensorMap*>(c->tmap_lo), c->vlo, c->U, c->p.capacity)) return false;
     c->tc_ready = 1;
     return true;
 }

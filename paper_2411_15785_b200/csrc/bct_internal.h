@@ -50,6 +50,7 @@ struct bct_cache {
     int tc_ready;    // tensor maps below are valid (bfloat16, head_dim 128)
     alignas(64) unsigned char tmap_k[128];  // CUtensorMap of the MK plane
     alignas(64) unsigned char tmap_v[128];  // CUtensorMap of the MV value plane
+    alignas(64) unsigned char tmap_lo[128]; // CUtensorMap of the MV residual plane
 };
 
 namespace bct {
@@ -69,6 +70,13 @@ bool tc_prepare(bct_cache* c);          // encode the planes' tensor maps; false
 bool tc_eligible(const bct_cache* c);   // this cache's decode steps run on the tensor path
 int launch_decode_tc(const bct_cache* c, const StepIO& io, int len, int do_write, cudaStream_t stream,
                      cudaError_t* err);
+
+// Chunked tensor-core stream kernel (full cache, bfloat16, head_dim 128, G <= 7, C <= 2048):
+// tokens per chunk for this cache, or 0 when the kernel does not apply.
+int stream_chunk_tokens(const bct_cache* c);
+// n_chunks whole chunks starting at token t_begin of the [B][T][H][d] step arrays.
+int launch_stream_tc(const bct_cache* c, const void* q, const void* k, const void* v, void* out, int64_t T,
+                     int64_t t_begin, int64_t n_chunks, cudaStream_t stream, cudaError_t* err);
 
 // Set the calling thread's bct_last_error() message (for entry points outside bct_api.cu).
 void set_last_error(const char* msg);

@@ -1,0 +1,591 @@
+// Chunked stream / prefill kernel of the bounded-cache attention layer on the sm_100a tensor path.
+//
+// Algorithm 1 never assigns MK, so the write weights ww_t = softmax(wq_t . MK^T) of all tokens of
+// a chunk are independent of one another ("Optimized for Parallelism": token-level parallel
+// accumulation).  For a chunk of Tc tokens against a full cache this turns Tc decode steps into
+// dense contractions over the resident tiles:
+//     Sr = Q MK^T, Sw = Kc MK^T            scores of the chunk's read and write queries
+//     Pr = softmax rows of Sr, WW = softmax rows of Sw
+//     A  = Pr WW^T                          what token t's read sees of token s's write
+//     O  = Pr MV + strict_tril(A) Vc        outputs: every token reads MV_{t-1}
+//     MV += WW^T Vc                         Method step 4 for the Tc tokens at once
+// One persistent CTA per (sequence, kv-head) unit at a time (C <= 2048 slots); per chunk the cache
+// streams through shared memory twice for MK (row statistics, then numerators) and once for MV
+// (value and residual planes), instead of twice per token, and every product runs as tcgen05.mma
+// with fp32 accumulators in tensor memory.  Numerators and write weights are kept as bfloat16
+// value + residual pairs, and MV is read as value + residual, so a long stream keeps the precision
+// of the per-token path.
+//   warp 4  producer : TMA loads (chunk operands, MK / MV tiles through a 3-stage ring)
+//   warp 5  MMA      : issues all tensor-core work, commits to mbarriers
+//   warps 0-3        : one thread per operand row: online row statistics, numerators, the write-back
+//                      of MV rows, the intra-chunk term and the epilogue
+// Every wait is bounded; a timeout sets the status word and the kernel runs to its end.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "bct_internal.h"
+#include "bct_tc.cuh"
+
+namespace bct {
+namespace {
+
+constexpr int kStThreads = 192;
+constexpr int kStS = 128;                // softmax threads = operand rows
+constexpr int kStTile = 128;             // slots per tile
+constexpr int kStHalf = 128 * 128;       // 64 columns (128 bytes) x 128 rows
+constexpr int kStTileBytes = 2 * kStHalf;
+constexpr int kStStages = 3;
+constexpr int kStMaxTc = 64;
+constexpr float kStNegBig = -3.0e38f;
+// tensor-memory columns
+constexpr int kColS0 = 0;     // score tile (pass 2, and buffer 0 of pass 1)
+constexpr int kColO = 128;    // outputs  [row (t,g)] x [d]
+constexpr int kColD = 256;    // MV increment of one tile [slot] x [d]; buffer 1 of the scores in pass 1
+constexpr int kColA = 384;    // A = Pr WW^T  [row (t,g)] x [write token]
+
+struct StArgs {
+    char* vhi;
+    char* vlo;
+    char* out;
+    int* status;
+    int C, Hq, Hkv, U, T, t_begin, n_chunks, Tc;
+    int wtr, out_f32;
+    float read_scale, write_scale;
+};
+
+struct StSmem {
+    int qall, vc, phi, plo, ring, bars, misc, total;
+};
+__host__ __device__ inline StSmem st_smem() {
+    StSmem L;
+    int off = 0;
+    L.qall = off;
+    off += kStTileBytes;        // [2 halves][128 rows][128 B]: G*Tc read queries, Tc write queries, zero rows
+    L.vc = off;
+    off += kStMaxTc * 256;      // [2 halves][Tc rows][128 B]: the chunk's write key-value vectors
+    L.phi = off;
+    off += kStTileBytes;        // numerators / write weights of one tile, bfloat16 value
+    L.plo = off;
+    off += kStTileBytes;        // ... and residual; reused for the masked A operand after the last tile
+    L.ring = off;
+    off += kStStages * kStTileBytes;
+    L.bars = off;
+    off += 32 * 8;
+    L.misc = off;
+    off += 64;
+    L.total = off + 1024;       // slack to align the base to 1024 bytes
+    return L;
+}
+
+__device__ __forceinline__ void st_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kStS) : "memory"); }
+
+// value / residual split of 8 floats into two 16-byte chunks of bfloat16
+__device__ __forceinline__ void split8(const float* e, uint4* hi, uint4* lo) {
+    *hi = Chunk<__nv_bfloat16>::pack(e);
+    float h[8], r[8];
+    Chunk<__nv_bfloat16>::unpack(*hi, h);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) r[i] = e[i] - h[i];
+    *lo = Chunk<__nv_bfloat16>::pack(r);
+}
+
+template <int G>
+__global__ void __launch_bounds__(kStThreads, 1)
+stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmVhi,
+                 const __grid_constant__ CUtensorMap tmVlo, const __grid_constant__ CUtensorMap tmQ,
+                 const __grid_constant__ CUtensorMap tmKin, const __grid_constant__ CUtensorMap tmVin,
+                 const StArgs a) {
+    extern __shared__ unsigned char st_smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(st_smem_raw) + 1023) & ~uintptr_t(1023));
+    const StSmem L = st_smem();
+    unsigned char* qall = smem + L.qall;
+    unsigned char* vc = smem + L.vc;
+    unsigned char* phi = smem + L.phi;
+    unsigned char* plo = smem + L.plo;
+    unsigned char* ring = smem + L.ring;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L.bars);
+    uint64_t* full = bars;            // [3] tile landed (TMA transaction bytes)
+    uint64_t* empty = bars + 3;       // [3] stage may be refilled (one arrival: MMA commit or softmax thread 0)
+    uint64_t* qfull = bars + 6;       // chunk operands landed
+    uint64_t* qfree = bars + 7;       // chunk operands no longer needed (128 arrivals)
+    uint64_t* sready = bars + 8;      // [2] score tile complete (commit)
+    uint64_t* sfree = bars + 10;      // [2] score tile consumed (128 arrivals)
+    uint64_t* pready = bars + 12;     // numerators of the tile written (128 arrivals)
+    uint64_t* pfree = bars + 13;      // MMAs that read them complete (commit)
+    uint64_t* dready = bars + 14;     // the tile's MV increment (and all earlier MMAs) complete (commit)
+    uint64_t* dfree = bars + 15;      // increment consumed (128 arrivals)
+    uint64_t* aready = bars + 16;     // masked A operand written (128 arrivals)
+    uint64_t* oready = bars + 17;     // outputs complete (commit)
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L.misc);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L.misc + 8);
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5;
+    const int lane = tid & 31;
+    const int Tc = a.Tc;
+    const int nt = (a.C + kStTile - 1) / kStTile;
+    const int n_read = Tc * G;         // rows [0, n_read): read queries (t, g); then Tc write rows
+    const int vc_half = Tc * 128;      // bytes between the two 64-column halves of Vc
+
+    if (tid == 0) {
+        for (int i = 0; i < 3; ++i) {
+            mbar_init(&full[i], 1);
+            mbar_init(&empty[i], 1);
+        }
+        mbar_init(qfull, 1);
+        mbar_init(qfree, kStS);
+        mbar_init(&sready[0], 1);
+        mbar_init(&sready[1], 1);
+        mbar_init(&sfree[0], kStS);
+        mbar_init(&sfree[1], kStS);
+        mbar_init(pready, kStS);
+        mbar_init(pfree, 1);
+        mbar_init(dready, 1);
+        mbar_init(dfree, kStS);
+        mbar_init(aready, kStS);
+        mbar_init(oready, 1);
+        *abort_flag = 0;
+        fence_mbar_init_cluster();
+    }
+    // rows of the query operand beyond the chunk's G*Tc + Tc stay zero for good
+    for (int i = tid; i < kStTileBytes / 16; i += kStThreads) reinterpret_cast<uint4*>(qall)[i] = make_uint4(0, 0, 0, 0);
+    if (warp == 5) tmem_alloc(tmem_slot, 512);
+    fence_proxy_async_smem();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+#define ST_WAIT(bar, parity, site)                                              \
+    if (!mbar_wait(bar, (parity) & 1, *abort_flag ? 1024u : kWaitLimit)) {      \
+        report_timeout(a.status, site);                                         \
+        *abort_flag = 1;                                                        \
+    }
+
+    if (warp == 4) {
+        // =========================== producer ===========================
+        if (lane == 0) {
+            uint32_t kc = 0, qn = 0;
+            auto load_tile = [&](const CUtensorMap* map, int u, int t) {
+                const int stage = kc % kStStages;
+                if (kc >= (uint32_t)kStStages) ST_WAIT(&empty[stage], (kc / kStStages) - 1, 31);
+                unsigned char* dst = ring + (size_t)stage * kStTileBytes;
+                mbar_arrive_expect_tx(&full[stage], kStTileBytes);
+                tma_load_3d(dst, map, 0, t * kStTile, u, &full[stage]);
+                tma_load_3d(dst + kStHalf, map, 64, t * kStTile, u, &full[stage]);
+                ++kc;
+            };
+            for (int u = blockIdx.x; u < a.U; u += gridDim.x) {
+                const int b = u / a.Hkv, h = u - b * a.Hkv;
+                for (int ch = 0; ch < a.n_chunks; ++ch, ++qn) {
+                    const int t0 = a.t_begin + ch * Tc;
+                    if (qn > 0) ST_WAIT(qfree, qn - 1, 32);
+                    mbar_arrive_expect_tx(qfull, (uint32_t)(Tc * (G + 2) * 256));
+                    tma_load_4d(qall, &tmQ, 0, h * G, t0, b, qfull);
+                    tma_load_4d(qall + kStHalf, &tmQ, 64, h * G, t0, b, qfull);
+                    tma_load_4d(qall + n_read * 128, &tmKin, 0, h, t0, b, qfull);
+                    tma_load_4d(qall + kStHalf + n_read * 128, &tmKin, 64, h, t0, b, qfull);
+                    tma_load_4d(vc, &tmVin, 0, h, t0, b, qfull);
+                    tma_load_4d(vc + vc_half, &tmVin, 64, h, t0, b, qfull);
+                    for (int t = 0; t < nt; ++t) load_tile(&tmK, u, t);  // pass 1: row statistics
+                    for (int t = 0; t < nt; ++t) {                       // pass 2: numerators, outputs, update
+                        load_tile(&tmK, u, t);
+                        load_tile(&tmVhi, u, t);
+                        load_tile(&tmVlo, u, t);
+                    }
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 5) {
+        // =========================== MMA issuer ===========================
+        if (lane == 0) {
+            constexpr uint32_t id_scores = instr_desc_mn(128, 128, false, false);  // Qall (K) x tile (K)
+            constexpr uint32_t id_out = instr_desc_mn(128, 128, false, true);      // P (K) x V tile (MN)
+            constexpr uint32_t id_delta = instr_desc_mn(128, 128, true, true);     // WW^T (MN) x Vc (MN)
+            const uint32_t id_a = instr_desc_mn(128, (uint32_t)(Tc < 16 ? 16 : Tc), false, false);  // P (K) x WW (K)
+            uint32_t kc = 0, qn = 0, su0 = 0, su1 = 0, np = 0, nd = 0;
+            const uint32_t qaddr = smem_u32(qall), vcaddr = smem_u32(vc), phiaddr = smem_u32(phi), ploaddr = smem_u32(plo);
+            auto scores = [&](uint32_t col, uint32_t taddr) {
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    const uint32_t o = (kk >> 2) * kStHalf + (kk & 3) * 32;
+                    umma_bf16(tmem_base + col, smem_desc(qaddr + o, 16, 1024), smem_desc(taddr + o, 16, 1024), id_scores,
+                              kk > 0);
+                }
+            };
+            for (int u = blockIdx.x; u < a.U; u += gridDim.x) {
+                for (int ch = 0; ch < a.n_chunks; ++ch, ++qn) {
+                    ST_WAIT(qfull, qn, 41);
+                    tc_fence_after();
+                    for (int t = 0; t < nt; ++t, ++kc) {  // pass 1
+                        const int stage = kc % kStStages;
+                        const int buf = t & 1;
+                        ST_WAIT(&full[stage], kc / kStStages, 42);
+                        uint32_t& su = buf ? su1 : su0;
+                        if (su > 0) ST_WAIT(&sfree[buf], su - 1, 43);
+                        tc_fence_after();
+                        scores(buf ? kColD : kColS0, smem_u32(ring + (size_t)stage * kStTileBytes));
+                        umma_commit(&sready[buf]);
+                        umma_commit(&empty[stage]);
+                        ++su;
+                    }
+                    for (int t = 0; t < nt; ++t) {  // pass 2
+                        const int ks = kc % kStStages;
+                        ST_WAIT(&full[ks], kc / kStStages, 44);
+                        if (su0 > 0) ST_WAIT(&sfree[0], su0 - 1, 45);
+                        tc_fence_after();
+                        scores(kColS0, smem_u32(ring + (size_t)ks * kStTileBytes));
+                        umma_commit(&sready[0]);
+                        umma_commit(&empty[ks]);
+                        ++su0;
+                        ++kc;
+                        const int vh = kc % kStStages;
+                        const uint32_t vh_par = kc / kStStages;
+                        ++kc;
+                        const int vl = kc % kStStages;
+                        const uint32_t vl_par = kc / kStStages;
+                        ++kc;
+                        ST_WAIT(pready, np, 46);
+                        ++np;
+                        ST_WAIT(&full[vh], vh_par, 47);
+                        ST_WAIT(&full[vl], vl_par, 48);
+                        if (nd > 0) ST_WAIT(dfree, nd - 1, 49);
+                        tc_fence_after();
+                        const uint32_t vhaddr = smem_u32(ring + (size_t)vh * kStTileBytes);
+                        const uint32_t vladdr = smem_u32(ring + (size_t)vl * kStTileBytes);
+                        // outputs: (P + P_residual) x MV_value + P x MV_residual, accumulated over the tiles
+#pragma unroll
+                        for (int kk = 0; kk < 8; ++kk) {
+                            const uint32_t po = (kk >> 2) * kStHalf + (kk & 3) * 32;
+                            const uint64_t vhd = smem_desc(vhaddr + kk * 2048, kStHalf, 1024);
+                            umma_bf16(tmem_base + kColO, smem_desc(phiaddr + po, 16, 1024), vhd, id_out, (t > 0) || (kk > 0));
+                            umma_bf16(tmem_base + kColO, smem_desc(ploaddr + po, 16, 1024), vhd, id_out, true);
+                            umma_bf16(tmem_base + kColO, smem_desc(phiaddr + po, 16, 1024),
+                                      smem_desc(vladdr + kk * 2048, kStHalf, 1024), id_out, true);
+                        }
+                        // A += P x WW^T over this tile's slots (write rows start at n_read)
+#pragma unroll
+                        for (int kk = 0; kk < 8; ++kk) {
+                            const uint32_t po = (kk >> 2) * kStHalf + (kk & 3) * 32;
+                            umma_bf16(tmem_base + kColA, smem_desc(phiaddr + po, 16, 1024),
+                                      smem_desc(phiaddr + n_read * 128 + po, 16, 1024), id_a, (t > 0) || (kk > 0));
+                        }
+                        // increment of this tile's MV rows: (WW + WW_residual)^T x Vc, 16 tokens per step
+                        for (int kk = 0; kk < Tc / 16; ++kk) {
+                            const uint64_t vd = smem_desc(vcaddr + kk * 2048, (uint32_t)vc_half, 1024);
+                            umma_bf16(tmem_base + kColD, smem_desc(phiaddr + n_read * 128 + kk * 2048, kStHalf, 1024), vd,
+                                      id_delta, kk > 0);
+                            umma_bf16(tmem_base + kColD, smem_desc(ploaddr + n_read * 128 + kk * 2048, kStHalf, 1024), vd,
+                                      id_delta, true);
+                        }
+                        umma_commit(dready);
+                        umma_commit(pfree);
+                        ++nd;
+                    }
+                    // intra-chunk term: O += strict_tril(A) x Vc
+                    ST_WAIT(aready, qn, 50);
+                    tc_fence_after();
+                    for (int kk = 0; kk < Tc / 16; ++kk)
+                        umma_bf16(tmem_base + kColO, smem_desc(ploaddr + kk * 32, 16, 1024),
+                                  smem_desc(vcaddr + kk * 2048, (uint32_t)vc_half, 1024), id_out, true);
+                    umma_commit(oready);
+                }
+            }
+        }
+        __syncwarp();
+    } else {
+        // =========================== row threads: statistics, numerators, write-back, epilogue ===========================
+        const int r = tid;                              // operand row = tensor-memory lane
+        const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
+        const bool is_read = r < n_read;
+        const bool is_write = !is_read && r < n_read + Tc;
+        const int my_t = is_read ? r / G : (is_write ? r - n_read : 0);  // token of the chunk this row belongs to
+        const int my_g = is_read ? r - my_t * G : 0;
+        const float scale = is_read ? a.read_scale : a.write_scale;
+        const int sw = r & 7;                           // swizzle phase of this row
+        uint32_t kc = 0, qn = 0, su0 = 0, su1 = 0, np = 0, nd = 0;
+        for (int u = blockIdx.x; u < a.U; u += gridDim.x) {
+            const int b = u / a.Hkv, h = u - b * a.Hkv;
+            for (int ch = 0; ch < a.n_chunks; ++ch, ++qn) {
+                const int t0 = a.t_begin + ch * Tc;
+                // ---- pass 1: online maximum and sum of this row's scaled scores over all C slots ----
+                float m = kStNegBig, l = 0.f;
+                for (int t = 0; t < nt; ++t, ++kc) {
+                    const int buf = t & 1;
+                    uint32_t& su = buf ? su1 : su0;
+                    ST_WAIT(&sready[buf], su, 61);
+                    ++su;
+                    tc_fence_after();
+                    const int n_valid = min(kStTile, a.C - t * kStTile);
+#pragma unroll 1
+                    for (int bch = 0; bch < 4; ++bch) {
+                        float x[32];
+                        tmem_ld32(lane_base + (buf ? kColD : kColS0) + bch * 32, x);
+                        float bm = kStNegBig;
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            x[i] = (bch * 32 + i < n_valid) ? x[i] * scale : kStNegBig;
+                            bm = fmaxf(bm, x[i]);
+                        }
+                        const float mn = fmaxf(m, bm);
+                        float s = 0.f;
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) s += __expf(x[i] - mn);
+                        l = l * __expf(m - mn) + s;
+                        m = mn;
+                    }
+                    tc_fence_before();
+                    mbar_arrive(&sfree[buf]);
+                }
+                const float inv_l = 1.f / l;
+                const float wmul = is_write ? inv_l : 1.f;  // write weights are stored normalised
+
+                // ---- pass 2: numerators (value + residual) of each tile, then the write-back of its MV rows ----
+                for (int t = 0; t < nt; ++t) {
+                    ST_WAIT(&sready[0], su0, 62);
+                    ++su0;
+                    ++kc;
+                    const int vh = kc % kStStages;
+                    const uint32_t vh_par = kc / kStStages;
+                    ++kc;
+                    const int vl = kc % kStStages;
+                    const uint32_t vl_par = kc / kStStages;
+                    ++kc;
+                    if (np > 0) ST_WAIT(pfree, np - 1, 63);
+                    tc_fence_after();
+                    const int n_valid = min(kStTile, a.C - t * kStTile);
+#pragma unroll 1
+                    for (int bch = 0; bch < 4; ++bch) {
+                        float x[32];
+                        tmem_ld32(lane_base + kColS0 + bch * 32, x);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            x[i] = ((is_read || is_write) && bch * 32 + i < n_valid) ? __expf(x[i] * scale - m) * wmul : 0.f;
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const int c = bch * 4 + j;  // 16-byte chunk = 8 slots
+                            uint4 hi, lo;
+                            split8(x + 8 * j, &hi, &lo);
+                            const int off = (c >> 3) * kStHalf + r * 128 + (((c & 7) ^ sw) * 16);
+                            *reinterpret_cast<uint4*>(phi + off) = hi;
+                            *reinterpret_cast<uint4*>(plo + off) = lo;
+                        }
+                    }
+                    tc_fence_before();
+                    mbar_arrive(&sfree[0]);
+                    fence_proxy_async_smem();
+                    mbar_arrive(pready);
+                    ++np;
+
+                    // the tile's MV rows: value + residual + increment, split again, stored
+                    ST_WAIT(&full[vh], vh_par, 64);
+                    ST_WAIT(&full[vl], vl_par, 65);
+                    ST_WAIT(dready, nd, 66);
+                    ++nd;
+                    tc_fence_after();
+                    const int slot = t * kStTile + r;
+                    const unsigned char* th = ring + (size_t)vh * kStTileBytes;
+                    const unsigned char* tl = ring + (size_t)vl * kStTileBytes;
+                    const size_t grow = ((size_t)u * a.C + slot) * 256;
+#pragma unroll 1
+                    for (int bch = 0; bch < 4; ++bch) {
+                        float dx[32];
+                        tmem_ld32(lane_base + kColD + bch * 32, dx);
+                        if (slot < a.C) {
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                const int c = bch * 4 + j;
+                                const int off = (c >> 3) * kStHalf + r * 128 + (((c & 7) ^ sw) * 16);
+                                float vh8[8], vl8[8], nv[8];
+                                Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(th + off), vh8);
+                                Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(tl + off), vl8);
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) nv[e] = (vh8[e] + vl8[e]) + dx[8 * j + e];
+                                uint4 hi, lo;
+                                split8(nv, &hi, &lo);
+                                *reinterpret_cast<uint4*>(a.vhi + grow + c * 16) = hi;
+                                *reinterpret_cast<uint4*>(a.vlo + grow + c * 16) = lo;
+                            }
+                        }
+                    }
+                    // later chunks read these rows back through TMA: order the stores before the async proxy
+                    asm volatile("fence.proxy.async.global;" ::: "memory");
+                    tc_fence_before();
+                    mbar_arrive(dfree);
+                    st_sync();  // every row of the two MV tiles has been read
+                    if (tid == 0) {
+                        mbar_arrive(&empty[vh]);
+                        mbar_arrive(&empty[vl]);
+                    }
+                }
+
+                // ---- intra-chunk term: row (t, g) sees the writes of tokens s < t (s <= t when the read
+                // ---- follows the write); A is masked, rounded to bfloat16 and handed back as an operand ----
+                {
+                    float av[kStMaxTc];
+#pragma unroll
+                    for (int bch = 0; bch < kStMaxTc / 32; ++bch)
+                        if (bch * 32 < Tc) tmem_ld32(lane_base + kColA + bch * 32, av + bch * 32);
+#pragma unroll
+                    for (int c = 0; c < kStMaxTc / 8; ++c) {
+                        if (c * 8 < Tc) {
+                            float z[8];
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) {
+                                const int s = c * 8 + e;
+                                const bool seen = is_read && s < Tc && (a.wtr ? s <= my_t : s < my_t);
+                                z[e] = seen ? av[s] : 0.f;
+                            }
+                            *reinterpret_cast<uint4*>(plo + r * 128 + ((c ^ sw) * 16)) = Chunk<__nv_bfloat16>::pack(z);
+                        }
+                    }
+                    tc_fence_before();
+                    fence_proxy_async_smem();
+                    mbar_arrive(aready);
+                }
+
+                // ---- epilogue: this row's outputs, normalised by its sum ----
+                ST_WAIT(oready, qn, 67);
+                tc_fence_after();
+                {
+                    const size_t orow = (((size_t)b * a.T + t0 + my_t) * a.Hq + (size_t)h * G + my_g) * 128;
+#pragma unroll 1
+                    for (int bch = 0; bch < 4; ++bch) {
+                        float o[32];
+                        tmem_ld32(lane_base + kColO + bch * 32, o);
+                        if (is_read && a.out != nullptr && !*abort_flag) {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) o[i] *= inv_l;
+                            if (a.out_f32) {
+                                float4* dst = reinterpret_cast<float4*>(a.out + (orow + bch * 32) * 4);
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) dst[j] = make_float4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+                            } else {
+                                uint4* dst = reinterpret_cast<uint4*>(a.out + (orow + bch * 32) * 2);
+#pragma unroll
+                                for (int j = 0; j < 4; ++j) dst[j] = Chunk<__nv_bfloat16>::pack(o + 8 * j);
+                            }
+                        }
+                    }
+                }
+                tc_fence_before();
+                mbar_arrive(qfree);  // the chunk's operands and accumulators may be reused
+            }
+        }
+    }
+#undef ST_WAIT
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 5) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+using StKernelFn = void (*)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap,
+                            const CUtensorMap, const CUtensorMap, const StArgs);
+
+StKernelFn pick_stream(int G) {
+    switch (G) {
+        case 1: return stream_tc_kernel<1>;
+        case 2: return stream_tc_kernel<2>;
+        case 3: return stream_tc_kernel<3>;
+        case 4: return stream_tc_kernel<4>;
+        case 5: return stream_tc_kernel<5>;
+        case 6: return stream_tc_kernel<6>;
+        case 7: return stream_tc_kernel<7>;
+        default: return nullptr;
+    }
+}
+
+typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                             const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                             CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeFn st_encode_fn() {
+    static EncodeFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeFn>(p);
+    }
+    return fn;
+}
+
+// Step vectors [B][T][H][128] bfloat16 as a 4-D tensor (d, head, token, sequence); one box is
+// 64 columns x `heads` heads x `tokens` tokens, landing as rows (token, head) with the 128-byte swizzle.
+bool make_step_map(CUtensorMap* map, const void* base, int B, int T, int H, int heads, int tokens) {
+    EncodeFn fn = st_encode_fn();
+    if (fn == nullptr) return false;
+    const cuuint64_t dims[4] = {128, (cuuint64_t)H, (cuuint64_t)T, (cuuint64_t)B};
+    const cuuint64_t strides[3] = {256, (cuuint64_t)H * 256, (cuuint64_t)T * H * 256};
+    const cuuint32_t box[4] = {64, (cuuint32_t)heads, (cuuint32_t)tokens, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+int stream_chunk_tokens(const bct_cache* c) {
+    const bct_params_t& p = c->p;
+    if (p.dtype != BCT_BF16 || p.head_dim != 128 || c->G > 7 || !c->tc_ready) return 0;
+    if (p.flags & BCT_FLAG_CUDA_CORES) return 0;
+    if (p.capacity < kStTile || p.capacity > 2048) return 0;
+    if (c->plane_bytes < (size_t)1 << 18) return 0;
+    return c->G == 1 ? 64 : (c->G <= 3 ? 32 : 16);
+}
+
+int launch_stream_tc(const bct_cache* c, const void* q, const void* k, const void* v, void* out, int64_t T,
+                     int64_t t_begin, int64_t n_chunks, cudaStream_t stream, cudaError_t* err) {
+    const bct_params_t& p = c->p;
+    StKernelFn fn = pick_stream(c->G);
+    const int Tc = stream_chunk_tokens(c);
+    if (fn == nullptr || Tc == 0 || T > (int64_t)1 << 30) {
+        *err = cudaErrorInvalidConfiguration;
+        return -1;
+    }
+    alignas(64) CUtensorMap mq, mk, mv;
+    if (!make_step_map(&mq, q, p.batch, (int)T, p.n_q_heads, c->G, Tc) ||
+        !make_step_map(&mk, k, p.batch, (int)T, p.n_kv_heads, 1, Tc) ||
+        !make_step_map(&mv, v, p.batch, (int)T, p.n_kv_heads, 1, Tc)) {
+        *err = cudaErrorInvalidValue;
+        return -1;
+    }
+    StArgs a;
+    a.vhi = c->vhi;
+    a.vlo = c->vlo;
+    a.out = static_cast<char*>(out);
+    a.status = c->status;
+    a.C = p.capacity;
+    a.Hq = p.n_q_heads;
+    a.Hkv = p.n_kv_heads;
+    a.U = c->U;
+    a.T = (int)T;
+    a.t_begin = (int)t_begin;
+    a.n_chunks = (int)n_chunks;
+    a.Tc = Tc;
+    a.wtr = (p.flags & BCT_FLAG_WRITE_THEN_READ) ? 1 : 0;
+    a.out_f32 = (p.flags & BCT_FLAG_OUT_F32) ? 1 : 0;
+    a.read_scale = p.read_scale;
+    a.write_scale = p.write_scale;
+    const int smem = st_smem().total;
+    *err = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (*err != cudaSuccess) return -1;
+    const int grid = c->U < c->sm_count ? c->U : c->sm_count;
+    fn<<<grid, kStThreads, smem, stream>>>(*reinterpret_cast<const CUtensorMap*>(c->tmap_k),
+                                           *reinterpret_cast<const CUtensorMap*>(c->tmap_v),
+                                           *reinterpret_cast<const CUtensorMap*>(c->tmap_lo), mq, mk, mv, a);
+    *err = cudaGetLastError();
+    return *err == cudaSuccess ? 1 : -1;
+}
+
+}  // namespace bct

@@ -1,0 +1,94 @@
+"""GPU parity of the chunked tensor-core stream kernel (bct_prefill_stream on a full bfloat16 cache,
+head_dim 128) against the CPU oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import bct_oracle as O
+from paper_2411_15785_b200 import binding as B
+from paper_2411_15785_b200 import build as bld
+from paper_2411_15785_b200 import workloads as W
+
+from _parity import TOL, compare_out, compare_state, make_pair, pick_units, _unit_slices
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    bld.build()
+    B.load()
+
+
+def _stream_parity(w, T, pieces, flags=0, oracle_flags=0, want_out=True):
+    units = pick_units(w, 8)
+    gpu, ora = make_pair(w, units, flags=flags, oracle_flags=oracle_flags)
+    q, k, v = W.stream_inputs(w, 0, T, "cuda")
+    launches0 = gpu.launches
+    outs, t = [], 0
+    for n in pieces:
+        sl = slice(t, t + n)
+        outs.append(gpu.prefill_stream(q[:, sl].contiguous(), k[:, sl].contiguous(), v[:, sl].contiguous(),
+                                       want_out=want_out))
+        t += n
+    assert t == T
+    gpu.check_status()
+    ref = ora.prefill_stream(*_unit_slices(w, units, q, k, v))
+    err = compare_out(w, units, torch.cat(outs, dim=1), ref) if want_out else 0.0
+    state = compare_state(w, units, gpu, ora)
+    n_launch = gpu.launches - launches0
+    gpu.destroy()
+    return err, state, n_launch
+
+
+@pytest.mark.parametrize("G,C,init_len,T,pieces", [
+    (1, 256, 256, 200, [200]),            # 3 chunks of 64 + 8 single tokens
+    (1, 1024, 1024, 256, [128, 128]),     # the long-stream shape, two calls
+    (1, 333, 300, 170, [170]),            # ragged capacity; 33 fill tokens first, then chunks
+    (2, 512, 512, 100, [64, 36]),         # chunks of 32
+    (3, 640, 640, 64, [64]),
+    (4, 520, 520, 50, [50]),              # chunks of 16
+    (7, 2048, 2048, 32, [32]),            # 16 tiles
+])
+def test_chunked_stream_matches_oracle(G, C, init_len, T, pieces):
+    d = 128
+    w = W.Workload("t", 2, 2 * G, 2, d, C, "bf16", init_len, T, 41, d ** -0.5, 1.0, 1.0, "stream")
+    w = w.scaled(batch=3 if C <= 512 else 2)
+    err, state, n_launch = _stream_parity(w, T, pieces)
+    assert err <= TOL["bf16"] and state <= TOL["bf16"], (err, state)
+    assert n_launch < T  # whole chunks went through the chunked kernel, not one launch per token
+
+
+@pytest.mark.parametrize("flags,oflags", [(B.FLAG_WRITE_THEN_READ, O.WRITE_THEN_READ), (B.FLAG_OUT_F32, 0),
+                                          (B.FLAG_SKIP_FIRST_WRITE, O.SKIP_FIRST_WRITE)])
+def test_chunked_stream_flags(flags, oflags):
+    d = 128
+    w = W.Workload("t", 3, 4, 2, d, 384, "bf16", 384, 150, 43, d ** -0.5, 1.0, 1.0, "stream", 1.0, 0.4)
+    err, state, _ = _stream_parity(w, 150, [150], flags=flags, oracle_flags=oflags)
+    assert err <= TOL["bf16"] and state <= TOL["bf16"], (err, state)
+
+
+def test_chunked_stream_state_only_and_diffuse_writes():
+    d = 128
+    w = W.Workload("t", 2, 2, 2, d, 256, "bf16", 256, 192, 47, d ** -0.5, 1.0, 1.0, "stream", 1.0, d ** -0.5)
+    err, state, _ = _stream_parity(w, 192, [192], want_out=False)
+    assert state <= 1e-3, state
+    err, state, _ = _stream_parity(w, 192, [192])
+    assert err <= TOL["bf16"] and state <= 1e-3, (err, state)
+
+
+def test_chunked_stream_tracks_decode_steps_on_a_long_run():
+    # the per-token path (tensor-core decode kernel) and the chunked path on the same 2048 tokens
+    d = 128
+    w = W.Workload("t", 1, 4, 4, d, 512, "bf16", 512, 2048, 53, d ** -0.5, 1.0, 1.0, "stream")
+    units = pick_units(w, 4)
+    a, ora = make_pair(w, units, flags=B.FLAG_OUT_F32)
+    b, _ = make_pair(w, units, flags=B.FLAG_OUT_F32)
+    q, k, v = W.stream_inputs(w, 0, w.steps, "cuda")
+    oa = a.prefill_stream(q, k, v)
+    ob = torch.stack([b.decode_step(q[:, t].contiguous(), k[:, t].contiguous(), v[:, t].contiguous())
+                      for t in range(w.steps)], dim=1)
+    ref = ora.prefill_stream(*_unit_slices(w, units, q, k, v))
+    ea, eb = compare_out(w, units, oa, ref), compare_out(w, units, ob, ref)
+    assert ea <= TOL["bf16"] and eb <= TOL["bf16"], (ea, eb)
+    assert compare_state(w, units, a, ora) <= TOL["bf16"]
