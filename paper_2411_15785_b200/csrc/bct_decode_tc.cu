@@ -259,7 +259,9 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     }
                     umma_commit(&empty[stage]);
                 }
-                umma_commit(oready);  // every V tile of the unit has been read
+                // (with no tile at all nothing is committed: the commit would complete at once, and a
+                // second one could follow before the first is observed)
+                if (nt > 0) umma_commit(oready);  // every V tile of the unit has been read
             }
         }
         __syncwarp();
@@ -450,7 +452,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             }
 
             // ---- epilogue: O[d][g] from tensor memory once every V tile has been read ----
-            if (!mbar_wait(oready, it & 1, *abort_flag ? 1024u : kWaitLimit)) {
+            if (nt > 0 && !mbar_wait(oready, it & 1, *abort_flag ? 1024u : kWaitLimit)) {
                 report_timeout(a.status, 19);
                 *abort_flag = 1;
             }
