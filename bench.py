@@ -30,6 +30,7 @@ from paper_2411_15785_b200 import workloads as W  # noqa: E402
 METRIC = "bounded-cache decode tokens/s"
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1400.0
 
 
 def _peaks():
@@ -109,6 +110,30 @@ TRAFFIC_PER_UNIT = {("mha7b", True): 1.2964e9 / 1184}
 def measured_traffic(w, tensor_path):
     per_unit = TRAFFIC_PER_UNIT.get((w.name.split("_")[0], bool(tensor_path)))
     return None if per_unit is None else per_unit * w.units
+
+
+def stream_roofline(w, tok_per_step, ms_step):
+    """Tensor-core roofline of stream_tc_kernel: the dense flops its MMAs execute per step (operand rows padded
+    to M = 128 included) against the measured bf16 matmul peak."""
+    Tc = 64 if w.group == 1 else (32 if w.group <= 3 else 16)
+    C, d = w.capacity, w.head_dim
+    per_chunk = 2 * (2 * 128 * C * d)          # scores of the 128 operand rows, two passes over MK
+    per_chunk += 3 * (2 * 128 * C * d)         # outputs: (P + P_lo) MV_hi + P MV_lo
+    per_chunk += 2 * 128 * C * Tc              # A = P WW^T
+    per_chunk += 2 * (2 * C * Tc * d)          # MV increment with value + residual weights
+    per_chunk += 2 * 128 * Tc * d              # strict_tril(A) Vc
+    flops = per_chunk * (tok_per_step // Tc) * w.units
+    peak = FALLBACK_BF16_TFLOPS
+    kind = "fallback"
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            peak, kind = float(json.load(open(path))["bf16_tflops_sustained"]), "measured"
+        except Exception:
+            pass
+    ach = flops / (ms_step * 1e-3) / 1e12
+    return {"bound": "tensor", "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak, "traffic": None,
+            "peak_kind": "of " + kind, "kernel": "stream_tc_kernel", "flops_per_launch": flops}
 
 
 def cpu_oracle_sample(w: W.Workload, budget_s: float = 25.0):
@@ -207,6 +232,8 @@ def main():
     ap.add_argument("--workload", default="mha7b_b64_c2048", choices=sorted(W.CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--write-scale", type=float, default=None, help="override the write score scale")
+    ap.add_argument("--stream-tokens", type=int, default=256,
+                    help="tokens per sequence pushed by one step of a stream workload")
     ap.add_argument("--write-eps", type=float, default=0.0, help="override write_eps (0 = library default 2^-24)")
     ap.add_argument("--flags", type=int, default=0, help="BCT_FLAG_* bits for the cache")
     ap.add_argument("--batch", type=int, default=None, help="override the batch (profiling on a smaller case)")
@@ -245,11 +272,29 @@ def main():
     mk, mv = W.initial_cache(wr, dev)
     cache = B.Cache(w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.capacity, w.torch_dtype,
                     read_scale=w.read_scale, write_scale=w.write_scale, init_len=w.init_len, mk_init=mk, mv_init=mv,
-                    write_eps=args.write_eps, flags=args.flags, device=dev)
+                    write_eps=args.write_eps, flags=args.flags, max_stream=(args.stream_tokens if w.api == "stream" else 1),
+                    device=dev)
     torch.cuda.synchronize()
     del mk, mv
-    pool = [W.step_inputs(wr, t, dev) for t in range(min(args.steps + args.warmup, 64))]
-    outs = [torch.empty_like(pool[0][0]) for _ in range(2)]
+    stream = (w.api == "stream")
+    tok_per_step = args.stream_tokens if stream else 1   # tokens per sequence in one step
+    if stream:
+        # fill the cache (untimed), then every step pushes one block of tokens through bct_prefill_stream
+        t_fill = 0
+        while cache.len < w.capacity:
+            n = min(256, w.capacity - cache.len)
+            cache.prefill_stream(*W.stream_inputs(wr, t_fill, n, dev), want_out=False)
+            t_fill += n
+        pool = [W.stream_inputs(wr, w.capacity + i * tok_per_step, tok_per_step, dev) for i in range(8)]
+    else:
+        pool = [W.step_inputs(wr, t, dev) for t in range(min(args.steps + args.warmup, 64))]
+    outs = [torch.empty_like(pool[0][0], dtype=cache.out_dtype) for _ in range(2)]
+
+    def step_dev(i):
+        if stream:
+            cache.prefill_stream(*pool[i % len(pool)], out=outs[i & 1])
+        else:
+            cache.decode_step(*pool[i % len(pool)], out=outs[i & 1])
 
     def sync_all():
         torch.cuda.synchronize()
@@ -259,7 +304,7 @@ def main():
 
     # ---------- device-resident timing ----------
     for i in range(args.warmup):
-        cache.decode_step(*pool[i % len(pool)], out=outs[i & 1])
+        step_dev(i)
     sync_all()
     sampler = ClockSampler(local)
     if rank == 0:
@@ -268,7 +313,7 @@ def main():
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for i in range(args.steps):
-        cache.decode_step(*pool[(args.warmup + i) % len(pool)], out=outs[i & 1])
+        step_dev(args.warmup + i)
     e1.record()
     sync_all()
     ms_total = e0.elapsed_time(e1)
@@ -278,14 +323,21 @@ def main():
 
     # ---------- end to end through the host-buffer entry point ----------
     hpool = [tuple(x.cpu().pin_memory() for x in pool[i]) for i in range(min(len(pool), 16))]
-    hout = [torch.empty_like(hpool[0][0]).pin_memory() for _ in range(2)]
+    hout = [torch.empty_like(hpool[0][0], dtype=cache.out_dtype).pin_memory() for _ in range(2)]
+
+    def step_host(i):
+        if stream:
+            cache.prefill_stream_host(*hpool[i % len(hpool)], hout[i & 1])
+        else:
+            cache.decode_step_host(*hpool[i % len(hpool)], hout[i & 1])
+
     for i in range(3):
-        cache.decode_step_host(*hpool[i % len(hpool)], hout[i & 1])
+        step_host(i)
     sync_all()
     e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e2.record()
     for i in range(args.steps):
-        cache.decode_step_host(*hpool[i % len(hpool)], hout[i & 1])
+        step_host(i)
     e3.record()
     sync_all()
     ms_e2e = e2.elapsed_time(e3)
@@ -301,9 +353,16 @@ def main():
     if rank == 0:
         peak, peak_kind = _peaks()
         ms_step = ms_total / args.steps
-        tokens = w.batch * world * args.steps
+        tokens = w.batch * world * args.steps * tok_per_step
         alg = algorithmic_bytes_per_step(w)
         achieved = alg / (ms_step * 1e-3) / 1e9
+        if stream:
+            roof = stream_roofline(w, tok_per_step, ms_step)
+        else:
+            roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                    "traffic": measured_traffic(w, cache.tensor_path), "peak_kind": "of " + peak_kind,
+                    "kernel": "decode_tc_kernel" if cache.tensor_path else "decode_kernel",
+                    "algorithmic_bytes_per_launch": alg, "frac_of_8TBps_nominal": achieved / 8000.0}
         line = {
             "metric": METRIC, "value": tokens / (ms_total * 1e-3), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
@@ -312,16 +371,15 @@ def main():
             "config": {"workload": w.name, "batch_per_gpu": w.batch, "n_q_heads": w.n_q_heads,
                        "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim, "capacity": w.capacity,
                        "write_scale": w.write_scale, "read_scale": w.read_scale,
-                       "l2": "cache planes streamed per step (%.2f GB) exceed L2" % (alg / 1e9),
+                       "tokens_per_step": tok_per_step,
+                       "l2": ("cache planes of all units (%.2f GB) exceed L2" % (1.5 * alg / 1e9)) if stream else
+                             ("cache planes streamed per step (%.2f GB) exceed L2" % (alg / 1e9)),
                        "parallelism": "independent units; replicas per GPU" if world > 1 else "1 GPU"},
             "clocks": clocks,
             "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.steps},
             "gpu_launches": launches,
-            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": measured_traffic(w, cache.tensor_path), "peak_kind": "of " + peak_kind,
-                         "kernel": "decode_tc_kernel" if cache.tensor_path else "decode_kernel",
-                         "algorithmic_bytes_per_launch": alg, "frac_of_8TBps_nominal": achieved / 8000.0},
+            "roofline": roof,
         }
         if world == 1 and not args.no_cpu_baseline:
             cb = cpu_oracle_sample(w)
