@@ -15,9 +15,9 @@
 // with fp32 accumulators in tensor memory.  Numerators and write weights are kept as bfloat16
 // value + residual pairs, and MV is read as value + residual, so a long stream keeps the precision
 // of the per-token path.
-//   warp 4  producer : TMA loads (chunk operands, MK / MV tiles through a 3-stage ring)
-//   warp 5  MMA      : issues all tensor-core work, commits to mbarriers
-//   warps 0-3        : one thread per operand row: online row statistics, numerators, the write-back
+//   warp 8  producer : TMA loads (chunk operands, MK / MV tiles through a 3-stage ring)
+//   warp 9  MMA      : issues all tensor-core work, commits to mbarriers
+//   warps 0-7        : two threads per operand row (64 accumulator columns each): online row statistics, numerators, the write-back
 //                      of MV rows, the intra-chunk term and the epilogue
 // Every wait is bounded; a timeout sets the status word and the kernel runs to its end.
 #include <cuda.h>
@@ -30,8 +30,8 @@
 namespace bct {
 namespace {
 
-constexpr int kStThreads = 192;
-constexpr int kStS = 128;                // softmax threads = operand rows
+constexpr int kStThreads = 320;
+constexpr int kStS = 256;                // row threads: two per operand row
 constexpr int kStTile = 128;             // slots per tile
 constexpr int kStHalf = 128 * 128;       // 64 columns (128 bytes) x 128 rows
 constexpr int kStTileBytes = 2 * kStHalf;
@@ -73,7 +73,7 @@ __host__ __device__ inline StSmem st_smem() {
     L.bars = off;
     off += 32 * 8;
     L.misc = off;
-    off += 64;
+    off += 64 + 2 * 128 * 2 * 4;  // flags, then (max, sum) of each half row
     L.total = off + 1024;       // slack to align the base to 1024 bytes
     return L;
 }
@@ -119,6 +119,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     uint64_t* oready = bars + 17;     // outputs complete (commit)
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L.misc);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L.misc + 8);
+    float* rowstat = reinterpret_cast<float*>(smem + L.misc + 64);
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
@@ -150,7 +151,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     }
     // rows of the query operand beyond the chunk's G*Tc + Tc stay zero for good
     for (int i = tid; i < kStTileBytes / 16; i += kStThreads) reinterpret_cast<uint4*>(qall)[i] = make_uint4(0, 0, 0, 0);
-    if (warp == 5) tmem_alloc(tmem_slot, 512);
+    if (warp == 9) tmem_alloc(tmem_slot, 512);
     fence_proxy_async_smem();
     tc_fence_before();
     __syncthreads();
@@ -163,7 +164,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         *abort_flag = 1;                                                        \
     }
 
-    if (warp == 4) {
+    if (warp == 8) {
         // =========================== producer ===========================
         if (lane == 0) {
             uint32_t kc = 0, qn = 0;
@@ -198,7 +199,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             }
         }
         __syncwarp();
-    } else if (warp == 5) {
+    } else if (warp == 9) {
         // =========================== MMA issuer ===========================
         if (lane == 0) {
             constexpr uint32_t id_scores = instr_desc_mn(128, 128, false, false);  // Qall (K) x tile (K)
@@ -297,8 +298,11 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         __syncwarp();
     } else {
         // =========================== row threads: statistics, numerators, write-back, epilogue ===========================
-        const int r = tid;                              // operand row = tensor-memory lane
-        const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
+        // Two threads per operand row (tensor-memory lane): thread half hf works on columns
+        // [64 hf, 64 hf + 64) of every 128-column accumulator.
+        const int r = tid & 127;
+        const int hf = tid >> 7;
+        const uint32_t lane_base = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + hf * 64;
         const bool is_read = r < n_read;
         const bool is_write = !is_read && r < n_read + Tc;
         const int my_t = is_read ? r / G : (is_write ? r - n_read : 0);  // token of the chunk this row belongs to
@@ -310,7 +314,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             const int b = u / a.Hkv, h = u - b * a.Hkv;
             for (int ch = 0; ch < a.n_chunks; ++ch, ++qn) {
                 const int t0 = a.t_begin + ch * Tc;
-                // ---- pass 1: online maximum and sum of this row's scaled scores over all C slots ----
+                // ---- pass 1: online maximum and sum of this half row's scaled scores over all C slots ----
                 float m = kStNegBig, l = 0.f;
                 for (int t = 0; t < nt; ++t, ++kc) {
                     const int buf = t & 1;
@@ -318,26 +322,36 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     ST_WAIT(&sready[buf], su, 61);
                     ++su;
                     tc_fence_after();
-                    const int n_valid = min(kStTile, a.C - t * kStTile);
-#pragma unroll 1
-                    for (int bch = 0; bch < 4; ++bch) {
-                        float x[32];
-                        tmem_ld32(lane_base + (buf ? kColD : kColS0) + bch * 32, x);
-                        float bm = kStNegBig;
+                    const int n_valid = min(kStTile, a.C - t * kStTile) - hf * 64;
+                    float x[64];
+                    tmem_ld64(lane_base + (buf ? kColD : kColS0), x);
+                    float bm = kStNegBig;
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) {
-                            x[i] = (bch * 32 + i < n_valid) ? x[i] * scale : kStNegBig;
-                            bm = fmaxf(bm, x[i]);
-                        }
-                        const float mn = fmaxf(m, bm);
-                        float s = 0.f;
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) s += __expf(x[i] - mn);
-                        l = l * __expf(m - mn) + s;
-                        m = mn;
+                    for (int i = 0; i < 64; ++i) {
+                        x[i] = (i < n_valid) ? x[i] * scale : kStNegBig;
+                        bm = fmaxf(bm, x[i]);
                     }
+                    const float mn = fmaxf(m, bm);
+                    float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+                    for (int i = 0; i < 64; i += 2) {
+                        s0 += __expf(x[i] - mn);
+                        s1 += __expf(x[i + 1] - mn);
+                    }
+                    l = l * __expf(m - mn) + (s0 + s1);
+                    m = mn;
                     tc_fence_before();
                     mbar_arrive(&sfree[buf]);
+                }
+                // combine the two halves of the row
+                rowstat[(hf * 128 + r) * 2] = m;
+                rowstat[(hf * 128 + r) * 2 + 1] = l;
+                st_sync();
+                {
+                    const float mo = rowstat[((hf ^ 1) * 128 + r) * 2], lo_ = rowstat[((hf ^ 1) * 128 + r) * 2 + 1];
+                    const float mn = fmaxf(m, mo);
+                    l = l * __expf(m - mn) + lo_ * __expf(mo - mn);
+                    m = mn;
                 }
                 const float inv_l = 1.f / l;
                 const float wmul = is_write ? inv_l : 1.f;  // write weights are stored normalised
@@ -355,49 +369,47 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     ++kc;
                     if (np > 0) ST_WAIT(pfree, np - 1, 63);
                     tc_fence_after();
-                    const int n_valid = min(kStTile, a.C - t * kStTile);
-#pragma unroll 1
-                    for (int bch = 0; bch < 4; ++bch) {
-                        float x[32];
-                        tmem_ld32(lane_base + kColS0 + bch * 32, x);
+                    {
+                        const int n_valid = min(kStTile, a.C - t * kStTile) - hf * 64;
+                        float x[64];
+                        tmem_ld64(lane_base + kColS0, x);
+                        tc_fence_before();
+                        mbar_arrive(&sfree[0]);  // the scores are in registers: the next tile's may be computed
 #pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            x[i] = ((is_read || is_write) && bch * 32 + i < n_valid) ? __expf(x[i] * scale - m) * wmul : 0.f;
+                        for (int i = 0; i < 64; ++i)
+                            x[i] = ((is_read || is_write) && i < n_valid) ? __expf(x[i] * scale - m) * wmul : 0.f;
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const int c = bch * 4 + j;  // 16-byte chunk = 8 slots
+                        for (int j = 0; j < 8; ++j) {  // 16-byte chunk j of this half = 8 slots
                             uint4 hi, lo;
                             split8(x + 8 * j, &hi, &lo);
-                            const int off = (c >> 3) * kStHalf + r * 128 + (((c & 7) ^ sw) * 16);
+                            const int off = hf * kStHalf + r * 128 + ((j ^ sw) * 16);
                             *reinterpret_cast<uint4*>(phi + off) = hi;
                             *reinterpret_cast<uint4*>(plo + off) = lo;
                         }
                     }
-                    tc_fence_before();
-                    mbar_arrive(&sfree[0]);
                     fence_proxy_async_smem();
                     mbar_arrive(pready);
                     ++np;
 
-                    // the tile's MV rows: value + residual + increment, split again, stored
+                    // the tile's MV rows: value + residual + increment, split again, stored (this thread: 64 of the 128 d)
                     ST_WAIT(&full[vh], vh_par, 64);
                     ST_WAIT(&full[vl], vl_par, 65);
                     ST_WAIT(dready, nd, 66);
                     ++nd;
                     tc_fence_after();
-                    const int slot = t * kStTile + r;
-                    const unsigned char* th = ring + (size_t)vh * kStTileBytes;
-                    const unsigned char* tl = ring + (size_t)vl * kStTileBytes;
-                    const size_t grow = ((size_t)u * a.C + slot) * 256;
-#pragma unroll 1
-                    for (int bch = 0; bch < 4; ++bch) {
-                        float dx[32];
-                        tmem_ld32(lane_base + kColD + bch * 32, dx);
+                    {
+                        const int slot = t * kStTile + r;
+                        const unsigned char* th = ring + (size_t)vh * kStTileBytes + hf * kStHalf + r * 128;
+                        const unsigned char* tl = ring + (size_t)vl * kStTileBytes + hf * kStHalf + r * 128;
+                        const size_t grow = ((size_t)u * a.C + slot) * 256 + hf * 128;
+                        float dx[64];
+                        tmem_ld64(lane_base + kColD, dx);
+                        tc_fence_before();
+                        mbar_arrive(dfree);
                         if (slot < a.C) {
 #pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                const int c = bch * 4 + j;
-                                const int off = (c >> 3) * kStHalf + r * 128 + (((c & 7) ^ sw) * 16);
+                            for (int j = 0; j < 8; ++j) {
+                                const int off = (j ^ sw) * 16;
                                 float vh8[8], vl8[8], nv[8];
                                 Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(th + off), vh8);
                                 Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(tl + off), vl8);
@@ -405,15 +417,13 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                                 for (int e = 0; e < 8; ++e) nv[e] = (vh8[e] + vl8[e]) + dx[8 * j + e];
                                 uint4 hi, lo;
                                 split8(nv, &hi, &lo);
-                                *reinterpret_cast<uint4*>(a.vhi + grow + c * 16) = hi;
-                                *reinterpret_cast<uint4*>(a.vlo + grow + c * 16) = lo;
+                                *reinterpret_cast<uint4*>(a.vhi + grow + j * 16) = hi;
+                                *reinterpret_cast<uint4*>(a.vlo + grow + j * 16) = lo;
                             }
                         }
                     }
                     // later chunks read these rows back through TMA: order the stores before the async proxy
                     asm volatile("fence.proxy.async.global;" ::: "memory");
-                    tc_fence_before();
-                    mbar_arrive(dfree);
                     st_sync();  // every row of the two MV tiles has been read
                     if (tid == 0) {
                         mbar_arrive(&empty[vh]);
@@ -424,21 +434,23 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 // ---- intra-chunk term: row (t, g) sees the writes of tokens s < t (s <= t when the read
                 // ---- follows the write); A is masked, rounded to bfloat16 and handed back as an operand ----
                 {
-                    float av[kStMaxTc];
+                    // thread half hf covers write tokens [32 hf, 32 hf + 32)
+                    float av[32];
+                    tmem_ld32(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + kColA + hf * 32, av);
+                    if (hf * 32 < Tc) {
 #pragma unroll
-                    for (int bch = 0; bch < kStMaxTc / 32; ++bch)
-                        if (bch * 32 < Tc) tmem_ld32(lane_base + kColA + bch * 32, av + bch * 32);
+                        for (int j = 0; j < 4; ++j) {
+                            const int c = hf * 4 + j;
+                            if (c * 8 < Tc) {
+                                float z[8];
 #pragma unroll
-                    for (int c = 0; c < kStMaxTc / 8; ++c) {
-                        if (c * 8 < Tc) {
-                            float z[8];
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) {
-                                const int s = c * 8 + e;
-                                const bool seen = is_read && s < Tc && (a.wtr ? s <= my_t : s < my_t);
-                                z[e] = seen ? av[s] : 0.f;
+                                for (int e = 0; e < 8; ++e) {
+                                    const int s = c * 8 + e;
+                                    const bool seen = is_read && (a.wtr ? s <= my_t : s < my_t);
+                                    z[e] = seen ? av[8 * j + e] : 0.f;
+                                }
+                                *reinterpret_cast<uint4*>(plo + r * 128 + ((c ^ sw) * 16)) = Chunk<__nv_bfloat16>::pack(z);
                             }
-                            *reinterpret_cast<uint4*>(plo + r * 128 + ((c ^ sw) * 16)) = Chunk<__nv_bfloat16>::pack(z);
                         }
                     }
                     tc_fence_before();
@@ -446,27 +458,24 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     mbar_arrive(aready);
                 }
 
-                // ---- epilogue: this row's outputs, normalised by its sum ----
+                // ---- epilogue: this row's outputs (this thread: 64 of the 128 d), normalised by the row sum ----
                 ST_WAIT(oready, qn, 67);
                 tc_fence_after();
                 {
-                    const size_t orow = (((size_t)b * a.T + t0 + my_t) * a.Hq + (size_t)h * G + my_g) * 128;
-#pragma unroll 1
-                    for (int bch = 0; bch < 4; ++bch) {
-                        float o[32];
-                        tmem_ld32(lane_base + kColO + bch * 32, o);
-                        if (is_read && a.out != nullptr && !*abort_flag) {
+                    const size_t orow = (((size_t)b * a.T + t0 + my_t) * a.Hq + (size_t)h * G + my_g) * 128 + hf * 64;
+                    float o[64];
+                    tmem_ld64(lane_base + kColO, o);
+                    if (is_read && a.out != nullptr && !*abort_flag) {
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) o[i] *= inv_l;
-                            if (a.out_f32) {
-                                float4* dst = reinterpret_cast<float4*>(a.out + (orow + bch * 32) * 4);
+                        for (int i = 0; i < 64; ++i) o[i] *= inv_l;
+                        if (a.out_f32) {
+                            float4* dst = reinterpret_cast<float4*>(a.out + orow * 4);
 #pragma unroll
-                                for (int j = 0; j < 8; ++j) dst[j] = make_float4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
-                            } else {
-                                uint4* dst = reinterpret_cast<uint4*>(a.out + (orow + bch * 32) * 2);
+                            for (int j = 0; j < 16; ++j) dst[j] = make_float4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+                        } else {
+                            uint4* dst = reinterpret_cast<uint4*>(a.out + orow * 2);
 #pragma unroll
-                                for (int j = 0; j < 4; ++j) dst[j] = Chunk<__nv_bfloat16>::pack(o + 8 * j);
-                            }
+                            for (int j = 0; j < 8; ++j) dst[j] = Chunk<__nv_bfloat16>::pack(o + 8 * j);
                         }
                     }
                 }
@@ -479,7 +488,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 
     tc_fence_before();
     __syncthreads();
-    if (warp == 5) {
+    if (warp == 9) {
         tc_fence_after();
         tmem_dealloc(tmem_base, 512);
     }
