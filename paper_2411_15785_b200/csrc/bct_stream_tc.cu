@@ -106,7 +106,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     unsigned char* ring = smem + L.ring;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L.bars);
     uint64_t* full = bars;            // [3] tile landed (TMA transaction bytes)
-    uint64_t* empty = bars + 3;       // [3] stage may be refilled (one arrival: MMA commit or softmax thread 0)
+    uint64_t* empty = bars + 3;       // [3] stage may be refilled (one arrival: MMA commit, or the producer after its store)
     uint64_t* qfull = bars + 6;       // chunk operands landed
     uint64_t* qfree = bars + 7;       // chunk operands no longer needed (128 arrivals)
     uint64_t* sready = bars + 8;      // [2] score tile complete (commit)
@@ -117,6 +117,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     uint64_t* dfree = bars + 15;      // increment consumed (128 arrivals)
     uint64_t* aready = bars + 16;     // masked A operand written (128 arrivals)
     uint64_t* oready = bars + 17;     // outputs complete (commit)
+    uint64_t* wready = bars + 18;     // rewritten MV rows of the tile are in their ring stages (256 arrivals)
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L.misc);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L.misc + 8);
     float* rowstat = reinterpret_cast<float*>(smem + L.misc + 64);
@@ -146,6 +147,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         mbar_init(dfree, kStS);
         mbar_init(aready, kStS);
         mbar_init(oready, 1);
+        mbar_init(wready, kStS);
         *abort_flag = 0;
         fence_mbar_init_cluster();
     }
@@ -167,7 +169,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     if (warp == 8) {
         // =========================== producer ===========================
         if (lane == 0) {
-            uint32_t kc = 0, qn = 0;
+            uint32_t kc = 0, qn = 0, nw = 0;
             auto load_tile = [&](const CUtensorMap* map, int u, int t) {
                 const int stage = kc % kStStages;
                 if (kc >= (uint32_t)kStStages) ST_WAIT(&empty[stage], (kc / kStStages) - 1, 31);
@@ -190,11 +192,33 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     tma_load_4d(vc, &tmVin, 0, h, t0, b, qfull);
                     tma_load_4d(vc + vc_half, &tmVin, 64, h, t0, b, qfull);
                     for (int t = 0; t < nt; ++t) load_tile(&tmK, u, t);  // pass 1: row statistics
-                    for (int t = 0; t < nt; ++t) {                       // pass 2: numerators, outputs, update
+                    // pass 2: numerators, outputs, update.  The row threads put the rewritten MV rows back
+                    // into the two ring stages the tile came in; they go home as TMA stores from here.
+                    int pvh = 0, pvl = 0;
+                    auto store_tile = [&](int t) {
+                        ST_WAIT(wready, nw, 33);
+                        ++nw;
+                        unsigned char* sh = ring + (size_t)pvh * kStTileBytes;
+                        unsigned char* sl = ring + (size_t)pvl * kStTileBytes;
+                        tma_store_3d(&tmVhi, 0, t * kStTile, u, sh);
+                        tma_store_3d(&tmVhi, 64, t * kStTile, u, sh + kStHalf);
+                        tma_store_3d(&tmVlo, 0, t * kStTile, u, sl);
+                        tma_store_3d(&tmVlo, 64, t * kStTile, u, sl + kStHalf);
+                        bulk_commit();
+                        bulk_wait_read();  // the stages have been read out: they may be refilled
+                        mbar_arrive(&empty[pvh]);
+                        mbar_arrive(&empty[pvl]);
+                    };
+                    for (int t = 0; t < nt; ++t) {
                         load_tile(&tmK, u, t);
+                        if (t > 0) store_tile(t - 1);
+                        pvh = kc % kStStages;
                         load_tile(&tmVhi, u, t);
+                        pvl = kc % kStStages;
                         load_tile(&tmVlo, u, t);
                     }
+                    store_tile(nt - 1);
+                    bulk_wait_all();  // the next chunk reads these rows again
                 }
             }
         }
@@ -398,15 +422,13 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     ++nd;
                     tc_fence_after();
                     {
-                        const int slot = t * kStTile + r;
-                        const unsigned char* th = ring + (size_t)vh * kStTileBytes + hf * kStHalf + r * 128;
-                        const unsigned char* tl = ring + (size_t)vl * kStTileBytes + hf * kStHalf + r * 128;
-                        const size_t grow = ((size_t)u * a.C + slot) * 256 + hf * 128;
+                        unsigned char* th = ring + (size_t)vh * kStTileBytes + hf * kStHalf + r * 128;
+                        unsigned char* tl = ring + (size_t)vl * kStTileBytes + hf * kStHalf + r * 128;
                         float dx[64];
                         tmem_ld64(lane_base + kColD, dx);
                         tc_fence_before();
                         mbar_arrive(dfree);
-                        if (slot < a.C) {
+                        {  // rows past C of a ragged last tile are clipped by the store
 #pragma unroll
                             for (int j = 0; j < 8; ++j) {
                                 const int off = (j ^ sw) * 16;
@@ -417,18 +439,13 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                                 for (int e = 0; e < 8; ++e) nv[e] = (vh8[e] + vl8[e]) + dx[8 * j + e];
                                 uint4 hi, lo;
                                 split8(nv, &hi, &lo);
-                                *reinterpret_cast<uint4*>(a.vhi + grow + j * 16) = hi;
-                                *reinterpret_cast<uint4*>(a.vlo + grow + j * 16) = lo;
+                                *reinterpret_cast<uint4*>(th + off) = hi;  // in place: the producer stores the stage
+                                *reinterpret_cast<uint4*>(tl + off) = lo;
                             }
                         }
                     }
-                    // later chunks read these rows back through TMA: order the stores before the async proxy
-                    asm volatile("fence.proxy.async.global;" ::: "memory");
-                    st_sync();  // every row of the two MV tiles has been read
-                    if (tid == 0) {
-                        mbar_arrive(&empty[vh]);
-                        mbar_arrive(&empty[vl]);
-                    }
+                    fence_proxy_async_smem();
+                    mbar_arrive(wready);
                 }
 
                 // ---- intra-chunk term: row (t, g) sees the writes of tokens s < t (s <= t when the read
