@@ -93,6 +93,23 @@ class ClockSampler:
                 "samples": len(mhz)}
 
 
+def max_over_ranks(values, device):
+    """Element-wise maximum of a list of floats over all ranks of the default process group
+    (the job is as slow as its slowest rank).  Works on any backend; a single process returns its own."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return list(values)
+    t = torch.tensor(list(values), device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def rank_workload(w, rank):
+    """The workload of one rank: the same per-GPU batch (weak scaling; units never interact, so there
+    is no data-path collective), drawn from a rank-specific seed."""
+    return w.scaled(seed=w.seed + 1000 * rank)
+
+
 def algorithmic_bytes_per_step(w: W.Workload) -> int:
     """Bytes the method must move per step: MK once + MV once per unit, plus the step vectors.
     The write-back of the few rows the update rule changes is left out (a conservative count)."""
@@ -268,7 +285,7 @@ def main():
     B.load()
 
     # per-rank workload: the same per-GPU batch on every rank (weak scaling), a different seed per rank
-    wr = w.scaled(seed=w.seed + 1000 * rank)
+    wr = rank_workload(w, rank)
     mk, mv = W.initial_cache(wr, dev)
     cache = B.Cache(w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.capacity, w.torch_dtype,
                     read_scale=w.read_scale, write_scale=w.write_scale, init_len=w.init_len, mk_init=mk, mv_init=mv,
@@ -346,9 +363,7 @@ def main():
     d2h = hout[0].numel() * hout[0].element_size()
 
     if world > 1:
-        t = torch.tensor([ms_total, ms_e2e], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total, ms_e2e = t.tolist()
+        ms_total, ms_e2e = max_over_ranks([ms_total, ms_e2e], dev)
 
     if rank == 0:
         peak, peak_kind = _peaks()
