@@ -57,6 +57,8 @@ def test_small_shapes_match_oracle(dtype, d, G, C, init_len, steps):
     (2, 3, 2500, 2500, 5),     # cluster of 2, ragged
     (40, 4, 300, 290, 14),     # more units than one pass of the persistent grid
     (1, 1, 16384, 16384, 3),   # cluster of 8, full slices
+    (2, 2, 2500, 2490, 14),    # cluster of 2, fill finishes inside the second CTA's slice
+    (1, 1, 4200, 2040, 12),    # cluster of 4, the appended slot crosses from one CTA's slice to the next
     (80, 1, 128, 0, 5),        # starts empty with more units than SMs: several tile-less units per CTA
 ])
 def test_tensor_core_and_cuda_core_kernels_match_oracle(cores, B_, G, C, init_len, steps):
