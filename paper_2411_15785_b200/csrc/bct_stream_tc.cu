@@ -45,8 +45,6 @@ constexpr int kColD = 256;    // MV increment of one tile [slot] x [d]; buffer 1
 constexpr int kColA = 384;    // A = Pr WW^T  [row (t,g)] x [write token]
 
 struct StArgs {
-    char* vhi;
-    char* vlo;
     char* out;
     int* status;
     int C, Hq, Hkv, U, T, t_begin, n_chunks, Tc;
@@ -587,8 +585,6 @@ int launch_stream_tc(const bct_cache* c, const void* q, const void* k, const voi
         return -1;
     }
     StArgs a;
-    a.vhi = c->vhi;
-    a.vlo = c->vlo;
     a.out = static_cast<char*>(out);
     a.status = c->status;
     a.C = p.capacity;
