@@ -35,14 +35,14 @@ constexpr int kSThreads = 128;
 constexpr int kTileRows = 128;
 constexpr int kHalfBytes = 128 * 128;          // 64 columns (128 bytes) x 128 rows
 constexpr int kTcTileBytes = 2 * kHalfBytes;   // one 128 x 128 bfloat16 tile
-constexpr int kMaxTiles = 16;                  // a CTA's slice holds at most 2048 slots
+constexpr int kMaxTiles = 16;                  // tiles per sub-slice: score tiles resident in tensor memory
+constexpr int kMaxSliceRows = 8192;            // slots per CTA: up to 4 sub-slices of 2048, streamed one after the other
 constexpr int kPTileBytes = 2048;              // P operand of one tile: 2 halves x (8 rows x 128 B)
 constexpr int kQBufBytes = 3072;               // Q operand (2 halves x 8 rows x 128 B) + 1 KiB of zeros
 constexpr int kScoreCols = 16;                 // tensor-memory columns per score tile (N = 16)
 constexpr int kOCol = kMaxTiles * kScoreCols;  // output accumulator behind the score tiles
 constexpr int kTmemCols = 512;
 constexpr int kMaxClusterTc = 8;
-constexpr int kLoCap = 80;                     // rewritten rows staged per round (more rows: more rounds)
 constexpr float kNegBigTc = -3.0e38f;
 
 struct TcArgs {
@@ -56,7 +56,7 @@ struct TcArgs {
     int* status;
     long long q_bs;
     long long kv_bs;
-    int C, len, slice_rows, S, Hkv, U, stages;
+    int C, len, slice_rows, S, Hkv, U, stages, lo_cap;  // lo_cap: rewritten rows staged per round
     int do_write, wtr, dense, out_f32;
     float read_scale, write_scale, write_eps;
 };
@@ -64,7 +64,8 @@ struct TcArgs {
 struct TcSmem {
     int ring, pbuf, qbuf, wsm, list, lostage, red, stat, wstat, merge, bars, total;
 };
-__host__ __device__ inline TcSmem tc_smem(int stages, int G, int S) {
+__host__ __device__ inline TcSmem tc_smem(int stages, int G, int S, int slice_rows, int lo_cap) {
+    const int rows = (slice_rows + kTileRows - 1) / kTileRows * kTileRows;
     TcSmem L;
     int off = 0;
     L.ring = off;
@@ -74,22 +75,23 @@ __host__ __device__ inline TcSmem tc_smem(int stages, int G, int S) {
     L.qbuf = off;
     off += 2 * kQBufBytes;
     L.wsm = off;
-    off += kMaxTiles * kTileRows * 4;
+    off += rows * 4;  // scaled write score of every slot of the slice
     L.list = off;     // slots the update rule rewrites this token, in no particular order
-    off += kMaxTiles * kTileRows * 2;
-    L.lostage = off;  // staged copies of up to kLoCap of those rows: value plane rows, then residual rows
-    off += 2 * kLoCap * 256;
+    off += rows * 2;
+    off = (off + 15) & ~15;
+    L.lostage = off;  // staged copies of up to lo_cap of those rows: value plane rows, then residual rows
+    off += 2 * lo_cap * 256;
     L.red = off;
     off += 4 * 16 * 4;
     L.stat = off;  // m[8], l[8], wd[8], ev[8], abort, tmem address
-    off += 4 * 8 * 4 + 16;
+    off += 256;
     L.wstat = off;
     off += 2 * kMaxClusterTc * 2 * 4;
     L.merge = off;
     off += (S > 1) ? 2 * (S - 1) * G * (128 + 3) * 4 : 0;
     off = (off + 15) & ~15;
     L.bars = off;
-    off += (2 * stages + 2 * kMaxTiles + 2 + 1 + 2 + 2) * 8;
+    off += (2 * stages + 2 * kMaxTiles + 2 + 1 + 2 + 2 + 1) * 8;
     L.total = ((off + 127) & ~127) + 1024;  // + slack to align the ring to 1024 bytes
     return L;
 }
@@ -105,7 +107,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int S = a.S;
     const int NST = a.stages;
-    const TcSmem L = tc_smem(NST, G, S);
+    const int kLoCap = a.lo_cap;
+    const TcSmem L = tc_smem(NST, G, S, a.slice_rows, kLoCap);
     unsigned char* ring = smem + L.ring;
     unsigned char* pbuf = smem + L.pbuf;
     unsigned char* qbuf = smem + L.qbuf;
@@ -121,6 +124,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     volatile int* abort_flag = reinterpret_cast<volatile int*>(st_m + 32);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(st_m + 33);
     int* lo_count = reinterpret_cast<int*>(st_m + 34);
+    float* st_alpha = st_m + 36;  // per head: exp(old maximum - new maximum) of the current sub-slice
     float* wstat = reinterpret_cast<float*>(smem + L.wstat);
     float* merge = reinterpret_cast<float*>(smem + L.merge);
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + L.bars);
@@ -131,6 +135,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     uint64_t* oready = qready + 2;
     uint64_t* xbar = oready + 1;            // [2]
     uint64_t* mbar = xbar + 2;              // [2]
+    uint64_t* subfree = mbar + 2;           // the score tiles of a sub-slice have been consumed (128 arrivals)
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
@@ -143,7 +148,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     const int n_slice = max(0, min(a.slice_rows, a.C - slice_start));
     const int n_stream = max(0, min(a.len - slice_start, n_slice));
     const bool has_virtual = (a.len < a.C) && (a.len >= slice_start) && (a.len < slice_start + n_slice);
-    const int nt = (n_stream + kTileRows - 1) / kTileRows;
+    const int nt = (n_stream + kTileRows - 1) / kTileRows;   // tiles of the slice
+    const int n_sub = (nt + kMaxTiles - 1) / kMaxTiles;       // sub-slices of up to kMaxTiles tiles
 
     if (tid == 0) {
         for (int i = 0; i < NST; ++i) {
@@ -157,6 +163,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         mbar_init(&qready[0], kSThreads);
         mbar_init(&qready[1], kSThreads);
         mbar_init(oready, 1);
+        mbar_init(subfree, kSThreads);
         mbar_init(&xbar[0], S);
         mbar_init(&xbar[1], S);
         mbar_init(&mbar[0], kSThreads * (S > 1 ? S - 1 : 1));
@@ -187,9 +194,10 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             uint32_t kc = 0;
             bool ok = true;
             for (int u = cid; u < a.U && ok; u += ncl) {
-                for (int ph = 0; ph < 2 && ok; ++ph) {
-                    const CUtensorMap* map = ph == 0 ? &tmK : &tmV;
-                    for (int t = 0; t < nt; ++t, ++kc) {
+                for (int ph = 0; ph < 2 * n_sub && ok; ++ph) {  // per sub-slice: its MK tiles, then its MV tiles
+                    const CUtensorMap* map = (ph & 1) == 0 ? &tmK : &tmV;
+                    const int t_begin = (ph >> 1) * kMaxTiles, t_end = min(nt, t_begin + kMaxTiles);
+                    for (int t = t_begin; t < t_end; ++t, ++kc) {
                         const int stage = kc % NST;
                         if (kc >= (uint32_t)NST &&
                             !mbar_wait(&empty[stage], ((kc / NST) - 1) & 1, *abort_flag ? 1024u : kWaitLimit)) {
@@ -212,7 +220,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         if (lane == 0) {
             constexpr uint32_t idesc_s = instr_desc(false);
             constexpr uint32_t idesc_o = instr_desc(true);
-            uint32_t kc = 0;
+            uint32_t kc = 0, sp = 0, nsf = 0;  // ring position, sub-slices so far, sub-slice hand-overs so far
             int it = 0;
             for (int u = cid; u < a.U; u += ncl, ++it) {
                 if (!mbar_wait(&qready[it & 1], (it >> 1) & 1, *abort_flag ? 1024u : kWaitLimit)) {
@@ -221,47 +229,56 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 }
                 tc_fence_after();
                 const uint32_t qaddr = smem_u32(qbuf + (it & 1) * kQBufBytes);
-                for (int t = 0; t < nt; ++t, ++kc) {  // scores: A = K tile (K-major), B = Q (K-major)
-                    const int stage = kc % NST;
-                    if (!mbar_wait(&full[stage], (kc / NST) & 1, *abort_flag ? 1024u : kWaitLimit)) {
-                        report_timeout(a.status, 13);
-                        *abort_flag = 1;
+                for (int sub = 0; sub < n_sub; ++sub, ++sp) {
+                    const int t_begin = sub * kMaxTiles, t_end = min(nt, t_begin + kMaxTiles);
+                    if (sub > 0) {  // the previous sub-slice's score tiles must have been consumed
+                        if (!mbar_wait(subfree, nsf & 1, *abort_flag ? 1024u : kWaitLimit)) {
+                            report_timeout(a.status, 22);
+                            *abort_flag = 1;
+                        }
+                        ++nsf;
+                        tc_fence_after();
                     }
-                    tc_fence_after();
-                    const uint32_t taddr = smem_u32(ring + (size_t)stage * kTcTileBytes);
+                    for (int t = t_begin; t < t_end; ++t, ++kc) {  // scores: A = K tile (K-major), B = Q (K-major)
+                        const int stage = kc % NST;
+                        if (!mbar_wait(&full[stage], (kc / NST) & 1, *abort_flag ? 1024u : kWaitLimit)) {
+                            report_timeout(a.status, 13);
+                            *abort_flag = 1;
+                        }
+                        tc_fence_after();
+                        const uint32_t taddr = smem_u32(ring + (size_t)stage * kTcTileBytes);
 #pragma unroll
-                    for (int kk = 0; kk < 8; ++kk) {
-                        const uint64_t ad = smem_desc(taddr + (kk >> 2) * kHalfBytes + (kk & 3) * 32, 16, 1024);
-                        const uint64_t bd = smem_desc(qaddr + (kk >> 2) * 1024 + (kk & 3) * 32, 16, 1024);
-                        umma_bf16(tmem_base + t * kScoreCols, ad, bd, idesc_s, kk > 0);
+                        for (int kk = 0; kk < 8; ++kk) {
+                            const uint64_t ad = smem_desc(taddr + (kk >> 2) * kHalfBytes + (kk & 3) * 32, 16, 1024);
+                            const uint64_t bd = smem_desc(qaddr + (kk >> 2) * 1024 + (kk & 3) * 32, 16, 1024);
+                            umma_bf16(tmem_base + (t - t_begin) * kScoreCols, ad, bd, idesc_s, kk > 0);
+                        }
+                        umma_commit(&sready[t - t_begin]);
+                        umma_commit(&empty[stage]);
                     }
-                    umma_commit(&sready[t]);
-                    umma_commit(&empty[stage]);
-                }
-                for (int t = 0; t < nt; ++t, ++kc) {  // outputs: A = V tile (MN-major), B = P (K-major)
-                    const int stage = kc % NST;
-                    if (!mbar_wait(&pready[t], it & 1, *abort_flag ? 1024u : kWaitLimit)) {
-                        report_timeout(a.status, 14);
-                        *abort_flag = 1;
-                    }
-                    if (!mbar_wait(&full[stage], (kc / NST) & 1, *abort_flag ? 1024u : kWaitLimit)) {
-                        report_timeout(a.status, 15);
-                        *abort_flag = 1;
-                    }
-                    tc_fence_after();
-                    const uint32_t taddr = smem_u32(ring + (size_t)stage * kTcTileBytes);
-                    const uint32_t paddr = smem_u32(pbuf + t * kPTileBytes);
+                    for (int t = t_begin; t < t_end; ++t, ++kc) {  // outputs: A = V tile (MN-major), B = P (K-major)
+                        const int stage = kc % NST;
+                        if (!mbar_wait(&pready[t - t_begin], sp & 1, *abort_flag ? 1024u : kWaitLimit)) {
+                            report_timeout(a.status, 14);
+                            *abort_flag = 1;
+                        }
+                        if (!mbar_wait(&full[stage], (kc / NST) & 1, *abort_flag ? 1024u : kWaitLimit)) {
+                            report_timeout(a.status, 15);
+                            *abort_flag = 1;
+                        }
+                        tc_fence_after();
+                        const uint32_t taddr = smem_u32(ring + (size_t)stage * kTcTileBytes);
+                        const uint32_t paddr = smem_u32(pbuf + (t - t_begin) * kPTileBytes);
 #pragma unroll
-                    for (int kk = 0; kk < 8; ++kk) {  // 16 slots per step
-                        const uint64_t ad = smem_desc(taddr + kk * 2048, kHalfBytes, 1024);
-                        const uint64_t bd = smem_desc(paddr + (kk >> 2) * 1024 + (kk & 3) * 32, 16, 1024);
-                        umma_bf16(tmem_base + kOCol, ad, bd, idesc_o, (t > 0) || (kk > 0));
+                        for (int kk = 0; kk < 8; ++kk) {  // 16 slots per step
+                            const uint64_t ad = smem_desc(taddr + kk * 2048, kHalfBytes, 1024);
+                            const uint64_t bd = smem_desc(paddr + (kk >> 2) * 1024 + (kk & 3) * 32, 16, 1024);
+                            umma_bf16(tmem_base + kOCol, ad, bd, idesc_o, (t > 0) || (kk > 0));
+                        }
+                        umma_commit(&empty[stage]);
                     }
-                    umma_commit(&empty[stage]);
+                    umma_commit(oready);  // every V tile of the sub-slice has been read
                 }
-                // (with no tile at all nothing is committed: the commit would complete at once, and a
-                // second one could follow before the first is observed)
-                if (nt > 0) umma_commit(oready);  // every V tile of the unit has been read
             }
         }
         __syncwarp();
@@ -289,6 +306,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         if (cid < a.U) write_q(cid, 0);
 
         int it = 0;
+        uint32_t sp = 0;  // sub-slices processed so far (phase of the per-tile barriers)
+        const int n_sub_rows = max(n_sub, 1);  // a unit with no tile still has its appended slot to look after
         for (int u = cid; u < a.U; u += ncl, ++it) {
             const int b = u / a.Hkv;
             const int h_kv = u - b * a.Hkv;
@@ -296,23 +315,6 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             const size_t kv_off = ((size_t)b * a.kv_bs + (size_t)h_kv * D) * 2;
             const size_t unit_off = (size_t)u * a.C * ROW_BYTES;
 
-            // ---- pass 1: row maxima of the raw scores, as the score tiles complete ----
-            float mx[8];
-#pragma unroll
-            for (int h = 0; h < 8; ++h) mx[h] = kNegBigTc;
-            for (int t = 0; t < nt; ++t) {
-                if (!mbar_wait(&sready[t], it & 1, *abort_flag ? 1024u : kWaitLimit)) {
-                    report_timeout(a.status, 16);
-                    *abort_flag = 1;
-                }
-                tc_fence_after();
-                float s[8];
-                tmem_ld8(lane_base + t * kScoreCols, s);
-                if (t * kTileRows + r < n_stream) {
-#pragma unroll
-                    for (int h = 0; h < 8; ++h) mx[h] = fmaxf(mx[h], s[h]);
-                }
-            }
             // the appended slot (fill phase) is scored from the step vectors
             float vq[G];
             const float kd = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(a.k + kv_off)[r]);
@@ -325,81 +327,135 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     vq[g] = warp_sum(qd * kd);
                 }
             }
-#pragma unroll
-            for (int h = 0; h < 8; ++h) {
-                mx[h] = warp_max(mx[h]);
-                if (lane == 0) red[warp * 16 + h] = mx[h];
-                if (lane == 0 && h < G) red[warp * 16 + 8 + h] = vq[h];
+            if (tid < 8) {  // running maximum, sum and read-write overlap of the unit, over its sub-slices
+                st_m[tid] = kNegBigTc;
+                st_l[tid] = 0.f;
+                st_wd[tid] = 0.f;
             }
-            s_sync();
-            if (tid < 8) {
-                const float scale = (tid < G) ? a.read_scale : a.write_scale;
-                float m = fmaxf(fmaxf(red[tid], red[16 + tid]), fmaxf(red[32 + tid], red[48 + tid]));
-                m = (m <= kNegBigTc) ? kNegBigTc : m * scale;
-                if (has_virtual && tid < G) {
-                    const float vs = (red[8 + tid] + red[24 + tid] + red[40 + tid] + red[56 + tid]) * a.read_scale;
-                    st_ev[tid] = vs;  // scaled score of the appended slot, turned into a numerator below
-                    m = fmaxf(m, vs);
-                }
-                st_m[tid] = m;
-            }
-            s_sync();
 
-            // ---- pass 2: numerators, row sums, P operand (bfloat16, swizzled), write numerators ----
-            float sum[8];
-            float wdacc[G];
+            // A slice longer than the tensor memory can score at once is taken in sub-slices of up to
+            // kMaxTiles tiles; maxima, sums and the output accumulator are rescaled from one to the next.
+            for (int sub = 0; sub < n_sub_rows; ++sub, ++sp) {
+                const int t_begin = sub * kMaxTiles, t_end = min(nt, t_begin + kMaxTiles);
+                const bool last_sub = (sub == n_sub_rows - 1);
+
+                // ---- pass 1: row maxima of the raw scores, as the score tiles complete ----
+                float mx[8];
 #pragma unroll
-            for (int h = 0; h < 8; ++h) sum[h] = 0.f;
+                for (int h = 0; h < 8; ++h) mx[h] = kNegBigTc;
+                for (int t = t_begin; t < t_end; ++t) {
+                    if (!mbar_wait(&sready[t - t_begin], sp & 1, *abort_flag ? 1024u : kWaitLimit)) {
+                        report_timeout(a.status, 16);
+                        *abort_flag = 1;
+                    }
+                    tc_fence_after();
+                    float s[8];
+                    tmem_ld8(lane_base + (t - t_begin) * kScoreCols, s);
+                    if (t * kTileRows + r < n_stream) {
 #pragma unroll
-            for (int g = 0; g < G; ++g) wdacc[g] = 0.f;
-            for (int t = 0; t < nt; ++t) {
-                float s[8];
-                tmem_ld8(lane_base + t * kScoreCols, s);
-                const bool valid = t * kTileRows + r < n_stream;
-                float e[8];
+                        for (int h = 0; h < 8; ++h) mx[h] = fmaxf(mx[h], s[h]);
+                    }
+                }
 #pragma unroll
                 for (int h = 0; h < 8; ++h) {
-                    const float scale = (h < G) ? a.read_scale : a.write_scale;
-                    e[h] = (valid && h <= G) ? __expf(s[h] * scale - st_m[h]) : 0.f;
-                    sum[h] += e[h];
+                    mx[h] = warp_max(mx[h]);
+                    if (lane == 0) red[warp * 16 + h] = mx[h];
+                    if (lane == 0 && h < G) red[warp * 16 + 8 + h] = vq[h];
                 }
-                unsigned char* prow = pbuf + t * kPTileBytes + (r >> 6) * 1024 + (r & 7) * 2;
-                const int c8 = (r & 63) >> 3;
+                s_sync();
+                if (tid < 8) {
+                    const float scale = (tid < G) ? a.read_scale : a.write_scale;
+                    float m = fmaxf(fmaxf(red[tid], red[16 + tid]), fmaxf(red[32 + tid], red[48 + tid]));
+                    m = (m <= kNegBigTc) ? kNegBigTc : m * scale;
+                    if (last_sub && has_virtual && tid < G) {
+                        const float vs = (red[8 + tid] + red[24 + tid] + red[40 + tid] + red[56 + tid]) * a.read_scale;
+                        st_ev[tid] = vs;  // scaled score of the appended slot, turned into a numerator below
+                        m = fmaxf(m, vs);
+                    }
+                    const float m_old = st_m[tid];
+                    const float m_new = fmaxf(m_old, m);
+                    st_alpha[tid] = (m_old <= kNegBigTc) ? 0.f : __expf(m_old - m_new);
+                    st_m[tid] = m_new;
+                }
+                s_sync();
+
+                // ---- the outputs accumulated so far refer to the old maxima: rescale them in tensor memory ----
+                if (sub > 0) {
+                    if (!mbar_wait(oready, (sp - 1) & 1, *abort_flag ? 1024u : kWaitLimit)) {
+                        report_timeout(a.status, 23);
+                        *abort_flag = 1;
+                    }
+                    tc_fence_after();
+                    float o[8];
+                    tmem_ld8(lane_base + kOCol, o);
 #pragma unroll
-                for (int h = 0; h < G; ++h)  // rows G..7 of the operand stay zero
-                    *reinterpret_cast<__nv_bfloat16*>(prow + h * 128 + ((c8 ^ h) * 16)) = __float2bfloat16_rn(e[h]);
-                wsm[t * kTileRows + r] = e[G];
+                    for (int h = 0; h < 8; ++h) o[h] *= st_alpha[h];
+                    tmem_st8(lane_base + kOCol, o);
+                    tc_fence_before();
+                }
+
+                // ---- pass 2: numerators, row sums, P operand (bfloat16, swizzled), scaled write scores ----
+                float sum[8];
+                float wdacc[G];
 #pragma unroll
-                for (int g = 0; g < G; ++g) wdacc[g] = fmaf(e[g], e[G], wdacc[g]);
-                fence_proxy_async_smem();
-                tc_fence_before();
-                mbar_arrive(&pready[t]);  // the V tile's MMAs may go as soon as its weights are in place
-            }
-            // the next unit's scores may start as soon as this unit's V tiles are through
-            if (u + ncl < a.U) write_q(u + ncl, (it + 1) & 1);
+                for (int h = 0; h < 8; ++h) sum[h] = 0.f;
+#pragma unroll
+                for (int g = 0; g < G; ++g) wdacc[g] = 0.f;
+                for (int t = t_begin; t < t_end; ++t) {
+                    float s[8];
+                    tmem_ld8(lane_base + (t - t_begin) * kScoreCols, s);
+                    const bool valid = t * kTileRows + r < n_stream;
+                    float e[8];
+#pragma unroll
+                    for (int h = 0; h < 8; ++h) {
+                        const float scale = (h < G) ? a.read_scale : a.write_scale;
+                        e[h] = (valid && h <= G) ? __expf(s[h] * scale - st_m[h]) : 0.f;
+                        sum[h] += e[h];
+                    }
+                    unsigned char* prow = pbuf + (t - t_begin) * kPTileBytes + (r >> 6) * 1024 + (r & 7) * 2;
+                    const int c8 = (r & 63) >> 3;
+#pragma unroll
+                    for (int h = 0; h < G; ++h)  // rows G..7 of the operand stay zero
+                        *reinterpret_cast<__nv_bfloat16*>(prow + h * 128 + ((c8 ^ h) * 16)) = __float2bfloat16_rn(e[h]);
+                    wsm[t * kTileRows + r] = valid ? s[G] * a.write_scale : kNegBigTc;
+#pragma unroll
+                    for (int g = 0; g < G; ++g) wdacc[g] = fmaf(e[g], e[G], wdacc[g]);
+                    fence_proxy_async_smem();
+                    tc_fence_before();
+                    mbar_arrive(&pready[t - t_begin]);  // the V tile's MMAs may go as soon as its weights are in place
+                }
+                if (last_sub) {
+                    // the next unit's scores may start as soon as this unit's V tiles are through
+                    if (u + ncl < a.U) write_q(u + ncl, (it + 1) & 1);
+                } else {
+                    tc_fence_before();
+                    mbar_arrive(subfree);  // this sub-slice's score tiles may be overwritten
+                }
 
 #pragma unroll
-            for (int h = 0; h < 8; ++h) {
-                sum[h] = warp_sum(sum[h]);
-                if (lane == 0) red[warp * 16 + h] = sum[h];
-            }
-#pragma unroll
-            for (int g = 0; g < G; ++g) {
-                wdacc[g] = warp_sum(wdacc[g]);
-                if (lane == 0) red[warp * 16 + 8 + g] = wdacc[g];
-            }
-            s_sync();
-            if (tid < 8) {
-                float l = red[tid] + red[16 + tid] + red[32 + tid] + red[48 + tid];
-                if (has_virtual && tid < G) {
-                    const float ev = __expf(st_ev[tid] - st_m[tid]);
-                    st_ev[tid] = ev;
-                    l += ev;
+                for (int h = 0; h < 8; ++h) {
+                    sum[h] = warp_sum(sum[h]);
+                    if (lane == 0) red[warp * 16 + h] = sum[h];
                 }
-                st_l[tid] = l;
-                st_wd[tid] = red[8 + tid] + red[24 + tid] + red[40 + tid] + red[56 + tid];
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    wdacc[g] = warp_sum(wdacc[g]);
+                    if (lane == 0) red[warp * 16 + 8 + g] = wdacc[g];
+                }
+                s_sync();
+                if (tid < 8) {
+                    float l = red[tid] + red[16 + tid] + red[32 + tid] + red[48 + tid];
+                    if (last_sub && has_virtual && tid < G) {
+                        const float ev = __expf(st_ev[tid] - st_m[tid]);
+                        st_ev[tid] = ev;
+                        l += ev;
+                    }
+                    st_l[tid] = st_l[tid] * st_alpha[tid] + l;
+                    st_wd[tid] = st_wd[tid] * st_alpha[tid] * st_alpha[G] +
+                                 (red[8 + tid] + red[24 + tid] + red[40 + tid] + red[56 + tid]);
+                }
+                s_sync();
             }
-            s_sync();
 
             // ---- write weights are normalised over ALL C slots: exchange across the cluster ----
             float wfac = 0.f;
@@ -443,7 +499,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             if (a.do_write) {
                 for (int t = 0; t < nt; ++t) {
                     const int row = t * kTileRows + r;
-                    if (row < n_stream && (a.dense || wsm[row] * wfac >= a.write_eps))
+                    if (row < n_stream && (a.dense || __expf(wsm[row] - st_m[G]) * wfac >= a.write_eps))
                         list[atomicAdd(lo_count, 1)] = (unsigned short)row;
                 }
                 s_sync();
@@ -452,7 +508,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             }
 
             // ---- epilogue: O[d][g] from tensor memory once every V tile has been read ----
-            if (nt > 0 && !mbar_wait(oready, it & 1, *abort_flag ? 1024u : kWaitLimit)) {
+            if (nt > 0 && !mbar_wait(oready, (sp - 1) & 1, *abort_flag ? 1024u : kWaitLimit)) {
                 report_timeout(a.status, 19);
                 *abort_flag = 1;
             }
@@ -541,7 +597,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     s_sync();  // every thread's staged chunks have landed
                     for (int i = tid >> 4; i < n; i += kSThreads / 16) {
                         const int row = list[base + i];
-                        const float ww = wsm[row] * wfac;
+                        const float ww = __expf(wsm[row] - st_m[G]) * wfac;
                         const size_t goff = unit_off + (size_t)(slice_start + row) * ROW_BYTES + c16 * 16;
                         float x[8], lo[8], nv[8], hf[8];
                         Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(histage + i * ROW_BYTES + c16 * 16), x);
@@ -633,7 +689,7 @@ bool tc_eligible(const bct_cache* c) {
     const bct_params_t& p = c->p;
     if (p.dtype != BCT_BF16 || p.head_dim != 128 || c->G > 7) return false;
     if (p.flags & BCT_FLAG_PRECISE_READ) return false;
-    if (p.capacity < kTileRows || p.capacity > kMaxClusterTc * kMaxTiles * kTileRows) return false;
+    if (p.capacity < kTileRows || p.capacity > kMaxClusterTc * kMaxSliceRows) return false;
     if (c->plane_bytes < (size_t)1 << 18) return false;  // tiny planes stay on the CUDA-core kernel
     return c->tc_ready != 0;
 }
@@ -657,9 +713,13 @@ int launch_decode_tc(const bct_cache* c, const StepIO& io, int len, int do_write
         *err = cudaErrorInvalidConfiguration;
         return -1;
     }
-    const int max_slice = kMaxTiles * kTileRows;
+    // Cluster size: clusters of 2 tile the whole chip (74 x 2 = 148 SMs), clusters of 4 and 8 only 132
+    // and 120 SMs, so a unit is split over at most 2 CTAs and a long slice is taken in sub-slices
+    // (up to kMaxSliceRows slots per CTA).  Only when there are too few units to fill the SMs is a unit
+    // spread wider.
     int S = 1;
-    while (S < kMaxClusterTc && (p.capacity + S - 1) / S > max_slice) S *= 2;
+    if (p.capacity > kMaxTiles * kTileRows) S = 2;
+    while (S < kMaxClusterTc && (p.capacity + S - 1) / S > kMaxSliceRows) S *= 2;
     while (S < kMaxClusterTc && (long long)c->U * S * 2 <= c->sm_count && (p.capacity + 2 * S - 1) / (2 * S) >= kTileRows)
         S *= 2;  // few units: spread each over more SMs
     int slice = (p.capacity + S - 1) / S;
@@ -669,8 +729,18 @@ int launch_decode_tc(const bct_cache* c, const StepIO& io, int len, int do_write
         const int v = atoi(e);
         if (v >= 2 && v <= 5) stages = v;
     }
-    while (stages > 2 && tc_smem(stages, c->G, S).total > c->smem_optin) --stages;
-    const int smem = tc_smem(stages, c->G, S).total;
+    int lo_cap = 80;
+    while (tc_smem(stages, c->G, S, slice, lo_cap).total > c->smem_optin && (stages > 3 || lo_cap > 32)) {
+        if (stages > 3)
+            --stages;
+        else
+            lo_cap -= 16;
+    }
+    const int smem = tc_smem(stages, c->G, S, slice, lo_cap).total;
+    if (smem > c->smem_optin) {
+        *err = cudaErrorInvalidConfiguration;
+        return -1;
+    }
 
     TcArgs a;
     a.vhi = c->vhi;
@@ -690,6 +760,7 @@ int launch_decode_tc(const bct_cache* c, const StepIO& io, int len, int do_write
     a.Hkv = p.n_kv_heads;
     a.U = c->U;
     a.stages = stages;
+    a.lo_cap = lo_cap;
     a.do_write = (len == p.capacity) && do_write;
     a.wtr = (p.flags & BCT_FLAG_WRITE_THEN_READ) ? 1 : 0;
     a.dense = (p.flags & BCT_FLAG_DENSE_WRITE) ? 1 : 0;

@@ -59,6 +59,9 @@ def test_small_shapes_match_oracle(dtype, d, G, C, init_len, steps):
     (1, 1, 16384, 16384, 3),   # cluster of 8, full slices
     (2, 2, 2500, 2490, 14),    # cluster of 2, fill finishes inside the second CTA's slice
     (1, 1, 4200, 2040, 12),    # cluster of 4, the appended slot crosses from one CTA's slice to the next
+    (20, 2, 5000, 5000, 4),    # cluster of 2, each CTA's 2560-slot slice in two sub-slices
+    (20, 1, 16384, 16384, 3),  # cluster of 2, 8192-slot slices in four sub-slices
+    (20, 3, 5000, 4993, 12),   # sub-slices while the cache is still filling
     (80, 1, 128, 0, 5),        # starts empty with more units than SMs: several tile-less units per CTA
 ])
 def test_tensor_core_and_cuda_core_kernels_match_oracle(cores, B_, G, C, init_len, steps):
@@ -73,10 +76,10 @@ def test_tensor_core_and_cuda_core_kernels_match_oracle(cores, B_, G, C, init_le
 
 @pytest.mark.parametrize("flag,oflag", [(B.FLAG_WRITE_THEN_READ, O.WRITE_THEN_READ), (B.FLAG_DENSE_WRITE, 0),
                                         (B.FLAG_OUT_F32, 0)])
-@pytest.mark.parametrize("C", [400, 5000])
-def test_tensor_core_kernel_flags(flag, oflag, C):
+@pytest.mark.parametrize("C,B_", [(400, 2), (5000, 2), (6000, 20)])
+def test_tensor_core_kernel_flags(flag, oflag, C, B_):
     d = 128
-    w = W.Workload("t", 2, 6, 2, d, C, "bf16", C, 6, 17, d ** -0.5, 1.0, 1.0, "decode", 1.0, 0.3)
+    w = W.Workload("t", B_, 6, 2, d, C, "bf16", C, 6, 17, d ** -0.5, 1.0, 1.0, "decode", 1.0, 0.3)
     out_err, state_err = run_decode_parity(w, pick_units(w, 4), flags=flag, oracle_flags=oflag,
                                            expect_tensor_path=True)
     assert out_err <= TOL["bf16"] and state_err <= TOL["bf16"], (out_err, state_err)
