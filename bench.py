@@ -129,13 +129,13 @@ def measured_traffic(w, tensor_path):
     return None if per_unit is None else per_unit * w.units
 
 
-def stream_roofline(w, tok_per_step, ms_step):
+def stream_roofline(w, tok_per_step, ms_step, precise=False):
     """Tensor-core roofline of stream_tc_kernel: the dense flops its MMAs execute per step (operand rows padded
     to M = 128 included) against the measured bf16 matmul peak."""
     Tc = 64 if w.group == 1 else (32 if w.group <= 3 else 16)
     C, d = w.capacity, w.head_dim
     per_chunk = 2 * (2 * 128 * C * d)          # scores of the 128 operand rows, two passes over MK
-    per_chunk += 3 * (2 * 128 * C * d)         # outputs: (P + P_lo) MV_hi + P MV_lo
+    per_chunk += (3 if precise else 1) * (2 * 128 * C * d)   # outputs: P MV_hi (+ P_lo MV_hi + P MV_lo with PRECISE_READ)
     per_chunk += 2 * 128 * C * Tc              # A = P WW^T
     per_chunk += 2 * (2 * C * Tc * d)          # MV increment with value + residual weights
     per_chunk += 2 * 128 * Tc * d              # strict_tril(A) Vc
@@ -372,7 +372,7 @@ def main():
         alg = algorithmic_bytes_per_step(w)
         achieved = alg / (ms_step * 1e-3) / 1e9
         if stream:
-            roof = stream_roofline(w, tok_per_step, ms_step)
+            roof = stream_roofline(w, tok_per_step, ms_step, precise=bool(args.flags & 16))
         else:
             roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                     "traffic": measured_traffic(w, cache.tensor_path), "peak_kind": "of " + peak_kind,

@@ -70,8 +70,10 @@ typedef enum bct_dtype {
 #define BCT_FLAG_WRITE_THEN_READ 2u  /* the token's read sees its own write */
 #define BCT_FLAG_DENSE_WRITE 4u      /* rewrite every slot, whatever its write weight */
 #define BCT_FLAG_PRECISE_READ 16u     /* bfloat16 cache: the read uses MV's value plus its
-                                        residual (one more plane streamed per token); for
-                                        states whose magnitude makes a bfloat16 ulp matter */
+                                        residual (one more plane streamed per token; in the
+                                        chunked stream kernel, value + residual numerators
+                                        as well); for states whose magnitude makes a
+                                        bfloat16 ulp matter */
 #define BCT_FLAG_CUDA_CORES 32u       /* keep every decode step on the CUDA-core kernel (the
                                         tensor-core kernel serves bfloat16, head_dim 128,
                                         G <= 7, C >= 128 by default) */

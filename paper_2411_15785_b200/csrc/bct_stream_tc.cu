@@ -12,9 +12,9 @@
 // One persistent CTA per (sequence, kv-head) unit at a time (C <= 2048 slots); per chunk the cache
 // streams through shared memory twice for MK (row statistics, then numerators) and once for MV
 // (value and residual planes), instead of twice per token, and every product runs as tcgen05.mma
-// with fp32 accumulators in tensor memory.  Numerators and write weights are kept as bfloat16
-// value + residual pairs, and MV is read as value + residual, so a long stream keeps the precision
-// of the per-token path.
+// with fp32 accumulators in tensor memory.  The write weights are always kept as bfloat16
+// value + residual pairs (the state must not drift); with BCT_FLAG_PRECISE_READ the read numerators
+// and MV are too, so that a long stream whose state grows large keeps the output precision.
 //   warp 8  producer : TMA loads (chunk operands, MK / MV tiles through a 3-stage ring)
 //   warp 9  MMA      : issues all tensor-core work, commits to mbarriers
 //   warps 0-7        : two threads per operand row (64 accumulator columns each): online row statistics, numerators, the write-back
@@ -48,7 +48,7 @@ struct StArgs {
     char* out;
     int* status;
     int C, Hq, Hkv, U, T, t_begin, n_chunks, Tc;
-    int wtr, out_f32;
+    int wtr, out_f32, precise;  // precise: the read uses value + residual of both the numerators and MV
     float read_scale, write_scale;
 };
 
@@ -284,9 +284,11 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                             const uint32_t po = (kk >> 2) * kStHalf + (kk & 3) * 32;
                             const uint64_t vhd = smem_desc(vhaddr + kk * 2048, kStHalf, 1024);
                             umma_bf16(tmem_base + kColO, smem_desc(phiaddr + po, 16, 1024), vhd, id_out, (t > 0) || (kk > 0));
-                            umma_bf16(tmem_base + kColO, smem_desc(ploaddr + po, 16, 1024), vhd, id_out, true);
-                            umma_bf16(tmem_base + kColO, smem_desc(phiaddr + po, 16, 1024),
-                                      smem_desc(vladdr + kk * 2048, kStHalf, 1024), id_out, true);
+                            if (a.precise) {
+                                umma_bf16(tmem_base + kColO, smem_desc(ploaddr + po, 16, 1024), vhd, id_out, true);
+                                umma_bf16(tmem_base + kColO, smem_desc(phiaddr + po, 16, 1024),
+                                          smem_desc(vladdr + kk * 2048, kStHalf, 1024), id_out, true);
+                            }
                         }
                         // A += P x WW^T over this tile's slots (write rows start at n_read)
 #pragma unroll
@@ -406,7 +408,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                             split8(x + 8 * j, &hi, &lo);
                             const int off = hf * kStHalf + r * 128 + ((j ^ sw) * 16);
                             *reinterpret_cast<uint4*>(phi + off) = hi;
-                            *reinterpret_cast<uint4*>(plo + off) = lo;
+                            if (is_write || a.precise) *reinterpret_cast<uint4*>(plo + off) = lo;  // write weights always keep it
                         }
                     }
                     fence_proxy_async_smem();
@@ -597,6 +599,7 @@ int launch_stream_tc(const bct_cache* c, const void* q, const void* k, const voi
     a.Tc = Tc;
     a.wtr = (p.flags & BCT_FLAG_WRITE_THEN_READ) ? 1 : 0;
     a.out_f32 = (p.flags & BCT_FLAG_OUT_F32) ? 1 : 0;
+    a.precise = (p.flags & BCT_FLAG_PRECISE_READ) ? 1 : 0;
     a.read_scale = p.read_scale;
     a.write_scale = p.write_scale;
     const int smem = st_smem().total;
