@@ -155,10 +155,12 @@ bct_status_t bct_prefill_stream(bct_cache_t *cache, const void *q, const void *k
 
 /*
  * Host-buffer forms of the two calls above: the same shapes, but q, k, v and out are
- * HOST pointers.  The inputs are copied into the workspace's staging area, the step
- * runs, and out is copied back, all on cuda_stream; the call returns without
- * synchronising, so out is valid once the stream has drained, and q, k, v must stay
- * unchanged until then.  T must not exceed the max_stream given at create.
+ * HOST pointers.  The inputs are copied into the workspace's staging area (two sets, used
+ * alternately, on a copy stream the handle owns, so that one call's copies overlap the
+ * previous call's kernel), the step runs on cuda_stream after them, and out is copied back
+ * on cuda_stream; the call returns without synchronising, so out is valid once cuda_stream
+ * has drained, and q, k, v must stay unchanged until then.  T must not exceed the
+ * max_stream given at create.
  */
 bct_status_t bct_decode_step_host(bct_cache_t *cache, const void *q, const void *k, const void *v,
                                   void *out, void *cuda_stream);

@@ -32,7 +32,7 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 // Offsets of the workspace sections.
 struct Carve {
-    size_t kplane, vhi, vlo, status, stage_q, stage_k, stage_v, stage_out, total;
+    size_t kplane, vhi, vlo, status, stage_q[2], stage_k[2], stage_v[2], stage_out[2], total;
     size_t plane_bytes, q_bytes, kv_bytes, out_bytes;  // staging for max_stream tokens
 };
 
@@ -81,14 +81,16 @@ Carve carve(const bct_params_t& p) {
     off += (p.dtype == BCT_BF16) ? round_up(c.plane_bytes, bct::kAlign) : 0;
     c.status = off;
     off += bct::kAlign;
-    c.stage_q = off;
-    off += round_up(c.q_bytes, bct::kAlign);
-    c.stage_k = off;
-    off += round_up(c.kv_bytes, bct::kAlign);
-    c.stage_v = off;
-    off += round_up(c.kv_bytes, bct::kAlign);
-    c.stage_out = off;
-    off += round_up(c.out_bytes, bct::kAlign);
+    for (int i = 0; i < 2; ++i) {  // two staging sets: one call's copies overlap the previous call's kernel
+        c.stage_q[i] = off;
+        off += round_up(c.q_bytes, bct::kAlign);
+        c.stage_k[i] = off;
+        off += round_up(c.kv_bytes, bct::kAlign);
+        c.stage_v[i] = off;
+        off += round_up(c.kv_bytes, bct::kAlign);
+        c.stage_out[i] = off;
+        off += round_up(c.out_bytes, bct::kAlign);
+    }
     c.total = off;
     return c;
 }
@@ -105,6 +107,16 @@ bct_status_t check_step_ptrs(const void* q, const void* k, const void* v, const 
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out))
         return fail(BCT_ERR_INVALID_ARG, "q, k, v and out must be 16-byte aligned");
     return BCT_OK;
+}
+
+void release_host_objects(bct_cache_t* c) {
+    for (int i = 0; i < 2; ++i) {
+        if (c->ev_in[i]) cudaEventDestroy(c->ev_in[i]);
+        if (c->ev_free[i]) cudaEventDestroy(c->ev_free[i]);
+        c->ev_in[i] = c->ev_free[i] = nullptr;
+    }
+    if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
+    c->copy_stream = nullptr;
 }
 
 // T tokens, one decode launch each.  Pointers are device pointers in [B][T][H][d].
@@ -211,10 +223,16 @@ bct_status_t bct_cache_create(const bct_params_t* params, void* workspace, size_
     c->vhi = c->ws + cv.vhi;
     c->vlo = p.dtype == BCT_BF16 ? c->ws + cv.vlo : nullptr;
     c->status = reinterpret_cast<int*>(c->ws + cv.status);
-    c->stage_q = c->ws + cv.stage_q;
-    c->stage_k = c->ws + cv.stage_k;
-    c->stage_v = c->ws + cv.stage_v;
-    c->stage_out = c->ws + cv.stage_out;
+    for (int i = 0; i < 2; ++i) {
+        c->stage_q[i] = c->ws + cv.stage_q[i];
+        c->stage_k[i] = c->ws + cv.stage_k[i];
+        c->stage_v[i] = c->ws + cv.stage_v[i];
+        c->stage_out[i] = c->ws + cv.stage_out[i];
+        c->ev_in[i] = nullptr;
+        c->ev_free[i] = nullptr;
+    }
+    c->copy_stream = nullptr;
+    c->host_calls = 0;
     c->len = p.init_len;
     c->n_full_tokens = 0;
     c->launches = 0;
@@ -222,12 +240,25 @@ bct_status_t bct_cache_create(const bct_params_t* params, void* workspace, size_
     c->sm_count = sms;
     c->smem_optin = optin;
 
+    // a stream and four events of the handle's own (host objects: no device memory)
+    e = cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking);
+    for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
+        e = cudaEventCreateWithFlags(&c->ev_in[i], cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_free[i], cudaEventDisableTiming);
+    }
+    if (e != cudaSuccess) {
+        release_host_objects(c);
+        c->magic = 0;
+        delete c;
+        return fail_cuda("stream / event creation", e);
+    }
     bct::tc_prepare(c);  // tensor maps of the planes; without them the CUDA-core kernel serves every shape
 
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     e = cudaMemsetAsync(c->status, 0, bct::kAlign, stream);
     if (e == cudaSuccess) e = bct::launch_import(c, mk_init, mv_init, p.dtype, p.init_len, stream);
     if (e != cudaSuccess) {
+        release_host_objects(c);
         c->magic = 0;
         delete c;
         return fail_cuda("state import", e);
@@ -269,17 +300,26 @@ bct_status_t bct_prefill_stream_host(bct_cache_t* c, const void* q, const void* 
     const size_t eb = (size_t)c->elem_bytes;
     const size_t qb = (size_t)c->p.batch * T * c->p.n_q_heads * c->p.head_dim * eb;
     const size_t kb = (size_t)c->p.batch * T * c->p.n_kv_heads * c->p.head_dim * eb;
-    cudaError_t e = cudaMemcpyAsync(c->stage_q, q, qb, cudaMemcpyHostToDevice, stream);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(c->stage_k, k, kb, cudaMemcpyHostToDevice, stream);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(c->stage_v, v, kb, cudaMemcpyHostToDevice, stream);
+    // The inputs go up on the handle's copy stream into the staging set that is not in use, so that
+    // they overlap the previous call's kernel; the step itself and the copy of `out` run on `stream`.
+    const int set = (int)(c->host_calls & 1);
+    cudaError_t e = cudaStreamWaitEvent(c->copy_stream, c->ev_free[set], 0);  // the set's last user is done
+    if (e == cudaSuccess) e = cudaMemcpyAsync(c->stage_q[set], q, qb, cudaMemcpyHostToDevice, c->copy_stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(c->stage_k[set], k, kb, cudaMemcpyHostToDevice, c->copy_stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(c->stage_v[set], v, kb, cudaMemcpyHostToDevice, c->copy_stream);
+    if (e == cudaSuccess) e = cudaEventRecord(c->ev_in[set], c->copy_stream);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, c->ev_in[set], 0);
     if (e != cudaSuccess) return fail_cuda("host-to-device copy", e);
-    st = run_tokens(c, c->stage_q, c->stage_k, c->stage_v, out ? c->stage_out : nullptr, T, stream);
+    c->host_calls += 1;
+    st = run_tokens(c, c->stage_q[set], c->stage_k[set], c->stage_v[set], out ? c->stage_out[set] : nullptr, T, stream);
     if (st != BCT_OK) return st;
     if (out != nullptr) {
         const size_t ob = (c->p.flags & BCT_FLAG_OUT_F32) ? qb / eb * 4 : qb;
-        e = cudaMemcpyAsync(out, c->stage_out, ob, cudaMemcpyDeviceToHost, stream);
+        e = cudaMemcpyAsync(out, c->stage_out[set], ob, cudaMemcpyDeviceToHost, stream);
         if (e != cudaSuccess) return fail_cuda("device-to-host copy", e);
     }
+    e = cudaEventRecord(c->ev_free[set], stream);
+    if (e != cudaSuccess) return fail_cuda("event record", e);
     return BCT_OK;
 }
 
@@ -363,6 +403,7 @@ bct_status_t bct_cache_launches(const bct_cache_t* c, int64_t* launches) {
 bct_status_t bct_cache_destroy(bct_cache_t* c) {
     if (c == nullptr) return BCT_OK;
     if (c->magic != bct::kMagic) return fail(BCT_ERR_STATE, "cache handle is destroyed or corrupted");
+    release_host_objects(c);
     c->magic = 0;
     delete c;
     return BCT_OK;

@@ -37,10 +37,14 @@ struct bct_cache {
     char* vhi;      // MV  [U][C][d] (value, or its bfloat16 head)
     char* vlo;      // MV residual plane (bfloat16 only), else NULL
     int* status;    // device status words
-    char* stage_q;  // staging of the host-buffer entry points
-    char* stage_k;
-    char* stage_v;
-    char* stage_out;
+    char* stage_q[2];  // staging of the host-buffer entry points, two sets used alternately
+    char* stage_k[2];
+    char* stage_v[2];
+    char* stage_out[2];
+    cudaStream_t copy_stream;  // host-to-device copies of the host-buffer entry points
+    cudaEvent_t ev_in[2];      // the set's inputs have landed
+    cudaEvent_t ev_free[2];    // the work that used the set has finished with it
+    uint64_t host_calls;
     int len;                // resident slots after the work enqueued so far
     int64_t n_full_tokens;  // full-phase tokens enqueued so far
     int64_t launches;
