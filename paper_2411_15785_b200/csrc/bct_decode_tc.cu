@@ -66,12 +66,13 @@ struct TcSmem {
 };
 __host__ __device__ inline TcSmem tc_smem(int stages, int G, int S, int slice_rows, int lo_cap) {
     const int rows = (slice_rows + kTileRows - 1) / kTileRows * kTileRows;
+    const int p_tiles = rows / kTileRows < kMaxTiles ? rows / kTileRows : kMaxTiles;  // tiles per sub-slice
     TcSmem L;
     int off = 0;
     L.ring = off;
     off += stages * kTcTileBytes;
     L.pbuf = off;
-    off += kMaxTiles * kPTileBytes + 1024;
+    off += p_tiles * kPTileBytes + 1024;
     L.qbuf = off;
     off += 2 * kQBufBytes;
     L.wsm = off;
@@ -175,7 +176,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     // zero the operands: rows G..7 of P and rows above the write query of Q stay zero for good,
     // and so do the dummy rows behind them that the N = 16 instruction shape reads
     for (int i = tid; i < 2 * kQBufBytes / 16; i += kTcThreads) reinterpret_cast<uint4*>(qbuf)[i] = make_uint4(0, 0, 0, 0);
-    for (int i = tid; i < (kMaxTiles * kPTileBytes + 1024) / 16; i += kTcThreads)
+    for (int i = tid; i < (L.qbuf - L.pbuf) / 16; i += kTcThreads)
         reinterpret_cast<uint4*>(pbuf)[i] = make_uint4(0, 0, 0, 0);
     if (warp == 5) tmem_alloc(tmem_slot, kTmemCols);
     fence_proxy_async_smem();
@@ -724,14 +725,17 @@ int launch_decode_tc(const bct_cache* c, const StepIO& io, int len, int do_write
         S *= 2;  // few units: spread each over more SMs
     int slice = (p.capacity + S - 1) / S;
     slice = (slice + kTileRows - 1) / kTileRows * kTileRows;  // whole tiles per CTA
-    int stages = 4;
-    if (const char* e = getenv("BCT_TC_STAGES")) {  // tuning knob: depth of the tile ring (2..5)
-        const int v = atoi(e);
-        if (v >= 2 && v <= 5) stages = v;
-    }
+    // Four ring stages and staging rounds of 80 rows where shared memory allows (slices up to 2048
+    // slots); longer slices keep more per-slot state and give up staging rows first, then a stage.
+    // (A deeper ring for short slices was measured: no gain, the softmax chain of a unit is the limit.)
     int lo_cap = 80;
+    int stages = 4;
+    if (const char* e = getenv("BCT_TC_STAGES")) {  // tuning knob: depth of the tile ring (2..8)
+        const int v = atoi(e);
+        if (v >= 2 && v <= 8) stages = v;
+    }
     while (tc_smem(stages, c->G, S, slice, lo_cap).total > c->smem_optin && (stages > 3 || lo_cap > 32)) {
-        if (stages > 3)
+        if (stages > 4 || (stages > 3 && lo_cap <= 48))
             --stages;
         else
             lo_cap -= 16;
