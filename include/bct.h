@@ -47,7 +47,7 @@ extern "C" {
 typedef enum bct_status {
     BCT_OK = 0,
     BCT_ERR_INVALID_ARG = 1, /* NULL / misaligned pointer, out-of-range size */
-    BCT_ERR_UNSUPPORTED = 2, /* a shape or flag this build has no kernel for */
+    BCT_ERR_UNSUPPORTED = 2, /* a shape or flag the library has no kernel for */
     BCT_ERR_STATE = 3,       /* destroyed or corrupted handle */
     BCT_ERR_CUDA = 4,        /* a CUDA runtime call failed; see bct_last_error() */
     BCT_ERR_TIMEOUT = 5      /* a bounded device-side wait gave up (bct_cache_status) */

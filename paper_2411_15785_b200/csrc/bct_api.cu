@@ -58,7 +58,7 @@ bct_status_t resolve_params(const bct_params_t* in, bct_params_t* p) {
     if ((long long)p->batch * p->n_kv_heads > (1LL << 24))
         return fail(BCT_ERR_INVALID_ARG, "batch * n_kv_heads too large");
     if (p->head_dim != 64 && p->head_dim != 128)
-        return fail(BCT_ERR_UNSUPPORTED, "head_dim %d: this build has kernels for 64 and 128", p->head_dim);
+        return fail(BCT_ERR_UNSUPPORTED, "head_dim %d: this library has kernels for 64 and 128", p->head_dim);
     if (p->n_q_heads / p->n_kv_heads > bct::kMaxGroup)
         return fail(BCT_ERR_UNSUPPORTED, "group size %d > %d", p->n_q_heads / p->n_kv_heads, bct::kMaxGroup);
     return BCT_OK;

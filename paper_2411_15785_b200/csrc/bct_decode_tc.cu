@@ -652,28 +652,10 @@ TcKernelFn pick_tc(int G) {
     }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-    }
-    return fn;
-}
-
 // [U][C][128] bfloat16 plane as a 3-D tensor (d, slot, unit); boxes of 64 x 128 x 1 with the
 // 128-byte swizzle; rows past C read as zeros.
 bool make_plane_map(CUtensorMap* map, void* base, int U, int C) {
-    EncodeTiledFn fn = encode_fn();
+    TensorMapEncodeFn fn = tensor_map_encode_fn();
     if (fn == nullptr) return false;
     const cuuint64_t dims[3] = {128, (cuuint64_t)C, (cuuint64_t)U};
     const cuuint64_t strides[2] = {256, (cuuint64_t)C * 256};
@@ -685,6 +667,21 @@ bool make_plane_map(CUtensorMap* map, void* base, int U, int C) {
 }
 
 }  // namespace
+
+// cuTensorMapEncodeTiled through the runtime's driver entry point lookup (no link against libcuda).
+TensorMapEncodeFn tensor_map_encode_fn() {
+    static TensorMapEncodeFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<TensorMapEncodeFn>(p);
+    }
+    return fn;
+}
 
 bool tc_eligible(const bct_cache* c) {
     const bct_params_t& p = c->p;

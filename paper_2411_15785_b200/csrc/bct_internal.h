@@ -66,7 +66,7 @@ namespace bct {
 int launch_decode(const bct_cache* c, const StepIO& io, int len, int do_write, cudaStream_t stream,
                   cudaError_t* err);
 
-// Whether launch_decode has a kernel for these parameters (shape limits of this build).
+// Whether launch_decode has a kernel for these parameters (shape limits of the library).
 bool decode_supported(const bct_params_t& p, int smem_optin, const char** why);
 
 // Tensor-core (tcgen05 + TMA) decode path: bfloat16, head_dim 128, group <= 7.

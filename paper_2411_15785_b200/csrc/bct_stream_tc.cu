@@ -527,28 +527,10 @@ StKernelFn pick_stream(int G) {
     }
 }
 
-typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                             const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                             CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeFn st_encode_fn() {
-    static EncodeFn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeFn>(p);
-    }
-    return fn;
-}
-
 // Step vectors [B][T][H][128] bfloat16 as a 4-D tensor (d, head, token, sequence); one box is
 // 64 columns x `heads` heads x `tokens` tokens, landing as rows (token, head) with the 128-byte swizzle.
 bool make_step_map(CUtensorMap* map, const void* base, int B, int T, int H, int heads, int tokens) {
-    EncodeFn fn = st_encode_fn();
+    TensorMapEncodeFn fn = tensor_map_encode_fn();
     if (fn == nullptr) return false;
     const cuuint64_t dims[4] = {128, (cuuint64_t)H, (cuuint64_t)T, (cuuint64_t)B};
     const cuuint64_t strides[3] = {256, (cuuint64_t)H * 256, (cuuint64_t)T * H * 256};
