@@ -135,10 +135,22 @@ bct_status_t run_tokens(bct_cache_t* c, const void* q, const void* k, const void
         if (Tc > 0 && full && do_write && T - t >= Tc) {
             const int64_t n_chunks = (T - t) / Tc;
             cudaError_t e = cudaSuccess;
-            const int n = bct::launch_stream_tc(c, q, k, v, out, T, t, n_chunks, stream, &e);
+            const int n = bct::launch_stream_tc(c, q, k, v, out, T, t, n_chunks, -1, stream, &e);
             if (n < 0) return fail_cuda("stream launch", e);
             c->launches += n;
             c->n_full_tokens += n_chunks * Tc;
+            t += n_chunks * Tc;
+            continue;
+        }
+        // whole chunks that still fit the free slots are appended by the same kernel in its fill mode
+        if (Tc > 0 && !full && T - t >= Tc && p.capacity - c->len >= Tc) {
+            const int64_t by_tokens = (T - t) / Tc, by_slots = (p.capacity - c->len) / Tc;
+            const int64_t n_chunks = by_tokens < by_slots ? by_tokens : by_slots;
+            cudaError_t e = cudaSuccess;
+            const int n = bct::launch_stream_tc(c, q, k, v, out, T, t, n_chunks, c->len, stream, &e);
+            if (n < 0) return fail_cuda("stream launch (fill)", e);
+            c->launches += n;
+            c->len += (int)(n_chunks * Tc);
             t += n_chunks * Tc;
             continue;
         }

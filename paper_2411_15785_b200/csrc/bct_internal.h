@@ -78,9 +78,11 @@ int launch_decode_tc(const bct_cache* c, const StepIO& io, int len, int do_write
 // Chunked tensor-core stream kernel (full cache, bfloat16, head_dim 128, G <= 7, C <= 2048):
 // tokens per chunk for this cache, or 0 when the kernel does not apply.
 int stream_chunk_tokens(const bct_cache* c);
-// n_chunks whole chunks starting at token t_begin of the [B][T][H][d] step arrays.
+// n_chunks whole chunks starting at token t_begin of the [B][T][H][d] step arrays.  fill_len < 0:
+// the cache is full and every token is a read plus a soft write; fill_len >= 0: the cache holds
+// fill_len slots, each chunk is appended (fill_len + n_chunks * Tc <= capacity) and read causally.
 int launch_stream_tc(const bct_cache* c, const void* q, const void* k, const void* v, void* out, int64_t T,
-                     int64_t t_begin, int64_t n_chunks, cudaStream_t stream, cudaError_t* err);
+                     int64_t t_begin, int64_t n_chunks, int fill_len, cudaStream_t stream, cudaError_t* err);
 
 // Set the calling thread's bct_last_error() message (for entry points outside bct_api.cu).
 void set_last_error(const char* msg);

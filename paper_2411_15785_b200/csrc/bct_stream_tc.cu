@@ -48,6 +48,7 @@ struct StArgs {
     char* out;
     int* status;
     int C, Hq, Hkv, U, T, t_begin, n_chunks, Tc;
+    int fill, len0;  // fill = 1: the cache holds len0 slots and each chunk is appended (no soft write)
     int wtr, out_f32, precise;  // precise: the read uses value + residual of both the numerators and MV
     float read_scale, write_scale;
 };
@@ -93,6 +94,7 @@ __global__ void __launch_bounds__(kStThreads, 1)
 stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmVhi,
                  const __grid_constant__ CUtensorMap tmVlo, const __grid_constant__ CUtensorMap tmQ,
                  const __grid_constant__ CUtensorMap tmKin, const __grid_constant__ CUtensorMap tmVin,
+                 const __grid_constant__ CUtensorMap tmKapp, const __grid_constant__ CUtensorMap tmVapp,
                  const StArgs a) {
     extern __shared__ unsigned char st_smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(st_smem_raw) + 1023) & ~uintptr_t(1023));
@@ -115,6 +117,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     uint64_t* dfree = bars + 15;      // increment consumed (128 arrivals)
     uint64_t* aready = bars + 16;     // masked A operand written (128 arrivals)
     uint64_t* oready = bars + 17;     // outputs complete (commit)
+    uint64_t* ccready = bars + 19;    // fill mode: scores of the chunk's queries against its own keys (commit)
     uint64_t* wready = bars + 18;     // rewritten MV rows of the tile are in their ring stages (256 arrivals)
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L.misc);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L.misc + 8);
@@ -124,7 +127,10 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     const int warp = tid >> 5;
     const int lane = tid & 31;
     const int Tc = a.Tc;
-    const int nt = (a.C + kStTile - 1) / kStTile;
+    const int nt_full = (a.C + kStTile - 1) / kStTile;
+    // resident slots and tiles seen by chunk ch: everything once the cache is full, len0 + ch*Tc while it fills
+    auto chunk_len = [&](int ch) { return a.fill ? a.len0 + ch * a.Tc : a.C; };
+    auto chunk_tiles = [&](int ch) { return a.fill ? (a.len0 + ch * a.Tc + kStTile - 1) / kStTile : nt_full; };
     const int n_read = Tc * G;         // rows [0, n_read): read queries (t, g); then Tc write rows
     const int vc_half = Tc * 128;      // bytes between the two 64-column halves of Vc
 
@@ -146,6 +152,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         mbar_init(aready, kStS);
         mbar_init(oready, 1);
         mbar_init(wready, kStS);
+        mbar_init(ccready, 1);
         *abort_flag = 0;
         fence_mbar_init_cluster();
     }
@@ -189,6 +196,18 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     tma_load_4d(qall + kStHalf + n_read * 128, &tmKin, 64, h, t0, b, qfull);
                     tma_load_4d(vc, &tmVin, 0, h, t0, b, qfull);
                     tma_load_4d(vc + vc_half, &tmVin, 64, h, t0, b, qfull);
+                    const int nt = chunk_tiles(ch);
+                    if (a.fill) {
+                        // fill phase: the chunk's keys and values are appended at slots len .. len + Tc - 1
+                        // straight from the operand buffers (the residual plane is zero there already)
+                        ST_WAIT(qfull, qn, 34);
+                        const int len = chunk_len(ch);
+                        tma_store_3d(&tmKapp, 0, len, u, qall + n_read * 128);
+                        tma_store_3d(&tmKapp, 64, len, u, qall + kStHalf + n_read * 128);
+                        tma_store_3d(&tmVapp, 0, len, u, vc);
+                        tma_store_3d(&tmVapp, 64, len, u, vc + vc_half);
+                        bulk_commit();
+                    }
                     for (int t = 0; t < nt; ++t) load_tile(&tmK, u, t);  // pass 1: row statistics
                     // pass 2: numerators, outputs, update.  The row threads put the rewritten MV rows back
                     // into the two ring stages the tile came in; they go home as TMA stores from here.
@@ -209,13 +228,13 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     };
                     for (int t = 0; t < nt; ++t) {
                         load_tile(&tmK, u, t);
-                        if (t > 0) store_tile(t - 1);
+                        if (t > 0 && !a.fill) store_tile(t - 1);
                         pvh = kc % kStStages;
                         load_tile(&tmVhi, u, t);
                         pvl = kc % kStStages;
                         load_tile(&tmVlo, u, t);
                     }
-                    store_tile(nt - 1);
+                    if (nt > 0 && !a.fill) store_tile(nt - 1);
                     bulk_wait_all();  // the next chunk reads these rows again
                 }
             }
@@ -242,6 +261,18 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 for (int ch = 0; ch < a.n_chunks; ++ch, ++qn) {
                     ST_WAIT(qfull, qn, 41);
                     tc_fence_after();
+                    const int nt = chunk_tiles(ch);
+                    if (a.fill) {
+                        // scores of the chunk's queries against the chunk's own keys (rows n_read.. of the
+                        // operand buffer), into the columns the full phase uses for A
+#pragma unroll
+                        for (int kk = 0; kk < 8; ++kk) {
+                            const uint32_t o = (kk >> 2) * kStHalf + (kk & 3) * 32;
+                            umma_bf16(tmem_base + kColA, smem_desc(qaddr + o, 16, 1024),
+                                      smem_desc(qaddr + n_read * 128 + o, 16, 1024), id_a, kk > 0);
+                        }
+                        umma_commit(ccready);
+                    }
                     for (int t = 0; t < nt; ++t, ++kc) {  // pass 1
                         const int stage = kc % kStStages;
                         const int buf = t & 1;
@@ -274,7 +305,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         ++np;
                         ST_WAIT(&full[vh], vh_par, 47);
                         ST_WAIT(&full[vl], vl_par, 48);
-                        if (nd > 0) ST_WAIT(dfree, nd - 1, 49);
+                        if (nd > 0 && !a.fill) ST_WAIT(dfree, nd - 1, 49);
                         tc_fence_after();
                         const uint32_t vhaddr = smem_u32(ring + (size_t)vh * kStTileBytes);
                         const uint32_t vladdr = smem_u32(ring + (size_t)vl * kStTileBytes);
@@ -289,6 +320,13 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                                 umma_bf16(tmem_base + kColO, smem_desc(phiaddr + po, 16, 1024),
                                           smem_desc(vladdr + kk * 2048, kStHalf, 1024), id_out, true);
                             }
+                        }
+                        if (a.fill) {
+                            // no soft write while the cache fills: the stages are free once the outputs are done
+                            umma_commit(pfree);
+                            umma_commit(&empty[vh]);
+                            umma_commit(&empty[vl]);
+                            continue;
                         }
                         // A += P x WW^T over this tile's slots (write rows start at n_read)
 #pragma unroll
@@ -309,12 +347,16 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         umma_commit(pfree);
                         ++nd;
                     }
-                    // intra-chunk term: O += strict_tril(A) x Vc
+                    // intra-chunk term: O += strict_tril(A) x Vc (fill phase: the causal numerators of the
+                    // chunk's own slots, value + residual, times Vc)
                     ST_WAIT(aready, qn, 50);
                     tc_fence_after();
-                    for (int kk = 0; kk < Tc / 16; ++kk)
-                        umma_bf16(tmem_base + kColO, smem_desc(ploaddr + kk * 32, 16, 1024),
-                                  smem_desc(vcaddr + kk * 2048, (uint32_t)vc_half, 1024), id_out, true);
+                    for (int kk = 0; kk < Tc / 16; ++kk) {
+                        const uint64_t vd = smem_desc(vcaddr + kk * 2048, (uint32_t)vc_half, 1024);
+                        umma_bf16(tmem_base + kColO, smem_desc(ploaddr + kk * 32, 16, 1024), vd, id_out, (nt > 0) || (kk > 0));
+                        if (a.fill && a.precise)
+                            umma_bf16(tmem_base + kColO, smem_desc(ploaddr + kStHalf + kk * 32, 16, 1024), vd, id_out, true);
+                    }
                     umma_commit(oready);
                 }
             }
@@ -338,7 +380,9 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             const int b = u / a.Hkv, h = u - b * a.Hkv;
             for (int ch = 0; ch < a.n_chunks; ++ch, ++qn) {
                 const int t0 = a.t_begin + ch * Tc;
-                // ---- pass 1: online maximum and sum of this half row's scaled scores over all C slots ----
+                const int nt = chunk_tiles(ch);
+                const int clen = chunk_len(ch);
+                // ---- pass 1: online maximum and sum of this half row's scaled scores over the resident slots ----
                 float m = kStNegBig, l = 0.f;
                 for (int t = 0; t < nt; ++t, ++kc) {
                     const int buf = t & 1;
@@ -346,7 +390,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     ST_WAIT(&sready[buf], su, 61);
                     ++su;
                     tc_fence_after();
-                    const int n_valid = min(kStTile, a.C - t * kStTile) - hf * 64;
+                    const int n_valid = min(kStTile, clen - t * kStTile) - hf * 64;
                     float x[64];
                     tmem_ld64(lane_base + (buf ? kColD : kColS0), x);
                     float bm = kStNegBig;
@@ -366,6 +410,27 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     m = mn;
                     tc_fence_before();
                     mbar_arrive(&sfree[buf]);
+                }
+                if (a.fill) {
+                    // fill phase: token t also sees the chunk's own slots s <= t (it is appended before it reads);
+                    // thread half hf covers chunk tokens [32 hf, 32 hf + 32)
+                    ST_WAIT(ccready, qn, 68);
+                    tc_fence_after();
+                    float cc[32];
+                    tmem_ld32(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + kColA + hf * 32, cc);
+                    float bm = kStNegBig;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const int s = hf * 32 + i;
+                        cc[i] = (is_read && s < Tc && s <= my_t) ? cc[i] * scale : kStNegBig;
+                        bm = fmaxf(bm, cc[i]);
+                    }
+                    const float mn = fmaxf(m, bm);
+                    float s0 = 0.f;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) s0 += (cc[i] > kStNegBig) ? __expf(cc[i] - mn) : 0.f;
+                    l = l * __expf(m - mn) + s0;
+                    m = mn;
                 }
                 // combine the two halves of the row
                 rowstat[(hf * 128 + r) * 2] = m;
@@ -394,14 +459,14 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     if (np > 0) ST_WAIT(pfree, np - 1, 63);
                     tc_fence_after();
                     {
-                        const int n_valid = min(kStTile, a.C - t * kStTile) - hf * 64;
+                        const int n_valid = min(kStTile, clen - t * kStTile) - hf * 64;
                         float x[64];
                         tmem_ld64(lane_base + kColS0, x);
                         tc_fence_before();
                         mbar_arrive(&sfree[0]);  // the scores are in registers: the next tile's may be computed
 #pragma unroll
                         for (int i = 0; i < 64; ++i)
-                            x[i] = ((is_read || is_write) && i < n_valid) ? __expf(x[i] * scale - m) * wmul : 0.f;
+                            x[i] = ((is_read || (is_write && !a.fill)) && i < n_valid) ? __expf(x[i] * scale - m) * wmul : 0.f;
 #pragma unroll
                         for (int j = 0; j < 8; ++j) {  // 16-byte chunk j of this half = 8 slots
                             uint4 hi, lo;
@@ -414,6 +479,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     fence_proxy_async_smem();
                     mbar_arrive(pready);
                     ++np;
+                    if (a.fill) continue;  // no soft write while the cache fills
 
                     // the tile's MV rows: value + residual + increment, split again, stored (this thread: 64 of the 128 d)
                     ST_WAIT(&full[vh], vh_par, 64);
@@ -450,7 +516,34 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 
                 // ---- intra-chunk term: row (t, g) sees the writes of tokens s < t (s <= t when the read
                 // ---- follows the write); A is masked, rounded to bfloat16 and handed back as an operand ----
-                {
+                if (a.fill) {
+                    // fill phase: numerators of the chunk's own slots, exp(score - m) for s <= t, as value + residual
+                    if (np > 0) ST_WAIT(pfree, np - 1, 69);  // the last tile's MMAs have read the residual buffer
+                    tc_fence_after();
+                    float cc[32];
+                    tmem_ld32(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + kColA + hf * 32, cc);
+                    if (hf * 32 < Tc) {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const int c = hf * 4 + j;
+                            if (c * 8 < Tc) {
+                                float z[8];
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) {
+                                    const int s = c * 8 + e;
+                                    z[e] = (is_read && s <= my_t) ? __expf(cc[8 * j + e] * scale - m) : 0.f;
+                                }
+                                uint4 hi, lo;
+                                split8(z, &hi, &lo);
+                                *reinterpret_cast<uint4*>(plo + r * 128 + ((c ^ sw) * 16)) = hi;
+                                if (a.precise) *reinterpret_cast<uint4*>(plo + kStHalf + r * 128 + ((c ^ sw) * 16)) = lo;
+                            }
+                        }
+                    }
+                    tc_fence_before();
+                    fence_proxy_async_smem();
+                    mbar_arrive(aready);
+                } else {
                     // thread half hf covers write tokens [32 hf, 32 hf + 32)
                     float av[32];
                     tmem_ld32(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + kColA + hf * 32, av);
@@ -512,7 +605,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 }
 
 using StKernelFn = void (*)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap,
-                            const CUtensorMap, const CUtensorMap, const StArgs);
+                            const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const StArgs);
 
 StKernelFn pick_stream(int G) {
     switch (G) {
@@ -541,6 +634,20 @@ bool make_step_map(CUtensorMap* map, const void* base, int B, int T, int H, int 
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// [U][C][128] bfloat16 plane as (d, slot, unit) with boxes of 64 columns x `rows` slots: the map
+// the fill phase appends a chunk's keys and values through.
+bool make_append_map(CUtensorMap* map, void* base, int U, int C, int rows) {
+    TensorMapEncodeFn fn = tensor_map_encode_fn();
+    if (fn == nullptr) return false;
+    const cuuint64_t dims[3] = {128, (cuuint64_t)C, (cuuint64_t)U};
+    const cuuint64_t strides[2] = {256, (cuuint64_t)C * 256};
+    const cuuint32_t box[3] = {64, (cuuint32_t)rows, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace
 
 int stream_chunk_tokens(const bct_cache* c) {
@@ -553,7 +660,7 @@ int stream_chunk_tokens(const bct_cache* c) {
 }
 
 int launch_stream_tc(const bct_cache* c, const void* q, const void* k, const void* v, void* out, int64_t T,
-                     int64_t t_begin, int64_t n_chunks, cudaStream_t stream, cudaError_t* err) {
+                     int64_t t_begin, int64_t n_chunks, int fill_len, cudaStream_t stream, cudaError_t* err) {
     const bct_params_t& p = c->p;
     StKernelFn fn = pick_stream(c->G);
     const int Tc = stream_chunk_tokens(c);
@@ -561,8 +668,13 @@ int launch_stream_tc(const bct_cache* c, const void* q, const void* k, const voi
         *err = cudaErrorInvalidConfiguration;
         return -1;
     }
-    alignas(64) CUtensorMap mq, mk, mv;
-    if (!make_step_map(&mq, q, p.batch, (int)T, p.n_q_heads, c->G, Tc) ||
+    if (fill_len >= 0 && fill_len + n_chunks * Tc > p.capacity) {
+        *err = cudaErrorInvalidValue;
+        return -1;
+    }
+    alignas(64) CUtensorMap mq, mk, mv, mka, mva;
+    if (!make_append_map(&mka, c->kplane, c->U, p.capacity, Tc) || !make_append_map(&mva, c->vhi, c->U, p.capacity, Tc) ||
+        !make_step_map(&mq, q, p.batch, (int)T, p.n_q_heads, c->G, Tc) ||
         !make_step_map(&mk, k, p.batch, (int)T, p.n_kv_heads, 1, Tc) ||
         !make_step_map(&mv, v, p.batch, (int)T, p.n_kv_heads, 1, Tc)) {
         *err = cudaErrorInvalidValue;
@@ -579,6 +691,8 @@ int launch_stream_tc(const bct_cache* c, const void* q, const void* k, const voi
     a.t_begin = (int)t_begin;
     a.n_chunks = (int)n_chunks;
     a.Tc = Tc;
+    a.fill = fill_len >= 0 ? 1 : 0;
+    a.len0 = fill_len >= 0 ? fill_len : 0;
     a.wtr = (p.flags & BCT_FLAG_WRITE_THEN_READ) ? 1 : 0;
     a.out_f32 = (p.flags & BCT_FLAG_OUT_F32) ? 1 : 0;
     a.precise = (p.flags & BCT_FLAG_PRECISE_READ) ? 1 : 0;
@@ -590,7 +704,7 @@ int launch_stream_tc(const bct_cache* c, const void* q, const void* k, const voi
     const int grid = c->U < c->sm_count ? c->U : c->sm_count;
     fn<<<grid, kStThreads, smem, stream>>>(*reinterpret_cast<const CUtensorMap*>(c->tmap_k),
                                            *reinterpret_cast<const CUtensorMap*>(c->tmap_v),
-                                           *reinterpret_cast<const CUtensorMap*>(c->tmap_lo), mq, mk, mv, a);
+                                           *reinterpret_cast<const CUtensorMap*>(c->tmap_lo), mq, mk, mv, mka, mva, a);
     *err = cudaGetLastError();
     return *err == cudaSuccess ? 1 : -1;
 }

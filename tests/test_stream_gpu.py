@@ -92,3 +92,41 @@ def test_chunked_stream_tracks_decode_steps_on_a_long_run():
     ea, eb = compare_out(w, units, oa, ref), compare_out(w, units, ob, ref)
     assert ea <= TOL["bf16"] and eb <= TOL["bf16"], (ea, eb)
     assert compare_state(w, units, a, ora) <= TOL["bf16"]
+
+
+@pytest.mark.parametrize("G,C,init_len,T,pieces,flags", [
+    (1, 1024, 0, 1200, [1200], 0),                 # from empty: 16 fill chunks of 64, then the full phase
+    (1, 333, 0, 400, [100, 300], 0),               # ragged capacity: 5 fill chunks, 13 single tokens, full phase
+    (2, 512, 100, 300, [300], 0),                  # starts inside tile 0; chunks of 32 cross tile borders
+    (3, 640, 37, 200, [70, 130], B.FLAG_OUT_F32),  # odd start, second call resumes the fill phase
+    (7, 2048, 1900, 140, [140], 0),                # chunks of 16 over 15 resident tiles
+    (1, 256, 192, 64, [64], B.FLAG_PRECISE_READ | B.FLAG_OUT_F32),  # exactly fills the cache
+])
+def test_fill_phase_chunks_match_oracle(G, C, init_len, T, pieces, flags):
+    d = 128
+    w = W.Workload("t", 2, 2 * G, 2, d, C, "bf16", init_len, T, 59, d ** -0.5, 1.0, 1.0, "stream")
+    w = w.scaled(batch=3 if C <= 512 else 2)
+    err, state, n_launch = _stream_parity(w, T, pieces, flags=flags)
+    tol = 2e-3 if flags & B.FLAG_PRECISE_READ else TOL["bf16"]
+    assert err <= tol and state <= TOL["bf16"], (err, state)
+    Tc = 64 if G == 1 else (32 if G <= 3 else 16)
+    assert n_launch <= len(pieces) * (2 + 2 * Tc)  # the fill phase went in chunks, not one launch per token
+
+
+def test_fill_phase_chunks_equal_single_tokens_in_the_cache():
+    # keys and values appended by the chunked kernel are the bits the per-token path appends
+    d = 128
+    w = W.Workload("t", 2, 2, 2, d, 512, "bf16", 0, 256, 61, d ** -0.5, 1.0, 1.0, "stream")
+    units = pick_units(w, 4)
+    a, _ = make_pair(w, units)
+    b, _ = make_pair(w, units)
+    q, k, v = W.stream_inputs(w, 0, 256, "cuda")
+    a.prefill_stream(q, k, v, want_out=False)
+    for t in range(256):
+        b.decode_step(q[:, t].contiguous(), k[:, t].contiguous(), v[:, t].contiguous())
+    assert a.len == b.len == 256
+    ka, va = a.export(v_dtype=torch.int32)
+    kb, vb = b.export(v_dtype=torch.int32)
+    assert torch.equal(ka, kb) and torch.equal(va, vb)
+    a.destroy()
+    b.destroy()
