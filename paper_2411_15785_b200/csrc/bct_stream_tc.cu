@@ -9,6 +9,9 @@
 //     A  = Pr WW^T                          what token t's read sees of token s's write
 //     O  = Pr MV + strict_tril(A) Vc        outputs: every token reads MV_{t-1}
 //     MV += WW^T Vc                         Method step 4 for the Tc tokens at once
+// While the cache still has Tc free slots the same kernel runs in fill mode: the chunk's keys and
+// values are appended (TMA stores from the operand buffers), token t reads the resident slots plus
+// the chunk's own slots s <= t (scores Q Kc^T, masked causally), and nothing is soft-written.
 // One persistent CTA per (sequence, kv-head) unit at a time (C <= 2048 slots); per chunk the cache
 // streams through shared memory twice for MK (row statistics, then numerators) and once for MV
 // (value and residual planes), instead of twice per token, and every product runs as tcgen05.mma
