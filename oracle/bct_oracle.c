@@ -28,6 +28,11 @@
  *   - Algorithm 1's "if t = 1" branch keeps MV_0 for the first token, while the
  *     exception-free formula of Method step 4 updates on every token.  Default:
  *     every token writes.  BCT_ORACLE_SKIP_FIRST_WRITE takes the branch literally.
+ *   - step size (Features, "Learning Rate Adaptation": the step size is adjusted
+ *     for each token; no formula is printed): eta_t multiplies the token's
+ *     increment, MV_t = MV_{t-1} + eta_t * ww_t^T . wv_t.  eta_t = 1 is Method
+ *     step 4 as printed.  How eta_t is produced is upstream of this layer: it is
+ *     an input.  The fill phase has no soft write and ignores it.
  *   - fill phase (not in the paper, whose MV_0 is full-size): while len < C the
  *     token's (k_t, v_t) is appended at slot len, the read then covers the
  *     len+1 resident slots (so the token sees itself), and no soft write happens.
@@ -72,10 +77,10 @@ static void read_head(const double *q, const double *MK, const double *MV, int64
         for (int e = 0; e < d; ++e) o[e] += p[j] * MV[j * d + e];
 }
 
-/* Write path: score = write_scale * wq . MK^T; ww = softmax(score); MV += ww^T . wv.
+/* Write path: score = write_scale * wq . MK^T; ww = softmax(score); MV += eta * ww^T . wv.
  * ww (length C) is left in `ww` for the caller. */
 static void write_update(const double *wq, const double *wv, const double *MK, double *MV,
-                         int64_t C, int d, double write_scale, double *s, double *ww) {
+                         int64_t C, int d, double write_scale, double eta, double *s, double *ww) {
     for (int64_t j = 0; j < C; ++j) {
         double dot = 0.0;
         for (int e = 0; e < d; ++e) dot += wq[e] * MK[j * d + e];
@@ -83,7 +88,7 @@ static void write_update(const double *wq, const double *wv, const double *MK, d
     }
     softmax(s, C, ww);
     for (int64_t j = 0; j < C; ++j)
-        for (int e = 0; e < d; ++e) MV[j * d + e] += ww[j] * wv[e];
+        for (int e = 0; e < d; ++e) MV[j * d + e] += eta * (ww[j] * wv[e]);
 }
 
 /*
@@ -94,8 +99,8 @@ static void write_update(const double *wq, const double *wv, const double *MK, d
  */
 static int64_t unit_token(int G, int d, int64_t C, int64_t len, double *MK, double *MV,
                           const double *q, const double *k, const double *v, double *out,
-                          double read_scale, double write_scale, unsigned flags, int do_write,
-                          double *s, double *p) {
+                          double read_scale, double write_scale, double eta, unsigned flags,
+                          int do_write, double *s, double *p) {
     if (len < C) { /* fill phase: append, then read over len+1 slots, no soft write */
         memcpy(MK + len * d, k, sizeof(double) * (size_t)d);
         memcpy(MV + len * d, v, sizeof(double) * (size_t)d);
@@ -106,12 +111,12 @@ static int64_t unit_token(int G, int d, int64_t C, int64_t len, double *MK, doub
         return len;
     }
     if ((flags & BCT_ORACLE_WRITE_THEN_READ) && do_write)
-        write_update(k, v, MK, MV, C, d, write_scale, s, p);
+        write_update(k, v, MK, MV, C, d, write_scale, eta, s, p);
     if (out)
         for (int g = 0; g < G; ++g)
             read_head(q + (int64_t)g * d, MK, MV, C, d, read_scale, s, p, out + (int64_t)g * d);
     if (!(flags & BCT_ORACLE_WRITE_THEN_READ) && do_write)
-        write_update(k, v, MK, MV, C, d, write_scale, s, p);
+        write_update(k, v, MK, MV, C, d, write_scale, eta, s, p);
     return len;
 }
 
@@ -123,16 +128,17 @@ static int64_t unit_token(int G, int d, int64_t C, int64_t len, double *MK, doub
  *   q       [U][T][G][d]
  *   k, v    [U][T][d]
  *   out     [U][T][G][d]   or NULL
+ *   eta     [U][T]         step size of each token's write, or NULL (all ones)
  * len_io        resident slots, the same for every unit (in/out)
  * n_written_io  soft writes applied so far per unit history (in/out); only its
  *               being zero matters (BCT_ORACLE_SKIP_FIRST_WRITE)
  * nthreads      OpenMP threads over units (<= 0: library default)
  * Returns the number of threads used, or -1 on bad arguments / allocation failure.
  */
-int bct_oracle_stream(int64_t U, int64_t T, int G, int d, int64_t C, int64_t *len_io,
-                      int64_t *n_written_io, double *MK, double *MV, const double *q,
-                      const double *k, const double *v, double *out, double read_scale,
-                      double write_scale, unsigned flags, int nthreads) {
+int bct_oracle_stream_eta(int64_t U, int64_t T, int G, int d, int64_t C, int64_t *len_io,
+                          int64_t *n_written_io, double *MK, double *MV, const double *q,
+                          const double *k, const double *v, const double *eta, double *out,
+                          double read_scale, double write_scale, unsigned flags, int nthreads) {
     if (U < 0 || T < 0 || G < 1 || d < 1 || C < 1 || !len_io || !n_written_io) return -1;
     if (*len_io < 0 || *len_io > C) return -1;
     int used = 1;
@@ -163,7 +169,7 @@ int bct_oracle_stream(int64_t U, int64_t T, int G, int d, int64_t C, int64_t *le
                 int full = (len == C);
                 int do_write = !((flags & BCT_ORACLE_SKIP_FIRST_WRITE) && nw == 0);
                 len = unit_token(G, d, C, len, mk, mv, qt, kt, vt, ot, read_scale, write_scale,
-                                 flags, do_write, s, p);
+                                 eta ? eta[u * T + t] : 1.0, flags, do_write, s, p);
                 if (full) nw += 1; /* counts full-phase tokens seen, written or skipped */
             }
         }
@@ -179,6 +185,15 @@ int bct_oracle_stream(int64_t U, int64_t T, int G, int d, int64_t C, int64_t *le
     *len_io = len;
     *n_written_io = nw;
     return used;
+}
+
+/* The same with every step size equal to one: Method step 4 as printed. */
+int bct_oracle_stream(int64_t U, int64_t T, int G, int d, int64_t C, int64_t *len_io,
+                      int64_t *n_written_io, double *MK, double *MV, const double *q,
+                      const double *k, const double *v, double *out, double read_scale,
+                      double write_scale, unsigned flags, int nthreads) {
+    return bct_oracle_stream_eta(U, T, G, d, C, len_io, n_written_io, MK, MV, q, k, v, NULL, out,
+                                 read_scale, write_scale, flags, nthreads);
 }
 
 /* The write weights ww = softmax(write_scale * wq . MK^T) of one unit, for tests

@@ -61,6 +61,11 @@ def _load():
             ctypes.c_int64, ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.c_int64,
             ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64),
             dp, dp, dp, dp, dp, dp, ctypes.c_double, ctypes.c_double, ctypes.c_uint, ctypes.c_int]
+        lib.bct_oracle_stream_eta.restype = ctypes.c_int
+        lib.bct_oracle_stream_eta.argtypes = [
+            ctypes.c_int64, ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.c_int64,
+            ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64),
+            dp, dp, dp, dp, dp, dp, dp, ctypes.c_double, ctypes.c_double, ctypes.c_uint, ctypes.c_int]
         lib.bct_oracle_write_weights.restype = ctypes.c_int
         lib.bct_oracle_write_weights.argtypes = [ctypes.c_int64, ctypes.c_int, dp, dp,
                                                  ctypes.c_double, dp]
@@ -146,8 +151,10 @@ class OracleCache:
         return self.MV.reshape(self.B, self.Hkv, self.C, self.d)
 
     # -- steps -------------------------------------------------------------------
-    def prefill_stream(self, q, k, v, want_out: bool = True):
-        """q ``[B, T, Hq, d]``, k, v ``[B, T, Hkv, d]`` -> out ``[B, T, Hq, d]`` (float64)."""
+    def prefill_stream(self, q, k, v, want_out: bool = True, eta=None):
+        """q ``[B, T, Hq, d]``, k, v ``[B, T, Hkv, d]`` -> out ``[B, T, Hq, d]`` (float64).
+
+        ``eta`` ``[B, T, Hkv]``: step size of each token's write (None = all ones)."""
         q = _f64(q)
         k = _f64(k)
         v = _f64(v)
@@ -164,9 +171,15 @@ class OracleCache:
         ou = np.empty((self.U, T, self.G, self.d), dtype=np.float64) if want_out else None
         ln = ctypes.c_int64(self.len)
         nw = ctypes.c_int64(self.n_written)
-        rc = _load().bct_oracle_stream(
+        eu = None
+        if eta is not None:
+            eta = _f64(eta)
+            assert eta.shape == (self.B, T, self.Hkv), eta.shape
+            eu = np.ascontiguousarray(eta.transpose(0, 2, 1)).reshape(self.U, T)
+        rc = _load().bct_oracle_stream_eta(
             self.U, T, self.G, self.d, self.C, ctypes.byref(ln), ctypes.byref(nw),
             _dptr(self.MK), _dptr(self.MV), _dptr(qu), _dptr(ku), _dptr(vu),
+            _dptr(eu) if eu is not None else None,
             _dptr(ou) if want_out else None, self.read_scale, self.write_scale,
             self.flags, self.nthreads)
         if rc < 0:
@@ -179,9 +192,9 @@ class OracleCache:
             ou.reshape(B, self.Hkv, T, self.G, self.d).transpose(0, 2, 1, 3, 4)
         ).reshape(B, T, self.Hq, self.d)
 
-    def decode_step(self, q, k, v):
-        """q ``[B, Hq, d]``, k, v ``[B, Hkv, d]`` -> out ``[B, Hq, d]``."""
+    def decode_step(self, q, k, v, eta=None):
+        """q ``[B, Hq, d]``, k, v ``[B, Hkv, d]``, eta ``[B, Hkv]`` or None -> out ``[B, Hq, d]``."""
         q = _f64(q)[:, None]
         k = _f64(k)[:, None]
         v = _f64(v)[:, None]
-        return self.prefill_stream(q, k, v)[:, 0]
+        return self.prefill_stream(q, k, v, eta=None if eta is None else _f64(eta)[:, None])[:, 0]

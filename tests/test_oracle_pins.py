@@ -367,3 +367,83 @@ def test_default_scales():
     ww = _np_softmax(k[0, 0, 0] @ mk[0, 0].T)                  # Algorithm 1 prints no write scale
     np.testing.assert_allclose(o[0, 0, 0], p @ mv0[0, 0], rtol=0, atol=1e-13)
     np.testing.assert_allclose(c.values()[0, 0], mv0[0, 0] + np.outer(ww, v[0, 0, 0]), rtol=0, atol=1e-13)
+
+
+# ---------------------------------------------------------------------------------------
+# Step size of each token's write (Features, "Learning Rate Adaptation"), read as
+#   MV_t = MV_{t-1} + eta_t * ww_t^T wv_t
+# ---------------------------------------------------------------------------------------
+def test_step_size_one_is_the_printed_rule_bit_for_bit():
+    B, Hq, Hkv, d, C, T = 2, 4, 2, 6, 5, 9
+    q, k, v = _rand(B, T, Hq, d), _rand(B, T, Hkv, d), _rand(B, T, Hkv, d)
+    a = O.OracleCache(B, Hq, Hkv, d, C)
+    b = O.OracleCache(B, Hq, Hkv, d, C)
+    np.testing.assert_array_equal(a.prefill_stream(q, k, v), b.prefill_stream(q, k, v, eta=np.ones((B, T, Hkv))))
+    np.testing.assert_array_equal(a.values(), b.values())
+
+
+def test_step_size_scales_the_mass_each_token_adds():
+    B, Hq, Hkv, d, C, T = 2, 2, 2, 8, 7, 6
+    mk, mv = _rand(B, Hkv, C, d), _rand(B, Hkv, C, d)
+    q, k, v = _rand(B, T, Hq, d), _rand(B, T, Hkv, d), _rand(B, T, Hkv, d)
+    eta = RNG.uniform(-0.5, 2.0, size=(B, T, Hkv))
+    c = O.OracleCache(B, Hq, Hkv, d, C, init_len=C, mk_init=mk, mv_init=mv)
+    prev = c.values().sum(axis=2).copy()
+    for t in range(T):
+        c.decode_step(q[:, t], k[:, t], v[:, t], eta=eta[:, t])
+        cur = c.values().sum(axis=2)
+        np.testing.assert_allclose(cur - prev, eta[:, t, :, None] * v[:, t], rtol=0, atol=1e-12)
+        prev = cur.copy()
+    np.testing.assert_array_equal(c.keys(), mk)
+
+
+@pytest.mark.parametrize("flags", [0, O.WRITE_THEN_READ])
+def test_step_size_dense_restatement(flags):
+    # MV_N = MV_0 + WW^T diag(eta) Vc ;  O = Pr MV_0 + tril(Pr WW^T) diag(eta) Vc
+    d, C, T, G = 8, 9, 12, 2
+    rs, ws = 0.4, 0.7
+    mk, mv0 = _rand(1, 1, C, d), _rand(1, 1, C, d)
+    q, k, v = _rand(1, T, G, d), _rand(1, T, 1, d), _rand(1, T, 1, d)
+    eta = RNG.uniform(0.0, 1.5, size=(1, T, 1))
+    c = O.OracleCache(1, G, 1, d, C, init_len=C, mk_init=mk, mv_init=mv0, read_scale=rs, write_scale=ws, flags=flags)
+    out = c.prefill_stream(q, k, v, eta=eta)
+    MK, MV0, Kc, Vc = mk[0, 0], mv0[0, 0], k[0, :, 0], v[0, :, 0]
+    EV = eta[0, :, 0, None] * Vc
+    WW = _np_softmax(ws * Kc @ MK.T)
+    np.testing.assert_allclose(c.values()[0, 0], MV0 + WW.T @ EV, rtol=0, atol=1e-12)
+    for g in range(G):
+        Pr = _np_softmax(rs * q[0, :, g] @ MK.T)
+        A = np.tril(Pr @ WW.T, 0 if flags else -1)
+        np.testing.assert_allclose(out[0, :, g], Pr @ MV0 + A @ EV, rtol=0, atol=1e-12)
+
+
+def test_step_size_zero_freezes_the_state_and_fill_phase_ignores_it():
+    B, Hq, Hkv, d, C, T = 1, 2, 1, 4, 6, 10
+    q, k, v = _rand(B, T, Hq, d), _rand(B, T, Hkv, d), _rand(B, T, Hkv, d)
+    eta = np.zeros((B, T, Hkv))
+    a = O.OracleCache(B, Hq, Hkv, d, C)
+    oa = a.prefill_stream(q, k, v, eta=eta)
+    # the six fill tokens are appended as they are; afterwards nothing changes
+    np.testing.assert_array_equal(a.keys()[0, 0], k[0, :C, 0])
+    np.testing.assert_array_equal(a.values()[0, 0], v[0, :C, 0])
+    for t in range(C, T):  # a frozen cache: plain attention over the six appended slots
+        for g in range(Hq):
+            p = _np_softmax(q[0, t, g] @ k[0, :C, 0].T / math.sqrt(d))
+            np.testing.assert_allclose(oa[0, t, g], p @ v[0, :C, 0], rtol=0, atol=1e-13)
+    b = O.OracleCache(B, Hq, Hkv, d, C)
+    ob = b.prefill_stream(q[:, :C], k[:, :C], v[:, :C])            # fill phase with and without eta
+    np.testing.assert_array_equal(oa[:, :C], ob)
+
+
+def test_step_size_equals_a_scaled_write_value_in_the_full_phase():
+    B, Hq, Hkv, d, C, T = 2, 4, 2, 5, 4, 7
+    mk, mv = _rand(B, Hkv, C, d), _rand(B, Hkv, C, d)
+    q, k, v = _rand(B, T, Hq, d), _rand(B, T, Hkv, d), _rand(B, T, Hkv, d)
+    eta = RNG.uniform(0.1, 3.0, size=(B, T, Hkv))
+    for flags in (0, O.WRITE_THEN_READ):
+        a = O.OracleCache(B, Hq, Hkv, d, C, init_len=C, mk_init=mk, mv_init=mv, flags=flags)
+        b = O.OracleCache(B, Hq, Hkv, d, C, init_len=C, mk_init=mk, mv_init=mv, flags=flags)
+        oa = a.prefill_stream(q, k, v, eta=eta)
+        ob = b.prefill_stream(q, k, eta[..., None] * v)
+        np.testing.assert_allclose(oa, ob, rtol=0, atol=1e-12)
+        np.testing.assert_allclose(a.values(), b.values(), rtol=0, atol=1e-12)
