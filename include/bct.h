@@ -154,6 +154,22 @@ bct_status_t bct_prefill_stream(bct_cache_t *cache, const void *q, const void *k
                                 void *out, int64_t T, void *cuda_stream);
 
 /*
+ * The two calls above with a step size for each token's write (Features, "Learning Rate
+ * Adaptation": the step size is adjusted for each token; the paper prints no formula, so
+ * the step size is an input and scales the increment of Method step 4):
+ *     MV_t = MV_{t-1} + eta_t * ww_t^T . wv_t
+ *   eta  DEVICE float [B][Hkv] (decode) / [B][T][Hkv] (stream), 4-byte aligned, read by
+ *        the kernels of this call only; NULL means all ones, which is the call above.
+ * Tokens of the fill phase are appended as they are and ignore eta; with
+ * BCT_FLAG_WRITE_THEN_READ the token's own read sees the scaled write.  write_eps is
+ * compared with ww_t, not with eta_t * ww_t.  Everything else as in the calls above.
+ */
+bct_status_t bct_decode_step_eta(bct_cache_t *cache, const void *q, const void *k, const void *v,
+                                 const float *eta, void *out, void *cuda_stream);
+bct_status_t bct_prefill_stream_eta(bct_cache_t *cache, const void *q, const void *k, const void *v,
+                                    const float *eta, void *out, int64_t T, void *cuda_stream);
+
+/*
  * Host-buffer forms of the two calls above: the same shapes, but q, k, v and out are
  * HOST pointers.  The inputs are copied into the workspace's staging area (two sets, used
  * alternately, on a copy stream the handle owns, so that one call's copies overlap the

@@ -23,7 +23,7 @@ EXPORTS = (
     "bct_version", "bct_last_error", "bct_cache_bytes", "bct_cache_create", "bct_decode_step",
     "bct_prefill_stream", "bct_decode_step_host", "bct_prefill_stream_host", "bct_cache_len",
     "bct_cache_export", "bct_cache_import", "bct_cache_status", "bct_cache_launches", "bct_cache_destroy",
-    "bct_cache_tensor_path", "bct_prefill_stream_host_static",
+    "bct_cache_tensor_path", "bct_prefill_stream_host_static", "bct_decode_step_eta", "bct_prefill_stream_eta",
 )
 STATIC_STAGE_BYTES = 8 << 20
 
@@ -64,6 +64,8 @@ def load() -> ctypes.CDLL:
     lib.bct_cache_create.argtypes = [pp, vp, ctypes.c_size_t, vp, vp, vp, ctypes.POINTER(vp)]
     lib.bct_decode_step.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.bct_prefill_stream.argtypes = [vp, vp, vp, vp, vp, i64, vp]
+    lib.bct_decode_step_eta.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    lib.bct_prefill_stream_eta.argtypes = [vp, vp, vp, vp, vp, vp, i64, vp]
     lib.bct_decode_step_host.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.bct_prefill_stream_host.argtypes = [vp, vp, vp, vp, vp, i64, vp]
     lib.bct_cache_len.argtypes = [vp, ctypes.POINTER(i32)]
@@ -116,6 +118,11 @@ def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
     return s.cuda_stream
 
 
+def _check_eta(eta: torch.Tensor, shape) -> None:
+    if eta.dtype != torch.float32 or tuple(eta.shape) != tuple(shape) or not eta.is_contiguous() or not eta.is_cuda:
+        raise ValueError("eta must be a contiguous float32 device tensor of shape %s" % (tuple(shape),))
+
+
 def _ptr(t: Optional[torch.Tensor]):
     return None if t is None else t.data_ptr()
 
@@ -150,19 +157,31 @@ class Cache:
                                              _ptr(mv_init), _stream_ptr(stream), ctypes.byref(self._h)))
 
     # ---- steps ----------------------------------------------------------------------
-    def decode_step(self, q, k, v, out=None, stream=None):
+    def decode_step(self, q, k, v, out=None, stream=None, eta=None):
+        """eta: float32 device tensor [B, Hkv], the step size of each unit's write (None = ones)."""
         if out is None:
             out = torch.empty_like(q, dtype=self.out_dtype)
-        _check(self.lib.bct_decode_step(self._h, q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
-                                        _stream_ptr(stream)))
+        if eta is None:
+            _check(self.lib.bct_decode_step(self._h, q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
+                                            _stream_ptr(stream)))
+        else:
+            _check_eta(eta, (self.B, self.Hkv))
+            _check(self.lib.bct_decode_step_eta(self._h, q.data_ptr(), k.data_ptr(), v.data_ptr(), eta.data_ptr(),
+                                                out.data_ptr(), _stream_ptr(stream)))
         return out
 
-    def prefill_stream(self, q, k, v, out=None, want_out=True, stream=None):
+    def prefill_stream(self, q, k, v, out=None, want_out=True, stream=None, eta=None):
+        """eta: float32 device tensor [B, T, Hkv], the step size of each token's write (None = ones)."""
         T = q.shape[1]
         if out is None and want_out:
             out = torch.empty_like(q, dtype=self.out_dtype)
-        _check(self.lib.bct_prefill_stream(self._h, q.data_ptr(), k.data_ptr(), v.data_ptr(), _ptr(out), T,
-                                           _stream_ptr(stream)))
+        if eta is None:
+            _check(self.lib.bct_prefill_stream(self._h, q.data_ptr(), k.data_ptr(), v.data_ptr(), _ptr(out), T,
+                                               _stream_ptr(stream)))
+        else:
+            _check_eta(eta, (self.B, T, self.Hkv))
+            _check(self.lib.bct_prefill_stream_eta(self._h, q.data_ptr(), k.data_ptr(), v.data_ptr(), eta.data_ptr(),
+                                                   _ptr(out), T, _stream_ptr(stream)))
         return out
 
     def decode_step_host(self, q, k, v, out, stream=None):

@@ -120,8 +120,9 @@ void release_host_objects(bct_cache_t* c) {
 }
 
 // T tokens, one decode launch each.  Pointers are device pointers in [B][T][H][d].
-bct_status_t run_tokens(bct_cache_t* c, const void* q, const void* k, const void* v, void* out, int64_t T,
-                        cudaStream_t stream) {
+// eta: [B][T][Hkv] floats on the device, or NULL.
+bct_status_t run_tokens(bct_cache_t* c, const void* q, const void* k, const void* v, const float* eta, void* out,
+                        int64_t T, cudaStream_t stream) {
     const bct_params_t& p = c->p;
     const size_t eb = (size_t)c->elem_bytes;
     const size_t q_tok = (size_t)p.n_q_heads * p.head_dim;   // elements per token per sequence
@@ -135,7 +136,7 @@ bct_status_t run_tokens(bct_cache_t* c, const void* q, const void* k, const void
         if (Tc > 0 && full && do_write && T - t >= Tc) {
             const int64_t n_chunks = (T - t) / Tc;
             cudaError_t e = cudaSuccess;
-            const int n = bct::launch_stream_tc(c, q, k, v, out, T, t, n_chunks, -1, stream, &e);
+            const int n = bct::launch_stream_tc(c, q, k, v, out, T, eta, t, n_chunks, -1, stream, &e);
             if (n < 0) return fail_cuda("stream launch", e);
             c->launches += n;
             c->n_full_tokens += n_chunks * Tc;
@@ -147,7 +148,7 @@ bct_status_t run_tokens(bct_cache_t* c, const void* q, const void* k, const void
             const int64_t by_tokens = (T - t) / Tc, by_slots = (p.capacity - c->len) / Tc;
             const int64_t n_chunks = by_tokens < by_slots ? by_tokens : by_slots;
             cudaError_t e = cudaSuccess;
-            const int n = bct::launch_stream_tc(c, q, k, v, out, T, t, n_chunks, c->len, stream, &e);
+            const int n = bct::launch_stream_tc(c, q, k, v, out, T, eta, t, n_chunks, c->len, stream, &e);
             if (n < 0) return fail_cuda("stream launch (fill)", e);
             c->launches += n;
             c->len += (int)(n_chunks * Tc);
@@ -162,6 +163,8 @@ bct_status_t run_tokens(bct_cache_t* c, const void* q, const void* k, const void
         io.out = out ? static_cast<char*>(out) + (size_t)t * q_tok * ob : nullptr;
         io.q_batch_stride = (int64_t)(T * q_tok);
         io.kv_batch_stride = (int64_t)(T * kv_tok);
+        io.eta = eta ? eta + (size_t)t * p.n_kv_heads : nullptr;
+        io.eta_batch_stride = (int64_t)T * p.n_kv_heads;
         cudaError_t e = cudaSuccess;
         const int n = bct::launch_decode(c, io, c->len, do_write, stream, &e);
         if (n < 0) return fail_cuda("decode launch", e);
@@ -286,7 +289,7 @@ bct_status_t bct_decode_step(bct_cache_t* c, const void* q, const void* k, const
     if (st != BCT_OK) return st;
     st = check_step_ptrs(q, k, v, out, false);
     if (st != BCT_OK) return st;
-    return run_tokens(c, q, k, v, out, 1, static_cast<cudaStream_t>(cuda_stream));
+    return run_tokens(c, q, k, v, nullptr, out, 1, static_cast<cudaStream_t>(cuda_stream));
 }
 
 bct_status_t bct_prefill_stream(bct_cache_t* c, const void* q, const void* k, const void* v, void* out, int64_t T,
@@ -296,7 +299,24 @@ bct_status_t bct_prefill_stream(bct_cache_t* c, const void* q, const void* k, co
     if (T < 1) return fail(BCT_ERR_INVALID_ARG, "T must be >= 1 (got %lld)", (long long)T);
     st = check_step_ptrs(q, k, v, out, true);
     if (st != BCT_OK) return st;
-    return run_tokens(c, q, k, v, out, T, static_cast<cudaStream_t>(cuda_stream));
+    return run_tokens(c, q, k, v, nullptr, out, T, static_cast<cudaStream_t>(cuda_stream));
+}
+
+bct_status_t bct_prefill_stream_eta(bct_cache_t* c, const void* q, const void* k, const void* v, const float* eta,
+                                    void* out, int64_t T, void* cuda_stream) {
+    bct_status_t st = check_handle(c);
+    if (st != BCT_OK) return st;
+    if (T < 1) return fail(BCT_ERR_INVALID_ARG, "T must be >= 1 (got %lld)", (long long)T);
+    st = check_step_ptrs(q, k, v, out, true);
+    if (st != BCT_OK) return st;
+    if ((reinterpret_cast<uintptr_t>(eta) & 3u) != 0) return fail(BCT_ERR_INVALID_ARG, "eta must be 4-byte aligned");
+    return run_tokens(c, q, k, v, eta, out, T, static_cast<cudaStream_t>(cuda_stream));
+}
+
+bct_status_t bct_decode_step_eta(bct_cache_t* c, const void* q, const void* k, const void* v, const float* eta,
+                                 void* out, void* cuda_stream) {
+    if (out == nullptr) return fail(BCT_ERR_INVALID_ARG, "out must not be NULL");
+    return bct_prefill_stream_eta(c, q, k, v, eta, out, 1, cuda_stream);
 }
 
 bct_status_t bct_prefill_stream_host(bct_cache_t* c, const void* q, const void* k, const void* v, void* out,
@@ -323,7 +343,8 @@ bct_status_t bct_prefill_stream_host(bct_cache_t* c, const void* q, const void* 
     if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, c->ev_in[set], 0);
     if (e != cudaSuccess) return fail_cuda("host-to-device copy", e);
     c->host_calls += 1;
-    st = run_tokens(c, c->stage_q[set], c->stage_k[set], c->stage_v[set], out ? c->stage_out[set] : nullptr, T, stream);
+    st = run_tokens(c, c->stage_q[set], c->stage_k[set], c->stage_v[set], nullptr, out ? c->stage_out[set] : nullptr, T,
+                    stream);
     if (st != BCT_OK) return st;
     if (out != nullptr) {
         const size_t ob = (c->p.flags & BCT_FLAG_OUT_F32) ? qb / eb * 4 : qb;

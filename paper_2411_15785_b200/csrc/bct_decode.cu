@@ -42,6 +42,8 @@ struct DecodeArgs {
     int* status;
     long long q_bs;   // elements between sequences in q / out
     long long kv_bs;  // elements between sequences in k / v
+    const float* eta; // step size of each unit's write, [sequence][kv-head], or NULL (all ones)
+    long long eta_bs; // elements between sequences in eta
     int C;
     int len;         // resident slots before this token
     int slice_rows;  // slots per CTA of the cluster
@@ -147,6 +149,8 @@ __global__ void __launch_bounds__(kThreads, (G <= 4 ? 2 : 1)) decode_kernel(cons
     const bool precise = (sizeof(T) == 2) && a.precise;
     const size_t q_off = ((size_t)b * a.q_bs + (size_t)h_kv * G * D) * sizeof(T);
     const size_t kv_off = ((size_t)b * a.kv_bs + (size_t)h_kv * D) * sizeof(T);
+    // step size of this token's write: MV_t = MV_{t-1} + eta_t ww_t^T wv_t (the write value is scaled once)
+    const float eta_u = (a.eta != nullptr && a.do_write) ? a.eta[(size_t)b * a.eta_bs + h_kv] : 1.f;
 
     if (tid == 0) {
         for (int i = 0; i < kStages; ++i) {
@@ -364,6 +368,8 @@ __global__ void __launch_bounds__(kThreads, (G <= 4 ? 2 : 1)) decode_kernel(cons
         }
         float vt[EPL];
         Ck::unpack(v_raw, vt);
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) vt[e] *= eta_u;
         for (int i = 0; i < nt; ++i) {
             const int item = precise ? nt + 2 * i : nt + i;
             const int stage = item % kStages;
@@ -493,7 +499,7 @@ __global__ void __launch_bounds__(kThreads, (G <= 4 ? 2 : 1)) decode_kernel(cons
                     const int g = idx / D, e = idx - g * D;
                     const float inv = 1.f / stat[(G + 1) + g];
                     float val = ofin[g * (D + 1) + e] * inv;
-                    if (add_own) val = fmaf(ofin[g * (D + 1) + D] * inv, (float)vin[e], val);
+                    if (add_own) val = fmaf(ofin[g * (D + 1) + D] * inv, (float)vin[e] * eta_u, val);
                     store_out<T>(a, q_off, idx, val);
                 }
             }
@@ -532,7 +538,7 @@ __global__ void __launch_bounds__(kThreads, (G <= 4 ? 2 : 1)) decode_kernel(cons
                     den = fmaf(mr[D + 2], f, den);
                 }
                 float val = num / den;
-                if (add_own) val = fmaf(own / den, (float)vin[e], val);
+                if (add_own) val = fmaf(own / den, (float)vin[e] * eta_u, val);
                 store_out<T>(a, q_off, idx, val);
             }
         }
@@ -639,6 +645,8 @@ int launch_decode(const bct_cache* c, const StepIO& io, int len, int do_write, c
     a.status = c->status;
     a.q_bs = io.q_batch_stride;
     a.kv_bs = io.kv_batch_stride;
+    a.eta = io.eta;
+    a.eta_bs = io.eta_batch_stride;
     a.C = p.capacity;
     a.len = len;
     a.slice_rows = pl.slice_rows;

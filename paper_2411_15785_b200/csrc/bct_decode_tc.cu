@@ -56,6 +56,8 @@ struct TcArgs {
     int* status;
     long long q_bs;
     long long kv_bs;
+    const float* eta;   // step size of each unit's write, [sequence][kv-head], or NULL (all ones)
+    long long eta_bs;
     int C, len, slice_rows, S, Hkv, U, stages, lo_cap;  // lo_cap: rewritten rows staged per round
     int do_write, wtr, dense, out_f32;
     float read_scale, write_scale, write_eps;
@@ -314,6 +316,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             const int h_kv = u - b * a.Hkv;
             const size_t q_off = ((size_t)b * a.q_bs + (size_t)h_kv * G * D) * 2;
             const size_t kv_off = ((size_t)b * a.kv_bs + (size_t)h_kv * D) * 2;
+            // step size of this token's write: MV_t = MV_{t-1} + eta_t ww_t^T wv_t
+            const float eta_u = (a.eta != nullptr && a.do_write) ? a.eta[(size_t)b * a.eta_bs + h_kv] : 1.f;
             const size_t unit_off = (size_t)u * a.C * ROW_BYTES;
 
             // the appended slot (fill phase) is scored from the step vectors
@@ -533,7 +537,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     for (int g = 0; g < G; ++g) {
                         const float inv = 1.f / st_l[g];
                         float val = o[g] * inv;
-                        if (add_own) val = fmaf(st_wd[g] * inv * wfac, vd, val);
+                        if (add_own) val = fmaf(st_wd[g] * inv * wfac, vd * eta_u, val);
                         if (a.out_f32)
                             reinterpret_cast<float*>(a.out + q_off * 2)[g * D + r] = val;
                         else
@@ -574,7 +578,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                                 den = fmaf(mr[D + 2], f, den);
                             }
                             float val = num / den;
-                            if (add_own) val = fmaf(own / den, vd, val);
+                            if (add_own) val = fmaf(own / den, vd * eta_u, val);
                             if (a.out_f32)
                                 reinterpret_cast<float*>(a.out + q_off * 2)[g * D + r] = val;
                             else
@@ -588,6 +592,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             if (a.do_write) {
                 float vt[8];
                 Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(a.v + kv_off + c16 * 16), vt);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) vt[e] *= eta_u;
                 for (int base = 0; base < n_touched; base += kLoCap) {
                     const int n = min(n_touched - base, kLoCap);
                     if (base > 0) {
@@ -754,6 +760,8 @@ int launch_decode_tc(const bct_cache* c, const StepIO& io, int len, int do_write
     a.status = c->status;
     a.q_bs = io.q_batch_stride;
     a.kv_bs = io.kv_batch_stride;
+    a.eta = io.eta;
+    a.eta_bs = io.eta_batch_stride;
     a.C = p.capacity;
     a.len = len;
     a.slice_rows = slice;

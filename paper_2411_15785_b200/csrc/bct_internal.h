@@ -19,6 +19,8 @@ struct StepIO {
     void* out;       // may be NULL in state-only streams
     int64_t q_batch_stride;   // elements between sequences in q / out
     int64_t kv_batch_stride;  // elements between sequences in k / v
+    const float* eta = nullptr;     // step size of the write per (sequence, kv-head), or NULL (all ones)
+    int64_t eta_batch_stride = 0;   // elements between sequences in eta
 };
 
 }  // namespace bct
@@ -81,8 +83,10 @@ int stream_chunk_tokens(const bct_cache* c);
 // n_chunks whole chunks starting at token t_begin of the [B][T][H][d] step arrays.  fill_len < 0:
 // the cache is full and every token is a read plus a soft write; fill_len >= 0: the cache holds
 // fill_len slots, each chunk is appended (fill_len + n_chunks * Tc <= capacity) and read causally.
+// eta: step size of each token's write, [B][T][Hkv] floats, or NULL.
 int launch_stream_tc(const bct_cache* c, const void* q, const void* k, const void* v, void* out, int64_t T,
-                     int64_t t_begin, int64_t n_chunks, int fill_len, cudaStream_t stream, cudaError_t* err);
+                     const float* eta, int64_t t_begin, int64_t n_chunks, int fill_len, cudaStream_t stream,
+                     cudaError_t* err);
 
 // Set the calling thread's bct_last_error() message (for entry points outside bct_api.cu).
 void set_last_error(const char* msg);

@@ -50,6 +50,7 @@ constexpr int kColA = 384;    // A = Pr WW^T  [row (t,g)] x [write token]
 struct StArgs {
     char* out;
     int* status;
+    const float* eta;  // step size of each token's write, [B][T][Hkv], or NULL (all ones)
     int C, Hq, Hkv, U, T, t_begin, n_chunks, Tc;
     int fill, len0;  // fill = 1: the cache holds len0 slots and each chunk is appended (no soft write)
     int wtr, out_f32, precise;  // precise: the read uses value + residual of both the numerators and MV
@@ -446,7 +447,13 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     m = mn;
                 }
                 const float inv_l = 1.f / l;
-                const float wmul = is_write ? inv_l : 1.f;  // write weights are stored normalised
+                // write weights are stored normalised and carry the token's step size:
+                // MV += sum_t eta_t ww_t^T wv_t, and A = Pr WW^T then holds eta_t as well
+                float wmul = 1.f;
+                if (is_write) {
+                    wmul = inv_l;
+                    if (a.eta != nullptr && !a.fill) wmul *= a.eta[((size_t)b * a.T + t0 + my_t) * a.Hkv + h];
+                }
 
                 // ---- pass 2: numerators (value + residual) of each tile, then the write-back of its MV rows ----
                 for (int t = 0; t < nt; ++t) {
@@ -663,7 +670,8 @@ int stream_chunk_tokens(const bct_cache* c) {
 }
 
 int launch_stream_tc(const bct_cache* c, const void* q, const void* k, const void* v, void* out, int64_t T,
-                     int64_t t_begin, int64_t n_chunks, int fill_len, cudaStream_t stream, cudaError_t* err) {
+                     const float* eta, int64_t t_begin, int64_t n_chunks, int fill_len, cudaStream_t stream,
+                     cudaError_t* err) {
     const bct_params_t& p = c->p;
     StKernelFn fn = pick_stream(c->G);
     const int Tc = stream_chunk_tokens(c);
@@ -686,6 +694,7 @@ int launch_stream_tc(const bct_cache* c, const void* q, const void* k, const voi
     StArgs a;
     a.out = static_cast<char*>(out);
     a.status = c->status;
+    a.eta = eta;
     a.C = p.capacity;
     a.Hq = p.n_q_heads;
     a.Hkv = p.n_kv_heads;
