@@ -18,9 +18,9 @@
 // with fp32 accumulators in tensor memory.  The write weights are always kept as bfloat16
 // value + residual pairs (the state must not drift); with BCT_FLAG_PRECISE_READ the read numerators
 // and MV are too, so that a long stream whose state grows large keeps the output precision.
-//   warp 8  producer : TMA loads (chunk operands, MK / MV tiles through a 3-stage ring)
-//   warp 9  MMA      : issues all tensor-core work, commits to mbarriers
-//   warps 0-7        : two threads per operand row (64 accumulator columns each): online row statistics, numerators, the write-back
+//   warp 16 producer : TMA loads (chunk operands, MK / MV tiles through a 3-stage ring)
+//   warp 17 MMA      : issues all tensor-core work, commits to mbarriers
+//   warps 0-15       : four threads per operand row (32 accumulator columns each): online row statistics, numerators, the write-back
 //                      of MV rows, the intra-chunk term and the epilogue
 // Every wait is bounded; a timeout sets the status word and the kernel runs to its end.
 #include <cuda.h>
@@ -33,8 +33,9 @@
 namespace bct {
 namespace {
 
-constexpr int kStThreads = 320;
-constexpr int kStS = 256;                // row threads: two per operand row
+constexpr int kStRowWarps = 16;
+constexpr int kStS = kStRowWarps * 32;   // row threads: four per operand row
+constexpr int kStThreads = kStS + 64;    // + producer warp + MMA warp
 constexpr int kStTile = 128;             // slots per tile
 constexpr int kStHalf = 128 * 128;       // 64 columns (128 bytes) x 128 rows
 constexpr int kStTileBytes = 2 * kStHalf;
@@ -76,9 +77,16 @@ __host__ __device__ inline StSmem st_smem() {
     L.bars = off;
     off += 32 * 8;
     L.misc = off;
-    off += 64 + 2 * 128 * 2 * 4;  // flags, then (max, sum) of each half row
+    off += 64 + 4 * 128 * 2 * 4;  // flags, then (max, sum) of each quarter row
     L.total = off + 1024;       // slack to align the base to 1024 bytes
     return L;
+}
+
+// 2^x (approximate, flushes denormals): every exponential of the kernel
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
 }
 
 __device__ __forceinline__ void st_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kStS) : "memory"); }
@@ -162,7 +170,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     }
     // rows of the query operand beyond the chunk's G*Tc + Tc stay zero for good
     for (int i = tid; i < kStTileBytes / 16; i += kStThreads) reinterpret_cast<uint4*>(qall)[i] = make_uint4(0, 0, 0, 0);
-    if (warp == 9) tmem_alloc(tmem_slot, 512);
+    if (warp == kStRowWarps + 1) tmem_alloc(tmem_slot, 512);
     fence_proxy_async_smem();
     tc_fence_before();
     __syncthreads();
@@ -175,7 +183,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         *abort_flag = 1;                                                        \
     }
 
-    if (warp == 8) {
+    if (warp == kStRowWarps) {
         // =========================== producer ===========================
         if (lane == 0) {
             uint32_t kc = 0, qn = 0, nw = 0;
@@ -244,7 +252,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             }
         }
         __syncwarp();
-    } else if (warp == 9) {
+    } else if (warp == kStRowWarps + 1) {
         // =========================== MMA issuer ===========================
         if (lane == 0) {
             constexpr uint32_t id_scores = instr_desc_mn(128, 128, false, false);  // Qall (K) x tile (K)
@@ -368,17 +376,21 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         __syncwarp();
     } else {
         // =========================== row threads: statistics, numerators, write-back, epilogue ===========================
-        // Two threads per operand row (tensor-memory lane): thread half hf works on columns
-        // [64 hf, 64 hf + 64) of every 128-column accumulator.
+        // Four threads per operand row (tensor-memory lane): thread quarter cq works on columns
+        // [32 cq, 32 cq + 32) of every 128-column accumulator.  Exponentials are taken in base 2:
+        // scores are multiplied by scale * log2(e) once, maxima are kept in that domain.
         const int r = tid & 127;
-        const int hf = tid >> 7;
-        const uint32_t lane_base = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + hf * 64;
+        const int cq = tid >> 7;
+        const uint32_t lane_base = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + cq * 32;
         const bool is_read = r < n_read;
         const bool is_write = !is_read && r < n_read + Tc;
         const int my_t = is_read ? r / G : (is_write ? r - n_read : 0);  // token of the chunk this row belongs to
         const int my_g = is_read ? r - my_t * G : 0;
-        const float scale = is_read ? a.read_scale : a.write_scale;
-        const int sw = r & 7;                           // swizzle phase of this row
+        const float c2 = (is_read ? a.read_scale : a.write_scale) * 1.4426950408889634f;
+        const int sw = r & 7;                                // swizzle phase of this row
+        const int poff = (cq >> 1) * kStHalf + r * 128;      // this thread's 64 bytes: chunks (cq & 1) * 4 + j
+        const int pch = (cq & 1) * 4;
+        const bool active = is_read || (is_write && !a.fill);  // rows that produce numerators
         uint32_t kc = 0, qn = 0, su0 = 0, su1 = 0, np = 0, nd = 0;
         for (int u = blockIdx.x; u < a.U; u += gridDim.x) {
             const int b = u / a.Hkv, h = u - b * a.Hkv;
@@ -386,7 +398,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 const int t0 = a.t_begin + ch * Tc;
                 const int nt = chunk_tiles(ch);
                 const int clen = chunk_len(ch);
-                // ---- pass 1: online maximum and sum of this half row's scaled scores over the resident slots ----
+                // ---- pass 1: online maximum and sum of this quarter row's scaled scores over the resident slots ----
                 float m = kStNegBig, l = 0.f;
                 for (int t = 0; t < nt; ++t, ++kc) {
                     const int buf = t & 1;
@@ -394,56 +406,75 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     ST_WAIT(&sready[buf], su, 61);
                     ++su;
                     tc_fence_after();
-                    const int n_valid = min(kStTile, clen - t * kStTile) - hf * 64;
-                    float x[64];
-                    tmem_ld64(lane_base + (buf ? kColD : kColS0), x);
-                    float bm = kStNegBig;
-#pragma unroll
-                    for (int i = 0; i < 64; ++i) {
-                        x[i] = (i < n_valid) ? x[i] * scale : kStNegBig;
-                        bm = fmaxf(bm, x[i]);
-                    }
-                    const float mn = fmaxf(m, bm);
-                    float s0 = 0.f, s1 = 0.f;
-#pragma unroll
-                    for (int i = 0; i < 64; i += 2) {
-                        s0 += __expf(x[i] - mn);
-                        s1 += __expf(x[i + 1] - mn);
-                    }
-                    l = l * __expf(m - mn) + (s0 + s1);
-                    m = mn;
+                    const int n_valid = min(kStTile, clen - t * kStTile) - cq * 32;
+                    float x[32];
+                    tmem_ld32(lane_base + (buf ? kColD : kColS0), x);
                     tc_fence_before();
-                    mbar_arrive(&sfree[buf]);
+                    mbar_arrive(&sfree[buf]);  // the scores are in registers
+                    if (n_valid >= 32) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) x[i] *= c2;
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) x[i] = (i < n_valid) ? x[i] * c2 : kStNegBig;
+                    }
+                    float b0 = fmaxf(x[0], x[1]), b1 = fmaxf(x[2], x[3]), b2 = fmaxf(x[4], x[5]), b3 = fmaxf(x[6], x[7]);
+#pragma unroll
+                    for (int i = 8; i < 32; i += 8) {
+                        b0 = fmaxf(b0, fmaxf(x[i], x[i + 1]));
+                        b1 = fmaxf(b1, fmaxf(x[i + 2], x[i + 3]));
+                        b2 = fmaxf(b2, fmaxf(x[i + 4], x[i + 5]));
+                        b3 = fmaxf(b3, fmaxf(x[i + 6], x[i + 7]));
+                    }
+                    const float mn = fmaxf(m, fmaxf(fmaxf(b0, b1), fmaxf(b2, b3)));
+                    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+                    for (int i = 0; i < 32; i += 4) {
+                        s0 += ex2(x[i] - mn);
+                        s1 += ex2(x[i + 1] - mn);
+                        s2 += ex2(x[i + 2] - mn);
+                        s3 += ex2(x[i + 3] - mn);
+                    }
+                    l = l * ex2(m - mn) + ((s0 + s1) + (s2 + s3));
+                    m = mn;
                 }
                 if (a.fill) {
                     // fill phase: token t also sees the chunk's own slots s <= t (it is appended before it reads);
-                    // thread half hf covers chunk tokens [32 hf, 32 hf + 32)
+                    // thread quarter cq covers chunk tokens [16 cq, 16 cq + 16)
                     ST_WAIT(ccready, qn, 68);
                     tc_fence_after();
-                    float cc[32];
-                    tmem_ld32(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + kColA + hf * 32, cc);
+                    float cc[16];
+                    const uint32_t cbase = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + kColA + cq * 16;
+                    tmem_ld8(cbase, cc);
+                    tmem_ld8(cbase + 8, cc + 8);
                     float bm = kStNegBig;
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        const int s = hf * 32 + i;
-                        cc[i] = (is_read && s < Tc && s <= my_t) ? cc[i] * scale : kStNegBig;
+                    for (int i = 0; i < 16; ++i) {
+                        const int s = cq * 16 + i;
+                        cc[i] = (is_read && s < Tc && s <= my_t) ? cc[i] * c2 : kStNegBig;
                         bm = fmaxf(bm, cc[i]);
                     }
                     const float mn = fmaxf(m, bm);
                     float s0 = 0.f;
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) s0 += (cc[i] > kStNegBig) ? __expf(cc[i] - mn) : 0.f;
-                    l = l * __expf(m - mn) + s0;
+                    for (int i = 0; i < 16; ++i) s0 += (cc[i] > kStNegBig) ? ex2(cc[i] - mn) : 0.f;
+                    l = l * ex2(m - mn) + s0;
                     m = mn;
                 }
-                // combine the two halves of the row
-                rowstat[(hf * 128 + r) * 2] = m;
-                rowstat[(hf * 128 + r) * 2 + 1] = l;
+                // combine the four quarters of the row
+                rowstat[(cq * 128 + r) * 2] = m;
+                rowstat[(cq * 128 + r) * 2 + 1] = l;
                 st_sync();
                 {
-                    const float mo = rowstat[((hf ^ 1) * 128 + r) * 2], lo_ = rowstat[((hf ^ 1) * 128 + r) * 2 + 1];
-                    const float mn = fmaxf(m, mo);
-                    l = l * __expf(m - mn) + lo_ * __expf(mo - mn);
+                    float mn = m;
+#pragma unroll
+                    for (int o = 1; o < 4; ++o) mn = fmaxf(mn, rowstat[(((cq + o) & 3) * 128 + r) * 2]);
+                    l *= ex2(m - mn);
+#pragma unroll
+                    for (int o = 1; o < 4; ++o) {
+                        const int idx = (((cq + o) & 3) * 128 + r) * 2;
+                        l += rowstat[idx + 1] * ex2(rowstat[idx] - mn);
+                    }
                     m = mn;
                 }
                 const float inv_l = 1.f / l;
@@ -466,24 +497,42 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     const int vl = kc % kStStages;
                     const uint32_t vl_par = kc / kStStages;
                     ++kc;
-                    if (np > 0) ST_WAIT(pfree, np - 1, 63);
                     tc_fence_after();
                     {
-                        const int n_valid = min(kStTile, clen - t * kStTile) - hf * 64;
-                        float x[64];
-                        tmem_ld64(lane_base + kColS0, x);
+                        const int n_valid = min(kStTile, clen - t * kStTile) - cq * 32;
+                        float x[32];
+                        tmem_ld32(lane_base + kColS0, x);
                         tc_fence_before();
                         mbar_arrive(&sfree[0]);  // the scores are in registers: the next tile's may be computed
+                        if (!active) {
 #pragma unroll
-                        for (int i = 0; i < 64; ++i)
-                            x[i] = ((is_read || (is_write && !a.fill)) && i < n_valid) ? __expf(x[i] * scale - m) * wmul : 0.f;
+                            for (int i = 0; i < 32; ++i) x[i] = 0.f;
+                        } else if (n_valid >= 32) {
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) {  // 16-byte chunk j of this half = 8 slots
-                            uint4 hi, lo;
-                            split8(x + 8 * j, &hi, &lo);
-                            const int off = hf * kStHalf + r * 128 + ((j ^ sw) * 16);
-                            *reinterpret_cast<uint4*>(phi + off) = hi;
-                            if (is_write || a.precise) *reinterpret_cast<uint4*>(plo + off) = lo;  // write weights always keep it
+                            for (int i = 0; i < 32; ++i) x[i] = ex2(fmaf(x[i], c2, -m));
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) x[i] = (i < n_valid) ? ex2(fmaf(x[i], c2, -m)) : 0.f;
+                        }
+                        if (is_write) {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) x[i] *= wmul;
+                        }
+                        if (np > 0) ST_WAIT(pfree, np - 1, 63);  // the previous tile's MMAs have read the operand buffers
+                        if (is_write || a.precise) {  // write weights always keep the residual
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {  // 16-byte chunk = 8 slots
+                                uint4 hi, lo;
+                                split8(x + 8 * j, &hi, &lo);
+                                const int off = poff + (((pch + j) ^ sw) * 16);
+                                *reinterpret_cast<uint4*>(phi + off) = hi;
+                                *reinterpret_cast<uint4*>(plo + off) = lo;
+                            }
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 4; ++j)
+                                *reinterpret_cast<uint4*>(phi + poff + (((pch + j) ^ sw) * 16)) =
+                                    Chunk<__nv_bfloat16>::pack(x + 8 * j);
                         }
                     }
                     fence_proxy_async_smem();
@@ -491,86 +540,85 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     ++np;
                     if (a.fill) continue;  // no soft write while the cache fills
 
-                    // the tile's MV rows: value + residual + increment, split again, stored (this thread: 64 of the 128 d)
+                    // the tile's MV rows: value + residual + increment, split again, stored (this thread: 32 of the 128 d)
                     ST_WAIT(&full[vh], vh_par, 64);
                     ST_WAIT(&full[vl], vl_par, 65);
                     ST_WAIT(dready, nd, 66);
                     ++nd;
                     tc_fence_after();
                     {
-                        unsigned char* th = ring + (size_t)vh * kStTileBytes + hf * kStHalf + r * 128;
-                        unsigned char* tl = ring + (size_t)vl * kStTileBytes + hf * kStHalf + r * 128;
-                        float dx[64];
-                        tmem_ld64(lane_base + kColD, dx);
+                        unsigned char* th = ring + (size_t)vh * kStTileBytes + poff;
+                        unsigned char* tl = ring + (size_t)vl * kStTileBytes + poff;
+                        float dx[32];
+                        tmem_ld32(lane_base + kColD, dx);
                         tc_fence_before();
                         mbar_arrive(dfree);
-                        {  // rows past C of a ragged last tile are clipped by the store
+                        // rows past C of a ragged last tile are clipped by the store
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) {
-                                const int off = (j ^ sw) * 16;
-                                float vh8[8], vl8[8], nv[8];
-                                Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(th + off), vh8);
-                                Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(tl + off), vl8);
+                        for (int j = 0; j < 4; ++j) {
+                            const int off = ((pch + j) ^ sw) * 16;
+                            float vh8[8], vl8[8], nv[8];
+                            Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(th + off), vh8);
+                            Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(tl + off), vl8);
 #pragma unroll
-                                for (int e = 0; e < 8; ++e) nv[e] = (vh8[e] + vl8[e]) + dx[8 * j + e];
-                                uint4 hi, lo;
-                                split8(nv, &hi, &lo);
-                                *reinterpret_cast<uint4*>(th + off) = hi;  // in place: the producer stores the stage
-                                *reinterpret_cast<uint4*>(tl + off) = lo;
-                            }
+                            for (int e = 0; e < 8; ++e) nv[e] = (vh8[e] + vl8[e]) + dx[8 * j + e];
+                            uint4 hi, lo;
+                            split8(nv, &hi, &lo);
+                            *reinterpret_cast<uint4*>(th + off) = hi;  // in place: the producer stores the stage
+                            *reinterpret_cast<uint4*>(tl + off) = lo;
                         }
                     }
                     fence_proxy_async_smem();
                     mbar_arrive(wready);
                 }
 
-                // ---- intra-chunk term: row (t, g) sees the writes of tokens s < t (s <= t when the read
-                // ---- follows the write); A is masked, rounded to bfloat16 and handed back as an operand ----
+                // ---- intra-chunk term: thread quarter cq covers chunk tokens [16 cq, 16 cq + 16) ----
                 if (a.fill) {
-                    // fill phase: numerators of the chunk's own slots, exp(score - m) for s <= t, as value + residual
+                    // fill phase: numerators of the chunk's own slots, 2^(score - m) for s <= t, as value + residual
                     if (np > 0) ST_WAIT(pfree, np - 1, 69);  // the last tile's MMAs have read the residual buffer
                     tc_fence_after();
-                    float cc[32];
-                    tmem_ld32(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + kColA + hf * 32, cc);
-                    if (hf * 32 < Tc) {
+                    if (cq * 16 < Tc) {
+                        float cc[16];
+                        const uint32_t cbase = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + kColA + cq * 16;
+                        tmem_ld8(cbase, cc);
+                        tmem_ld8(cbase + 8, cc + 8);
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const int c = hf * 4 + j;
-                            if (c * 8 < Tc) {
-                                float z[8];
+                        for (int j = 0; j < 2; ++j) {
+                            const int c = cq * 2 + j;
+                            float z[8];
 #pragma unroll
-                                for (int e = 0; e < 8; ++e) {
-                                    const int s = c * 8 + e;
-                                    z[e] = (is_read && s <= my_t) ? __expf(cc[8 * j + e] * scale - m) : 0.f;
-                                }
-                                uint4 hi, lo;
-                                split8(z, &hi, &lo);
-                                *reinterpret_cast<uint4*>(plo + r * 128 + ((c ^ sw) * 16)) = hi;
-                                if (a.precise) *reinterpret_cast<uint4*>(plo + kStHalf + r * 128 + ((c ^ sw) * 16)) = lo;
+                            for (int e = 0; e < 8; ++e) {
+                                const int s = c * 8 + e;
+                                z[e] = (is_read && s <= my_t) ? ex2(fmaf(cc[8 * j + e], c2, -m)) : 0.f;
                             }
+                            uint4 hi, lo;
+                            split8(z, &hi, &lo);
+                            *reinterpret_cast<uint4*>(plo + r * 128 + ((c ^ sw) * 16)) = hi;
+                            if (a.precise) *reinterpret_cast<uint4*>(plo + kStHalf + r * 128 + ((c ^ sw) * 16)) = lo;
                         }
                     }
                     tc_fence_before();
                     fence_proxy_async_smem();
                     mbar_arrive(aready);
                 } else {
-                    // thread half hf covers write tokens [32 hf, 32 hf + 32)
-                    float av[32];
-                    tmem_ld32(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + kColA + hf * 32, av);
-                    if (hf * 32 < Tc) {
+                    // row (t, g) sees the writes of tokens s < t (s <= t when the read follows the write);
+                    // A is masked, rounded to bfloat16 and handed back as an operand
+                    if (cq * 16 < Tc) {
+                        float av[16];
+                        const uint32_t abase = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + kColA + cq * 16;
+                        tmem_ld8(abase, av);
+                        tmem_ld8(abase + 8, av + 8);
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const int c = hf * 4 + j;
-                            if (c * 8 < Tc) {
-                                float z[8];
+                        for (int j = 0; j < 2; ++j) {
+                            const int c = cq * 2 + j;
+                            float z[8];
 #pragma unroll
-                                for (int e = 0; e < 8; ++e) {
-                                    const int s = c * 8 + e;
-                                    const bool seen = is_read && (a.wtr ? s <= my_t : s < my_t);
-                                    z[e] = seen ? av[8 * j + e] : 0.f;
-                                }
-                                *reinterpret_cast<uint4*>(plo + r * 128 + ((c ^ sw) * 16)) = Chunk<__nv_bfloat16>::pack(z);
+                            for (int e = 0; e < 8; ++e) {
+                                const int s = c * 8 + e;
+                                const bool seen = is_read && (a.wtr ? s <= my_t : s < my_t);
+                                z[e] = seen ? av[8 * j + e] : 0.f;
                             }
+                            *reinterpret_cast<uint4*>(plo + r * 128 + ((c ^ sw) * 16)) = Chunk<__nv_bfloat16>::pack(z);
                         }
                     }
                     tc_fence_before();
@@ -578,24 +626,24 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     mbar_arrive(aready);
                 }
 
-                // ---- epilogue: this row's outputs (this thread: 64 of the 128 d), normalised by the row sum ----
+                // ---- epilogue: this row's outputs (this thread: 32 of the 128 d), normalised by the row sum ----
                 ST_WAIT(oready, qn, 67);
                 tc_fence_after();
                 {
-                    const size_t orow = (((size_t)b * a.T + t0 + my_t) * a.Hq + (size_t)h * G + my_g) * 128 + hf * 64;
-                    float o[64];
-                    tmem_ld64(lane_base + kColO, o);
+                    const size_t orow = (((size_t)b * a.T + t0 + my_t) * a.Hq + (size_t)h * G + my_g) * 128 + cq * 32;
+                    float o[32];
+                    tmem_ld32(lane_base + kColO, o);
                     if (is_read && a.out != nullptr && !*abort_flag) {
 #pragma unroll
-                        for (int i = 0; i < 64; ++i) o[i] *= inv_l;
+                        for (int i = 0; i < 32; ++i) o[i] *= inv_l;
                         if (a.out_f32) {
                             float4* dst = reinterpret_cast<float4*>(a.out + orow * 4);
 #pragma unroll
-                            for (int j = 0; j < 16; ++j) dst[j] = make_float4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+                            for (int j = 0; j < 8; ++j) dst[j] = make_float4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
                         } else {
                             uint4* dst = reinterpret_cast<uint4*>(a.out + orow * 2);
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) dst[j] = Chunk<__nv_bfloat16>::pack(o + 8 * j);
+                            for (int j = 0; j < 4; ++j) dst[j] = Chunk<__nv_bfloat16>::pack(o + 8 * j);
                         }
                     }
                 }
@@ -608,7 +656,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 
     tc_fence_before();
     __syncthreads();
-    if (warp == 9) {
+    if (warp == kStRowWarps + 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, 512);
     }
