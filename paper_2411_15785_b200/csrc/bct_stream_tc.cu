@@ -297,22 +297,29 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         umma_commit(&empty[stage]);
                         ++su;
                     }
-                    for (int t = 0; t < nt; ++t) {  // pass 2
-                        const int ks = kc % kStStages;
-                        ST_WAIT(&full[ks], kc / kStStages, 44);
+                    // pass 2: the scores of tile t + 1 are issued before the products of tile t, so that the row
+                    // threads turn them into numerators while the tensor pipe works on tile t
+                    const uint32_t kc0 = kc;  // ring position of the pass's first tile: K, MV value, MV residual per tile
+                    auto issue_scores = [&](int t) {
+                        const uint32_t ki = kc0 + 3u * (uint32_t)t;
+                        const int ks = ki % kStStages;
+                        ST_WAIT(&full[ks], ki / kStStages, 44);
                         if (su0 > 0) ST_WAIT(&sfree[0], su0 - 1, 45);
                         tc_fence_after();
                         scores(kColS0, smem_u32(ring + (size_t)ks * kStTileBytes));
                         umma_commit(&sready[0]);
                         umma_commit(&empty[ks]);
                         ++su0;
-                        ++kc;
-                        const int vh = kc % kStStages;
-                        const uint32_t vh_par = kc / kStStages;
-                        ++kc;
-                        const int vl = kc % kStStages;
-                        const uint32_t vl_par = kc / kStStages;
-                        ++kc;
+                    };
+                    if (nt > 0) issue_scores(0);
+                    kc = kc0 + 3u * (uint32_t)nt;
+                    for (int t = 0; t < nt; ++t) {
+                        if (t + 1 < nt) issue_scores(t + 1);
+                        const uint32_t vi = kc0 + 3u * (uint32_t)t + 1u;
+                        const int vh = vi % kStStages;
+                        const uint32_t vh_par = vi / kStStages;
+                        const int vl = (vi + 1u) % kStStages;
+                        const uint32_t vl_par = (vi + 1u) / kStStages;
                         ST_WAIT(pready, np, 46);
                         ++np;
                         ST_WAIT(&full[vh], vh_par, 47);
@@ -340,13 +347,6 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                             umma_commit(&empty[vl]);
                             continue;
                         }
-                        // A += P x WW^T over this tile's slots (write rows start at n_read)
-#pragma unroll
-                        for (int kk = 0; kk < 8; ++kk) {
-                            const uint32_t po = (kk >> 2) * kStHalf + (kk & 3) * 32;
-                            umma_bf16(tmem_base + kColA, smem_desc(phiaddr + po, 16, 1024),
-                                      smem_desc(phiaddr + n_read * 128 + po, 16, 1024), id_a, (t > 0) || (kk > 0));
-                        }
                         // increment of this tile's MV rows: (WW + WW_residual)^T x Vc, 16 tokens per step
                         for (int kk = 0; kk < Tc / 16; ++kk) {
                             const uint64_t vd = smem_desc(vcaddr + kk * 2048, (uint32_t)vc_half, 1024);
@@ -355,7 +355,14 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                             umma_bf16(tmem_base + kColD, smem_desc(ploaddr + n_read * 128 + kk * 2048, kStHalf, 1024), vd,
                                       id_delta, true);
                         }
-                        umma_commit(dready);
+                        umma_commit(dready);  // the write-back may start: outputs and increment are complete
+                        // A += P x WW^T over this tile's slots (write rows start at n_read)
+#pragma unroll
+                        for (int kk = 0; kk < 8; ++kk) {
+                            const uint32_t po = (kk >> 2) * kStHalf + (kk & 3) * 32;
+                            umma_bf16(tmem_base + kColA, smem_desc(phiaddr + po, 16, 1024),
+                                      smem_desc(phiaddr + n_read * 128 + po, 16, 1024), id_a, (t > 0) || (kk > 0));
+                        }
                         umma_commit(pfree);
                         ++nd;
                     }
@@ -486,86 +493,93 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     if (a.eta != nullptr && !a.fill) wmul *= a.eta[((size_t)b * a.T + t0 + my_t) * a.Hkv + h];
                 }
 
-                // ---- pass 2: numerators (value + residual) of each tile, then the write-back of its MV rows ----
-                for (int t = 0; t < nt; ++t) {
+                // ---- pass 2: numerators of each tile, then the write-back of its MV rows.  The numerators of
+                // ---- tile t + 1 are taken (into registers) while the tensor pipe works on tile t ----
+                const uint32_t kc0 = kc;  // ring position of the pass's first tile: K, MV value, MV residual per tile
+                kc = kc0 + 3u * (uint32_t)nt;
+                float e[32];
+                auto numerators = [&](int t) {
                     ST_WAIT(&sready[0], su0, 62);
                     ++su0;
-                    ++kc;
-                    const int vh = kc % kStStages;
-                    const uint32_t vh_par = kc / kStStages;
-                    ++kc;
-                    const int vl = kc % kStStages;
-                    const uint32_t vl_par = kc / kStStages;
-                    ++kc;
                     tc_fence_after();
-                    {
-                        const int n_valid = min(kStTile, clen - t * kStTile) - cq * 32;
-                        float x[32];
-                        tmem_ld32(lane_base + kColS0, x);
-                        tc_fence_before();
-                        mbar_arrive(&sfree[0]);  // the scores are in registers: the next tile's may be computed
-                        if (!active) {
+                    const int n_valid = min(kStTile, clen - t * kStTile) - cq * 32;
+                    tmem_ld32(lane_base + kColS0, e);
+                    tc_fence_before();
+                    mbar_arrive(&sfree[0]);  // the scores are in registers: the next tile's may be computed
+                    if (!active) {
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) x[i] = 0.f;
-                        } else if (n_valid >= 32) {
+                        for (int i = 0; i < 32; ++i) e[i] = 0.f;
+                    } else if (n_valid >= 32) {
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) x[i] = ex2(fmaf(x[i], c2, -m));
-                        } else {
+                        for (int i = 0; i < 32; ++i) e[i] = ex2(fmaf(e[i], c2, -m));
+                    } else {
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) x[i] = (i < n_valid) ? ex2(fmaf(x[i], c2, -m)) : 0.f;
+                        for (int i = 0; i < 32; ++i) e[i] = (i < n_valid) ? ex2(fmaf(e[i], c2, -m)) : 0.f;
+                    }
+                    if (is_write) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) e[i] *= wmul;
+                    }
+                };
+                if (nt > 0) numerators(0);
+                for (int t = 0; t < nt; ++t) {
+                    if (np > 0) ST_WAIT(pfree, np - 1, 63);  // the previous tile's MMAs have read the operand buffers
+                    if (is_write || a.precise) {  // write weights always keep the residual
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {  // 16-byte chunk = 8 slots
+                            uint4 hi, lo;
+                            split8(e + 8 * j, &hi, &lo);
+                            const int off = poff + (((pch + j) ^ sw) * 16);
+                            *reinterpret_cast<uint4*>(phi + off) = hi;
+                            *reinterpret_cast<uint4*>(plo + off) = lo;
                         }
-                        if (is_write) {
+                    } else {
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) x[i] *= wmul;
-                        }
-                        if (np > 0) ST_WAIT(pfree, np - 1, 63);  // the previous tile's MMAs have read the operand buffers
-                        if (is_write || a.precise) {  // write weights always keep the residual
-#pragma unroll
-                            for (int j = 0; j < 4; ++j) {  // 16-byte chunk = 8 slots
-                                uint4 hi, lo;
-                                split8(x + 8 * j, &hi, &lo);
-                                const int off = poff + (((pch + j) ^ sw) * 16);
-                                *reinterpret_cast<uint4*>(phi + off) = hi;
-                                *reinterpret_cast<uint4*>(plo + off) = lo;
-                            }
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 4; ++j)
-                                *reinterpret_cast<uint4*>(phi + poff + (((pch + j) ^ sw) * 16)) =
-                                    Chunk<__nv_bfloat16>::pack(x + 8 * j);
-                        }
+                        for (int j = 0; j < 4; ++j)
+                            *reinterpret_cast<uint4*>(phi + poff + (((pch + j) ^ sw) * 16)) =
+                                Chunk<__nv_bfloat16>::pack(e + 8 * j);
                     }
                     fence_proxy_async_smem();
                     mbar_arrive(pready);
                     ++np;
+                    if (t + 1 < nt) numerators(t + 1);  // overlaps the tensor-core work on tile t
                     if (a.fill) continue;  // no soft write while the cache fills
 
                     // the tile's MV rows: value + residual + increment, split again, stored (this thread: 32 of the 128 d)
-                    ST_WAIT(&full[vh], vh_par, 64);
-                    ST_WAIT(&full[vl], vl_par, 65);
+                    const uint32_t vi = kc0 + 3u * (uint32_t)t + 1u;
+                    const int vh = vi % kStStages;
+                    const int vl = (vi + 1u) % kStStages;
+                    ST_WAIT(&full[vh], vi / kStStages, 64);
+                    ST_WAIT(&full[vl], (vi + 1u) / kStStages, 65);
                     ST_WAIT(dready, nd, 66);
                     ++nd;
                     tc_fence_after();
                     {
                         unsigned char* th = ring + (size_t)vh * kStTileBytes + poff;
                         unsigned char* tl = ring + (size_t)vl * kStTileBytes + poff;
-                        float dx[32];
-                        tmem_ld32(lane_base + kColD, dx);
-                        tc_fence_before();
-                        mbar_arrive(dfree);
                         // rows past C of a ragged last tile are clipped by the store
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const int off = ((pch + j) ^ sw) * 16;
-                            float vh8[8], vl8[8], nv[8];
-                            Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(th + off), vh8);
-                            Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(tl + off), vl8);
+                        for (int hh = 0; hh < 2; ++hh) {  // 16 columns at a time: the next tile's numerators stay in registers
+                            float dx[16];
+                            tmem_ld8(lane_base + kColD + hh * 16, dx);
+                            tmem_ld8(lane_base + kColD + hh * 16 + 8, dx + 8);
+                            if (hh == 1) {
+                                tc_fence_before();
+                                mbar_arrive(dfree);
+                            }
 #pragma unroll
-                            for (int e = 0; e < 8; ++e) nv[e] = (vh8[e] + vl8[e]) + dx[8 * j + e];
-                            uint4 hi, lo;
-                            split8(nv, &hi, &lo);
-                            *reinterpret_cast<uint4*>(th + off) = hi;  // in place: the producer stores the stage
-                            *reinterpret_cast<uint4*>(tl + off) = lo;
+                            for (int jj = 0; jj < 2; ++jj) {
+                                const int off = ((pch + hh * 2 + jj) ^ sw) * 16;
+                                float vh8[8], vl8[8], nv[8];
+                                Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(th + off), vh8);
+                                Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(tl + off), vl8);
+#pragma unroll
+                                for (int q8 = 0; q8 < 8; ++q8) nv[q8] = (vh8[q8] + vl8[q8]) + dx[8 * jj + q8];
+                                uint4 hi, lo;
+                                split8(nv, &hi, &lo);
+                                *reinterpret_cast<uint4*>(th + off) = hi;  // in place: the producer stores the stage
+                                *reinterpret_cast<uint4*>(tl + off) = lo;
+                            }
                         }
                     }
                     fence_proxy_async_smem();
@@ -603,6 +617,8 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 } else {
                     // row (t, g) sees the writes of tokens s < t (s <= t when the read follows the write);
                     // A is masked, rounded to bfloat16 and handed back as an operand
+                    if (np > 0) ST_WAIT(pfree, np - 1, 70);  // the last tile's A products are complete
+                    tc_fence_after();
                     if (cq * 16 < Tc) {
                         float av[16];
                         const uint32_t abase = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + kColA + cq * 16;
