@@ -39,7 +39,7 @@ constexpr int kStThreads = kStS + 64;    // + producer warp + MMA warp
 constexpr int kStTile = 128;             // slots per tile
 constexpr int kStHalf = 128 * 128;       // 64 columns (128 bytes) x 128 rows
 constexpr int kStTileBytes = 2 * kStHalf;
-constexpr int kStStages = 3;
+constexpr int kStMaxStages = 4;
 constexpr int kStMaxTc = 64;
 constexpr float kStNegBig = -3.0e38f;
 // tensor-memory columns
@@ -60,9 +60,16 @@ struct StArgs {
 
 struct StSmem {
     int qall, vc, phi, plo, ring, bars, misc, total;
+    int stages;    // ring stages of one tile each
+    int plo_half;  // bytes between the two 64-column halves of the residual operand
 };
-__host__ __device__ inline StSmem st_smem() {
+// Shared-memory carve-up, the same on host and device.  With PRECISE_READ every operand row keeps
+// its residual (a full second operand buffer) and the ring has three stages; otherwise only the
+// write rows do (at most 64 rows), and the 16 KiB saved buy a fourth stage.
+__host__ __device__ inline StSmem st_smem(int precise) {
     StSmem L;
+    L.stages = precise ? 3 : kStMaxStages;
+    L.plo_half = precise ? kStHalf : kStMaxTc * 128;
     int off = 0;
     L.qall = off;
     off += kStTileBytes;        // [2 halves][128 rows][128 B]: G*Tc read queries, Tc write queries, zero rows
@@ -71,15 +78,25 @@ __host__ __device__ inline StSmem st_smem() {
     L.phi = off;
     off += kStTileBytes;        // numerators / write weights of one tile, bfloat16 value
     L.plo = off;
-    off += kStTileBytes;        // ... and residual; reused for the masked A operand after the last tile
+    off += 2 * L.plo_half;      // ... and residual; reused for the row statistics and, after the last tile, the masked A operand
     L.ring = off;
-    off += kStStages * kStTileBytes;
+    off += L.stages * kStTileBytes;
     L.bars = off;
     off += 32 * 8;
     L.misc = off;
-    off += 64 + 4 * 128 * 2 * 4;  // flags, then (max, sum) of each quarter row
+    off += 64;                  // flags
     L.total = off + 1024;       // slack to align the base to 1024 bytes
     return L;
+}
+
+// use[s] of a stage picked at run time, without indexing the register array dynamically
+__device__ __forceinline__ uint32_t& use_at(uint32_t (&u)[kStMaxStages], int s) {
+    switch (s) {
+        case 0: return u[0];
+        case 1: return u[1];
+        case 2: return u[2];
+        default: return u[3];
+    }
 }
 
 // 2^x (approximate, flushes denormals): every exponential of the kernel
@@ -110,15 +127,16 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                  const StArgs a) {
     extern __shared__ unsigned char st_smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(st_smem_raw) + 1023) & ~uintptr_t(1023));
-    const StSmem L = st_smem();
+    const StSmem L = st_smem(a.precise);
+    const int ns = L.stages;
     unsigned char* qall = smem + L.qall;
     unsigned char* vc = smem + L.vc;
     unsigned char* phi = smem + L.phi;
     unsigned char* plo = smem + L.plo;
     unsigned char* ring = smem + L.ring;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L.bars);
-    uint64_t* full = bars;            // [3] tile landed (TMA transaction bytes)
-    uint64_t* empty = bars + 3;       // [3] stage may be refilled (one arrival: MMA commit, or the producer after its store)
+    uint64_t* full = bars;            // [4] tile landed (TMA transaction bytes)
+    uint64_t* empty = bars + 20;      // [4] stage may be refilled (one arrival: MMA commit, or the producer after its store)
     uint64_t* qfull = bars + 6;       // chunk operands landed
     uint64_t* qfree = bars + 7;       // chunk operands no longer needed (128 arrivals)
     uint64_t* sready = bars + 8;      // [2] score tile complete (commit)
@@ -133,7 +151,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     uint64_t* wready = bars + 18;     // rewritten MV rows of the tile are in their ring stages (256 arrivals)
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L.misc);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L.misc + 8);
-    float* rowstat = reinterpret_cast<float*>(smem + L.misc + 64);
+    float* rowstat = reinterpret_cast<float*>(plo);  // [4 quarters][128 rows](max, sum): between the two passes only
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
@@ -145,9 +163,34 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     auto chunk_tiles = [&](int ch) { return a.fill ? (a.len0 + ch * a.Tc + kStTile - 1) / kStTile : nt_full; };
     const int n_read = Tc * G;         // rows [0, n_read): read queries (t, g); then Tc write rows
     const int vc_half = Tc * 128;      // bytes between the two 64-column halves of Vc
+    // Ring use.  Pass 1 streams the MK tiles round the stages.  In pass 2 stage 0 takes the MK tiles, the
+    // last stage the residual tiles of MV, and the stages between them the value tiles of MV: two of
+    // them with four stages, so that tile t + 1's values arrive while tile t is rebuilt and stored.
+    // use[s] counts the loads into stage s; every role walks the same sequence.
+    const int st_vl = ns - 1;
+    auto st_vh = [&](int t) { return ns == kStMaxStages ? 1 + (t & 1) : 1; };
+    const bool load_vl = !a.fill || a.precise;  // the residual tiles feed the write-back and the precise read only
+    auto pass1_advance = [&](uint32_t (&use)[kStMaxStages], int nt) {
+#pragma unroll
+        for (int st = 0; st < kStMaxStages; ++st)
+            if (st < ns && nt > st) use[st] += (uint32_t)((nt - st + ns - 1) / ns);
+    };
+    auto pass2_advance = [&](uint32_t (&use)[kStMaxStages], int nt) {
+        use[0] += nt;
+        if (ns == kStMaxStages) {
+            use[1] += (nt + 1) >> 1;
+            use[2] += nt >> 1;
+        } else {
+            use[1] += nt;
+        }
+        if (load_vl) use_at(use, st_vl) += nt;
+    };
+    auto vh_use = [&](uint32_t (&use)[kStMaxStages], int t) {
+        return ns == kStMaxStages ? ((t & 1) ? use[2] : use[1]) + (uint32_t)(t >> 1) : use[1] + (uint32_t)t;
+    };
 
     if (tid == 0) {
-        for (int i = 0; i < 3; ++i) {
+        for (int i = 0; i < kStMaxStages; ++i) {
             mbar_init(&full[i], 1);
             mbar_init(&empty[i], 1);
         }
@@ -186,20 +229,24 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     if (warp == kStRowWarps) {
         // =========================== producer ===========================
         if (lane == 0) {
-            uint32_t kc = 0, qn = 0, nw = 0;
-            auto load_tile = [&](const CUtensorMap* map, int u, int t) {
-                const int stage = kc % kStStages;
-                if (kc >= (uint32_t)kStStages) ST_WAIT(&empty[stage], (kc / kStStages) - 1, 31);
+            uint32_t qn = 0, nw = 0;
+            uint32_t use[kStMaxStages] = {0, 0, 0, 0};
+            auto load_tile = [&](const CUtensorMap* map, int u, int t, int stage) {
+                const uint32_t n = use_at(use, stage)++;
+                if (n > 0) ST_WAIT(&empty[stage], n - 1, 31);
                 unsigned char* dst = ring + (size_t)stage * kStTileBytes;
                 mbar_arrive_expect_tx(&full[stage], kStTileBytes);
                 tma_load_3d(dst, map, 0, t * kStTile, u, &full[stage]);
                 tma_load_3d(dst + kStHalf, map, 64, t * kStTile, u, &full[stage]);
-                ++kc;
             };
             for (int u = blockIdx.x; u < a.U; u += gridDim.x) {
                 const int b = u / a.Hkv, h = u - b * a.Hkv;
                 for (int ch = 0; ch < a.n_chunks; ++ch, ++qn) {
                     const int t0 = a.t_begin + ch * Tc;
+                    const int nt = chunk_tiles(ch);
+                    // the first MK tiles of pass 1 do not depend on the chunk's operands: ask for them first
+                    const int n_early = nt < ns - 1 ? nt : ns - 1;
+                    for (int t = 0; t < n_early; ++t) load_tile(&tmK, u, t, t % ns);
                     if (qn > 0) ST_WAIT(qfree, qn - 1, 32);
                     mbar_arrive_expect_tx(qfull, (uint32_t)(Tc * (G + 2) * 256));
                     tma_load_4d(qall, &tmQ, 0, h * G, t0, b, qfull);
@@ -208,7 +255,6 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     tma_load_4d(qall + kStHalf + n_read * 128, &tmKin, 64, h, t0, b, qfull);
                     tma_load_4d(vc, &tmVin, 0, h, t0, b, qfull);
                     tma_load_4d(vc + vc_half, &tmVin, 64, h, t0, b, qfull);
-                    const int nt = chunk_tiles(ch);
                     if (a.fill) {
                         // fill phase: the chunk's keys and values are appended at slots len .. len + Tc - 1
                         // straight from the operand buffers (the residual plane is zero there already)
@@ -220,33 +266,49 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         tma_store_3d(&tmVapp, 64, len, u, vc + vc_half);
                         bulk_commit();
                     }
-                    for (int t = 0; t < nt; ++t) load_tile(&tmK, u, t);  // pass 1: row statistics
+                    for (int t = n_early; t < nt; ++t) load_tile(&tmK, u, t, t % ns);  // pass 1: row statistics
                     // pass 2: numerators, outputs, update.  The row threads put the rewritten MV rows back
                     // into the two ring stages the tile came in; they go home as TMA stores from here.
-                    int pvh = 0, pvl = 0;
-                    auto store_tile = [&](int t) {
-                        ST_WAIT(wready, nw, 33);
-                        ++nw;
-                        unsigned char* sh = ring + (size_t)pvh * kStTileBytes;
-                        unsigned char* sl = ring + (size_t)pvl * kStTileBytes;
-                        tma_store_3d(&tmVhi, 0, t * kStTile, u, sh);
-                        tma_store_3d(&tmVhi, 64, t * kStTile, u, sh + kStHalf);
-                        tma_store_3d(&tmVlo, 0, t * kStTile, u, sl);
-                        tma_store_3d(&tmVlo, 64, t * kStTile, u, sl + kStHalf);
-                        bulk_commit();
-                        bulk_wait_read();  // the stages have been read out: they may be refilled
-                        mbar_arrive(&empty[pvh]);
-                        mbar_arrive(&empty[pvl]);
-                    };
-                    for (int t = 0; t < nt; ++t) {
-                        load_tile(&tmK, u, t);
-                        if (t > 0 && !a.fill) store_tile(t - 1);
-                        pvh = kc % kStStages;
-                        load_tile(&tmVhi, u, t);
-                        pvl = kc % kStStages;
-                        load_tile(&tmVlo, u, t);
+                    // The MK tile is asked for two tiles ahead (its stage is free as soon as the scores of the
+                    // tile before it are issued, long before tile t is stored), the values one tile ahead when
+                    // there are two value stages.  The residual stage is stored and refilled first: the next
+                    // tile's write-back waits for it.
+                    const bool two_vh = ns == kStMaxStages;
+                    if (nt > 0) {
+                        load_tile(&tmK, u, 0, 0);
+                        load_tile(&tmVhi, u, 0, st_vh(0));
+                        if (load_vl) load_tile(&tmVlo, u, 0, st_vl);
+                        if (nt > 1) load_tile(&tmK, u, 1, 0);
+                        if (nt > 1 && two_vh) load_tile(&tmVhi, u, 1, st_vh(1));
                     }
-                    if (nt > 0 && !a.fill) store_tile(nt - 1);
+                    for (int t = 0; t < nt; ++t) {
+                        if (t + 2 < nt) load_tile(&tmK, u, t + 2, 0);
+                        const int pvh = st_vh(t);
+                        if (!a.fill) {
+                            ST_WAIT(wready, nw, 33);
+                            ++nw;
+                            unsigned char* sh = ring + (size_t)pvh * kStTileBytes;
+                            unsigned char* sl = ring + (size_t)st_vl * kStTileBytes;
+                            tma_store_3d(&tmVlo, 0, t * kStTile, u, sl);
+                            tma_store_3d(&tmVlo, 64, t * kStTile, u, sl + kStHalf);
+                            bulk_commit();
+                            tma_store_3d(&tmVhi, 0, t * kStTile, u, sh);
+                            tma_store_3d(&tmVhi, 64, t * kStTile, u, sh + kStHalf);
+                            bulk_commit();
+                            bulk_wait_read_but_one();  // the residual stage has been read out: it may be refilled
+                            mbar_arrive(&empty[st_vl]);
+                        }
+                        if (t + 1 < nt && load_vl) load_tile(&tmVlo, u, t + 1, st_vl);
+                        if (!a.fill) {
+                            bulk_wait_read();
+                            mbar_arrive(&empty[pvh]);
+                        }
+                        if (two_vh) {
+                            if (t + 2 < nt) load_tile(&tmVhi, u, t + 2, st_vh(t + 2));
+                        } else if (t + 1 < nt) {
+                            load_tile(&tmVhi, u, t + 1, st_vh(t + 1));
+                        }
+                    }
                     bulk_wait_all();  // the next chunk reads these rows again
                 }
             }
@@ -259,7 +321,9 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             constexpr uint32_t id_out = instr_desc_mn(128, 128, false, true);      // P (K) x V tile (MN)
             constexpr uint32_t id_delta = instr_desc_mn(128, 128, true, true);     // WW^T (MN) x Vc (MN)
             const uint32_t id_a = instr_desc_mn(128, (uint32_t)(Tc < 16 ? 16 : Tc), false, false);  // P (K) x WW (K)
-            uint32_t kc = 0, qn = 0, su0 = 0, su1 = 0, np = 0, nd = 0;
+            uint32_t qn = 0, su0 = 0, su1 = 0, np = 0, nd = 0;
+            uint32_t use[kStMaxStages] = {0, 0, 0, 0};
+            const uint32_t plo_row0 = a.precise ? 0u : (uint32_t)n_read;  // first operand row the residual buffer holds
             const uint32_t qaddr = smem_u32(qall), vcaddr = smem_u32(vc), phiaddr = smem_u32(phi), ploaddr = smem_u32(plo);
             auto scores = [&](uint32_t col, uint32_t taddr) {
 #pragma unroll
@@ -285,10 +349,11 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         }
                         umma_commit(ccready);
                     }
-                    for (int t = 0; t < nt; ++t, ++kc) {  // pass 1
-                        const int stage = kc % kStStages;
+                    for (int t = 0; t < nt; ++t) {  // pass 1
+                        const int stage = t % ns;
                         const int buf = t & 1;
-                        ST_WAIT(&full[stage], kc / kStStages, 42);
+                        ST_WAIT(&full[stage], use_at(use, stage), 42);
+                        ++use_at(use, stage);
                         uint32_t& su = buf ? su1 : su0;
                         if (su > 0) ST_WAIT(&sfree[buf], su - 1, 43);
                         tc_fence_after();
@@ -299,31 +364,23 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     }
                     // pass 2: the scores of tile t + 1 are issued before the products of tile t, so that the row
                     // threads turn them into numerators while the tensor pipe works on tile t
-                    const uint32_t kc0 = kc;  // ring position of the pass's first tile: K, MV value, MV residual per tile
                     auto issue_scores = [&](int t) {
-                        const uint32_t ki = kc0 + 3u * (uint32_t)t;
-                        const int ks = ki % kStStages;
-                        ST_WAIT(&full[ks], ki / kStStages, 44);
+                        ST_WAIT(&full[0], use[0] + (uint32_t)t, 44);
                         if (su0 > 0) ST_WAIT(&sfree[0], su0 - 1, 45);
                         tc_fence_after();
-                        scores(kColS0, smem_u32(ring + (size_t)ks * kStTileBytes));
+                        scores(kColS0, smem_u32(ring));
                         umma_commit(&sready[0]);
-                        umma_commit(&empty[ks]);
+                        umma_commit(&empty[0]);
                         ++su0;
                     };
                     if (nt > 0) issue_scores(0);
-                    kc = kc0 + 3u * (uint32_t)nt;
                     for (int t = 0; t < nt; ++t) {
                         if (t + 1 < nt) issue_scores(t + 1);
-                        const uint32_t vi = kc0 + 3u * (uint32_t)t + 1u;
-                        const int vh = vi % kStStages;
-                        const uint32_t vh_par = vi / kStStages;
-                        const int vl = (vi + 1u) % kStStages;
-                        const uint32_t vl_par = (vi + 1u) / kStStages;
+                        const int vh = st_vh(t), vl = st_vl;
                         ST_WAIT(pready, np, 46);
                         ++np;
-                        ST_WAIT(&full[vh], vh_par, 47);
-                        ST_WAIT(&full[vl], vl_par, 48);
+                        ST_WAIT(&full[vh], vh_use(use, t), 47);
+                        if (a.precise) ST_WAIT(&full[vl], use_at(use, vl) + (uint32_t)t, 48);
                         if (nd > 0 && !a.fill) ST_WAIT(dfree, nd - 1, 49);
                         tc_fence_after();
                         const uint32_t vhaddr = smem_u32(ring + (size_t)vh * kStTileBytes);
@@ -344,7 +401,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                             // no soft write while the cache fills: the stages are free once the outputs are done
                             umma_commit(pfree);
                             umma_commit(&empty[vh]);
-                            umma_commit(&empty[vl]);
+                            if (load_vl) umma_commit(&empty[vl]);
                             continue;
                         }
                         // increment of this tile's MV rows: (WW + WW_residual)^T x Vc, 16 tokens per step
@@ -352,7 +409,8 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                             const uint64_t vd = smem_desc(vcaddr + kk * 2048, (uint32_t)vc_half, 1024);
                             umma_bf16(tmem_base + kColD, smem_desc(phiaddr + n_read * 128 + kk * 2048, kStHalf, 1024), vd,
                                       id_delta, kk > 0);
-                            umma_bf16(tmem_base + kColD, smem_desc(ploaddr + n_read * 128 + kk * 2048, kStHalf, 1024), vd,
+                            umma_bf16(tmem_base + kColD,
+                                      smem_desc(ploaddr + ((uint32_t)n_read - plo_row0) * 128 + kk * 2048, (uint32_t)L.plo_half, 1024), vd,
                                       id_delta, true);
                         }
                         umma_commit(dready);  // the write-back may start: outputs and increment are complete
@@ -366,6 +424,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         umma_commit(pfree);
                         ++nd;
                     }
+                    pass2_advance(use, nt);
                     // intra-chunk term: O += strict_tril(A) x Vc (fill phase: the causal numerators of the
                     // chunk's own slots, value + residual, times Vc)
                     ST_WAIT(aready, qn, 50);
@@ -398,7 +457,9 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         const int poff = (cq >> 1) * kStHalf + r * 128;      // this thread's 64 bytes: chunks (cq & 1) * 4 + j
         const int pch = (cq & 1) * 4;
         const bool active = is_read || (is_write && !a.fill);  // rows that produce numerators
-        uint32_t kc = 0, qn = 0, su0 = 0, su1 = 0, np = 0, nd = 0;
+        uint32_t qn = 0, su0 = 0, su1 = 0, np = 0, nd = 0;
+        uint32_t use[kStMaxStages] = {0, 0, 0, 0};
+        const int lo_off = (cq >> 1) * L.plo_half + (r - (a.precise ? 0 : n_read)) * 128;  // residual buffer: write rows only unless precise
         for (int u = blockIdx.x; u < a.U; u += gridDim.x) {
             const int b = u / a.Hkv, h = u - b * a.Hkv;
             for (int ch = 0; ch < a.n_chunks; ++ch, ++qn) {
@@ -407,7 +468,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 const int clen = chunk_len(ch);
                 // ---- pass 1: online maximum and sum of this quarter row's scaled scores over the resident slots ----
                 float m = kStNegBig, l = 0.f;
-                for (int t = 0; t < nt; ++t, ++kc) {
+                for (int t = 0; t < nt; ++t) {
                     const int buf = t & 1;
                     uint32_t& su = buf ? su1 : su0;
                     ST_WAIT(&sready[buf], su, 61);
@@ -484,6 +545,8 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     }
                     m = mn;
                 }
+                st_sync();  // the statistics have been read: the buffer goes back to the residual operand
+                pass1_advance(use, nt);
                 const float inv_l = 1.f / l;
                 // write weights are stored normalised and carry the token's step size:
                 // MV += sum_t eta_t ww_t^T wv_t, and A = Pr WW^T then holds eta_t as well
@@ -495,8 +558,6 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 
                 // ---- pass 2: numerators of each tile, then the write-back of its MV rows.  The numerators of
                 // ---- tile t + 1 are taken (into registers) while the tensor pipe works on tile t ----
-                const uint32_t kc0 = kc;  // ring position of the pass's first tile: K, MV value, MV residual per tile
-                kc = kc0 + 3u * (uint32_t)nt;
                 float e[32];
                 auto numerators = [&](int t) {
                     ST_WAIT(&sready[0], su0, 62);
@@ -531,7 +592,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                             split8(e + 8 * j, &hi, &lo);
                             const int off = poff + (((pch + j) ^ sw) * 16);
                             *reinterpret_cast<uint4*>(phi + off) = hi;
-                            *reinterpret_cast<uint4*>(plo + off) = lo;
+                            *reinterpret_cast<uint4*>(plo + lo_off + (((pch + j) ^ sw) * 16)) = lo;
                         }
                     } else {
 #pragma unroll
@@ -546,11 +607,9 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     if (a.fill) continue;  // no soft write while the cache fills
 
                     // the tile's MV rows: value + residual + increment, split again, stored (this thread: 32 of the 128 d)
-                    const uint32_t vi = kc0 + 3u * (uint32_t)t + 1u;
-                    const int vh = vi % kStStages;
-                    const int vl = (vi + 1u) % kStStages;
-                    ST_WAIT(&full[vh], vi / kStStages, 64);
-                    ST_WAIT(&full[vl], (vi + 1u) / kStStages, 65);
+                    const int vh = st_vh(t), vl = st_vl;
+                    ST_WAIT(&full[vh], vh_use(use, t), 64);
+                    ST_WAIT(&full[vl], use_at(use, vl) + (uint32_t)t, 65);
                     ST_WAIT(dready, nd, 66);
                     ++nd;
                     tc_fence_after();
@@ -585,6 +644,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     fence_proxy_async_smem();
                     mbar_arrive(wready);
                 }
+                pass2_advance(use, nt);
 
                 // ---- intra-chunk term: thread quarter cq covers chunk tokens [16 cq, 16 cq + 16) ----
                 if (a.fill) {
@@ -774,7 +834,7 @@ int launch_stream_tc(const bct_cache* c, const void* q, const void* k, const voi
     a.precise = (p.flags & BCT_FLAG_PRECISE_READ) ? 1 : 0;
     a.read_scale = p.read_scale;
     a.write_scale = p.write_scale;
-    const int smem = st_smem().total;
+    const int smem = st_smem(a.precise).total;
     *err = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (*err != cudaSuccess) return -1;
     const int grid = c->U < c->sm_count ? c->U : c->sm_count;
