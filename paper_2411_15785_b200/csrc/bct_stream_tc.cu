@@ -137,8 +137,10 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L.bars);
     uint64_t* full = bars;            // [4] tile landed (TMA transaction bytes)
     uint64_t* empty = bars + 20;      // [4] stage may be refilled (one arrival: MMA commit, or the producer after its store)
-    uint64_t* qfull = bars + 6;       // chunk operands landed
-    uint64_t* qfree = bars + 7;       // chunk operands no longer needed (128 arrivals)
+    uint64_t* qfull = bars + 6;       // the chunk's read and write queries landed
+    uint64_t* vfull = bars + 5;       // the chunk's write key-value vectors landed
+    uint64_t* qfree_q = bars + 4;     // every product that reads the query operand has been issued and is complete (commit)
+    uint64_t* qfree = bars + 7;       // the chunk's outputs have been read from tensor memory (row-thread arrivals)
     uint64_t* sready = bars + 8;      // [2] score tile complete (commit)
     uint64_t* sfree = bars + 10;      // [2] score tile consumed (128 arrivals)
     uint64_t* pready = bars + 12;     // numerators of the tile written (128 arrivals)
@@ -195,6 +197,8 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             mbar_init(&empty[i], 1);
         }
         mbar_init(qfull, 1);
+        mbar_init(vfull, 1);
+        mbar_init(qfree_q, 1);
         mbar_init(qfree, kStS);
         mbar_init(&sready[0], 1);
         mbar_init(&sready[1], 1);
@@ -239,6 +243,29 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 tma_load_3d(dst, map, 0, t * kStTile, u, &full[stage]);
                 tma_load_3d(dst + kStHalf, map, 64, t * kStTile, u, &full[stage]);
             };
+            // read and write queries of chunk ch of unit u into the query operand
+            auto load_queries = [&](int u, int ch) {
+                const int b = u / a.Hkv, h = u - b * a.Hkv;
+                const int t0 = a.t_begin + ch * Tc;
+                mbar_arrive_expect_tx(qfull, (uint32_t)(Tc * (G + 1) * 256));
+                tma_load_4d(qall, &tmQ, 0, h * G, t0, b, qfull);
+                tma_load_4d(qall + kStHalf, &tmQ, 64, h * G, t0, b, qfull);
+                tma_load_4d(qall + n_read * 128, &tmKin, 0, h, t0, b, qfull);
+                tma_load_4d(qall + kStHalf + n_read * 128, &tmKin, 64, h, t0, b, qfull);
+            };
+            // The query operand is free once the last scores of a chunk are complete, well before the
+            // chunk's last tile is stored: the next chunk's queries are asked for at that point.
+            auto next_queries = [&](int u, int ch) {
+                int u2 = u, ch2 = ch + 1;
+                if (ch2 == a.n_chunks) {
+                    u2 = u + gridDim.x;
+                    ch2 = 0;
+                }
+                if (u2 >= a.U) return;
+                ST_WAIT(qfree_q, qn, 32);
+                if (a.fill) bulk_wait_read();  // the appended keys have been read out of the operand
+                load_queries(u2, ch2);
+            };
             for (int u = blockIdx.x; u < a.U; u += gridDim.x) {
                 const int b = u / a.Hkv, h = u - b * a.Hkv;
                 for (int ch = 0; ch < a.n_chunks; ++ch, ++qn) {
@@ -247,18 +274,16 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     // the first MK tiles of pass 1 do not depend on the chunk's operands: ask for them first
                     const int n_early = nt < ns - 1 ? nt : ns - 1;
                     for (int t = 0; t < n_early; ++t) load_tile(&tmK, u, t, t % ns);
-                    if (qn > 0) ST_WAIT(qfree, qn - 1, 32);
-                    mbar_arrive_expect_tx(qfull, (uint32_t)(Tc * (G + 2) * 256));
-                    tma_load_4d(qall, &tmQ, 0, h * G, t0, b, qfull);
-                    tma_load_4d(qall + kStHalf, &tmQ, 64, h * G, t0, b, qfull);
-                    tma_load_4d(qall + n_read * 128, &tmKin, 0, h, t0, b, qfull);
-                    tma_load_4d(qall + kStHalf + n_read * 128, &tmKin, 64, h, t0, b, qfull);
-                    tma_load_4d(vc, &tmVin, 0, h, t0, b, qfull);
-                    tma_load_4d(vc + vc_half, &tmVin, 64, h, t0, b, qfull);
+                    if (qn == 0) load_queries(u, ch);
+                    if (qn > 0) ST_WAIT(oready, qn - 1, 35);  // the previous chunk's last product has read Vc
+                    mbar_arrive_expect_tx(vfull, (uint32_t)(Tc * 256));
+                    tma_load_4d(vc, &tmVin, 0, h, t0, b, vfull);
+                    tma_load_4d(vc + vc_half, &tmVin, 64, h, t0, b, vfull);
                     if (a.fill) {
                         // fill phase: the chunk's keys and values are appended at slots len .. len + Tc - 1
                         // straight from the operand buffers (the residual plane is zero there already)
                         ST_WAIT(qfull, qn, 34);
+                        ST_WAIT(vfull, qn, 36);
                         const int len = chunk_len(ch);
                         tma_store_3d(&tmKapp, 0, len, u, qall + n_read * 128);
                         tma_store_3d(&tmKapp, 64, len, u, qall + kStHalf + n_read * 128);
@@ -281,8 +306,10 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         if (nt > 1) load_tile(&tmK, u, 1, 0);
                         if (nt > 1 && two_vh) load_tile(&tmVhi, u, 1, st_vh(1));
                     }
+                    if (nt == 0) next_queries(u, ch);
                     for (int t = 0; t < nt; ++t) {
                         if (t + 2 < nt) load_tile(&tmK, u, t + 2, 0);
+                        if (t == nt - 1) next_queries(u, ch);
                         const int pvh = st_vh(t);
                         if (!a.fill) {
                             ST_WAIT(wready, nw, 33);
@@ -348,6 +375,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                                       smem_desc(qaddr + n_read * 128 + o, 16, 1024), id_a, kk > 0);
                         }
                         umma_commit(ccready);
+                        if (nt == 0) umma_commit(qfree_q);  // nothing else reads the query operand
                     }
                     for (int t = 0; t < nt; ++t) {  // pass 1
                         const int stage = t % ns;
@@ -356,6 +384,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         ++use_at(use, stage);
                         uint32_t& su = buf ? su1 : su0;
                         if (su > 0) ST_WAIT(&sfree[buf], su - 1, 43);
+                        if (buf == 1 && nd > 0) ST_WAIT(dfree, nd - 1, 51);  // buffer 1 is the increment's columns
                         tc_fence_after();
                         scores(buf ? kColD : kColS0, smem_u32(ring + (size_t)stage * kStTileBytes));
                         umma_commit(&sready[buf]);
@@ -371,8 +400,13 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         scores(kColS0, smem_u32(ring));
                         umma_commit(&sready[0]);
                         umma_commit(&empty[0]);
+                        if (t == nt - 1) umma_commit(qfree_q);  // the last product that reads the query operand
                         ++su0;
                     };
+                    // the previous chunk's outputs have left tensor memory; this chunk's Vc has landed
+                    if (qn > 0) ST_WAIT(qfree, qn - 1, 52);
+                    ST_WAIT(vfull, qn, 53);
+                    tc_fence_after();
                     if (nt > 0) issue_scores(0);
                     for (int t = 0; t < nt; ++t) {
                         if (t + 1 < nt) issue_scores(t + 1);
