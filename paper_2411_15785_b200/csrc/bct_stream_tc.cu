@@ -326,6 +326,14 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                             mbar_arrive(&empty[st_vl]);
                         }
                         if (t + 1 < nt && load_vl) load_tile(&tmVlo, u, t + 1, st_vl);
+                        if (t + 2 < nt && load_vl) {  // and the one after it towards L2: its load must not wait for HBM
+                            tma_prefetch_3d(&tmVlo, 0, (t + 2) * kStTile, u);
+                            tma_prefetch_3d(&tmVlo, 64, (t + 2) * kStTile, u);
+                            if (!two_vh) {  // one value stage: the same for the values
+                                tma_prefetch_3d(&tmVhi, 0, (t + 2) * kStTile, u);
+                                tma_prefetch_3d(&tmVhi, 64, (t + 2) * kStTile, u);
+                            }
+                        }
                         if (!a.fill) {
                             bulk_wait_read();
                             mbar_arrive(&empty[pvh]);
