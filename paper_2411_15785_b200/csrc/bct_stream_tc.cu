@@ -537,6 +537,10 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         b3 = fmaxf(b3, fmaxf(x[i + 6], x[i + 7]));
                     }
                     const float mn = fmaxf(m, fmaxf(fmaxf(b0, b1), fmaxf(b2, b3)));
+                    if (!is_write) {  // read rows need only the maximum here: their sum is taken from the numerators of pass 2
+                        m = mn;
+                        continue;
+                    }
                     float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
                     for (int i = 0; i < 32; i += 4) {
@@ -555,8 +559,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     tc_fence_after();
                     float cc[16];
                     const uint32_t cbase = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + kColA + cq * 16;
-                    tmem_ld8(cbase, cc);
-                    tmem_ld8(cbase + 8, cc + 8);
+                    tmem_ld16(cbase, cc);
                     float bm = kStNegBig;
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
@@ -564,12 +567,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         cc[i] = (is_read && s < Tc && s <= my_t) ? cc[i] * c2 : kStNegBig;
                         bm = fmaxf(bm, cc[i]);
                     }
-                    const float mn = fmaxf(m, bm);
-                    float s0 = 0.f;
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) s0 += (cc[i] > kStNegBig) ? ex2(cc[i] - mn) : 0.f;
-                    l = l * ex2(m - mn) + s0;
-                    m = mn;
+                    m = fmaxf(m, bm);  // read rows only (write rows see nothing here): the sum comes with the numerators
                 }
                 // combine the four quarters of the row
                 rowstat[(cq * 128 + r) * 2] = m;
@@ -589,12 +587,12 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 }
                 st_sync();  // the statistics have been read: the buffer goes back to the residual operand
                 pass1_advance(use, nt);
-                const float inv_l = 1.f / l;
+                float lr = 0.f;  // read rows: sum of this thread's numerators
                 // write weights are stored normalised and carry the token's step size:
                 // MV += sum_t eta_t ww_t^T wv_t, and A = Pr WW^T then holds eta_t as well
                 float wmul = 1.f;
-                if (is_write) {
-                    wmul = inv_l;
+                if (is_write && !a.fill) {
+                    wmul = 1.f / l;
                     if (a.eta != nullptr && !a.fill) wmul *= a.eta[((size_t)b * a.T + t0 + my_t) * a.Hkv + h];
                 }
 
@@ -622,6 +620,16 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     if (is_write) {
 #pragma unroll
                         for (int i = 0; i < 32; ++i) e[i] *= wmul;
+                    } else {
+                        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+                        for (int i = 0; i < 32; i += 4) {
+                            s0 += e[i];
+                            s1 += e[i + 1];
+                            s2 += e[i + 2];
+                            s3 += e[i + 3];
+                        }
+                        lr += (s0 + s1) + (s2 + s3);
                     }
                 };
                 if (nt > 0) numerators(0);
@@ -662,8 +670,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 #pragma unroll
                         for (int hh = 0; hh < 2; ++hh) {  // 16 columns at a time: the next tile's numerators stay in registers
                             float dx[16];
-                            tmem_ld8(lane_base + kColD + hh * 16, dx);
-                            tmem_ld8(lane_base + kColD + hh * 16 + 8, dx + 8);
+                            tmem_ld16(lane_base + kColD + hh * 16, dx);
                             if (hh == 1) {
                                 tc_fence_before();
                                 mbar_arrive(dfree);
@@ -696,8 +703,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     if (cq * 16 < Tc) {
                         float cc[16];
                         const uint32_t cbase = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + kColA + cq * 16;
-                        tmem_ld8(cbase, cc);
-                        tmem_ld8(cbase + 8, cc + 8);
+                        tmem_ld16(cbase, cc);
 #pragma unroll
                         for (int j = 0; j < 2; ++j) {
                             const int c = cq * 2 + j;
@@ -706,6 +712,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                             for (int e = 0; e < 8; ++e) {
                                 const int s = c * 8 + e;
                                 z[e] = (is_read && s <= my_t) ? ex2(fmaf(cc[8 * j + e], c2, -m)) : 0.f;
+                                lr += z[e];
                             }
                             uint4 hi, lo;
                             split8(z, &hi, &lo);
@@ -724,8 +731,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     if (cq * 16 < Tc) {
                         float av[16];
                         const uint32_t abase = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + kColA + cq * 16;
-                        tmem_ld8(abase, av);
-                        tmem_ld8(abase + 8, av + 8);
+                        tmem_ld16(abase, av);
 #pragma unroll
                         for (int j = 0; j < 2; ++j) {
                             const int c = cq * 2 + j;
@@ -747,6 +753,11 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 // ---- epilogue: this row's outputs (this thread: 32 of the 128 d), normalised by the row sum ----
                 ST_WAIT(oready, qn, 67);
                 tc_fence_after();
+                // the row sum of a read row: its four quarters' sums of numerators (the residual operand is free again)
+                rowstat[cq * 128 + r] = lr;
+                st_sync();
+                const float inv_l = 1.f / ((rowstat[r] + rowstat[128 + r]) + (rowstat[256 + r] + rowstat[384 + r]));
+                st_sync();
                 {
                     const size_t orow = (((size_t)b * a.T + t0 + my_t) * a.Hq + (size_t)h * G + my_g) * 128 + cq * 32;
                     float o[32];
