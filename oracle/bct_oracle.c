@@ -228,3 +228,29 @@ int bct_oracle_read_weights(int64_t n, int d, const double *MK, const double *q,
     free(s);
     return 0;
 }
+
+/*
+ * The projections in front of the layer (Algorithm 1, "Compute write query" and "Compute
+ * write key-value vector": wq_t = W_wq x_t, wv_t = W_wv x_t; the read query of the
+ * attention layer is projected the same way):
+ *     y[m][n] = sum_k x[m][k] * W[n][k]
+ * x [M][K] one row per token, W [N][K] one row per output feature, y [M][N].
+ * Returns the number of threads used, or -1 on bad arguments.
+ */
+int bct_oracle_project(int64_t M, int64_t K, int64_t N, const double *x, const double *W, double *y,
+                       int nthreads) {
+    if (M < 0 || K < 1 || N < 1 || !x || !W || !y) return -1;
+    int used = 1;
+#ifdef _OPENMP
+    if (nthreads > 0) omp_set_num_threads(nthreads);
+    used = omp_get_max_threads();
+#pragma omp parallel for schedule(static)
+#endif
+    for (int64_t m = 0; m < M; ++m)
+        for (int64_t n = 0; n < N; ++n) {
+            double acc = 0.0;
+            for (int64_t k = 0; k < K; ++k) acc += x[m * K + k] * W[n * K + k];
+            y[m * N + n] = acc;
+        }
+    return used;
+}

@@ -66,6 +66,8 @@ def _load():
             ctypes.c_int64, ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.c_int64,
             ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64),
             dp, dp, dp, dp, dp, dp, dp, ctypes.c_double, ctypes.c_double, ctypes.c_uint, ctypes.c_int]
+        lib.bct_oracle_project.restype = ctypes.c_int
+        lib.bct_oracle_project.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, dp, dp, dp, ctypes.c_int]
         lib.bct_oracle_write_weights.restype = ctypes.c_int
         lib.bct_oracle_write_weights.argtypes = [ctypes.c_int64, ctypes.c_int, dp, dp,
                                                  ctypes.c_double, dp]
@@ -106,6 +108,43 @@ def read_weights(MK, q, read_scale: float) -> np.ndarray:
     if rc != 0:
         raise RuntimeError("bct_oracle_read_weights failed")
     return p
+
+
+def project(x, W, nthreads: int = 0) -> np.ndarray:
+    """y = x . W^T: x ``[..., K]`` (one row per token), W ``[N, K]`` (one row per output feature)
+    -> ``[..., N]`` float64 (Algorithm 1: wq_t = W_wq x_t, wv_t = W_wv x_t)."""
+    x = _f64(x)
+    W = _f64(W)
+    K = x.shape[-1]
+    N = W.shape[0]
+    assert W.shape == (N, K), (W.shape, K)
+    x2 = np.ascontiguousarray(x.reshape(-1, K))
+    y = np.empty((x2.shape[0], N), dtype=np.float64)
+    rc = _load().bct_oracle_project(x2.shape[0], K, N, _dptr(x2), _dptr(W), _dptr(y), int(nthreads))
+    if rc < 0:
+        raise RuntimeError("bct_oracle_project failed")
+    return y.reshape(x.shape[:-1] + (N,))
+
+
+def round_bf16(a) -> np.ndarray:
+    """Round to the nearest bfloat16 (ties to even), returned as float64: the storage type of the
+    step vectors when the cache is bfloat16."""
+    f = np.ascontiguousarray(np.asarray(a, dtype=np.float32))
+    u = f.view(np.uint32).astype(np.uint64)
+    u = (u + 0x7FFF + ((u >> 16) & 1)) & 0xFFFF0000
+    return u.astype(np.uint32).view(np.float32).astype(np.float64).reshape(f.shape)
+
+
+def layer_step_inputs(x, Wq, Wwq, Wwv, n_q_heads, n_kv_heads, head_dim, bf16: bool = True):
+    """Projections of a block of tokens x ``[B, T, d_model]`` into the step vectors of the layer:
+    q ``[B, T, Hq, d]``, k (= wq) and v (= wv) ``[B, T, Hkv, d]``, rounded to the step-vector
+    storage type."""
+    B, T = x.shape[0], x.shape[1]
+    rnd = round_bf16 if bf16 else (lambda z: np.asarray(z, dtype=np.float32).astype(np.float64))
+    q = rnd(project(x, Wq)).reshape(B, T, n_q_heads, head_dim)
+    k = rnd(project(x, Wwq)).reshape(B, T, n_kv_heads, head_dim)
+    v = rnd(project(x, Wwv)).reshape(B, T, n_kv_heads, head_dim)
+    return q, k, v
 
 
 class OracleCache:

@@ -447,3 +447,52 @@ def test_step_size_equals_a_scaled_write_value_in_the_full_phase():
         ob = b.prefill_stream(q, k, eta[..., None] * v)
         np.testing.assert_allclose(oa, ob, rtol=0, atol=1e-12)
         np.testing.assert_allclose(a.values(), b.values(), rtol=0, atol=1e-12)
+
+
+# ---------------------------------------------------------------------------------------
+# Projections in front of the layer (Algorithm 1: wq_t = W_wq x_t, wv_t = W_wv x_t)
+# ---------------------------------------------------------------------------------------
+def test_projection_brute_force_and_operand_roles():
+    M, K, N = 3, 4, 5                               # all different: a transposed operand cannot pass
+    x, W = _rand(M, K), _rand(N, K)
+    y = O.project(x, W)
+    assert y.shape == (M, N)
+    for m in range(M):
+        for n in range(N):
+            acc = 0.0
+            for k in range(K):
+                acc += float(x[m, k]) * float(W[n, k])
+            assert abs(y[m, n] - acc) <= 1e-14
+    # one-hot token picks a column of W; identity weights return the token
+    e = np.zeros((1, K)); e[0, 2] = 1.0
+    np.testing.assert_array_equal(O.project(e, W)[0], W[:, 2])
+    np.testing.assert_array_equal(O.project(x, np.eye(K)), x)
+    # linear in both arguments, leading dimensions kept
+    x3 = _rand(2, 3, K)
+    np.testing.assert_allclose(O.project(2.0 * x3 + 1.0, W), 2.0 * O.project(x3, W) + W.sum(axis=1), rtol=0, atol=1e-13)
+    assert O.project(x3, W).shape == (2, 3, N)
+
+
+def test_round_bf16_is_nearest_even_on_the_bfloat16_grid():
+    vals = np.array([1.0, 1.0 + 2.0 ** -8, 1.0 + 2.0 ** -7, 1.0 + 3 * 2.0 ** -8, -0.3, 1e-3, 255.5, 0.0])
+    got = O.round_bf16(vals)
+    # ties go to the even mantissa: 1 + 2^-8 -> 1, 1 + 3 * 2^-8 -> 1 + 2^-6
+    assert got[0] == 1.0 and got[1] == 1.0 and got[2] == 1.0 + 2.0 ** -7 and got[3] == 1.0 + 2.0 ** -6
+    ref = torch.tensor(vals, dtype=torch.float32).to(torch.bfloat16).double().numpy()
+    np.testing.assert_array_equal(got, ref)
+    assert np.all(np.abs(got - vals) <= np.abs(vals) * 2.0 ** -8)
+
+
+def test_layer_step_inputs_feed_the_layer():
+    # a layer with identity-like projections is the plain layer on the tokens themselves
+    B, T, Hq, Hkv, d, C = 1, 5, 1, 1, 4, 3
+    x = _rand(B, T, d)
+    I = np.eye(d)
+    q, k, v = O.layer_step_inputs(x, I, 2.0 * I, -I, Hq, Hkv, d, bf16=False)
+    f32 = x.astype(np.float32).astype(np.float64)
+    np.testing.assert_array_equal(q[:, :, 0], f32)
+    np.testing.assert_allclose(k[:, :, 0], 2.0 * f32, rtol=1e-7)
+    np.testing.assert_allclose(v[:, :, 0], -f32, rtol=1e-7)
+    a = O.OracleCache(B, Hq, Hkv, d, C)
+    b = O.OracleCache(B, Hq, Hkv, d, C)
+    np.testing.assert_array_equal(a.prefill_stream(q, k, v), b.prefill_stream(f32[:, :, None], 2 * f32[:, :, None], -f32[:, :, None]))
