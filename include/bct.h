@@ -170,7 +170,39 @@ bct_status_t bct_prefill_stream_eta(bct_cache_t *cache, const void *q, const voi
                                     const float *eta, void *out, int64_t T, void *cuda_stream);
 
 /*
- * Host-buffer forms of the two calls above: the same shapes, but q, k, v and out are
+ * The projections in front of the layer (Algorithm 1, "Compute write query" wq_t = W_wq x_t and
+ * "Compute write key-value vector" wv_t = W_wv x_t; the read query q_t = W_q x_t of the attention
+ * layer likewise), for a block of tokens, as one tensor-core contraction:
+ *     q = x W_q^T   [n_tokens][n_q]      k = x W_wq^T, v = x W_wv^T   [n_tokens][n_kv]
+ *   x      DEVICE bfloat16 [n_tokens][d_model]      one row per token (tokens of all sequences, [B][T] order)
+ *   w_q    DEVICE bfloat16 [n_q][d_model]           one row per output feature, n_q = Hq * head_dim
+ *   w_wq   DEVICE bfloat16 [n_kv][d_model]          n_kv = Hkv * head_dim
+ *   w_wv   DEVICE bfloat16 [n_kv][d_model]
+ *   q,k,v  DEVICE bfloat16, written by the call: exactly the step arrays bct_prefill_stream reads
+ * fp32 accumulation, one rounding to bfloat16.  d_model a multiple of 8, n_q and n_kv multiples of 32,
+ * every pointer 16-byte aligned; sm_100 devices only (BCT_ERR_UNSUPPORTED elsewhere).  Asynchronous on
+ * cuda_stream; allocates nothing.
+ */
+bct_status_t bct_project_qkv(int64_t n_tokens, int32_t d_model, int32_t n_q, int32_t n_kv, const void *x,
+                             const void *w_q, const void *w_wq, const void *w_wv, void *q, void *k, void *v,
+                             void *cuda_stream);
+
+/*
+ * One layer call on the tokens themselves: the projections above, then bct_prefill_stream_eta on
+ * their results (Algorithm 1's loop body from x_t to MV_t, plus the read).  bfloat16 caches only.
+ *   x        DEVICE bfloat16 [B][T][d_model]
+ *   eta      DEVICE float [B][T][Hkv] or NULL (all ones)
+ *   scratch  DEVICE, 256-byte aligned, at least bct_layer_scratch_bytes(cache, T) bytes: holds q, k, v
+ *            between the two steps; owned by the caller, free for reuse once the stream has passed the call
+ *   out      DEVICE [B][T][Hq][d] or NULL
+ */
+bct_status_t bct_layer_scratch_bytes(const bct_cache_t *cache, int64_t T, size_t *bytes);
+bct_status_t bct_layer_forward(bct_cache_t *cache, const void *x, const void *w_q, const void *w_wq,
+                               const void *w_wv, int32_t d_model, const float *eta, void *scratch,
+                               size_t scratch_bytes, void *out, int64_t T, void *cuda_stream);
+
+/*
+ * Host-buffer forms of bct_decode_step and bct_prefill_stream: the same shapes, but q, k, v and out are
  * HOST pointers.  The inputs are copied into the workspace's staging area (two sets, used
  * alternately, on a copy stream the handle owns, so that one call's copies overlap the
  * previous call's kernel), the step runs on cuda_stream after them, and out is copied back

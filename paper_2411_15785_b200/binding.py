@@ -24,6 +24,7 @@ EXPORTS = (
     "bct_prefill_stream", "bct_decode_step_host", "bct_prefill_stream_host", "bct_cache_len",
     "bct_cache_export", "bct_cache_import", "bct_cache_status", "bct_cache_launches", "bct_cache_destroy",
     "bct_cache_tensor_path", "bct_prefill_stream_host_static", "bct_decode_step_eta", "bct_prefill_stream_eta",
+    "bct_project_qkv", "bct_layer_scratch_bytes", "bct_layer_forward",
 )
 STATIC_STAGE_BYTES = 8 << 20
 
@@ -66,6 +67,9 @@ def load() -> ctypes.CDLL:
     lib.bct_prefill_stream.argtypes = [vp, vp, vp, vp, vp, i64, vp]
     lib.bct_decode_step_eta.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     lib.bct_prefill_stream_eta.argtypes = [vp, vp, vp, vp, vp, vp, i64, vp]
+    lib.bct_project_qkv.argtypes = [i64, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.bct_layer_scratch_bytes.argtypes = [vp, i64, ctypes.POINTER(ctypes.c_size_t)]
+    lib.bct_layer_forward.argtypes = [vp, vp, vp, vp, vp, i32, vp, vp, ctypes.c_size_t, vp, i64, vp]
     lib.bct_decode_step_host.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.bct_prefill_stream_host.argtypes = [vp, vp, vp, vp, vp, i64, vp]
     lib.bct_cache_len.argtypes = [vp, ctypes.POINTER(i32)]
@@ -127,6 +131,24 @@ def _ptr(t: Optional[torch.Tensor]):
     return None if t is None else t.data_ptr()
 
 
+def project_qkv(x, w_q, w_wq, w_wv, stream=None):
+    """q = x W_q^T, k = x W_wq^T, v = x W_wv^T: x ``[..., d_model]`` bfloat16 on the device, weights
+    ``[features, d_model]``; returns q ``[..., n_q]``, k, v ``[..., n_kv]`` (bfloat16)."""
+    lib = load()
+    d_model = x.shape[-1]
+    n_tokens = x.numel() // d_model
+    for t in (x, w_q, w_wq, w_wv):
+        if t.dtype != torch.bfloat16 or not t.is_cuda or not t.is_contiguous():
+            raise ValueError("x and the weights must be contiguous bfloat16 device tensors")
+    n_q, n_kv = w_q.shape[0], w_wq.shape[0]
+    q = torch.empty(x.shape[:-1] + (n_q,), dtype=torch.bfloat16, device=x.device)
+    k = torch.empty(x.shape[:-1] + (n_kv,), dtype=torch.bfloat16, device=x.device)
+    v = torch.empty_like(k)
+    _check(lib.bct_project_qkv(n_tokens, d_model, n_q, n_kv, x.data_ptr(), w_q.data_ptr(), w_wq.data_ptr(),
+                               w_wv.data_ptr(), q.data_ptr(), k.data_ptr(), v.data_ptr(), _stream_ptr(stream)))
+    return q, k, v
+
+
 class Cache:
     """A bounded cache over a torch-allocated workspace.  Methods map 1:1 to the C calls."""
 
@@ -182,6 +204,25 @@ class Cache:
             _check_eta(eta, (self.B, T, self.Hkv))
             _check(self.lib.bct_prefill_stream_eta(self._h, q.data_ptr(), k.data_ptr(), v.data_ptr(), eta.data_ptr(),
                                                    _ptr(out), T, _stream_ptr(stream)))
+        return out
+
+    def layer_scratch_bytes(self, T: int) -> int:
+        n = ctypes.c_size_t(0)
+        _check(self.lib.bct_layer_scratch_bytes(self._h, T, ctypes.byref(n)))
+        return n.value
+
+    def layer_forward(self, x, w_q, w_wq, w_wv, out=None, want_out=True, eta=None, scratch=None, stream=None):
+        """x ``[B, T, d_model]`` bfloat16: projections, then the stream call on their results."""
+        T, d_model = x.shape[1], x.shape[2]
+        if scratch is None:
+            scratch = torch.empty(self.layer_scratch_bytes(T), dtype=torch.uint8, device=self.device)
+        if out is None and want_out:
+            out = torch.empty((self.B, T, self.Hq, self.d), dtype=self.out_dtype, device=self.device)
+        if eta is not None:
+            _check_eta(eta, (self.B, T, self.Hkv))
+        _check(self.lib.bct_layer_forward(self._h, x.data_ptr(), w_q.data_ptr(), w_wq.data_ptr(), w_wv.data_ptr(),
+                                          d_model, _ptr(eta), scratch.data_ptr(), scratch.numel(), _ptr(out), T,
+                                          _stream_ptr(stream)))
         return out
 
     def decode_step_host(self, q, k, v, out, stream=None):

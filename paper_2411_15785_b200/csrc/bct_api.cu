@@ -319,6 +319,98 @@ bct_status_t bct_decode_step_eta(bct_cache_t* c, const void* q, const void* k, c
     return bct_prefill_stream_eta(c, q, k, v, eta, out, 1, cuda_stream);
 }
 
+namespace {
+
+bct_status_t check_project_args(int64_t n_tokens, int32_t d_model, int32_t n_q, int32_t n_kv, const void* x,
+                                const void* w_q, const void* w_wq, const void* w_wv, const void* q, const void* k,
+                                const void* v) {
+    if (n_tokens < 1 || n_tokens > ((int64_t)1 << 31) - 256)
+        return fail(BCT_ERR_INVALID_ARG, "n_tokens must be in [1, 2^31 - 256] (got %lld)", (long long)n_tokens);
+    if (d_model < 8 || d_model % 8 != 0)
+        return fail(BCT_ERR_INVALID_ARG, "d_model must be a positive multiple of 8 (got %d)", d_model);
+    if (n_q < 32 || n_q % 32 != 0 || n_kv < 32 || n_kv % 32 != 0)
+        return fail(BCT_ERR_UNSUPPORTED, "output features must be positive multiples of 32 (got %d and %d)", n_q, n_kv);
+    if (!x || !w_q || !w_wq || !w_wv || !q || !k || !v) return fail(BCT_ERR_INVALID_ARG, "no pointer may be NULL");
+    if (!aligned16(x) || !aligned16(w_q) || !aligned16(w_wq) || !aligned16(w_wv) || !aligned16(q) || !aligned16(k) ||
+        !aligned16(v))
+        return fail(BCT_ERR_INVALID_ARG, "every pointer must be 16-byte aligned");
+    return BCT_OK;
+}
+
+// SM count and opt-in shared memory of the current device, which must offer the sm_100 tensor path.
+bct_status_t tensor_device(int* sm_count, int* smem_optin) {
+    int dev = 0, major = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(sm_count, cudaDevAttrMultiProcessorCount, dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    if (e != cudaSuccess) return fail_cuda("device query", e);
+    if (major != 10) return fail(BCT_ERR_UNSUPPORTED, "the projections need an sm_100 device");
+    return BCT_OK;
+}
+
+inline size_t round256(size_t x) { return (x + 255) / 256 * 256; }
+
+}  // namespace
+
+bct_status_t bct_project_qkv(int64_t n_tokens, int32_t d_model, int32_t n_q, int32_t n_kv, const void* x,
+                             const void* w_q, const void* w_wq, const void* w_wv, void* q, void* k, void* v,
+                             void* cuda_stream) {
+    bct_status_t st = check_project_args(n_tokens, d_model, n_q, n_kv, x, w_q, w_wq, w_wv, q, k, v);
+    if (st != BCT_OK) return st;
+    int sm_count = 0, smem_optin = 0;
+    st = tensor_device(&sm_count, &smem_optin);
+    if (st != BCT_OK) return st;
+    cudaError_t e = bct::launch_project(n_tokens, d_model, n_q, n_kv, x, w_q, w_wq, w_wv, q, k, v, nullptr, sm_count,
+                                        smem_optin, static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return fail_cuda("projection launch", e);
+    return BCT_OK;
+}
+
+bct_status_t bct_layer_scratch_bytes(const bct_cache_t* c, int64_t T, size_t* bytes) {
+    bct_status_t st = check_handle(c);
+    if (st != BCT_OK) return st;
+    if (T < 1 || bytes == nullptr) return fail(BCT_ERR_INVALID_ARG, "T must be >= 1 and bytes not NULL");
+    const size_t eb = (size_t)c->elem_bytes;
+    const size_t qb = (size_t)c->p.batch * (size_t)T * c->p.n_q_heads * c->p.head_dim * eb;
+    const size_t kb = (size_t)c->p.batch * (size_t)T * c->p.n_kv_heads * c->p.head_dim * eb;
+    *bytes = round256(qb) + 2 * round256(kb);
+    return BCT_OK;
+}
+
+bct_status_t bct_layer_forward(bct_cache_t* c, const void* x, const void* w_q, const void* w_wq, const void* w_wv,
+                               int32_t d_model, const float* eta, void* scratch, size_t scratch_bytes, void* out,
+                               int64_t T, void* cuda_stream) {
+    bct_status_t st = check_handle(c);
+    if (st != BCT_OK) return st;
+    if (c->p.dtype != BCT_BF16) return fail(BCT_ERR_UNSUPPORTED, "the fused projections serve bfloat16 caches only");
+    if (T < 1) return fail(BCT_ERR_INVALID_ARG, "T must be >= 1 (got %lld)", (long long)T);
+    size_t need = 0;
+    st = bct_layer_scratch_bytes(c, T, &need);
+    if (st != BCT_OK) return st;
+    if (scratch == nullptr || scratch_bytes < need || (reinterpret_cast<uintptr_t>(scratch) & 255u) != 0)
+        return fail(BCT_ERR_INVALID_ARG, "scratch must be 256-byte aligned and hold %zu bytes (got %zu)", need,
+                    scratch_bytes);
+    const bct_params_t& p = c->p;
+    const int n_q = p.n_q_heads * p.head_dim, n_kv = p.n_kv_heads * p.head_dim;
+    const int64_t n_tokens = (int64_t)p.batch * T;
+    const size_t qb = round256((size_t)n_tokens * n_q * 2), kb = round256((size_t)n_tokens * n_kv * 2);
+    char* q = static_cast<char*>(scratch);
+    char* k = q + qb;
+    char* v = k + kb;
+    st = check_project_args(n_tokens, d_model, n_q, n_kv, x, w_q, w_wq, w_wv, q, k, v);
+    if (st != BCT_OK) return st;
+    if (out != nullptr && !aligned16(out)) return fail(BCT_ERR_INVALID_ARG, "out must be 16-byte aligned");
+    if ((reinterpret_cast<uintptr_t>(eta) & 3u) != 0) return fail(BCT_ERR_INVALID_ARG, "eta must be 4-byte aligned");
+    if (!c->tc_ready) return fail(BCT_ERR_UNSUPPORTED, "the projections need the driver's tensor-map encoder");
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e = bct::launch_project(n_tokens, d_model, n_q, n_kv, x, w_q, w_wq, w_wv, q, k, v, c->status,
+                                        c->sm_count, c->smem_optin, stream);
+    if (e != cudaSuccess) return fail_cuda("projection launch", e);
+    c->launches += 1;
+    return run_tokens(c, q, k, v, eta, out, T, stream);
+}
+
 bct_status_t bct_prefill_stream_host(bct_cache_t* c, const void* q, const void* k, const void* v, void* out,
                                      int64_t T, void* cuda_stream) {
     bct_status_t st = check_handle(c);

@@ -1,0 +1,267 @@
+// The projections in front of the bounded-cache layer on the sm_100a tensor path.
+//
+// Algorithm 1 starts every token with two products, wq_t = W_wq x_t ("Compute write query") and
+// wv_t = W_wv x_t ("Compute write key-value vector"); the read query of the attention layer is a
+// third product of the same token.  For a block of tokens they are one contraction
+//     [q | k | v][m][n] = sum_c x[m][c] * W[n][c]        W = W_q, W_wq, W_wv stacked over n
+// with bfloat16 operands, fp32 accumulation in tensor memory and bfloat16 results, written straight
+// into the three step-vector arrays the layer reads.
+//
+// One persistent CTA per SM over 128 x BN output tiles (BN = 128 for blocks of tokens, 32 for a
+// decode step, where the weights stream once from HBM and more, smaller tiles fill the SMs):
+//   warp 0      producer : TMA loads of x and W tiles (64 columns = 128 bytes per row, 128-byte swizzle)
+//                          into a ring of stages
+//   warp 1      MMA      : tcgen05.mma (M = 128, N = BN, K = 16) four times per stage; its commit frees the
+//                          stage; two accumulators in tensor memory, so that the epilogue of one tile
+//                          overlaps the products of the next
+//   warps 2-5   epilogue : one thread per output row: tcgen05.ld, round to bfloat16, 64-byte stores
+// Rows past the last token and columns past d_model are zero-filled by the TMA unit.
+// Every wait is bounded; a timeout sets the status word and the kernel runs to its end.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+#include <cstdio>
+
+#include "bct_internal.h"
+#include "bct_tc.cuh"
+
+namespace bct {
+namespace {
+
+constexpr int kPjThreads = 192;
+constexpr int kPjBM = 128;
+constexpr int kPjBK = 64;                      // columns per stage: 128 bytes per row
+constexpr int kPjABytes = kPjBM * kPjBK * 2;   // 16 KiB
+constexpr int kPjMaxStages = 8;
+
+struct PjArgs {
+    __nv_bfloat16* out[3];   // q, k, v
+    int* status;             // may be NULL (no cache at hand): timeouts are then only counted in the return path
+    int n_seg[3];            // output features of each segment (multiples of BN)
+    long long M;             // tokens
+    int K;                   // d_model
+    int stages;
+};
+
+__host__ __device__ constexpr int pj_stage_bytes(int BN) { return kPjABytes + BN * kPjBK * 2; }
+
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
+        : "memory");
+}
+
+template <int BN>
+__global__ void __launch_bounds__(kPjThreads, 1)
+project_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW0,
+               const __grid_constant__ CUtensorMap tmW1, const __grid_constant__ CUtensorMap tmW2, const PjArgs a) {
+    extern __shared__ unsigned char pj_smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(pj_smem_raw) + 1023) & ~uintptr_t(1023));
+    constexpr int kStage = pj_stage_bytes(BN);
+    constexpr uint32_t kTmemCols = (2 * BN < 32) ? 32 : 2 * BN;   // two accumulators (a power of two)
+    unsigned char* ring = smem;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)a.stages * kStage);
+    uint64_t* full = bars;                        // [stages] tile pair landed (TMA transaction bytes)
+    uint64_t* empty = bars + kPjMaxStages;        // [stages] products that read the stage complete (commit)
+    uint64_t* acc_full = bars + 2 * kPjMaxStages;     // [2] accumulator complete (commit)
+    uint64_t* acc_empty = bars + 2 * kPjMaxStages + 2;  // [2] accumulator read out (128 arrivals)
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 2 * kPjMaxStages + 4);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kPjMaxStages + 5);
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5;
+    const int lane = tid & 31;
+    const int m_tiles = (int)((a.M + kPjBM - 1) / kPjBM);
+    const int nt0 = a.n_seg[0] / BN, nt1 = a.n_seg[1] / BN, nt2 = a.n_seg[2] / BN;
+    const int n_tiles = (nt0 + nt1 + nt2) * m_tiles;
+    const int kb_count = (a.K + kPjBK - 1) / kPjBK;
+
+    if (tid == 0) {
+        for (int i = 0; i < a.stages; ++i) {
+            mbar_init(&full[i], 1);
+            mbar_init(&empty[i], 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&acc_full[i], 1);
+            mbar_init(&acc_empty[i], 128);
+        }
+        *abort_flag = 0;
+        fence_mbar_init_cluster();
+    }
+    if (warp == 1) tmem_alloc(tmem_slot, kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+#define PJ_WAIT(bar, parity, site)                                                  \
+    if (!mbar_wait(bar, (parity) & 1, *abort_flag ? 1024u : kWaitLimit)) {          \
+        if (a.status != nullptr) report_timeout(a.status, site);                    \
+        *abort_flag = 1;                                                            \
+    }
+
+    // tile id -> (segment, first feature of the tile within the segment, first token)
+    auto locate = [&](int tile, int* seg, int* n0, int* m0) {
+        const int nt = tile / m_tiles;
+        *m0 = (tile - nt * m_tiles) * kPjBM;
+        if (nt < nt0) {
+            *seg = 0;
+            *n0 = nt * BN;
+        } else if (nt < nt0 + nt1) {
+            *seg = 1;
+            *n0 = (nt - nt0) * BN;
+        } else {
+            *seg = 2;
+            *n0 = (nt - nt0 - nt1) * BN;
+        }
+    };
+
+    if (warp == 0) {
+        // =========================== producer ===========================
+        if (lane == 0) {
+            uint32_t it = 0;  // stage uses so far
+            for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+                int seg, n0, m0;
+                locate(tile, &seg, &n0, &m0);
+                const CUtensorMap* tw = seg == 0 ? &tmW0 : (seg == 1 ? &tmW1 : &tmW2);
+                for (int kb = 0; kb < kb_count; ++kb, ++it) {
+                    const int s = it % a.stages;
+                    if (it >= (uint32_t)a.stages) PJ_WAIT(&empty[s], it / a.stages - 1, 81);
+                    unsigned char* dst = ring + (size_t)s * kStage;
+                    mbar_arrive_expect_tx(&full[s], (uint32_t)kStage);
+                    tma_load_2d(dst, &tmX, kb * kPjBK, m0, &full[s]);
+                    tma_load_2d(dst + kPjABytes, tw, kb * kPjBK, n0, &full[s]);
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // =========================== MMA issuer ===========================
+        if (lane == 0) {
+            constexpr uint32_t idesc = instr_desc_mn(128, BN, false, false);  // x tile (K-major) x W tile (K-major)
+            uint32_t it = 0, nacc = 0;
+            for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++nacc) {
+                const int buf = nacc & 1;
+                if (nacc >= 2) PJ_WAIT(&acc_empty[buf], nacc / 2 - 1, 82);
+                tc_fence_after();
+                const uint32_t dcol = tmem_base + (uint32_t)(buf * BN);
+                for (int kb = 0; kb < kb_count; ++kb, ++it) {
+                    const int s = it % a.stages;
+                    PJ_WAIT(&full[s], it / a.stages, 83);
+                    tc_fence_after();
+                    const uint32_t aaddr = smem_u32(ring + (size_t)s * kStage);
+                    const uint32_t baddr = aaddr + kPjABytes;
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)
+                        umma_bf16(dcol, smem_desc(aaddr + kk * 32, 16, 1024), smem_desc(baddr + kk * 32, 16, 1024), idesc,
+                                  (kb > 0) || (kk > 0));
+                    umma_commit(&empty[s]);
+                }
+                umma_commit(&acc_full[buf]);
+            }
+        }
+        __syncwarp();
+    } else {
+        // =========================== epilogue: one thread per output row ===========================
+        const int quarter = warp & 3;  // the tensor-memory lanes this warp may read
+        const int row = quarter * 32 + lane;
+        uint32_t nacc = 0;
+        for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++nacc) {
+            int seg, n0, m0;
+            locate(tile, &seg, &n0, &m0);
+            const int buf = nacc & 1;
+            PJ_WAIT(&acc_full[buf], nacc / 2, 84);
+            tc_fence_after();
+            const long long m = (long long)m0 + row;
+            __nv_bfloat16* obase = seg == 0 ? a.out[0] : (seg == 1 ? a.out[1] : a.out[2]);
+            const int n_feat = seg == 0 ? a.n_seg[0] : (seg == 1 ? a.n_seg[1] : a.n_seg[2]);
+            __nv_bfloat16* dst = obase + (size_t)m * n_feat + n0;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN);
+#pragma unroll
+            for (int c = 0; c < BN / 32; ++c) {
+                float y[32];
+                tmem_ld32(taddr + c * 32, y);
+                if (m < a.M && !*abort_flag) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        reinterpret_cast<uint4*>(dst + c * 32)[j] = Chunk<__nv_bfloat16>::pack(y + 8 * j);
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(&acc_empty[buf]);
+        }
+    }
+#undef PJ_WAIT
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// [rows][K] bfloat16, row-major, as a 2-D tensor (column, row); boxes of 64 columns x `box_rows` rows
+// with the 128-byte swizzle; what lies outside reads as zeros.
+bool make_matrix_map(CUtensorMap* map, const void* base, long long rows, int K, int box_rows) {
+    TensorMapEncodeFn fn = tensor_map_encode_fn();
+    if (fn == nullptr) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kPjBK, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int BN>
+cudaError_t launch_bn(const CUtensorMap& mx, const CUtensorMap& m0, const CUtensorMap& m1, const CUtensorMap& m2,
+                      PjArgs a, int sm_count, int smem_optin, cudaStream_t stream) {
+    constexpr int kStage = pj_stage_bytes(BN);
+    int stages = (smem_optin - 2048) / kStage;
+    if (stages > kPjMaxStages) stages = kPjMaxStages;
+    if (stages < 2) return cudaErrorInvalidConfiguration;
+    a.stages = stages;
+    const int smem = stages * kStage + (2 * kPjMaxStages + 8) * 8 + 1024;
+    auto fn = project_kernel<BN>;
+    cudaError_t e = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    const long long m_tiles = (a.M + kPjBM - 1) / kPjBM;
+    const long long tiles = m_tiles * ((a.n_seg[0] + a.n_seg[1] + a.n_seg[2]) / BN);
+    const int grid = (int)(tiles < sm_count ? tiles : sm_count);
+    fn<<<grid, kPjThreads, smem, stream>>>(mx, m0, m1, m2, a);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+// q = x W_q^T, k = x W_wq^T, v = x W_wv^T for n_tokens rows of x.  Returns the CUDA error of the launch.
+cudaError_t launch_project(long long n_tokens, int d_model, int n_q, int n_kv, const void* x, const void* w_q,
+                           const void* w_wq, const void* w_wv, void* q, void* k, void* v, int* status, int sm_count,
+                           int smem_optin, cudaStream_t stream) {
+    const bool big = n_tokens > 256 && n_q % 128 == 0 && n_kv % 128 == 0;
+    const int BN = big ? 128 : 32;
+    alignas(64) CUtensorMap mx, m0, m1, m2;
+    if (!make_matrix_map(&mx, x, n_tokens, d_model, kPjBM) || !make_matrix_map(&m0, w_q, n_q, d_model, BN) ||
+        !make_matrix_map(&m1, w_wq, n_kv, d_model, BN) || !make_matrix_map(&m2, w_wv, n_kv, d_model, BN))
+        return cudaErrorInvalidValue;
+    PjArgs a;
+    a.out[0] = static_cast<__nv_bfloat16*>(q);
+    a.out[1] = static_cast<__nv_bfloat16*>(k);
+    a.out[2] = static_cast<__nv_bfloat16*>(v);
+    a.status = status;
+    a.n_seg[0] = n_q;
+    a.n_seg[1] = n_kv;
+    a.n_seg[2] = n_kv;
+    a.M = n_tokens;
+    a.K = d_model;
+    a.stages = 0;
+    return big ? launch_bn<128>(mx, m0, m1, m2, a, sm_count, smem_optin, stream)
+               : launch_bn<32>(mx, m0, m1, m2, a, sm_count, smem_optin, stream);
+}
+
+}  // namespace bct
