@@ -241,6 +241,66 @@ def run_reference(args, w):
     print(json.dumps(line))
 
 
+def run_project(args, w):
+    """Times bct_project_qkv alone (the projections in front of the layer) for --project-tokens rows of
+    x with the workload's head counts: one step = one launch.  Two weight sets are used alternately so
+    that the weights of a step (100 MB at d_model 4096) do not come from L2."""
+    from paper_2411_15785_b200 import binding as B
+    from paper_2411_15785_b200 import build as bld
+    bld.build()
+    B.load()
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    M, K = args.project_tokens, args.d_model
+    n_q, n_kv = w.n_q_heads * w.head_dim, w.n_kv_heads * w.head_dim
+    g = torch.Generator(device=dev).manual_seed(w.seed)
+    sets = [tuple((torch.randn((n, K), generator=g, device=dev) * K ** -0.5).to(torch.bfloat16) for n in (n_q, n_kv, n_kv))
+            for _ in range(2)]
+    xs = [torch.randn((M, K), generator=g, device=dev).to(torch.bfloat16) for _ in range(4)]
+    warm = max(args.warmup, 3)
+    for i in range(warm):
+        B.project_qkv(xs[i % 4], *sets[i & 1])
+    torch.cuda.synchronize()
+    sampler = ClockSampler(dev.index)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        B.project_qkv(xs[i % 4], *sets[i & 1])
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms_step = e0.elapsed_time(e1) / args.steps
+    n_out = n_q + 2 * n_kv
+    flops = 2.0 * M * n_out * K
+    nbytes = 2.0 * (n_out * K + M * K + M * n_out)
+    hbm_peak, kind = _peaks()
+    tf_peak = FALLBACK_BF16_TFLOPS
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            tf_peak = float(json.load(open(path))["bf16_tflops_sustained"])
+        except Exception:
+            pass
+    t_hbm, t_tensor = nbytes / (hbm_peak * 1e9), flops / (tf_peak * 1e12)
+    if t_hbm >= t_tensor:
+        ach = nbytes / (ms_step * 1e-3) / 1e9
+        roof = {"bound": "hbm", "achieved": ach, "peak": hbm_peak, "unit": "GB/s", "frac": ach / hbm_peak,
+                "algorithmic_bytes_per_launch": nbytes}
+    else:
+        ach = flops / (ms_step * 1e-3) / 1e12
+        roof = {"bound": "tensor", "achieved": ach, "peak": tf_peak, "unit": "TFLOP/s", "frac": ach / tf_peak,
+                "flops_per_launch": flops}
+    roof.update({"traffic": None, "peak_kind": "of " + kind, "kernel": "project_kernel"})
+    print(json.dumps({
+        "metric": "projection tokens/s", "value": M / (ms_step * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+        "warmup": warm, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16, f32 accumulate", "data": "synthetic",
+        "config": {"workload": "project_qkv", "tokens": M, "d_model": K, "n_q": n_q, "n_kv": n_kv,
+                   "l2": "two weight sets used alternately (%.0f MB each)" % (2e-6 * n_out * K)},
+        "clocks": clocks, "gpu_launches": args.steps, "roofline": roof}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -255,6 +315,9 @@ def main():
     ap.add_argument("--flags", type=int, default=0, help="BCT_FLAG_* bits for the cache")
     ap.add_argument("--batch", type=int, default=None, help="override the batch (profiling on a smaller case)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--project-tokens", type=int, default=0,
+                    help="time bct_project_qkv alone on this many tokens (the workload gives the head counts)")
+    ap.add_argument("--d-model", type=int, default=4096, help="model width of the projections")
     args = ap.parse_args()
     w = W.CONFIGS[args.workload]
     if args.write_scale is not None:
@@ -263,6 +326,9 @@ def main():
         w = w.scaled(batch=args.batch, name="%s@batch%d" % (w.name, args.batch))
     if args.impl == "reference":
         run_reference(args, w)
+        return
+    if args.project_tokens > 0:
+        run_project(args, w)
         return
     if args.warmup < 3:
         args.warmup = 3

@@ -15,7 +15,8 @@
 //                          stage; two accumulators in tensor memory, so that the epilogue of one tile
 //                          overlaps the products of the next
 //   warps 2-5   epilogue : one thread per output row: tcgen05.ld, round to bfloat16, 64-byte stores
-// Rows past the last token and columns past d_model are zero-filled by the TMA unit.
+// Rows past the last token and columns past d_model are zero-filled by the TMA unit (with fewer than
+// 128 tokens the box of x is shorter and the rows below it are never read back).
 // Every wait is bounded; a timeout sets the status word and the kernel runs to its end.
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -34,7 +35,7 @@ constexpr int kPjThreads = 192;
 constexpr int kPjBM = 128;
 constexpr int kPjBK = 64;                      // columns per stage: 128 bytes per row
 constexpr int kPjABytes = kPjBM * kPjBK * 2;   // 16 KiB
-constexpr int kPjMaxStages = 8;
+constexpr int kPjMaxStages = 16;
 
 struct PjArgs {
     __nv_bfloat16* out[3];   // q, k, v
@@ -43,9 +44,10 @@ struct PjArgs {
     long long M;             // tokens
     int K;                   // d_model
     int stages;
+    int a_rows;              // rows of x one TMA box brings (128, or fewer when there are fewer tokens)
+    int a_bytes;             // a_rows * 128: the x part of a stage; the W part (BN * 128 bytes) follows it
 };
 
-__host__ __device__ constexpr int pj_stage_bytes(int BN) { return kPjABytes + BN * kPjBK * 2; }
 
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
     asm volatile(
@@ -60,10 +62,12 @@ project_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                const __grid_constant__ CUtensorMap tmW1, const __grid_constant__ CUtensorMap tmW2, const PjArgs a) {
     extern __shared__ unsigned char pj_smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(pj_smem_raw) + 1023) & ~uintptr_t(1023));
-    constexpr int kStage = pj_stage_bytes(BN);
+    const int kStage = a.a_bytes + BN * kPjBK * 2;  // a short block of tokens leaves room for more stages in flight
     constexpr uint32_t kTmemCols = (2 * BN < 32) ? 32 : 2 * BN;   // two accumulators (a power of two)
     unsigned char* ring = smem;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)a.stages * kStage);
+    // The MMA always reads 128 rows of x: with a shorter box the rows below it are whatever follows in
+    // shared memory (their output rows are never stored), so the last stage is followed by that much padding.
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)a.stages * kStage + (kPjABytes - a.a_bytes));
     uint64_t* full = bars;                        // [stages] tile pair landed (TMA transaction bytes)
     uint64_t* empty = bars + kPjMaxStages;        // [stages] products that read the stage complete (commit)
     uint64_t* acc_full = bars + 2 * kPjMaxStages;     // [2] accumulator complete (commit)
@@ -97,10 +101,14 @@ project_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-#define PJ_WAIT(bar, parity, site)                                                  \
-    if (!mbar_wait(bar, (parity) & 1, *abort_flag ? 1024u : kWaitLimit)) {          \
-        if (a.status != nullptr) report_timeout(a.status, site);                    \
-        *abort_flag = 1;                                                            \
+    // One try first: the single threads of the producer and MMA warps run these loops with nothing to
+    // hide latency behind, so the usual case (the phase is already complete) must cost one instruction.
+#define PJ_WAIT(bar, parity, site)                                                      \
+    if (!mbar_try_wait(bar, (parity) & 1)) {                                            \
+        if (!mbar_wait(bar, (parity) & 1, *abort_flag ? 1024u : kWaitLimit)) {          \
+            if (a.status != nullptr) report_timeout(a.status, site);                    \
+            *abort_flag = 1;                                                            \
+        }                                                                               \
     }
 
     // tile id -> (segment, first feature of the tile within the segment, first token)
@@ -122,18 +130,30 @@ project_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     if (warp == 0) {
         // =========================== producer ===========================
         if (lane == 0) {
-            uint32_t it = 0;  // stage uses so far
+            int s = 0;        // stage of the next load
+            uint32_t ph = 0;  // parity of the ring pass: pass p waits for the commits of pass p - 1
+            bool first_pass = true;
             for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
                 int seg, n0, m0;
                 locate(tile, &seg, &n0, &m0);
                 const CUtensorMap* tw = seg == 0 ? &tmW0 : (seg == 1 ? &tmW1 : &tmW2);
-                for (int kb = 0; kb < kb_count; ++kb, ++it) {
-                    const int s = it % a.stages;
-                    if (it >= (uint32_t)a.stages) PJ_WAIT(&empty[s], it / a.stages - 1, 81);
+                // every CTA starts its walk over d_model at another column block: otherwise all of them ask
+                // L2 for the same lines of x at the same time
+                const int kb0 = (int)(((unsigned)blockIdx.x * 5u + (unsigned)tile) % (unsigned)kb_count);
+                // Column blocks are asked for in groups: a row of W is 128 bytes per block, and neighbouring
+                // blocks requested together let one DRAM page visit serve several of them.
+                for (int i = 0; i < kb_count; ++i) {
+                    const int kb = kb0 + i < kb_count ? kb0 + i : kb0 + i - kb_count;
+                    if (!first_pass) PJ_WAIT(&empty[s], ph ^ 1u, 81);
                     unsigned char* dst = ring + (size_t)s * kStage;
                     mbar_arrive_expect_tx(&full[s], (uint32_t)kStage);
+                    tma_load_2d(dst + a.a_bytes, tw, kb * kPjBK, n0, &full[s]);
                     tma_load_2d(dst, &tmX, kb * kPjBK, m0, &full[s]);
-                    tma_load_2d(dst + kPjABytes, tw, kb * kPjBK, n0, &full[s]);
+                    if (++s == a.stages) {
+                        s = 0;
+                        ph ^= 1u;
+                        first_pass = false;
+                    }
                 }
             }
         }
@@ -142,23 +162,30 @@ project_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         // =========================== MMA issuer ===========================
         if (lane == 0) {
             constexpr uint32_t idesc = instr_desc_mn(128, BN, false, false);  // x tile (K-major) x W tile (K-major)
-            uint32_t it = 0, nacc = 0;
+            uint32_t nacc = 0, ph = 0;
+            int s = 0;
+            const uint32_t ring_addr = smem_u32(ring);
+            // descriptor of a K-major 128-byte-swizzled operand at shared address 0: the address field is added per use
+            const uint64_t desc0 = smem_desc(0, 16, 1024);
             for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++nacc) {
                 const int buf = nacc & 1;
-                if (nacc >= 2) PJ_WAIT(&acc_empty[buf], nacc / 2 - 1, 82);
+                if (nacc >= 2) PJ_WAIT(&acc_empty[buf], (nacc >> 1) - 1, 82);
                 tc_fence_after();
                 const uint32_t dcol = tmem_base + (uint32_t)(buf * BN);
-                for (int kb = 0; kb < kb_count; ++kb, ++it) {
-                    const int s = it % a.stages;
-                    PJ_WAIT(&full[s], it / a.stages, 83);
+                for (int kb = 0; kb < kb_count; ++kb) {
+                    PJ_WAIT(&full[s], ph, 83);
                     tc_fence_after();
-                    const uint32_t aaddr = smem_u32(ring + (size_t)s * kStage);
-                    const uint32_t baddr = aaddr + kPjABytes;
+                    const uint32_t aaddr = ring_addr + (uint32_t)s * (uint32_t)kStage;
+                    const uint64_t ad = desc0 + (uint64_t)(aaddr >> 4);
+                    const uint64_t bd = desc0 + (uint64_t)((aaddr + (uint32_t)a.a_bytes) >> 4);
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk)
-                        umma_bf16(dcol, smem_desc(aaddr + kk * 32, 16, 1024), smem_desc(baddr + kk * 32, 16, 1024), idesc,
-                                  (kb > 0) || (kk > 0));
+                    for (int kk = 0; kk < 4; ++kk)  // 16 columns = 32 bytes = 2 units of the address field
+                        umma_bf16(dcol, ad + 2 * kk, bd + 2 * kk, idesc, (kb > 0) || (kk > 0));
                     umma_commit(&empty[s]);
+                    if (++s == a.stages) {
+                        s = 0;
+                        ph ^= 1u;
+                    }
                 }
                 umma_commit(&acc_full[buf]);
             }
@@ -207,6 +234,7 @@ project_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
 // [rows][K] bfloat16, row-major, as a 2-D tensor (column, row); boxes of 64 columns x `box_rows` rows
 // with the 128-byte swizzle; what lies outside reads as zeros.
 bool make_matrix_map(CUtensorMap* map, const void* base, long long rows, int K, int box_rows) {
+    if (box_rows > 256) return false;
     TensorMapEncodeFn fn = tensor_map_encode_fn();
     if (fn == nullptr) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
@@ -221,12 +249,13 @@ bool make_matrix_map(CUtensorMap* map, const void* base, long long rows, int K, 
 template <int BN>
 cudaError_t launch_bn(const CUtensorMap& mx, const CUtensorMap& m0, const CUtensorMap& m1, const CUtensorMap& m2,
                       PjArgs a, int sm_count, int smem_optin, cudaStream_t stream) {
-    constexpr int kStage = pj_stage_bytes(BN);
-    int stages = (smem_optin - 2048) / kStage;
+    const int kStage = a.a_bytes + BN * kPjBK * 2;
+    const int pad = kPjABytes - a.a_bytes;  // the 128-row operand read of the last stage stays inside the allocation
+    int stages = (smem_optin - 2048 - pad) / kStage;
     if (stages > kPjMaxStages) stages = kPjMaxStages;
     if (stages < 2) return cudaErrorInvalidConfiguration;
     a.stages = stages;
-    const int smem = stages * kStage + (2 * kPjMaxStages + 8) * 8 + 1024;
+    const int smem = stages * kStage + pad + (2 * kPjMaxStages + 8) * 8 + 1024;
     auto fn = project_kernel<BN>;
     cudaError_t e = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
@@ -243,10 +272,14 @@ cudaError_t launch_bn(const CUtensorMap& mx, const CUtensorMap& m0, const CUtens
 cudaError_t launch_project(long long n_tokens, int d_model, int n_q, int n_kv, const void* x, const void* w_q,
                            const void* w_wq, const void* w_wv, void* q, void* k, void* v, int* status, int sm_count,
                            int smem_optin, cudaStream_t stream) {
-    const bool big = n_tokens > 256 && n_q % 128 == 0 && n_kv % 128 == 0;
-    const int BN = big ? 128 : 32;
+    // feature tiles: 256 wide for long blocks of tokens (fewest operand bytes per product), 128 for
+    // shorter ones, 32 for a decode step (more tiles than SMs while the weights stream once)
+    int BN = 32;
+    if (n_tokens > 256 && n_q % 128 == 0 && n_kv % 128 == 0) BN = 128;
+    if (n_tokens >= 1024 && n_q % 256 == 0 && n_kv % 256 == 0) BN = 256;
+    const int a_rows = n_tokens >= kPjBM ? kPjBM : (int)((n_tokens + 7) / 8 * 8);
     alignas(64) CUtensorMap mx, m0, m1, m2;
-    if (!make_matrix_map(&mx, x, n_tokens, d_model, kPjBM) || !make_matrix_map(&m0, w_q, n_q, d_model, BN) ||
+    if (!make_matrix_map(&mx, x, n_tokens, d_model, a_rows) || !make_matrix_map(&m0, w_q, n_q, d_model, BN) ||
         !make_matrix_map(&m1, w_wq, n_kv, d_model, BN) || !make_matrix_map(&m2, w_wv, n_kv, d_model, BN))
         return cudaErrorInvalidValue;
     PjArgs a;
@@ -260,8 +293,11 @@ cudaError_t launch_project(long long n_tokens, int d_model, int n_q, int n_kv, c
     a.M = n_tokens;
     a.K = d_model;
     a.stages = 0;
-    return big ? launch_bn<128>(mx, m0, m1, m2, a, sm_count, smem_optin, stream)
-               : launch_bn<32>(mx, m0, m1, m2, a, sm_count, smem_optin, stream);
+    a.a_rows = a_rows;
+    a.a_bytes = a_rows * kPjBK * 2;
+    if (BN == 256) return launch_bn<256>(mx, m0, m1, m2, a, sm_count, smem_optin, stream);
+    if (BN == 128) return launch_bn<128>(mx, m0, m1, m2, a, sm_count, smem_optin, stream);
+    return launch_bn<32>(mx, m0, m1, m2, a, sm_count, smem_optin, stream);
 }
 
 }  // namespace bct
