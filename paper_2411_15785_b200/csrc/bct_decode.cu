@@ -176,7 +176,7 @@ __global__ void __launch_bounds__(kThreads, (G <= 4 ? 2 : 1)) decode_kernel(cons
                 const int stage = item % kStages;
                 if (item >= kStages) {
                     const uint32_t parity = ((item / kStages) - 1) & 1;
-                    if (!mbar_wait(&empty[stage], parity, *abort_flag ? 1024u : kWaitLimit)) {
+                    if (!mbar_wait_abortable(&empty[stage], parity, abort_flag)) {
                         report_timeout(a.status, 1);
                         *abort_flag = 1;
                         break;
@@ -220,7 +220,7 @@ __global__ void __launch_bounds__(kThreads, (G <= 4 ? 2 : 1)) decode_kernel(cons
         // ---- phase K: scores of every resident slot of the slice ----
         for (int i = 0; i < nt; ++i) {
             const int stage = i % kStages;
-            if (!mbar_wait(&full[stage], (i / kStages) & 1, *abort_flag ? 1024u : kWaitLimit)) {
+            if (!mbar_wait_abortable(&full[stage], (i / kStages) & 1, abort_flag)) {
                 report_timeout(a.status, 2);
                 *abort_flag = 1;
             }
@@ -343,7 +343,7 @@ __global__ void __launch_bounds__(kThreads, (G <= 4 ? 2 : 1)) decode_kernel(cons
                         mbar_arrive_remote(map_to_rank(xbar, r));
                     }
                 }
-                if (!mbar_wait<true>(xbar, 0, *abort_flag ? 1024u : kWaitLimit)) {
+                if (!mbar_wait_abortable<true>(xbar, 0, abort_flag)) {
                     report_timeout(a.status, 3);
                     *abort_flag = 1;
                 }
@@ -373,12 +373,12 @@ __global__ void __launch_bounds__(kThreads, (G <= 4 ? 2 : 1)) decode_kernel(cons
         for (int i = 0; i < nt; ++i) {
             const int item = precise ? nt + 2 * i : nt + i;
             const int stage = item % kStages;
-            if (!mbar_wait(&full[stage], (item / kStages) & 1, *abort_flag ? 1024u : kWaitLimit)) {
+            if (!mbar_wait_abortable(&full[stage], (item / kStages) & 1, abort_flag)) {
                 report_timeout(a.status, 4);
                 *abort_flag = 1;
             }
             const int stage_lo = (item + 1) % kStages;
-            if (precise && !mbar_wait(&full[stage_lo], ((item + 1) / kStages) & 1, *abort_flag ? 1024u : kWaitLimit)) {
+            if (precise && !mbar_wait_abortable(&full[stage_lo], ((item + 1) / kStages) & 1, abort_flag)) {
                 report_timeout(a.status, 5);
                 *abort_flag = 1;
             }

@@ -203,7 +203,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     for (int t = t_begin; t < t_end; ++t, ++kc) {
                         const int stage = kc % NST;
                         if (kc >= (uint32_t)NST &&
-                            !mbar_wait(&empty[stage], ((kc / NST) - 1) & 1, *abort_flag ? 1024u : kWaitLimit)) {
+                            !mbar_wait_abortable(&empty[stage], ((kc / NST) - 1) & 1, abort_flag)) {
                             report_timeout(a.status, 11);
                             *abort_flag = 1;
                             ok = false;
@@ -226,7 +226,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             uint32_t kc = 0, sp = 0, nsf = 0;  // ring position, sub-slices so far, sub-slice hand-overs so far
             int it = 0;
             for (int u = cid; u < a.U; u += ncl, ++it) {
-                if (!mbar_wait(&qready[it & 1], (it >> 1) & 1, *abort_flag ? 1024u : kWaitLimit)) {
+                if (!mbar_wait_abortable(&qready[it & 1], (it >> 1) & 1, abort_flag)) {
                     report_timeout(a.status, 12);
                     *abort_flag = 1;
                 }
@@ -235,7 +235,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 for (int sub = 0; sub < n_sub; ++sub, ++sp) {
                     const int t_begin = sub * kMaxTiles, t_end = min(nt, t_begin + kMaxTiles);
                     if (sub > 0) {  // the previous sub-slice's score tiles must have been consumed
-                        if (!mbar_wait(subfree, nsf & 1, *abort_flag ? 1024u : kWaitLimit)) {
+                        if (!mbar_wait_abortable(subfree, nsf & 1, abort_flag)) {
                             report_timeout(a.status, 22);
                             *abort_flag = 1;
                         }
@@ -244,7 +244,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     }
                     for (int t = t_begin; t < t_end; ++t, ++kc) {  // scores: A = K tile (K-major), B = Q (K-major)
                         const int stage = kc % NST;
-                        if (!mbar_wait(&full[stage], (kc / NST) & 1, *abort_flag ? 1024u : kWaitLimit)) {
+                        if (!mbar_wait_abortable(&full[stage], (kc / NST) & 1, abort_flag)) {
                             report_timeout(a.status, 13);
                             *abort_flag = 1;
                         }
@@ -261,11 +261,11 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     }
                     for (int t = t_begin; t < t_end; ++t, ++kc) {  // outputs: A = V tile (MN-major), B = P (K-major)
                         const int stage = kc % NST;
-                        if (!mbar_wait(&pready[t - t_begin], sp & 1, *abort_flag ? 1024u : kWaitLimit)) {
+                        if (!mbar_wait_abortable(&pready[t - t_begin], sp & 1, abort_flag)) {
                             report_timeout(a.status, 14);
                             *abort_flag = 1;
                         }
-                        if (!mbar_wait(&full[stage], (kc / NST) & 1, *abort_flag ? 1024u : kWaitLimit)) {
+                        if (!mbar_wait_abortable(&full[stage], (kc / NST) & 1, abort_flag)) {
                             report_timeout(a.status, 15);
                             *abort_flag = 1;
                         }
@@ -349,7 +349,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 #pragma unroll
                 for (int h = 0; h < 8; ++h) mx[h] = kNegBigTc;
                 for (int t = t_begin; t < t_end; ++t) {
-                    if (!mbar_wait(&sready[t - t_begin], sp & 1, *abort_flag ? 1024u : kWaitLimit)) {
+                    if (!mbar_wait_abortable(&sready[t - t_begin], sp & 1, abort_flag)) {
                         report_timeout(a.status, 16);
                         *abort_flag = 1;
                     }
@@ -386,7 +386,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 
                 // ---- the outputs accumulated so far refer to the old maxima: rescale them in tensor memory ----
                 if (sub > 0) {
-                    if (!mbar_wait(oready, (sp - 1) & 1, *abort_flag ? 1024u : kWaitLimit)) {
+                    if (!mbar_wait_abortable(oready, (sp - 1) & 1, abort_flag)) {
                         report_timeout(a.status, 23);
                         *abort_flag = 1;
                     }
@@ -475,7 +475,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                             mbar_arrive_remote(map_to_rank(&xbar[it & 1], rr));
                         }
                     }
-                    if (!mbar_wait<true>(&xbar[it & 1], (it >> 1) & 1, *abort_flag ? 1024u : kWaitLimit)) {
+                    if (!mbar_wait_abortable<true>(&xbar[it & 1], (it >> 1) & 1, abort_flag)) {
                         report_timeout(a.status, 17);
                         *abort_flag = 1;
                     }
@@ -513,7 +513,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             }
 
             // ---- epilogue: O[d][g] from tensor memory once every V tile has been read ----
-            if (nt > 0 && !mbar_wait(oready, (sp - 1) & 1, *abort_flag ? 1024u : kWaitLimit)) {
+            if (nt > 0 && !mbar_wait_abortable(oready, (sp - 1) & 1, abort_flag)) {
                 report_timeout(a.status, 19);
                 *abort_flag = 1;
             }
@@ -559,7 +559,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     }
                     mbar_arrive_remote(map_to_rank(&mbar[it & 1], 0));
                 } else {
-                    if (!mbar_wait<true>(&mbar[it & 1], (it >> 1) & 1, *abort_flag ? 1024u : kWaitLimit)) {
+                    if (!mbar_wait_abortable<true>(&mbar[it & 1], (it >> 1) & 1, abort_flag)) {
                         report_timeout(a.status, 20);
                         *abort_flag = 1;
                     }

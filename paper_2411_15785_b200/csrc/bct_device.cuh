@@ -77,6 +77,16 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32
     return false;
 }
 
+// The same for kernels that keep an abort flag in shared memory (set after the first timeout, so that
+// the waits that follow give up quickly).  One try comes first: the usual case, a phase that is
+// already complete, then costs a single instruction and no read of the flag, which matters in the
+// single-thread producer and MMA loops that have nothing to hide latency behind.
+template <bool kCluster = false>
+__device__ __forceinline__ bool mbar_wait_abortable(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    if (kCluster ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
+    return mbar_wait<kCluster>(bar, parity, *abort_flag ? 1024u : kWaitLimit);
+}
+
 __device__ __forceinline__ void report_timeout(int* status, int where) {
     if (atomicCAS(status, kStatusOk, kStatusTimeout) == kStatusOk) status[1] = where;
 }

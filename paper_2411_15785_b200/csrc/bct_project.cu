@@ -101,14 +101,10 @@ project_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    // One try first: the single threads of the producer and MMA warps run these loops with nothing to
-    // hide latency behind, so the usual case (the phase is already complete) must cost one instruction.
-#define PJ_WAIT(bar, parity, site)                                                      \
-    if (!mbar_try_wait(bar, (parity) & 1)) {                                            \
-        if (!mbar_wait(bar, (parity) & 1, *abort_flag ? 1024u : kWaitLimit)) {          \
-            if (a.status != nullptr) report_timeout(a.status, site);                    \
-            *abort_flag = 1;                                                            \
-        }                                                                               \
+#define PJ_WAIT(bar, parity, site)                                      \
+    if (!mbar_wait_abortable(bar, (parity) & 1, abort_flag)) {          \
+        if (a.status != nullptr) report_timeout(a.status, site);        \
+        *abort_flag = 1;                                                \
     }
 
     // tile id -> (segment, first feature of the tile within the segment, first token)

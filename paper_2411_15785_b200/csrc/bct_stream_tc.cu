@@ -225,7 +225,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     const uint32_t tmem_base = *tmem_slot;
 
 #define ST_WAIT(bar, parity, site)                                              \
-    if (!mbar_wait(bar, (parity) & 1, *abort_flag ? 1024u : kWaitLimit)) {      \
+    if (!mbar_wait_abortable(bar, (parity) & 1, abort_flag)) {      \
         report_timeout(a.status, site);                                         \
         *abort_flag = 1;                                                        \
     }
