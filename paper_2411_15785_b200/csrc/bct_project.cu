@@ -24,6 +24,7 @@
 
 #include <cstdint>
 #include <cstdio>
+#include <cstdlib>
 
 #include "bct_internal.h"
 #include "bct_tc.cuh"
@@ -56,13 +57,14 @@ __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, i
         : "memory");
 }
 
-template <int BN>
+template <int BN, int KPER>
 __global__ void __launch_bounds__(kPjThreads, 1)
 project_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW0,
                const __grid_constant__ CUtensorMap tmW1, const __grid_constant__ CUtensorMap tmW2, const PjArgs a) {
     extern __shared__ unsigned char pj_smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(pj_smem_raw) + 1023) & ~uintptr_t(1023));
-    const int kStage = a.a_bytes + BN * kPjBK * 2;  // a short block of tokens leaves room for more stages in flight
+    const int kBlock = a.a_bytes + BN * kPjBK * 2;  // one 64-column block: x part, then W part
+    const int kStage = KPER * kBlock;               // small blocks travel several to a stage: fewer hand-overs
     constexpr uint32_t kTmemCols = (2 * BN < 32) ? 32 : 2 * BN;   // two accumulators (a power of two)
     unsigned char* ring = smem;
     // The MMA always reads 128 rows of x: with a shorter box the rows below it are whatever follows in
@@ -138,13 +140,17 @@ project_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 const int kb0 = (int)(((unsigned)blockIdx.x * 5u + (unsigned)tile) % (unsigned)kb_count);
                 // Column blocks are asked for in groups: a row of W is 128 bytes per block, and neighbouring
                 // blocks requested together let one DRAM page visit serve several of them.
-                for (int i = 0; i < kb_count; ++i) {
-                    const int kb = kb0 + i < kb_count ? kb0 + i : kb0 + i - kb_count;
+                for (int i0 = 0; i0 < kb_count; i0 += KPER) {
+                    const int nblk = min(KPER, kb_count - i0);
                     if (!first_pass) PJ_WAIT(&empty[s], ph ^ 1u, 81);
-                    unsigned char* dst = ring + (size_t)s * kStage;
-                    mbar_arrive_expect_tx(&full[s], (uint32_t)kStage);
-                    tma_load_2d(dst + a.a_bytes, tw, kb * kPjBK, n0, &full[s]);
-                    tma_load_2d(dst, &tmX, kb * kPjBK, m0, &full[s]);
+                    mbar_arrive_expect_tx(&full[s], (uint32_t)(nblk * kBlock));
+                    for (int j = 0; j < nblk; ++j) {
+                        const int i = i0 + j;
+                        const int kb = kb0 + i < kb_count ? kb0 + i : kb0 + i - kb_count;
+                        unsigned char* dst = ring + (size_t)s * kStage + (size_t)j * kBlock;
+                        tma_load_2d(dst + a.a_bytes, tw, kb * kPjBK, n0, &full[s]);
+                        tma_load_2d(dst, &tmX, kb * kPjBK, m0, &full[s]);
+                    }
                     if (++s == a.stages) {
                         s = 0;
                         ph ^= 1u;
@@ -168,15 +174,20 @@ project_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
                 if (nacc >= 2) PJ_WAIT(&acc_empty[buf], (nacc >> 1) - 1, 82);
                 tc_fence_after();
                 const uint32_t dcol = tmem_base + (uint32_t)(buf * BN);
-                for (int kb = 0; kb < kb_count; ++kb) {
+                for (int i0 = 0; i0 < kb_count; i0 += KPER) {
+                    const int nblk = min(KPER, kb_count - i0);
                     PJ_WAIT(&full[s], ph, 83);
                     tc_fence_after();
-                    const uint32_t aaddr = ring_addr + (uint32_t)s * (uint32_t)kStage;
-                    const uint64_t ad = desc0 + (uint64_t)(aaddr >> 4);
-                    const uint64_t bd = desc0 + (uint64_t)((aaddr + (uint32_t)a.a_bytes) >> 4);
+                    uint32_t aaddr = ring_addr + (uint32_t)s * (uint32_t)kStage;
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk)  // 16 columns = 32 bytes = 2 units of the address field
-                        umma_bf16(dcol, ad + 2 * kk, bd + 2 * kk, idesc, (kb > 0) || (kk > 0));
+                    for (int j = 0; j < KPER; ++j, aaddr += (uint32_t)kBlock) {
+                        if (j >= nblk) break;
+                        const uint64_t ad = desc0 + (uint64_t)(aaddr >> 4);
+                        const uint64_t bd = desc0 + (uint64_t)((aaddr + (uint32_t)a.a_bytes) >> 4);
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk)  // 16 columns = 32 bytes = 2 units of the address field
+                            umma_bf16(dcol, ad + 2 * kk, bd + 2 * kk, idesc, (i0 > 0) || (j > 0) || (kk > 0));
+                    }
                     umma_commit(&empty[s]);
                     if (++s == a.stages) {
                         s = 0;
@@ -242,17 +253,17 @@ bool make_matrix_map(CUtensorMap* map, const void* base, long long rows, int K, 
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BN>
+template <int BN, int KPER>
 cudaError_t launch_bn(const CUtensorMap& mx, const CUtensorMap& m0, const CUtensorMap& m1, const CUtensorMap& m2,
                       PjArgs a, int sm_count, int smem_optin, cudaStream_t stream) {
-    const int kStage = a.a_bytes + BN * kPjBK * 2;
+    const int kStage = KPER * (a.a_bytes + BN * kPjBK * 2);
     const int pad = kPjABytes - a.a_bytes;  // the 128-row operand read of the last stage stays inside the allocation
     int stages = (smem_optin - 2048 - pad) / kStage;
     if (stages > kPjMaxStages) stages = kPjMaxStages;
     if (stages < 2) return cudaErrorInvalidConfiguration;
     a.stages = stages;
     const int smem = stages * kStage + pad + (2 * kPjMaxStages + 8) * 8 + 1024;
-    auto fn = project_kernel<BN>;
+    auto fn = project_kernel<BN, KPER>;
     cudaError_t e = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     const long long m_tiles = (a.M + kPjBM - 1) / kPjBM;
@@ -269,10 +280,19 @@ cudaError_t launch_project(long long n_tokens, int d_model, int n_q, int n_kv, c
                            const void* w_wq, const void* w_wv, void* q, void* k, void* v, int* status, int sm_count,
                            int smem_optin, cudaStream_t stream) {
     // feature tiles: 256 wide for long blocks of tokens (fewest operand bytes per product), 128 for
-    // shorter ones, 32 for a decode step (more tiles than SMs while the weights stream once)
+    // shorter ones, 64 (else 32) for a decode step (more tiles than SMs while the weights stream once)
     int BN = 32;
-    if (n_tokens > 256 && n_q % 128 == 0 && n_kv % 128 == 0) BN = 128;
+    if (n_q % 64 == 0 && n_kv % 64 == 0) BN = 64;
+    const long long m_tiles = (n_tokens + kPjBM - 1) / kPjBM;
+    // 128 wide when that still leaves about two thirds of the SMs a tile (a decode step of a model with
+    // 12288 output features: 96 tiles on 148 SMs), or when there are several row tiles anyway
+    if (n_q % 128 == 0 && n_kv % 128 == 0 && (n_tokens > 256 || m_tiles * ((n_q + 2 * n_kv) / 128) * 8 >= 5LL * sm_count))
+        BN = 128;
     if (n_tokens >= 1024 && n_q % 256 == 0 && n_kv % 256 == 0) BN = 256;
+    if (const char* e = getenv("BCT_PJ_BN")) {  // tuning knob: width of the feature tiles
+        const int v = atoi(e);
+        if ((v == 32 || v == 64 || v == 128 || v == 256) && n_q % v == 0 && n_kv % v == 0) BN = v;
+    }
     const int a_rows = n_tokens >= kPjBM ? kPjBM : (int)((n_tokens + 7) / 8 * 8);
     alignas(64) CUtensorMap mx, m0, m1, m2;
     if (!make_matrix_map(&mx, x, n_tokens, d_model, a_rows) || !make_matrix_map(&m0, w_q, n_q, d_model, BN) ||
@@ -291,9 +311,29 @@ cudaError_t launch_project(long long n_tokens, int d_model, int n_q, int n_kv, c
     a.stages = 0;
     a.a_rows = a_rows;
     a.a_bytes = a_rows * kPjBK * 2;
-    if (BN == 256) return launch_bn<256>(mx, m0, m1, m2, a, sm_count, smem_optin, stream);
-    if (BN == 128) return launch_bn<128>(mx, m0, m1, m2, a, sm_count, smem_optin, stream);
-    return launch_bn<32>(mx, m0, m1, m2, a, sm_count, smem_optin, stream);
+    // Small blocks travel four or two to a stage while three stages still fit: measured at 64 tokens,
+    // d_model 4096, 12288 features, every halving of the hand-overs per byte paid (64-wide tiles:
+    // 57.6 / 43.1 / 34.8 us with 1 / 2 / 4 blocks per stage; 128-wide: 33.0 / 28.1 us with 1 / 2).
+    const int block = a.a_bytes + BN * kPjBK * 2;
+    int kper = 12 * block <= 200 * 1024 ? 4 : (6 * block <= 200 * 1024 ? 2 : 1);
+    if (const char* e = getenv("BCT_PJ_KPER")) {  // tuning knob: 64-column blocks per stage (1, 2, 4)
+        const int v = atoi(e);
+        if (v == 1 || v == 2 || v == 4) kper = v;
+    }
+#define PJ_LAUNCH(bn, kp) \
+    if (BN == bn && kper == kp) return launch_bn<bn, kp>(mx, m0, m1, m2, a, sm_count, smem_optin, stream);
+    PJ_LAUNCH(256, 1)
+    PJ_LAUNCH(256, 2)
+    PJ_LAUNCH(128, 1)
+    PJ_LAUNCH(128, 2)
+    PJ_LAUNCH(64, 1)
+    PJ_LAUNCH(64, 2)
+    PJ_LAUNCH(64, 4)
+    PJ_LAUNCH(32, 1)
+    PJ_LAUNCH(32, 2)
+    PJ_LAUNCH(32, 4)
+#undef PJ_LAUNCH
+    return cudaErrorInvalidConfiguration;
 }
 
 }  // namespace bct
