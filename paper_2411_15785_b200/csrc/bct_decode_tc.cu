@@ -194,16 +194,16 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     if (warp == 4) {
         // =========================== producer ===========================
         if (lane == 0) {
-            uint32_t kc = 0;
+            int stage = 0;        // ring position without divisions: this thread has nothing to hide their latency behind
+            uint32_t rph = 0;     // parity of the ring pass
+            bool first_pass = true;
             bool ok = true;
             for (int u = cid; u < a.U && ok; u += ncl) {
                 for (int ph = 0; ph < 2 * n_sub && ok; ++ph) {  // per sub-slice: its MK tiles, then its MV tiles
                     const CUtensorMap* map = (ph & 1) == 0 ? &tmK : &tmV;
                     const int t_begin = (ph >> 1) * kMaxTiles, t_end = min(nt, t_begin + kMaxTiles);
-                    for (int t = t_begin; t < t_end; ++t, ++kc) {
-                        const int stage = kc % NST;
-                        if (kc >= (uint32_t)NST &&
-                            !mbar_wait_abortable(&empty[stage], ((kc / NST) - 1) & 1, abort_flag)) {
+                    for (int t = t_begin; t < t_end; ++t) {
+                        if (!first_pass && !mbar_wait_abortable(&empty[stage], rph ^ 1u, abort_flag)) {
                             report_timeout(a.status, 11);
                             *abort_flag = 1;
                             ok = false;
@@ -213,6 +213,11 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         mbar_arrive_expect_tx(&full[stage], kTcTileBytes);
                         tma_load_3d(dst, map, 0, slice_start + t * kTileRows, u, &full[stage]);
                         tma_load_3d(dst + kHalfBytes, map, 64, slice_start + t * kTileRows, u, &full[stage]);
+                        if (++stage == NST) {
+                            stage = 0;
+                            rph ^= 1u;
+                            first_pass = false;
+                        }
                     }
                 }
             }
@@ -223,7 +228,11 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         if (lane == 0) {
             constexpr uint32_t idesc_s = instr_desc(false);
             constexpr uint32_t idesc_o = instr_desc(true);
-            uint32_t kc = 0, sp = 0, nsf = 0;  // ring position, sub-slices so far, sub-slice hand-overs so far
+            uint32_t sp = 0, nsf = 0;  // sub-slices so far, sub-slice hand-overs so far
+            int stage = 0;             // ring position and the parity of its pass
+            uint32_t rph = 0;
+            // descriptors at shared address 0: the address field is added per use (addresses stay below 256 KiB)
+            const uint64_t dk0 = smem_desc(0, 16, 1024), dmn0 = smem_desc(0, kHalfBytes, 1024);
             int it = 0;
             for (int u = cid; u < a.U; u += ncl, ++it) {
                 if (!mbar_wait_abortable(&qready[it & 1], (it >> 1) & 1, abort_flag)) {
@@ -242,9 +251,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         ++nsf;
                         tc_fence_after();
                     }
-                    for (int t = t_begin; t < t_end; ++t, ++kc) {  // scores: A = K tile (K-major), B = Q (K-major)
-                        const int stage = kc % NST;
-                        if (!mbar_wait_abortable(&full[stage], (kc / NST) & 1, abort_flag)) {
+                    for (int t = t_begin; t < t_end; ++t) {  // scores: A = K tile (K-major), B = Q (K-major)
+                        if (!mbar_wait_abortable(&full[stage], rph, abort_flag)) {
                             report_timeout(a.status, 13);
                             *abort_flag = 1;
                         }
@@ -252,20 +260,23 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         const uint32_t taddr = smem_u32(ring + (size_t)stage * kTcTileBytes);
 #pragma unroll
                         for (int kk = 0; kk < 8; ++kk) {
-                            const uint64_t ad = smem_desc(taddr + (kk >> 2) * kHalfBytes + (kk & 3) * 32, 16, 1024);
-                            const uint64_t bd = smem_desc(qaddr + (kk >> 2) * 1024 + (kk & 3) * 32, 16, 1024);
+                            const uint64_t ad = desc_at(dk0, taddr + (kk >> 2) * kHalfBytes + (kk & 3) * 32);
+                            const uint64_t bd = desc_at(dk0, qaddr + (kk >> 2) * 1024 + (kk & 3) * 32);
                             umma_bf16(tmem_base + (t - t_begin) * kScoreCols, ad, bd, idesc_s, kk > 0);
                         }
                         umma_commit(&sready[t - t_begin]);
                         umma_commit(&empty[stage]);
+                        if (++stage == NST) {
+                            stage = 0;
+                            rph ^= 1u;
+                        }
                     }
-                    for (int t = t_begin; t < t_end; ++t, ++kc) {  // outputs: A = V tile (MN-major), B = P (K-major)
-                        const int stage = kc % NST;
+                    for (int t = t_begin; t < t_end; ++t) {  // outputs: A = V tile (MN-major), B = P (K-major)
                         if (!mbar_wait_abortable(&pready[t - t_begin], sp & 1, abort_flag)) {
                             report_timeout(a.status, 14);
                             *abort_flag = 1;
                         }
-                        if (!mbar_wait_abortable(&full[stage], (kc / NST) & 1, abort_flag)) {
+                        if (!mbar_wait_abortable(&full[stage], rph, abort_flag)) {
                             report_timeout(a.status, 15);
                             *abort_flag = 1;
                         }
@@ -274,11 +285,15 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         const uint32_t paddr = smem_u32(pbuf + (t - t_begin) * kPTileBytes);
 #pragma unroll
                         for (int kk = 0; kk < 8; ++kk) {  // 16 slots per step
-                            const uint64_t ad = smem_desc(taddr + kk * 2048, kHalfBytes, 1024);
-                            const uint64_t bd = smem_desc(paddr + (kk >> 2) * 1024 + (kk & 3) * 32, 16, 1024);
+                            const uint64_t ad = desc_at(dmn0, taddr + kk * 2048);
+                            const uint64_t bd = desc_at(dk0, paddr + (kk >> 2) * 1024 + (kk & 3) * 32);
                             umma_bf16(tmem_base + kOCol, ad, bd, idesc_o, (t > 0) || (kk > 0));
                         }
                         umma_commit(&empty[stage]);
+                        if (++stage == NST) {
+                            stage = 0;
+                            rph ^= 1u;
+                        }
                     }
                     umma_commit(oready);  // every V tile of the sub-slice has been read
                 }

@@ -182,8 +182,8 @@ project_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
 #pragma unroll
                     for (int j = 0; j < KPER; ++j, aaddr += (uint32_t)kBlock) {
                         if (j >= nblk) break;
-                        const uint64_t ad = desc0 + (uint64_t)(aaddr >> 4);
-                        const uint64_t bd = desc0 + (uint64_t)((aaddr + (uint32_t)a.a_bytes) >> 4);
+                        const uint64_t ad = desc_at(desc0, aaddr);
+                        const uint64_t bd = desc_at(desc0, aaddr + (uint32_t)a.a_bytes);
 #pragma unroll
                         for (int kk = 0; kk < 4; ++kk)  // 16 columns = 32 bytes = 2 units of the address field
                             umma_bf16(dcol, ad + 2 * kk, bd + 2 * kk, idesc, (i0 > 0) || (j > 0) || (kk > 0));

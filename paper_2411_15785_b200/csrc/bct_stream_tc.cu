@@ -359,12 +359,16 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             uint32_t qn = 0, su0 = 0, su1 = 0, np = 0, nd = 0;
             uint32_t use[kStMaxStages] = {0, 0, 0, 0};
             const uint32_t plo_row0 = a.precise ? 0u : (uint32_t)n_read;  // first operand row the residual buffer holds
+            // descriptors at shared address 0 (K-major; MN-major with the half strides of the tiles, of Vc and of
+            // the residual operand): the address field is added per use, addresses stay below 256 KiB
+            const uint64_t dk0 = smem_desc(0, 16, 1024), dmn0 = smem_desc(0, kStHalf, 1024);
+            const uint64_t dvc0 = smem_desc(0, (uint32_t)vc_half, 1024), dpl0 = smem_desc(0, (uint32_t)L.plo_half, 1024);
             const uint32_t qaddr = smem_u32(qall), vcaddr = smem_u32(vc), phiaddr = smem_u32(phi), ploaddr = smem_u32(plo);
             auto scores = [&](uint32_t col, uint32_t taddr) {
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk) {
                     const uint32_t o = (kk >> 2) * kStHalf + (kk & 3) * 32;
-                    umma_bf16(tmem_base + col, smem_desc(qaddr + o, 16, 1024), smem_desc(taddr + o, 16, 1024), id_scores,
+                    umma_bf16(tmem_base + col, desc_at(dk0, qaddr + o), desc_at(dk0, taddr + o), id_scores,
                               kk > 0);
                 }
             };
@@ -379,8 +383,8 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 #pragma unroll
                         for (int kk = 0; kk < 8; ++kk) {
                             const uint32_t o = (kk >> 2) * kStHalf + (kk & 3) * 32;
-                            umma_bf16(tmem_base + kColA, smem_desc(qaddr + o, 16, 1024),
-                                      smem_desc(qaddr + n_read * 128 + o, 16, 1024), id_a, kk > 0);
+                            umma_bf16(tmem_base + kColA, desc_at(dk0, qaddr + o),
+                                      desc_at(dk0, qaddr + n_read * 128 + o), id_a, kk > 0);
                         }
                         umma_commit(ccready);
                         if (nt == 0) umma_commit(qfree_q);  // nothing else reads the query operand
@@ -431,12 +435,12 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 #pragma unroll
                         for (int kk = 0; kk < 8; ++kk) {
                             const uint32_t po = (kk >> 2) * kStHalf + (kk & 3) * 32;
-                            const uint64_t vhd = smem_desc(vhaddr + kk * 2048, kStHalf, 1024);
-                            umma_bf16(tmem_base + kColO, smem_desc(phiaddr + po, 16, 1024), vhd, id_out, (t > 0) || (kk > 0));
+                            const uint64_t vhd = desc_at(dmn0, vhaddr + kk * 2048);
+                            umma_bf16(tmem_base + kColO, desc_at(dk0, phiaddr + po), vhd, id_out, (t > 0) || (kk > 0));
                             if (a.precise) {
-                                umma_bf16(tmem_base + kColO, smem_desc(ploaddr + po, 16, 1024), vhd, id_out, true);
-                                umma_bf16(tmem_base + kColO, smem_desc(phiaddr + po, 16, 1024),
-                                          smem_desc(vladdr + kk * 2048, kStHalf, 1024), id_out, true);
+                                umma_bf16(tmem_base + kColO, desc_at(dk0, ploaddr + po), vhd, id_out, true);
+                                umma_bf16(tmem_base + kColO, desc_at(dk0, phiaddr + po),
+                                          desc_at(dmn0, vladdr + kk * 2048), id_out, true);
                             }
                         }
                         if (a.fill) {
@@ -448,11 +452,11 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         }
                         // increment of this tile's MV rows: (WW + WW_residual)^T x Vc, 16 tokens per step
                         for (int kk = 0; kk < Tc / 16; ++kk) {
-                            const uint64_t vd = smem_desc(vcaddr + kk * 2048, (uint32_t)vc_half, 1024);
-                            umma_bf16(tmem_base + kColD, smem_desc(phiaddr + n_read * 128 + kk * 2048, kStHalf, 1024), vd,
+                            const uint64_t vd = desc_at(dvc0, vcaddr + kk * 2048);
+                            umma_bf16(tmem_base + kColD, desc_at(dmn0, phiaddr + n_read * 128 + kk * 2048), vd,
                                       id_delta, kk > 0);
                             umma_bf16(tmem_base + kColD,
-                                      smem_desc(ploaddr + ((uint32_t)n_read - plo_row0) * 128 + kk * 2048, (uint32_t)L.plo_half, 1024), vd,
+                                      desc_at(dpl0, ploaddr + ((uint32_t)n_read - plo_row0) * 128 + kk * 2048), vd,
                                       id_delta, true);
                         }
                         umma_commit(dready);  // the write-back may start: outputs and increment are complete
@@ -460,8 +464,8 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 #pragma unroll
                         for (int kk = 0; kk < 8; ++kk) {
                             const uint32_t po = (kk >> 2) * kStHalf + (kk & 3) * 32;
-                            umma_bf16(tmem_base + kColA, smem_desc(phiaddr + po, 16, 1024),
-                                      smem_desc(phiaddr + n_read * 128 + po, 16, 1024), id_a, (t > 0) || (kk > 0));
+                            umma_bf16(tmem_base + kColA, desc_at(dk0, phiaddr + po),
+                                      desc_at(dk0, phiaddr + n_read * 128 + po), id_a, (t > 0) || (kk > 0));
                         }
                         umma_commit(pfree);
                         ++nd;
@@ -472,10 +476,10 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     ST_WAIT(aready, qn, 50);
                     tc_fence_after();
                     for (int kk = 0; kk < Tc / 16; ++kk) {
-                        const uint64_t vd = smem_desc(vcaddr + kk * 2048, (uint32_t)vc_half, 1024);
-                        umma_bf16(tmem_base + kColO, smem_desc(ploaddr + kk * 32, 16, 1024), vd, id_out, (nt > 0) || (kk > 0));
+                        const uint64_t vd = desc_at(dvc0, vcaddr + kk * 2048);
+                        umma_bf16(tmem_base + kColO, desc_at(dk0, ploaddr + kk * 32), vd, id_out, (nt > 0) || (kk > 0));
                         if (a.fill && a.precise)
-                            umma_bf16(tmem_base + kColO, smem_desc(ploaddr + kStHalf + kk * 32, 16, 1024), vd, id_out, true);
+                            umma_bf16(tmem_base + kColO, desc_at(dk0, ploaddr + kStHalf + kk * 32), vd, id_out, true);
                     }
                     umma_commit(oready);
                 }

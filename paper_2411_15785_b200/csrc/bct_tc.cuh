@@ -80,6 +80,10 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes
     d |= (uint64_t)2 << 61;
     return d;
 }
+// The descriptor d0 = smem_desc(0, lbo, sbo) moved to shared address saddr: one mask, shift and add
+// instead of the whole construction, for the single-thread MMA loops.  (The mask matters: in a cluster
+// launch the shared address of a CTA carries its rank above the 18 address bits.)
+__device__ __forceinline__ uint64_t desc_at(uint64_t d0, uint32_t saddr) { return d0 + (uint64_t)((saddr & 0x3FFFFu) >> 4); }
 // Instruction descriptor: bf16 x bf16 -> f32, M = 128, N = 16; A K-major or MN-major, B K-major.
 __host__ __device__ constexpr uint32_t instr_desc(bool a_mn_major) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn_major ? 1u : 0u) << 15) | ((16u >> 3) << 17) |
