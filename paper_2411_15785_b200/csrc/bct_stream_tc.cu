@@ -273,7 +273,11 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     const int nt = chunk_tiles(ch);
                     // the first MK tiles of pass 1 do not depend on the chunk's operands: ask for them first
                     const int n_early = nt < ns - 1 ? nt : ns - 1;
-                    for (int t = 0; t < n_early; ++t) load_tile(&tmK, u, t, t % ns);
+                    int st1 = 0;  // pass-1 stage of the next tile, t mod ns without the division
+                    for (int t = 0; t < n_early; ++t) {
+                        load_tile(&tmK, u, t, st1);
+                        if (++st1 == ns) st1 = 0;
+                    }
                     if (qn == 0) load_queries(u, ch);
                     if (qn > 0) ST_WAIT(oready, qn - 1, 35);  // the previous chunk's last product has read Vc
                     mbar_arrive_expect_tx(vfull, (uint32_t)(Tc * 256));
@@ -291,7 +295,10 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         tma_store_3d(&tmVapp, 64, len, u, vc + vc_half);
                         bulk_commit();
                     }
-                    for (int t = n_early; t < nt; ++t) load_tile(&tmK, u, t, t % ns);  // pass 1: row statistics
+                    for (int t = n_early; t < nt; ++t) {  // pass 1: row statistics
+                        load_tile(&tmK, u, t, st1);
+                        if (++st1 == ns) st1 = 0;
+                    }
                     // pass 2: numerators, outputs, update.  The row threads put the rewritten MV rows back
                     // into the two ring stages the tile came in; they go home as TMA stores from here.
                     // The MK tile is asked for two tiles ahead (its stage is free as soon as the scores of the
@@ -389,8 +396,8 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         umma_commit(ccready);
                         if (nt == 0) umma_commit(qfree_q);  // nothing else reads the query operand
                     }
-                    for (int t = 0; t < nt; ++t) {  // pass 1
-                        const int stage = t % ns;
+                    for (int t = 0, st1 = 0; t < nt; ++t, st1 = (st1 + 1 == ns ? 0 : st1 + 1)) {  // pass 1
+                        const int stage = st1;
                         const int buf = t & 1;
                         ST_WAIT(&full[stage], use_at(use, stage), 42);
                         ++use_at(use, stage);
