@@ -231,6 +231,13 @@ class OracleCache:
             ou.reshape(B, self.Hkv, T, self.G, self.d).transpose(0, 2, 1, 3, 4)
         ).reshape(B, T, self.Hq, self.d)
 
+    def update_kv(self, k, v, eta=None):
+        """Algorithm 1 itself (procedure UpdateKV): the write queries k and write key-value vectors v
+        ``[B, T, Hkv, d]`` of T tokens go into the state, nothing is read."""
+        k = _f64(k)
+        q = np.zeros((k.shape[0], k.shape[1], self.Hq, self.d), dtype=np.float64)  # unused: no output is asked for
+        self.prefill_stream(q, k, v, want_out=False, eta=eta)
+
     def decode_step(self, q, k, v, eta=None):
         """q ``[B, Hq, d]``, k, v ``[B, Hkv, d]``, eta ``[B, Hkv]`` or None -> out ``[B, Hq, d]``."""
         q = _f64(q)[:, None]

@@ -496,3 +496,18 @@ def test_layer_step_inputs_feed_the_layer():
     a = O.OracleCache(B, Hq, Hkv, d, C)
     b = O.OracleCache(B, Hq, Hkv, d, C)
     np.testing.assert_array_equal(a.prefill_stream(q, k, v), b.prefill_stream(f32[:, :, None], 2 * f32[:, :, None], -f32[:, :, None]))
+
+
+def test_update_kv_is_algorithm_1():
+    # UpdateKV(x_1..x_N, MV_0, MK, ...) returns MV_N = MV_0 + sum_t ww_t^T wv_t, reads nothing, leaves MK alone
+    B, Hq, Hkv, d, C, T = 2, 4, 2, 6, 5, 11
+    mk, mv = _rand(B, Hkv, C, d), _rand(B, Hkv, C, d)
+    k, v = _rand(B, T, Hkv, d), _rand(B, T, Hkv, d)
+    c = O.OracleCache(B, Hq, Hkv, d, C, init_len=C, mk_init=mk, mv_init=mv, write_scale=0.7)
+    c.update_kv(k, v)
+    for b in range(B):
+        for h in range(Hkv):
+            WW = _np_softmax(0.7 * k[b, :, h] @ mk[b, h].T)
+            np.testing.assert_allclose(c.values()[b, h], mv[b, h] + WW.T @ v[b, :, h], rtol=0, atol=1e-12)
+    np.testing.assert_array_equal(c.keys(), mk)
+    assert c.len == C and c.n_written == T
