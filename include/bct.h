@@ -170,6 +170,21 @@ bct_status_t bct_prefill_stream_eta(bct_cache_t *cache, const void *q, const voi
                                     const float *eta, void *out, int64_t T, void *cuda_stream);
 
 /*
+ * Algorithm 1 itself, procedure UpdateKV: the write queries and write key-value vectors of T tokens
+ * go into the state, MV_N = MV_0 + sum_t eta_t ww_t^T wv_t, and nothing is read.  The same state as
+ * bct_prefill_stream_eta with out == NULL (within rounding), in chunks of up to 128 tokens whose
+ * write weights are formed together ("token-level parallel training": MK is never assigned, so the
+ * tokens' write weights do not depend on one another).
+ *   wq   DEVICE [B][T][Hkv][d]  write queries     wv  DEVICE [B][T][Hkv][d]  write key-value vectors
+ *   eta  DEVICE float [B][T][Hkv] or NULL (all ones)
+ * Needs a full cache (the paper's full-size MV_0; BCT_ERR_STATE otherwise) of the shape the chunked
+ * tensor-core kernel serves: bfloat16, head_dim 128, 128..2048 slots, no BCT_FLAG_SKIP_FIRST_WRITE
+ * (BCT_ERR_UNSUPPORTED otherwise: use bct_prefill_stream with out == NULL).
+ */
+bct_status_t bct_update_kv(bct_cache_t *cache, const void *wq, const void *wv, const float *eta, int64_t T,
+                           void *cuda_stream);
+
+/*
  * The projections in front of the layer (Algorithm 1, "Compute write query" wq_t = W_wq x_t and
  * "Compute write key-value vector" wv_t = W_wv x_t; the read query q_t = W_q x_t of the attention
  * layer likewise), for a block of tokens, as one tensor-core contraction:

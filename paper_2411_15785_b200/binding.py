@@ -24,7 +24,7 @@ EXPORTS = (
     "bct_prefill_stream", "bct_decode_step_host", "bct_prefill_stream_host", "bct_cache_len",
     "bct_cache_export", "bct_cache_import", "bct_cache_status", "bct_cache_launches", "bct_cache_destroy",
     "bct_cache_tensor_path", "bct_prefill_stream_host_static", "bct_decode_step_eta", "bct_prefill_stream_eta",
-    "bct_project_qkv", "bct_layer_scratch_bytes", "bct_layer_forward",
+    "bct_project_qkv", "bct_layer_scratch_bytes", "bct_layer_forward", "bct_update_kv",
 )
 STATIC_STAGE_BYTES = 8 << 20
 
@@ -67,6 +67,7 @@ def load() -> ctypes.CDLL:
     lib.bct_prefill_stream.argtypes = [vp, vp, vp, vp, vp, i64, vp]
     lib.bct_decode_step_eta.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     lib.bct_prefill_stream_eta.argtypes = [vp, vp, vp, vp, vp, vp, i64, vp]
+    lib.bct_update_kv.argtypes = [vp, vp, vp, vp, i64, vp]
     lib.bct_project_qkv.argtypes = [i64, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.bct_layer_scratch_bytes.argtypes = [vp, i64, ctypes.POINTER(ctypes.c_size_t)]
     lib.bct_layer_forward.argtypes = [vp, vp, vp, vp, vp, i32, vp, vp, ctypes.c_size_t, vp, i64, vp]
@@ -205,6 +206,13 @@ class Cache:
             _check(self.lib.bct_prefill_stream_eta(self._h, q.data_ptr(), k.data_ptr(), v.data_ptr(), eta.data_ptr(),
                                                    _ptr(out), T, _stream_ptr(stream)))
         return out
+
+    def update_kv(self, wq, wv, eta=None, stream=None):
+        """Algorithm 1's UpdateKV: wq, wv ``[B, T, Hkv, d]`` go into the state, nothing is read."""
+        T = wq.shape[1]
+        if eta is not None:
+            _check_eta(eta, (self.B, T, self.Hkv))
+        _check(self.lib.bct_update_kv(self._h, wq.data_ptr(), wv.data_ptr(), _ptr(eta), T, _stream_ptr(stream)))
 
     def layer_scratch_bytes(self, T: int) -> int:
         n = ctypes.c_size_t(0)

@@ -136,7 +136,7 @@ bct_status_t run_tokens(bct_cache_t* c, const void* q, const void* k, const void
         if (Tc > 0 && full && do_write && T - t >= Tc) {
             const int64_t n_chunks = (T - t) / Tc;
             cudaError_t e = cudaSuccess;
-            const int n = bct::launch_stream_tc(c, q, k, v, out, T, eta, t, n_chunks, -1, stream, &e);
+            const int n = bct::launch_stream_tc(c, q, k, v, out, T, eta, t, n_chunks, -1, 0, stream, &e);
             if (n < 0) return fail_cuda("stream launch", e);
             c->launches += n;
             c->n_full_tokens += n_chunks * Tc;
@@ -148,7 +148,7 @@ bct_status_t run_tokens(bct_cache_t* c, const void* q, const void* k, const void
             const int64_t by_tokens = (T - t) / Tc, by_slots = (p.capacity - c->len) / Tc;
             const int64_t n_chunks = by_tokens < by_slots ? by_tokens : by_slots;
             cudaError_t e = cudaSuccess;
-            const int n = bct::launch_stream_tc(c, q, k, v, out, T, eta, t, n_chunks, c->len, stream, &e);
+            const int n = bct::launch_stream_tc(c, q, k, v, out, T, eta, t, n_chunks, c->len, 0, stream, &e);
             if (n < 0) return fail_cuda("stream launch (fill)", e);
             c->launches += n;
             c->len += (int)(n_chunks * Tc);
@@ -311,6 +311,39 @@ bct_status_t bct_prefill_stream_eta(bct_cache_t* c, const void* q, const void* k
     if (st != BCT_OK) return st;
     if ((reinterpret_cast<uintptr_t>(eta) & 3u) != 0) return fail(BCT_ERR_INVALID_ARG, "eta must be 4-byte aligned");
     return run_tokens(c, q, k, v, eta, out, T, static_cast<cudaStream_t>(cuda_stream));
+}
+
+bct_status_t bct_update_kv(bct_cache_t* c, const void* wq, const void* wv, const float* eta, int64_t T,
+                           void* cuda_stream) {
+    bct_status_t st = check_handle(c);
+    if (st != BCT_OK) return st;
+    if (T < 1) return fail(BCT_ERR_INVALID_ARG, "T must be >= 1 (got %lld)", (long long)T);
+    if (wq == nullptr || wv == nullptr) return fail(BCT_ERR_INVALID_ARG, "wq and wv must not be NULL");
+    if (!aligned16(wq) || !aligned16(wv)) return fail(BCT_ERR_INVALID_ARG, "wq and wv must be 16-byte aligned");
+    if ((reinterpret_cast<uintptr_t>(eta) & 3u) != 0) return fail(BCT_ERR_INVALID_ARG, "eta must be 4-byte aligned");
+    if (c->len != c->p.capacity)
+        return fail(BCT_ERR_STATE, "UpdateKV works on a full-size MV_0: the cache holds %d of %d slots", c->len,
+                    c->p.capacity);
+    if (bct::stream_chunk_tokens(c) == 0 || (c->p.flags & BCT_FLAG_SKIP_FIRST_WRITE))
+        return fail(BCT_ERR_UNSUPPORTED,
+                    "the write-only form serves bfloat16 caches with head_dim 128 and 128..2048 slots, without "
+                    "SKIP_FIRST_WRITE; use bct_prefill_stream with out = NULL");
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const int64_t whole = T / 128, rest = T - whole * 128;
+    cudaError_t e = cudaSuccess;
+    if (whole > 0) {
+        const int n = bct::launch_stream_tc(c, nullptr, wq, wv, nullptr, T, eta, 0, whole, -1, 128, stream, &e);
+        if (n < 0) return fail_cuda("write-only stream launch", e);
+        c->launches += n;
+    }
+    if (rest > 0) {  // one shorter chunk; its rows past the last token read as zeros
+        const int tc = (int)((rest + 15) / 16 * 16);
+        const int n = bct::launch_stream_tc(c, nullptr, wq, wv, nullptr, T, eta, whole * 128, 1, -1, tc, stream, &e);
+        if (n < 0) return fail_cuda("write-only stream launch", e);
+        c->launches += n;
+    }
+    c->n_full_tokens += T;
+    return BCT_OK;
 }
 
 bct_status_t bct_decode_step_eta(bct_cache_t* c, const void* q, const void* k, const void* v, const float* eta,

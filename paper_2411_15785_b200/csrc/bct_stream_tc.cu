@@ -65,16 +65,17 @@ struct StSmem {
 };
 // Shared-memory carve-up, the same on host and device.  With PRECISE_READ every operand row keeps
 // its residual (a full second operand buffer) and the ring has three stages; otherwise only the
-// write rows do (at most 64 rows), and the 16 KiB saved buy a fourth stage.
-__host__ __device__ inline StSmem st_smem(int precise) {
+// write rows do (at most 64 rows), and the 16 KiB saved buy a fourth stage.  `wide`: chunks of more
+// than 64 tokens (the write-only form, up to 128 write rows): a full residual buffer and twice the Vc.
+__host__ __device__ inline StSmem st_smem(int precise, int wide) {
     StSmem L;
-    L.stages = precise ? 3 : kStMaxStages;
-    L.plo_half = precise ? kStHalf : kStMaxTc * 128;
+    L.stages = (precise || wide) ? 3 : kStMaxStages;
+    L.plo_half = (precise || wide) ? kStHalf : kStMaxTc * 128;
     int off = 0;
     L.qall = off;
     off += kStTileBytes;        // [2 halves][128 rows][128 B]: G*Tc read queries, Tc write queries, zero rows
     L.vc = off;
-    off += kStMaxTc * 256;      // [2 halves][Tc rows][128 B]: the chunk's write key-value vectors
+    off += (wide ? 2 : 1) * kStMaxTc * 256;  // [2 halves][Tc rows][128 B]: the chunk's write key-value vectors
     L.phi = off;
     off += kStTileBytes;        // numerators / write weights of one tile, bfloat16 value
     L.plo = off;
@@ -127,7 +128,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                  const StArgs a) {
     extern __shared__ unsigned char st_smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(st_smem_raw) + 1023) & ~uintptr_t(1023));
-    const StSmem L = st_smem(a.precise);
+    const StSmem L = st_smem(a.precise, a.Tc > kStMaxTc);
     const int ns = L.stages;
     unsigned char* qall = smem + L.qall;
     unsigned char* vc = smem + L.vc;
@@ -248,8 +249,10 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 const int b = u / a.Hkv, h = u - b * a.Hkv;
                 const int t0 = a.t_begin + ch * Tc;
                 mbar_arrive_expect_tx(qfull, (uint32_t)(Tc * (G + 1) * 256));
-                tma_load_4d(qall, &tmQ, 0, h * G, t0, b, qfull);
-                tma_load_4d(qall + kStHalf, &tmQ, 64, h * G, t0, b, qfull);
+                if (G > 0) {
+                    tma_load_4d(qall, &tmQ, 0, h * G, t0, b, qfull);
+                    tma_load_4d(qall + kStHalf, &tmQ, 64, h * G, t0, b, qfull);
+                }
                 tma_load_4d(qall + n_read * 128, &tmKin, 0, h, t0, b, qfull);
                 tma_load_4d(qall + kStHalf + n_read * 128, &tmKin, 64, h, t0, b, qfull);
             };
@@ -362,7 +365,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             constexpr uint32_t id_scores = instr_desc_mn(128, 128, false, false);  // Qall (K) x tile (K)
             constexpr uint32_t id_out = instr_desc_mn(128, 128, false, true);      // P (K) x V tile (MN)
             constexpr uint32_t id_delta = instr_desc_mn(128, 128, true, true);     // WW^T (MN) x Vc (MN)
-            const uint32_t id_a = instr_desc_mn(128, (uint32_t)(Tc < 16 ? 16 : Tc), false, false);  // P (K) x WW (K)
+            const uint32_t id_a = instr_desc_mn(128, (uint32_t)(Tc < 16 ? 16 : (Tc > kStMaxTc ? kStMaxTc : Tc)), false, false);  // P (K) x WW (K)
             uint32_t qn = 0, su0 = 0, su1 = 0, np = 0, nd = 0;
             uint32_t use[kStMaxStages] = {0, 0, 0, 0};
             const uint32_t plo_row0 = a.precise ? 0u : (uint32_t)n_read;  // first operand row the residual buffer holds
@@ -439,8 +442,9 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         const uint32_t vhaddr = smem_u32(ring + (size_t)vh * kStTileBytes);
                         const uint32_t vladdr = smem_u32(ring + (size_t)vl * kStTileBytes);
                         // outputs: (P + P_residual) x MV_value + P x MV_residual, accumulated over the tiles
+                        // (none in the write-only form, G = 0)
 #pragma unroll
-                        for (int kk = 0; kk < 8; ++kk) {
+                        for (int kk = 0; kk < (G > 0 ? 8 : 0); ++kk) {
                             const uint32_t po = (kk >> 2) * kStHalf + (kk & 3) * 32;
                             const uint64_t vhd = desc_at(dmn0, vhaddr + kk * 2048);
                             umma_bf16(tmem_base + kColO, desc_at(dk0, phiaddr + po), vhd, id_out, (t > 0) || (kk > 0));
@@ -469,7 +473,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         umma_commit(dready);  // the write-back may start: outputs and increment are complete
                         // A += P x WW^T over this tile's slots (write rows start at n_read)
 #pragma unroll
-                        for (int kk = 0; kk < 8; ++kk) {
+                        for (int kk = 0; kk < (G > 0 ? 8 : 0); ++kk) {
                             const uint32_t po = (kk >> 2) * kStHalf + (kk & 3) * 32;
                             umma_bf16(tmem_base + kColA, desc_at(dk0, phiaddr + po),
                                       desc_at(dk0, phiaddr + n_read * 128 + po), id_a, (t > 0) || (kk > 0));
@@ -482,7 +486,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     // chunk's own slots, value + residual, times Vc)
                     ST_WAIT(aready, qn, 50);
                     tc_fence_after();
-                    for (int kk = 0; kk < Tc / 16; ++kk) {
+                    for (int kk = 0; kk < (G > 0 ? Tc / 16 : 0); ++kk) {
                         const uint64_t vd = desc_at(dvc0, vcaddr + kk * 2048);
                         umma_bf16(tmem_base + kColO, desc_at(dk0, ploaddr + kk * 32), vd, id_out, (nt > 0) || (kk > 0));
                         if (a.fill && a.precise)
@@ -503,7 +507,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         const uint32_t lane_base = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + cq * 32;
         const bool is_read = r < n_read;
         const bool is_write = !is_read && r < n_read + Tc;
-        const int my_t = is_read ? r / G : (is_write ? r - n_read : 0);  // token of the chunk this row belongs to
+        const int my_t = is_read ? r / (G > 0 ? G : 1) : (is_write ? r - n_read : 0);  // token of the chunk this row belongs to
         const int my_g = is_read ? r - my_t * G : 0;
         const float c2 = (is_read ? a.read_scale : a.write_scale) * 1.4426950408889634f;
         const int sw = r & 7;                                // swizzle phase of this row
@@ -604,7 +608,8 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 float wmul = 1.f;
                 if (is_write && !a.fill) {
                     wmul = 1.f / l;
-                    if (a.eta != nullptr && !a.fill) wmul *= a.eta[((size_t)b * a.T + t0 + my_t) * a.Hkv + h];
+                    // (a ragged last chunk of the write-only form has rows past the last token: their Vc rows are zero)
+                    if (a.eta != nullptr && !a.fill && t0 + my_t < a.T) wmul *= a.eta[((size_t)b * a.T + t0 + my_t) * a.Hkv + h];
                 }
 
                 // ---- pass 2: numerators of each tile, then the write-back of its MV rows.  The numerators of
@@ -739,7 +744,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     // A is masked, rounded to bfloat16 and handed back as an operand
                     if (np > 0) ST_WAIT(pfree, np - 1, 70);  // the last tile's A products are complete
                     tc_fence_after();
-                    if (cq * 16 < Tc) {
+                    if (G > 0 && cq * 16 < Tc) {
                         float av[16];
                         const uint32_t abase = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + kColA + cq * 16;
                         tmem_ld16(abase, av);
@@ -765,11 +770,14 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 ST_WAIT(oready, qn, 67);
                 tc_fence_after();
                 // the row sum of a read row: its four quarters' sums of numerators (the residual operand is free again)
-                rowstat[cq * 128 + r] = lr;
-                st_sync();
-                const float inv_l = 1.f / ((rowstat[r] + rowstat[128 + r]) + (rowstat[256 + r] + rowstat[384 + r]));
-                st_sync();
-                {
+                float inv_l = 1.f;
+                if (G > 0) {
+                    rowstat[cq * 128 + r] = lr;
+                    st_sync();
+                    inv_l = 1.f / ((rowstat[r] + rowstat[128 + r]) + (rowstat[256 + r] + rowstat[384 + r]));
+                    st_sync();
+                }
+                if (G > 0) {
                     const size_t orow = (((size_t)b * a.T + t0 + my_t) * a.Hq + (size_t)h * G + my_g) * 128 + cq * 32;
                     float o[32];
                     tmem_ld32(lane_base + kColO, o);
@@ -807,6 +815,7 @@ using StKernelFn = void (*)(const CUtensorMap, const CUtensorMap, const CUtensor
 
 StKernelFn pick_stream(int G) {
     switch (G) {
+        case 0: return stream_tc_kernel<0>;  // the write-only form
         case 1: return stream_tc_kernel<1>;
         case 2: return stream_tc_kernel<2>;
         case 3: return stream_tc_kernel<3>;
@@ -858,12 +867,16 @@ int stream_chunk_tokens(const bct_cache* c) {
 }
 
 int launch_stream_tc(const bct_cache* c, const void* q, const void* k, const void* v, void* out, int64_t T,
-                     const float* eta, int64_t t_begin, int64_t n_chunks, int fill_len, cudaStream_t stream,
-                     cudaError_t* err) {
+                     const float* eta, int64_t t_begin, int64_t n_chunks, int fill_len, int write_only_tc,
+                     cudaStream_t stream, cudaError_t* err) {
     const bct_params_t& p = c->p;
-    StKernelFn fn = pick_stream(c->G);
-    const int Tc = stream_chunk_tokens(c);
-    if (fn == nullptr || Tc == 0 || T > (int64_t)1 << 30) {
+    // write_only_tc > 0: the form without read queries (Algorithm 1's UpdateKV), chunks of that many tokens
+    const bool write_only = write_only_tc > 0;
+    const int G = write_only ? 0 : c->G;
+    StKernelFn fn = pick_stream(G);
+    const int Tc = write_only ? write_only_tc : stream_chunk_tokens(c);
+    if (fn == nullptr || Tc == 0 || stream_chunk_tokens(c) == 0 || T > (int64_t)1 << 30 || Tc % 16 != 0 || Tc > 128 ||
+        (write_only && fill_len >= 0)) {
         *err = cudaErrorInvalidConfiguration;
         return -1;
     }
@@ -873,7 +886,8 @@ int launch_stream_tc(const bct_cache* c, const void* q, const void* k, const voi
     }
     alignas(64) CUtensorMap mq, mk, mv, mka, mva;
     if (!make_append_map(&mka, c->kplane, c->U, p.capacity, Tc) || !make_append_map(&mva, c->vhi, c->U, p.capacity, Tc) ||
-        !make_step_map(&mq, q, p.batch, (int)T, p.n_q_heads, c->G, Tc) ||
+        !make_step_map(&mq, write_only ? k : q, p.batch, (int)T, write_only ? p.n_kv_heads : p.n_q_heads,
+                       write_only ? 1 : c->G, Tc) ||
         !make_step_map(&mk, k, p.batch, (int)T, p.n_kv_heads, 1, Tc) ||
         !make_step_map(&mv, v, p.batch, (int)T, p.n_kv_heads, 1, Tc)) {
         *err = cudaErrorInvalidValue;
@@ -898,7 +912,7 @@ int launch_stream_tc(const bct_cache* c, const void* q, const void* k, const voi
     a.precise = (p.flags & BCT_FLAG_PRECISE_READ) ? 1 : 0;
     a.read_scale = p.read_scale;
     a.write_scale = p.write_scale;
-    const int smem = st_smem(a.precise).total;
+    const int smem = st_smem(a.precise, Tc > kStMaxTc).total;
     *err = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (*err != cudaSuccess) return -1;
     const int grid = c->U < c->sm_count ? c->U : c->sm_count;
