@@ -129,16 +129,20 @@ def measured_traffic(w, tensor_path):
     return None if per_unit is None else per_unit * w.units
 
 
-def stream_roofline(w, tok_per_step, ms_step, precise=False):
+def stream_roofline(w, tok_per_step, ms_step, precise=False, write_only=False):
     """Tensor-core roofline of stream_tc_kernel: the dense flops its MMAs execute per step (operand rows padded
     to M = 128 included) against the measured bf16 matmul peak."""
     Tc = 64 if w.group == 1 else (32 if w.group <= 3 else 16)
     C, d = w.capacity, w.head_dim
-    per_chunk = 2 * (2 * 128 * C * d)          # scores of the 128 operand rows, two passes over MK
-    per_chunk += (3 if precise else 1) * (2 * 128 * C * d)   # outputs: P MV_hi (+ P_lo MV_hi + P MV_lo with PRECISE_READ)
-    per_chunk += 2 * 128 * C * Tc              # A = P WW^T
-    per_chunk += 2 * (2 * C * Tc * d)          # MV increment with value + residual weights
-    per_chunk += 2 * 128 * Tc * d              # strict_tril(A) Vc
+    if write_only:                                 # bct_update_kv: chunks of 128 write rows, no outputs
+        Tc = 128
+        per_chunk = 2 * (2 * 128 * C * d) + 2 * (2 * C * Tc * d)
+    else:
+        per_chunk = 2 * (2 * 128 * C * d)          # scores of the 128 operand rows, two passes over MK
+        per_chunk += (3 if precise else 1) * (2 * 128 * C * d)   # outputs: P MV_hi (+ P_lo MV_hi + P MV_lo with PRECISE_READ)
+        per_chunk += 2 * 128 * C * Tc              # A = P WW^T
+        per_chunk += 2 * (2 * C * Tc * d)          # MV increment with value + residual weights
+        per_chunk += 2 * 128 * Tc * d              # strict_tril(A) Vc
     flops = per_chunk * (tok_per_step // Tc) * w.units
     peak = FALLBACK_BF16_TFLOPS
     kind = "fallback"
@@ -315,6 +319,8 @@ def main():
     ap.add_argument("--flags", type=int, default=0, help="BCT_FLAG_* bits for the cache")
     ap.add_argument("--batch", type=int, default=None, help="override the batch (profiling on a smaller case)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--update-kv", action="store_true",
+                    help="stream workloads: time bct_update_kv (Algorithm 1's UpdateKV, state only) instead of bct_prefill_stream")
     ap.add_argument("--project-tokens", type=int, default=0,
                     help="time bct_project_qkv alone on this many tokens (the workload gives the head counts)")
     ap.add_argument("--d-model", type=int, default=4096, help="model width of the projections")
@@ -373,8 +379,12 @@ def main():
         pool = [W.step_inputs(wr, t, dev) for t in range(min(args.steps + args.warmup, 64))]
     outs = [torch.empty_like(pool[0][0], dtype=cache.out_dtype) for _ in range(2)]
 
+    update_only = stream and args.update_kv
+
     def step_dev(i):
-        if stream:
+        if update_only:
+            cache.update_kv(pool[i % len(pool)][1], pool[i % len(pool)][2])
+        elif stream:
             cache.prefill_stream(*pool[i % len(pool)], out=outs[i & 1])
         else:
             cache.decode_step(*pool[i % len(pool)], out=outs[i & 1])
@@ -409,7 +419,9 @@ def main():
     hout = [torch.empty_like(hpool[0][0], dtype=cache.out_dtype).pin_memory() for _ in range(2)]
 
     def step_host(i):
-        if stream:
+        if update_only:   # no host-buffer form of UpdateKV: the stream call without outputs
+            cache.prefill_stream_host(*hpool[i % len(hpool)], None)
+        elif stream:
             cache.prefill_stream_host(*hpool[i % len(hpool)], hout[i & 1])
         else:
             cache.decode_step_host(*hpool[i % len(hpool)], hout[i & 1])
@@ -426,7 +438,7 @@ def main():
     ms_e2e = e2.elapsed_time(e3)
     cache.check_status()
     h2d = sum(x.numel() * x.element_size() for x in hpool[0])
-    d2h = hout[0].numel() * hout[0].element_size()
+    d2h = 0 if update_only else hout[0].numel() * hout[0].element_size()
 
     if world > 1:
         ms_total, ms_e2e = max_over_ranks([ms_total, ms_e2e], dev)
@@ -438,7 +450,7 @@ def main():
         alg = algorithmic_bytes_per_step(w)
         achieved = alg / (ms_step * 1e-3) / 1e9
         if stream:
-            roof = stream_roofline(w, tok_per_step, ms_step, precise=bool(args.flags & 16))
+            roof = stream_roofline(w, tok_per_step, ms_step, precise=bool(args.flags & 16), write_only=update_only)
         else:
             roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                     "traffic": measured_traffic(w, cache.tensor_path), "peak_kind": "of " + peak_kind,
@@ -452,7 +464,8 @@ def main():
             "config": {"workload": w.name, "batch_per_gpu": w.batch, "n_q_heads": w.n_q_heads,
                        "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim, "capacity": w.capacity,
                        "write_scale": w.write_scale, "read_scale": w.read_scale,
-                       "tokens_per_step": tok_per_step,
+                       "tokens_per_step": tok_per_step, "call": "bct_update_kv" if update_only else (
+                           "bct_prefill_stream" if stream else "bct_decode_step"),
                        "l2": ("cache planes of all units (%.2f GB) exceed L2" % (1.5 * alg / 1e9)) if stream else
                              ("cache planes streamed per step (%.2f GB) exceed L2" % (alg / 1e9)),
                        "parallelism": "independent units; replicas per GPU" if world > 1 else "1 GPU"},
