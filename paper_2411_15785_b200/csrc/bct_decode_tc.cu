@@ -43,6 +43,7 @@ constexpr int kScoreCols = 16;                 // tensor-memory columns per scor
 constexpr int kOCol = kMaxTiles * kScoreCols;  // output accumulator behind the score tiles
 constexpr int kTmemCols = 512;
 constexpr int kMaxClusterTc = 8;
+constexpr int kLwwCap = 512;                   // rewritten rows whose weights are kept for the deferred update
 constexpr float kNegBigTc = -3.0e38f;
 
 struct TcArgs {
@@ -64,7 +65,7 @@ struct TcArgs {
 };
 
 struct TcSmem {
-    int ring, pbuf, qbuf, wsm, list, lostage, red, stat, wstat, merge, bars, total;
+    int ring, pbuf, qbuf, wsm, list, lww, lostage, red, stat, wstat, merge, bars, total;
 };
 __host__ __device__ inline TcSmem tc_smem(int stages, int G, int S, int slice_rows, int lo_cap) {
     const int rows = (slice_rows + kTileRows - 1) / kTileRows * kTileRows;
@@ -82,6 +83,8 @@ __host__ __device__ inline TcSmem tc_smem(int stages, int G, int S, int slice_ro
     L.list = off;     // slots the update rule rewrites this token, in no particular order
     off += rows * 2;
     off = (off + 15) & ~15;
+    L.lww = off;      // write weights of the first kLwwCap listed slots (the update is applied one unit late)
+    off += kLwwCap * 4;
     L.lostage = off;  // staged copies of up to lo_cap of those rows: value plane rows, then residual rows
     off += 2 * lo_cap * 256;
     L.red = off;
@@ -117,6 +120,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     unsigned char* qbuf = smem + L.qbuf;
     float* wsm = reinterpret_cast<float*>(smem + L.wsm);
     unsigned short* list = reinterpret_cast<unsigned short*>(smem + L.list);
+    float* lww = reinterpret_cast<float*>(smem + L.lww);
     unsigned char* histage = smem + L.lostage;
     unsigned char* lostage = histage + kLoCap * ROW_BYTES;
     float* red = reinterpret_cast<float*>(smem + L.red);
@@ -325,6 +329,10 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 
         int it = 0;
         uint32_t sp = 0;  // sub-slices processed so far (phase of the per-tile barriers)
+        // update of the previous unit, applied during this unit's turn: rows listed, plane offset, v_t * eta_t
+        int pend_n = 0;
+        size_t pend_off = 0;
+        float pend_vt[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
         const int n_sub_rows = max(n_sub, 1);  // a unit with no tile still has its appended slot to look after
         for (int u = cid; u < a.U; u += ncl, ++it) {
             const int b = u / a.Hkv;
@@ -507,24 +515,67 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             // ---- list the slots the rule rewrites and stage copies of their value and residual rows with
             // ---- 16-byte asynchronous copies, so that no global-memory latency is left for the update ----
             const int c16 = tid & 15;  // 16-byte chunk of a 256-byte row
-            auto stage_rows = [&](int base, int n) {
+            auto stage_rows = [&](size_t uoff, int base, int n) {
                 for (int i = tid >> 4; i < n; i += kSThreads / 16) {
-                    const size_t goff = unit_off + (size_t)(slice_start + list[base + i]) * ROW_BYTES + c16 * 16;
+                    const size_t goff = uoff + (size_t)(slice_start + list[base + i]) * ROW_BYTES + c16 * 16;
                     cp_async16(histage + i * ROW_BYTES + c16 * 16, a.vhi + goff);
                     cp_async16(lostage + i * ROW_BYTES + c16 * 16, a.vlo + goff);
                 }
                 cp_async_commit();
             };
+            // The update rule MV_t = MV_{t-1} + ww_t^T . wv_t on the rows it changes: rounds of kLoCap staged
+            // rows.  `late`: the rows are those of the previous unit (weights kept in lww), whose first round
+            // has been in flight since that unit's epilogue.
+            auto apply_update = [&](int n_rows, size_t uoff, const float* vtv, bool late) {
+                for (int base = 0; base < n_rows; base += kLoCap) {
+                    const int n = min(n_rows - base, kLoCap);
+                    if (base > 0) {
+                        s_sync();  // the previous round's staged rows have been consumed
+                        stage_rows(uoff, base, n);
+                    }
+                    cp_async_wait_all();
+                    s_sync();  // every thread's staged chunks have landed
+                    for (int i = tid >> 4; i < n; i += kSThreads / 16) {
+                        const int row = list[base + i];
+                        const float ww = late ? lww[base + i] : __expf(wsm[row] - st_m[G]) * wfac;
+                        const size_t goff = uoff + (size_t)(slice_start + row) * ROW_BYTES + c16 * 16;
+                        float x[8], lo[8], nv[8], hf[8];
+                        Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(histage + i * ROW_BYTES + c16 * 16), x);
+                        Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(lostage + i * ROW_BYTES + c16 * 16), lo);
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) nv[e] = fmaf(ww, vtv[e], x[e] + lo[e]);
+                        const uint4 hi_new = Chunk<__nv_bfloat16>::pack(nv);
+                        Chunk<__nv_bfloat16>::unpack(hi_new, hf);
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) nv[e] -= hf[e];
+                        *reinterpret_cast<uint4*>(a.vhi + goff) = hi_new;
+                        *reinterpret_cast<uint4*>(a.vlo + goff) = Chunk<__nv_bfloat16>::pack(nv);
+                    }
+                }
+            };
+            // The previous unit's rows first: their staged copies had this unit's whole softmax to arrive,
+            // and this unit's V tiles are being multiplied meanwhile.  (Units are independent memories.)
+            if (pend_n > 0) {
+                apply_update(pend_n, pend_off, pend_vt, true);
+                pend_n = 0;
+                s_sync();  // the list and the staging rows are free for this unit
+                if (tid == 0) *lo_count = 0;
+                s_sync();
+            }
             int n_touched = 0;
             if (a.do_write) {
                 for (int t = 0; t < nt; ++t) {
                     const int row = t * kTileRows + r;
-                    if (row < n_stream && (a.dense || __expf(wsm[row] - st_m[G]) * wfac >= a.write_eps))
-                        list[atomicAdd(lo_count, 1)] = (unsigned short)row;
+                    const float ww = (row < n_stream) ? __expf(wsm[row] - st_m[G]) * wfac : 0.f;
+                    if (row < n_stream && (a.dense || ww >= a.write_eps)) {
+                        const int idx = atomicAdd(lo_count, 1);
+                        list[idx] = (unsigned short)row;
+                        if (idx < kLwwCap) lww[idx] = ww;
+                    }
                 }
                 s_sync();
                 n_touched = *lo_count;
-                stage_rows(0, min(n_touched, kLoCap));
+                stage_rows(unit_off, 0, min(n_touched, kLoCap));
             }
 
             // ---- epilogue: O[d][g] from tensor memory once every V tile has been read ----
@@ -603,36 +654,20 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 }
             }
 
-            // ---- the update rule MV_t = MV_{t-1} + ww_t^T . wv_t on the rows it changes ----
-            if (a.do_write) {
+            // ---- the update: deferred to the next unit's turn (its weights are in lww), unless it rewrites
+            // ---- more rows than lww keeps (diffuse write weights): then it is applied here ----
+            if (a.do_write && n_touched > 0) {
                 float vt[8];
                 Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(a.v + kv_off + c16 * 16), vt);
 #pragma unroll
                 for (int e = 0; e < 8; ++e) vt[e] *= eta_u;
-                for (int base = 0; base < n_touched; base += kLoCap) {
-                    const int n = min(n_touched - base, kLoCap);
-                    if (base > 0) {
-                        s_sync();  // the previous round's staged rows have been consumed
-                        stage_rows(base, n);
-                    }
-                    cp_async_wait_all();
-                    s_sync();  // every thread's staged chunks have landed
-                    for (int i = tid >> 4; i < n; i += kSThreads / 16) {
-                        const int row = list[base + i];
-                        const float ww = __expf(wsm[row] - st_m[G]) * wfac;
-                        const size_t goff = unit_off + (size_t)(slice_start + row) * ROW_BYTES + c16 * 16;
-                        float x[8], lo[8], nv[8], hf[8];
-                        Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(histage + i * ROW_BYTES + c16 * 16), x);
-                        Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(lostage + i * ROW_BYTES + c16 * 16), lo);
+                if (n_touched <= kLwwCap) {
+                    pend_n = n_touched;
+                    pend_off = unit_off;
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) nv[e] = fmaf(ww, vt[e], x[e] + lo[e]);
-                        const uint4 hi_new = Chunk<__nv_bfloat16>::pack(nv);
-                        Chunk<__nv_bfloat16>::unpack(hi_new, hf);
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) nv[e] -= hf[e];
-                        *reinterpret_cast<uint4*>(a.vhi + goff) = hi_new;
-                        *reinterpret_cast<uint4*>(a.vlo + goff) = Chunk<__nv_bfloat16>::pack(nv);
-                    }
+                    for (int e = 0; e < 8; ++e) pend_vt[e] = vt[e];
+                } else {
+                    apply_update(n_touched, unit_off, vt, false);
                 }
             }
             if (has_virtual && tid < 16) {  // store the appended slot
@@ -641,8 +676,41 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 *reinterpret_cast<uint4*>(a.vhi + off) = *reinterpret_cast<const uint4*>(a.v + kv_off + tid * 16);
                 *reinterpret_cast<uint4*>(a.vlo + off) = make_uint4(0, 0, 0, 0);
             }
-            s_sync();  // st_*, red, wsm, the list and the staging rows are reused by the next unit
-            if (tid == 0) *lo_count = 0;
+            s_sync();  // st_*, red and wsm are reused by the next unit (the list and the staging rows: after its deferred update)
+            if (pend_n == 0 && tid == 0) *lo_count = 0;
+        }
+        if (pend_n > 0) {  // the last unit's rows
+            const int c16 = tid & 15;
+            for (int base = 0; base < pend_n; base += kLoCap) {
+                const int n = min(pend_n - base, kLoCap);
+                if (base > 0) {
+                    s_sync();
+                    for (int i = tid >> 4; i < n; i += kSThreads / 16) {
+                        const size_t goff = pend_off + (size_t)(slice_start + list[base + i]) * ROW_BYTES + c16 * 16;
+                        cp_async16(histage + i * ROW_BYTES + c16 * 16, a.vhi + goff);
+                        cp_async16(lostage + i * ROW_BYTES + c16 * 16, a.vlo + goff);
+                    }
+                    cp_async_commit();
+                }
+                cp_async_wait_all();
+                s_sync();
+                for (int i = tid >> 4; i < n; i += kSThreads / 16) {
+                    const int row = list[base + i];
+                    const float ww = lww[base + i];
+                    const size_t goff = pend_off + (size_t)(slice_start + row) * ROW_BYTES + c16 * 16;
+                    float x[8], lo[8], nv[8], hf[8];
+                    Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(histage + i * ROW_BYTES + c16 * 16), x);
+                    Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(lostage + i * ROW_BYTES + c16 * 16), lo);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) nv[e] = fmaf(ww, pend_vt[e], x[e] + lo[e]);
+                    const uint4 hi_new = Chunk<__nv_bfloat16>::pack(nv);
+                    Chunk<__nv_bfloat16>::unpack(hi_new, hf);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) nv[e] -= hf[e];
+                    *reinterpret_cast<uint4*>(a.vhi + goff) = hi_new;
+                    *reinterpret_cast<uint4*>(a.vlo + goff) = Chunk<__nv_bfloat16>::pack(nv);
+                }
+            }
         }
     }
 
