@@ -524,9 +524,9 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 cp_async_commit();
             };
             // The update rule MV_t = MV_{t-1} + ww_t^T . wv_t on the rows it changes: rounds of kLoCap staged
-            // rows.  `late`: the rows are those of the previous unit (weights kept in lww), whose first round
-            // has been in flight since that unit's epilogue.
-            auto apply_update = [&](int n_rows, size_t uoff, const float* vtv, bool late) {
+            // rows of the previous unit (weights kept in lww), whose first round has been in flight since that
+            // unit's epilogue.
+            auto apply_update = [&](int n_rows, size_t uoff, const float* vtv) {
                 for (int base = 0; base < n_rows; base += kLoCap) {
                     const int n = min(n_rows - base, kLoCap);
                     if (base > 0) {
@@ -537,7 +537,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     s_sync();  // every thread's staged chunks have landed
                     for (int i = tid >> 4; i < n; i += kSThreads / 16) {
                         const int row = list[base + i];
-                        const float ww = late ? lww[base + i] : __expf(wsm[row] - st_m[G]) * wfac;
+                        const float ww = lww[base + i];
                         const size_t goff = uoff + (size_t)(slice_start + row) * ROW_BYTES + c16 * 16;
                         float x[8], lo[8], nv[8], hf[8];
                         Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(histage + i * ROW_BYTES + c16 * 16), x);
@@ -556,7 +556,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             // The previous unit's rows first: their staged copies had this unit's whole softmax to arrive,
             // and this unit's V tiles are being multiplied meanwhile.  (Units are independent memories.)
             if (pend_n > 0) {
-                apply_update(pend_n, pend_off, pend_vt, true);
+                apply_update(pend_n, pend_off, pend_vt);
                 pend_n = 0;
                 s_sync();  // the list and the staging rows are free for this unit
                 if (tid == 0) *lo_count = 0;
@@ -575,7 +575,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 }
                 s_sync();
                 n_touched = *lo_count;
-                stage_rows(unit_off, 0, min(n_touched, kLoCap));
+                // (a unit that rewrites more rows than lww keeps goes in double-buffered half rounds, below)
+                stage_rows(unit_off, 0, min(n_touched, n_touched > kLwwCap ? kLoCap / 2 : kLoCap));
             }
 
             // ---- epilogue: O[d][g] from tensor memory once every V tile has been read ----
@@ -667,7 +668,44 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 #pragma unroll
                     for (int e = 0; e < 8; ++e) pend_vt[e] = vt[e];
                 } else {
-                    apply_update(n_touched, unit_off, vt, false);
+                    // Diffuse write weights: most rows of the slice.  Half rounds alternate between the two
+                    // halves of the staging area, so that one half round is rewritten while the next arrives.
+                    const int hcap = kLoCap / 2;
+                    const int n_rounds = (n_touched + hcap - 1) / hcap;
+                    for (int rd = 0; rd < n_rounds; ++rd) {
+                        const int base = rd * hcap, n = min(n_touched - base, hcap);
+                        const int sbase = (rd & 1) * hcap;  // first staging row of this half round
+                        if (rd + 1 < n_rounds) {  // ask for the next half round (its half was consumed a round ago)
+                            const int nb = base + hcap, nn = min(n_touched - nb, hcap), nsb = ((rd + 1) & 1) * hcap;
+                            for (int i = tid >> 4; i < nn; i += kSThreads / 16) {
+                                const size_t goff = unit_off + (size_t)(slice_start + list[nb + i]) * ROW_BYTES + c16 * 16;
+                                cp_async16(histage + (nsb + i) * ROW_BYTES + c16 * 16, a.vhi + goff);
+                                cp_async16(lostage + (nsb + i) * ROW_BYTES + c16 * 16, a.vlo + goff);
+                            }
+                            cp_async_commit();
+                            cp_async_wait_but_one();
+                        } else {
+                            cp_async_wait_all();
+                        }
+                        s_sync();  // this half round's chunks have landed for every thread
+                        for (int i = tid >> 4; i < n; i += kSThreads / 16) {
+                            const int row = list[base + i];
+                            const float ww = __expf(wsm[row] - st_m[G]) * wfac;
+                            const size_t goff = unit_off + (size_t)(slice_start + row) * ROW_BYTES + c16 * 16;
+                            float x[8], lo[8], nv[8], hf[8];
+                            Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(histage + (sbase + i) * ROW_BYTES + c16 * 16), x);
+                            Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(lostage + (sbase + i) * ROW_BYTES + c16 * 16), lo);
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) nv[e] = fmaf(ww, vt[e], x[e] + lo[e]);
+                            const uint4 hi_new = Chunk<__nv_bfloat16>::pack(nv);
+                            Chunk<__nv_bfloat16>::unpack(hi_new, hf);
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) nv[e] -= hf[e];
+                            *reinterpret_cast<uint4*>(a.vhi + goff) = hi_new;
+                            *reinterpret_cast<uint4*>(a.vlo + goff) = Chunk<__nv_bfloat16>::pack(nv);
+                        }
+                        s_sync();  // the half is free for the round after next
+                    }
                 }
             }
             if (has_virtual && tid < 16) {  // store the appended slot

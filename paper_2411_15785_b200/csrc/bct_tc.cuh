@@ -95,6 +95,8 @@ __device__ __forceinline__ void cp_async16(void* dst_smem, const void* src_gmem)
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+// all but the most recent group of 16-byte copies have landed
+__device__ __forceinline__ void cp_async_wait_but_one() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
 
 
 // General form: M in {64,128}, N a multiple of 16 (for M = 128), each operand K-major or MN-major.
