@@ -178,7 +178,7 @@ bct_status_t bct_prefill_stream_eta(bct_cache_t *cache, const void *q, const voi
  *   wq   DEVICE [B][T][Hkv][d]  write queries     wv  DEVICE [B][T][Hkv][d]  write key-value vectors
  *   eta  DEVICE float [B][T][Hkv] or NULL (all ones)
  * Needs a full cache (the paper's full-size MV_0; BCT_ERR_STATE otherwise) of the shape the chunked
- * tensor-core kernel serves: bfloat16, head_dim 128, 128..2048 slots, no BCT_FLAG_SKIP_FIRST_WRITE
+ * tensor-core kernel serves: bfloat16, head_dim 128, 128..16384 slots, no BCT_FLAG_SKIP_FIRST_WRITE
  * (BCT_ERR_UNSUPPORTED otherwise: use bct_prefill_stream with out == NULL).
  */
 bct_status_t bct_update_kv(bct_cache_t *cache, const void *wq, const void *wv, const float *eta, int64_t T,

@@ -326,7 +326,7 @@ bct_status_t bct_update_kv(bct_cache_t* c, const void* wq, const void* wv, const
                     c->p.capacity);
     if (bct::stream_chunk_tokens(c) == 0 || (c->p.flags & BCT_FLAG_SKIP_FIRST_WRITE))
         return fail(BCT_ERR_UNSUPPORTED,
-                    "the write-only form serves bfloat16 caches with head_dim 128 and 128..2048 slots, without "
+                    "the write-only form serves bfloat16 caches with head_dim 128 and 128..16384 slots, without "
                     "SKIP_FIRST_WRITE; use bct_prefill_stream with out = NULL");
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const int64_t whole = T / 128, rest = T - whole * 128;

@@ -12,7 +12,7 @@
 // While the cache still has Tc free slots the same kernel runs in fill mode: the chunk's keys and
 // values are appended (TMA stores from the operand buffers), token t reads the resident slots plus
 // the chunk's own slots s <= t (scores Q Kc^T, masked causally), and nothing is soft-written.
-// One persistent CTA per (sequence, kv-head) unit at a time (C <= 2048 slots); per chunk the cache
+// One persistent CTA per (sequence, kv-head) unit at a time (C <= 16384 slots); per chunk the cache
 // streams through shared memory twice for MK (row statistics, then numerators) and once for MV
 // (value and residual planes), instead of twice per token, and every product runs as tcgen05.mma
 // with fp32 accumulators in tensor memory.  The write weights are always kept as bfloat16
@@ -41,6 +41,7 @@ constexpr int kStHalf = 128 * 128;       // 64 columns (128 bytes) x 128 rows
 constexpr int kStTileBytes = 2 * kStHalf;
 constexpr int kStMaxStages = 4;
 constexpr int kStMaxTc = 64;
+constexpr int kStMaxCapacity = 16384;    // slots per unit: one CTA walks all tiles of a unit, twice per chunk
 constexpr float kStNegBig = -3.0e38f;
 // tensor-memory columns
 constexpr int kColS0 = 0;     // score tile (pass 2, and buffer 0 of pass 1)
@@ -861,7 +862,7 @@ int stream_chunk_tokens(const bct_cache* c) {
     const bct_params_t& p = c->p;
     if (p.dtype != BCT_BF16 || p.head_dim != 128 || c->G > 7 || !c->tc_ready) return 0;
     if (p.flags & BCT_FLAG_CUDA_CORES) return 0;
-    if (p.capacity < kStTile || p.capacity > 2048) return 0;
+    if (p.capacity < kStTile || p.capacity > kStMaxCapacity) return 0;
     if (c->plane_bytes < (size_t)1 << 18) return 0;
     return c->G == 1 ? 64 : (c->G <= 3 ? 32 : 16);
 }

@@ -49,6 +49,8 @@ def _stream_parity(w, T, pieces, flags=0, oracle_flags=0, want_out=True):
     (3, 640, 640, 64, [64]),
     (4, 520, 520, 50, [50]),              # chunks of 16
     (7, 2048, 2048, 32, [32]),            # 16 tiles
+    (4, 4096, 4096, 40, [40]),            # 32 tiles per unit: beyond one decode CTA's slice
+    (1, 3000, 3000, 130, [130]),          # ragged capacity above 2048
 ])
 def test_chunked_stream_matches_oracle(G, C, init_len, T, pieces):
     d = 128
@@ -100,6 +102,7 @@ def test_chunked_stream_tracks_decode_steps_on_a_long_run():
     (2, 512, 100, 300, [300], 0),                  # starts inside tile 0; chunks of 32 cross tile borders
     (3, 640, 37, 200, [70, 130], B.FLAG_OUT_F32),  # odd start, second call resumes the fill phase
     (7, 2048, 1900, 140, [140], 0),                # chunks of 16 over 15 resident tiles
+    (2, 2500, 2400, 160, [160], 0),                # fill chunks above 2048 slots, then soft writes
     (1, 256, 192, 64, [64], B.FLAG_PRECISE_READ | B.FLAG_OUT_F32),  # exactly fills the cache
 ])
 def test_fill_phase_chunks_match_oracle(G, C, init_len, T, pieces, flags):
