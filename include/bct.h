@@ -76,7 +76,7 @@ typedef enum bct_dtype {
                                         bfloat16 ulp matter */
 #define BCT_FLAG_CUDA_CORES 32u       /* keep every decode step on the CUDA-core kernel (the
                                         tensor-core kernel serves bfloat16, head_dim 128,
-                                        G <= 7, C >= 128 by default) */
+                                        G <= 15, C >= 128 by default) */
 #define BCT_FLAG_OUT_F32 8u          /* `out` is float (the fp32 accumulator, unrounded)
                                         whatever the cache dtype */
 
@@ -294,7 +294,7 @@ bct_status_t bct_cache_import(bct_cache_t *cache, const void *k_in, const void *
 bct_status_t bct_cache_status(bct_cache_t *cache, void *cuda_stream);
 
 /* *yes = 1 if this cache's decode steps run on the tensor-core kernel (tcgen05 + TMA tensor
- * copies: bfloat16, head_dim 128, G <= 7, 128 <= C <= 65536, no PRECISE_READ / CUDA_CORES
+ * copies: bfloat16, head_dim 128, G <= 15, 128 <= C <= 65536, no PRECISE_READ / CUDA_CORES
  * flag), 0 if on the CUDA-core kernel.  Both compute the same step (Algorithm 1 + read). */
 bct_status_t bct_cache_tensor_path(const bct_cache_t *cache, int32_t *yes);
 

@@ -59,8 +59,8 @@ bct_status_t resolve_params(const bct_params_t* in, bct_params_t* p) {
         return fail(BCT_ERR_INVALID_ARG, "batch * n_kv_heads too large");
     if (p->head_dim != 64 && p->head_dim != 128)
         return fail(BCT_ERR_UNSUPPORTED, "head_dim %d: this library has kernels for 64 and 128", p->head_dim);
-    if (p->n_q_heads / p->n_kv_heads > bct::kMaxGroup)
-        return fail(BCT_ERR_UNSUPPORTED, "group size %d > %d", p->n_q_heads / p->n_kv_heads, bct::kMaxGroup);
+    if (p->n_q_heads / p->n_kv_heads > bct::kMaxGroupTc)
+        return fail(BCT_ERR_UNSUPPORTED, "group size %d > %d", p->n_q_heads / p->n_kv_heads, bct::kMaxGroupTc);
     return BCT_OK;
 }
 
@@ -221,7 +221,8 @@ bct_status_t bct_cache_create(const bct_params_t* params, void* workspace, size_
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
     if (e != cudaSuccess) return fail_cuda("device query", e);
     const char* why = "";
-    if (!bct::decode_supported(p, optin, &why)) return fail(BCT_ERR_UNSUPPORTED, "%s", why);
+    const bool tc_only = p.n_q_heads / p.n_kv_heads > bct::kMaxGroup;  // 9..15 query heads per kv-head: tensor-core kernel only
+    if (!tc_only && !bct::decode_supported(p, optin, &why)) return fail(BCT_ERR_UNSUPPORTED, "%s", why);
 
     bct_cache_t* c = new (std::nothrow) bct_cache_t();
     if (c == nullptr) return fail(BCT_ERR_STATE, "out of host memory");
@@ -268,6 +269,14 @@ bct_status_t bct_cache_create(const bct_params_t* params, void* workspace, size_
         return fail_cuda("stream / event creation", e);
     }
     bct::tc_prepare(c);  // tensor maps of the planes; without them the CUDA-core kernel serves every shape
+    if (tc_only && (!bct::tc_eligible(c) || (p.flags & BCT_FLAG_CUDA_CORES))) {
+        release_host_objects(c);
+        c->magic = 0;
+        delete c;
+        return fail(BCT_ERR_UNSUPPORTED,
+                    "group sizes 9..15 are served by the tensor-core kernel only: bfloat16, head_dim 128, 128 <= capacity "
+                    "<= 65536, K plane >= 256 KiB, no PRECISE_READ / CUDA_CORES");
+    }
 
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     e = cudaMemsetAsync(c->status, 0, bct::kAlign, stream);

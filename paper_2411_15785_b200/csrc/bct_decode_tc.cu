@@ -37,8 +37,14 @@ constexpr int kHalfBytes = 128 * 128;          // 64 columns (128 bytes) x 128 r
 constexpr int kTcTileBytes = 2 * kHalfBytes;   // one 128 x 128 bfloat16 tile
 constexpr int kMaxTiles = 16;                  // tiles per sub-slice: score tiles resident in tensor memory
 constexpr int kMaxSliceRows = 8192;            // slots per CTA: up to 4 sub-slices of 2048, streamed one after the other
-constexpr int kPTileBytes = 2048;              // P operand of one tile: 2 halves x (8 rows x 128 B)
-constexpr int kQBufBytes = 3072;               // Q operand (2 halves x 8 rows x 128 B) + 1 KiB of zeros
+// Operand rows of the small operands (queries, softmax numerators): the N = 16 instruction shape reads 16
+// rows; with up to 7 read heads 8 rows are kept and the upper 8 are whatever follows (their score / output
+// columns are never read), with 8 to 15 read heads all 16 are kept.
+__host__ __device__ constexpr int tc_rows(int G) { return G + 1 <= 8 ? 8 : 16; }
+__host__ __device__ constexpr int tc_ptile_bytes(int G) { return 2 * tc_rows(G) * 128; }  // P operand of one tile: 2 halves
+__host__ __device__ constexpr int tc_qbuf_bytes(int G) {  // Q operand: 2 halves (+ 1 KiB of zeros behind 8-row halves)
+    return 2 * tc_rows(G) * 128 + (tc_rows(G) == 8 ? 1024 : 0);
+}
 constexpr int kScoreCols = 16;                 // tensor-memory columns per score tile (N = 16)
 constexpr int kOCol = kMaxTiles * kScoreCols;  // output accumulator behind the score tiles
 constexpr int kTmemCols = 512;
@@ -75,9 +81,9 @@ __host__ __device__ inline TcSmem tc_smem(int stages, int G, int S, int slice_ro
     L.ring = off;
     off += stages * kTcTileBytes;
     L.pbuf = off;
-    off += p_tiles * kPTileBytes + 1024;
+    off += p_tiles * tc_ptile_bytes(G) + 1024;
     L.qbuf = off;
-    off += 2 * kQBufBytes;
+    off += 2 * tc_qbuf_bytes(G);
     L.wsm = off;
     off += rows * 4;  // scaled write score of every slot of the slice
     L.list = off;     // slots the update rule rewrites this token, in no particular order
@@ -88,9 +94,9 @@ __host__ __device__ inline TcSmem tc_smem(int stages, int G, int S, int slice_ro
     L.lostage = off;  // staged copies of up to lo_cap of those rows: value plane rows, then residual rows
     off += 2 * lo_cap * 256;
     L.red = off;
-    off += 4 * 16 * 4;
-    L.stat = off;  // m[8], l[8], wd[8], ev[8], abort, tmem address
-    off += 256;
+    off += 4 * 32 * 4;  // per softmax warp: 16 partial maxima / sums, 16 partial appended-slot scores / overlaps
+    L.stat = off;  // m[16], l[16], wd[16], ev[16], alpha[16], abort, tmem address, list count
+    off += 512;
     L.wstat = off;
     off += 2 * kMaxClusterTc * 2 * 4;
     L.merge = off;
@@ -102,6 +108,21 @@ __host__ __device__ inline TcSmem tc_smem(int stages, int G, int S, int slice_ro
     return L;
 }
 
+// N = 8 or 16 consecutive columns of this thread's tensor-memory lane
+template <int N>
+__device__ __forceinline__ void tmem_ld_rows(uint32_t taddr, float* x) {
+    if constexpr (N == 8) {
+        tmem_ld8(taddr, x);
+    } else {
+        tmem_ld16(taddr, x);
+    }
+}
+template <int N>
+__device__ __forceinline__ void tmem_st_rows(uint32_t taddr, const float* x) {
+    tmem_st8(taddr, x);
+    if constexpr (N == 16) tmem_st8(taddr + 8, x + 8);
+}
+
 __device__ __forceinline__ void s_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kSThreads) : "memory"); }
 
 template <int G>
@@ -109,6 +130,9 @@ __global__ void __launch_bounds__(kTcThreads, 1)
 decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const TcArgs a) {
     constexpr int D = 128;
     constexpr int ROW_BYTES = 256;
+    constexpr int NR = tc_rows(G);                 // operand rows kept: read heads, write query, zero rows
+    constexpr int kQHalf = NR * 128, kPHalf = NR * 128;  // bytes between the two 64-column halves
+    constexpr int kQBufBytes = tc_qbuf_bytes(G), kPTileBytes = tc_ptile_bytes(G);
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int S = a.S;
@@ -125,13 +149,13 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     unsigned char* lostage = histage + kLoCap * ROW_BYTES;
     float* red = reinterpret_cast<float*>(smem + L.red);
     float* st_m = reinterpret_cast<float*>(smem + L.stat);
-    float* st_l = st_m + 8;
-    float* st_wd = st_m + 16;
-    float* st_ev = st_m + 24;
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(st_m + 32);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(st_m + 33);
-    int* lo_count = reinterpret_cast<int*>(st_m + 34);
-    float* st_alpha = st_m + 36;  // per head: exp(old maximum - new maximum) of the current sub-slice
+    float* st_l = st_m + 16;
+    float* st_wd = st_m + 32;
+    float* st_ev = st_m + 48;
+    float* st_alpha = st_m + 64;  // per head: exp(old maximum - new maximum) of the current sub-slice
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(st_m + 80);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(st_m + 81);
+    int* lo_count = reinterpret_cast<int*>(st_m + 82);
     float* wstat = reinterpret_cast<float*>(smem + L.wstat);
     float* merge = reinterpret_cast<float*>(smem + L.merge);
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + L.bars);
@@ -265,7 +289,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 #pragma unroll
                         for (int kk = 0; kk < 8; ++kk) {
                             const uint64_t ad = desc_at(dk0, taddr + (kk >> 2) * kHalfBytes + (kk & 3) * 32);
-                            const uint64_t bd = desc_at(dk0, qaddr + (kk >> 2) * 1024 + (kk & 3) * 32);
+                            const uint64_t bd = desc_at(dk0, qaddr + (kk >> 2) * kQHalf + (kk & 3) * 32);
                             umma_bf16(tmem_base + (t - t_begin) * kScoreCols, ad, bd, idesc_s, kk > 0);
                         }
                         umma_commit(&sready[t - t_begin]);
@@ -290,7 +314,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 #pragma unroll
                         for (int kk = 0; kk < 8; ++kk) {  // 16 slots per step
                             const uint64_t ad = desc_at(dmn0, taddr + kk * 2048);
-                            const uint64_t bd = desc_at(dk0, paddr + (kk >> 2) * 1024 + (kk & 3) * 32);
+                            const uint64_t bd = desc_at(dk0, paddr + (kk >> 2) * kPHalf + (kk & 3) * 32);
                             umma_bf16(tmem_base + kOCol, ad, bd, idesc_o, (t > 0) || (kk > 0));
                         }
                         umma_commit(&empty[stage]);
@@ -313,12 +337,13 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         auto write_q = [&](int u, int buf) {
             const int b = u / a.Hkv;
             const int h_kv = u - b * a.Hkv;
-            const int h = tid >> 4, c = tid & 15;
-            if (h <= G) {
+            const int c = tid & 15;
+#pragma unroll
+            for (int h = tid >> 4; h <= G; h += kSThreads / 16) {  // 8 rows per sweep of the 128 threads
                 const char* src = (h < G) ? a.q + ((size_t)b * a.q_bs + (size_t)h_kv * G * D) * 2 + (size_t)h * ROW_BYTES
                                           : a.k + ((size_t)b * a.kv_bs + (size_t)h_kv * D) * 2;
                 const uint4 w = *reinterpret_cast<const uint4*>(src + c * 16);
-                unsigned char* dst = qbuf + buf * kQBufBytes + (c >> 3) * 1024 + h * 128 + (((c & 7) ^ h) * 16);
+                unsigned char* dst = qbuf + buf * kQBufBytes + (c >> 3) * kQHalf + h * 128 + (((c & 7) ^ (h & 7)) * 16);
                 *reinterpret_cast<uint4*>(dst) = w;
             }
             fence_proxy_async_smem();
@@ -355,7 +380,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     vq[g] = warp_sum(qd * kd);
                 }
             }
-            if (tid < 8) {  // running maximum, sum and read-write overlap of the unit, over its sub-slices
+            if (tid < NR) {  // running maximum, sum and read-write overlap of the unit, over its sub-slices
                 st_m[tid] = kNegBigTc;
                 st_l[tid] = 0.f;
                 st_wd[tid] = 0.f;
@@ -368,35 +393,35 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 const bool last_sub = (sub == n_sub_rows - 1);
 
                 // ---- pass 1: row maxima of the raw scores, as the score tiles complete ----
-                float mx[8];
+                float mx[NR];
 #pragma unroll
-                for (int h = 0; h < 8; ++h) mx[h] = kNegBigTc;
+                for (int h = 0; h < NR; ++h) mx[h] = kNegBigTc;
                 for (int t = t_begin; t < t_end; ++t) {
                     if (!mbar_wait_abortable(&sready[t - t_begin], sp & 1, abort_flag)) {
                         report_timeout(a.status, 16);
                         *abort_flag = 1;
                     }
                     tc_fence_after();
-                    float s[8];
-                    tmem_ld8(lane_base + (t - t_begin) * kScoreCols, s);
+                    float s[NR];
+                    tmem_ld_rows<NR>(lane_base + (t - t_begin) * kScoreCols, s);
                     if (t * kTileRows + r < n_stream) {
 #pragma unroll
-                        for (int h = 0; h < 8; ++h) mx[h] = fmaxf(mx[h], s[h]);
+                        for (int h = 0; h < NR; ++h) mx[h] = fmaxf(mx[h], s[h]);
                     }
                 }
 #pragma unroll
-                for (int h = 0; h < 8; ++h) {
+                for (int h = 0; h < NR; ++h) {
                     mx[h] = warp_max(mx[h]);
-                    if (lane == 0) red[warp * 16 + h] = mx[h];
-                    if (lane == 0 && h < G) red[warp * 16 + 8 + h] = vq[h];
+                    if (lane == 0) red[warp * 32 + h] = mx[h];
+                    if (lane == 0 && h < G) red[warp * 32 + 16 + h] = vq[h];
                 }
                 s_sync();
-                if (tid < 8) {
+                if (tid < NR) {
                     const float scale = (tid < G) ? a.read_scale : a.write_scale;
-                    float m = fmaxf(fmaxf(red[tid], red[16 + tid]), fmaxf(red[32 + tid], red[48 + tid]));
+                    float m = fmaxf(fmaxf(red[tid], red[32 + tid]), fmaxf(red[64 + tid], red[96 + tid]));
                     m = (m <= kNegBigTc) ? kNegBigTc : m * scale;
                     if (last_sub && has_virtual && tid < G) {
-                        const float vs = (red[8 + tid] + red[24 + tid] + red[40 + tid] + red[56 + tid]) * a.read_scale;
+                        const float vs = (red[16 + tid] + red[48 + tid] + red[80 + tid] + red[112 + tid]) * a.read_scale;
                         st_ev[tid] = vs;  // scaled score of the appended slot, turned into a numerator below
                         m = fmaxf(m, vs);
                     }
@@ -414,37 +439,37 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         *abort_flag = 1;
                     }
                     tc_fence_after();
-                    float o[8];
-                    tmem_ld8(lane_base + kOCol, o);
+                    float o[NR];
+                    tmem_ld_rows<NR>(lane_base + kOCol, o);
 #pragma unroll
-                    for (int h = 0; h < 8; ++h) o[h] *= st_alpha[h];
-                    tmem_st8(lane_base + kOCol, o);
+                    for (int h = 0; h < NR; ++h) o[h] *= st_alpha[h];
+                    tmem_st_rows<NR>(lane_base + kOCol, o);
                     tc_fence_before();
                 }
 
                 // ---- pass 2: numerators, row sums, P operand (bfloat16, swizzled), scaled write scores ----
-                float sum[8];
+                float sum[NR];
                 float wdacc[G];
 #pragma unroll
-                for (int h = 0; h < 8; ++h) sum[h] = 0.f;
+                for (int h = 0; h < NR; ++h) sum[h] = 0.f;
 #pragma unroll
                 for (int g = 0; g < G; ++g) wdacc[g] = 0.f;
                 for (int t = t_begin; t < t_end; ++t) {
-                    float s[8];
-                    tmem_ld8(lane_base + (t - t_begin) * kScoreCols, s);
+                    float s[NR];
+                    tmem_ld_rows<NR>(lane_base + (t - t_begin) * kScoreCols, s);
                     const bool valid = t * kTileRows + r < n_stream;
-                    float e[8];
+                    float e[NR];
 #pragma unroll
-                    for (int h = 0; h < 8; ++h) {
+                    for (int h = 0; h < NR; ++h) {
                         const float scale = (h < G) ? a.read_scale : a.write_scale;
                         e[h] = (valid && h <= G) ? __expf(s[h] * scale - st_m[h]) : 0.f;
                         sum[h] += e[h];
                     }
-                    unsigned char* prow = pbuf + (t - t_begin) * kPTileBytes + (r >> 6) * 1024 + (r & 7) * 2;
+                    unsigned char* prow = pbuf + (t - t_begin) * kPTileBytes + (r >> 6) * kPHalf + (r & 7) * 2;
                     const int c8 = (r & 63) >> 3;
 #pragma unroll
                     for (int h = 0; h < G; ++h)  // rows G..7 of the operand stay zero
-                        *reinterpret_cast<__nv_bfloat16*>(prow + h * 128 + ((c8 ^ h) * 16)) = __float2bfloat16_rn(e[h]);
+                        *reinterpret_cast<__nv_bfloat16*>(prow + h * 128 + ((c8 ^ (h & 7)) * 16)) = __float2bfloat16_rn(e[h]);
                     wsm[t * kTileRows + r] = valid ? s[G] * a.write_scale : kNegBigTc;
 #pragma unroll
                     for (int g = 0; g < G; ++g) wdacc[g] = fmaf(e[g], e[G], wdacc[g]);
@@ -461,18 +486,18 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 }
 
 #pragma unroll
-                for (int h = 0; h < 8; ++h) {
+                for (int h = 0; h < NR; ++h) {
                     sum[h] = warp_sum(sum[h]);
-                    if (lane == 0) red[warp * 16 + h] = sum[h];
+                    if (lane == 0) red[warp * 32 + h] = sum[h];
                 }
 #pragma unroll
                 for (int g = 0; g < G; ++g) {
                     wdacc[g] = warp_sum(wdacc[g]);
-                    if (lane == 0) red[warp * 16 + 8 + g] = wdacc[g];
+                    if (lane == 0) red[warp * 32 + 16 + g] = wdacc[g];
                 }
                 s_sync();
-                if (tid < 8) {
-                    float l = red[tid] + red[16 + tid] + red[32 + tid] + red[48 + tid];
+                if (tid < NR) {
+                    float l = red[tid] + red[32 + tid] + red[64 + tid] + red[96 + tid];
                     if (last_sub && has_virtual && tid < G) {
                         const float ev = __expf(st_ev[tid] - st_m[tid]);
                         st_ev[tid] = ev;
@@ -480,7 +505,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     }
                     st_l[tid] = st_l[tid] * st_alpha[tid] + l;
                     st_wd[tid] = st_wd[tid] * st_alpha[tid] * st_alpha[G] +
-                                 (red[8 + tid] + red[24 + tid] + red[40 + tid] + red[56 + tid]);
+                                 (red[16 + tid] + red[48 + tid] + red[80 + tid] + red[112 + tid]);
                 }
                 s_sync();
             }
@@ -585,12 +610,12 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 *abort_flag = 1;
             }
             tc_fence_after();
-            float o[8];
+            float o[NR];
             if (nt > 0) {
-                tmem_ld8(lane_base + kOCol, o);
+                tmem_ld_rows<NR>(lane_base + kOCol, o);
             } else {
 #pragma unroll
-                for (int h = 0; h < 8; ++h) o[h] = 0.f;
+                for (int h = 0; h < NR; ++h) o[h] = 0.f;
             }
             tc_fence_before();
             if (has_virtual) {
@@ -775,6 +800,14 @@ TcKernelFn pick_tc(int G) {
         case 5: return decode_tc_kernel<5>;
         case 6: return decode_tc_kernel<6>;
         case 7: return decode_tc_kernel<7>;
+        case 8: return decode_tc_kernel<8>;
+        case 9: return decode_tc_kernel<9>;
+        case 10: return decode_tc_kernel<10>;
+        case 11: return decode_tc_kernel<11>;
+        case 12: return decode_tc_kernel<12>;
+        case 13: return decode_tc_kernel<13>;
+        case 14: return decode_tc_kernel<14>;
+        case 15: return decode_tc_kernel<15>;
         default: return nullptr;
     }
 }
@@ -812,7 +845,7 @@ TensorMapEncodeFn tensor_map_encode_fn() {
 
 bool tc_eligible(const bct_cache* c) {
     const bct_params_t& p = c->p;
-    if (p.dtype != BCT_BF16 || p.head_dim != 128 || c->G > 7) return false;
+    if (p.dtype != BCT_BF16 || p.head_dim != 128 || c->G > 15) return false;
     if (p.flags & BCT_FLAG_PRECISE_READ) return false;
     if (p.capacity < kTileRows || p.capacity > kMaxClusterTc * kMaxSliceRows) return false;
     if (c->plane_bytes < (size_t)1 << 18) return false;  // tiny planes stay on the CUDA-core kernel
@@ -845,8 +878,14 @@ int launch_decode_tc(const bct_cache* c, const StepIO& io, int len, int do_write
     int S = 1;
     if (p.capacity > kMaxTiles * kTileRows) S = 2;
     while (S < kMaxClusterTc && (p.capacity + S - 1) / S > kMaxSliceRows) S *= 2;
-    while (S < kMaxClusterTc && (long long)c->U * S * 2 <= c->sm_count && (p.capacity + 2 * S - 1) / (2 * S) >= kTileRows)
-        S *= 2;  // few units: spread each over more SMs
+    // few units: spread each over more SMs, as long as the merge buffer of the wider cluster (it grows with
+    // the cluster size times the group size) still leaves room for the smallest ring and staging area
+    while (S < kMaxClusterTc && (long long)c->U * S * 2 <= c->sm_count && (p.capacity + 2 * S - 1) / (2 * S) >= kTileRows) {
+        const int s2 = 2 * S;
+        const int slice2 = ((p.capacity + s2 - 1) / s2 + kTileRows - 1) / kTileRows * kTileRows;
+        if (tc_smem(3, c->G, s2, slice2, 32).total > c->smem_optin) break;
+        S = s2;
+    }
     int slice = (p.capacity + S - 1) / S;
     slice = (slice + kTileRows - 1) / kTileRows * kTileRows;  // whole tiles per CTA
     // Four ring stages and staging rounds of 80 rows where shared memory allows (slices up to 2048

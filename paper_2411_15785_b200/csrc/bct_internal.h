@@ -9,7 +9,8 @@ namespace bct {
 
 constexpr uint64_t kMagic = 0x4243545f43414348ull;  // "BCT_CACH"
 constexpr size_t kAlign = 256;                      // alignment of every workspace section
-constexpr int kMaxGroup = 8;
+constexpr int kMaxGroup = 8;     // query heads per kv-head on the CUDA-core kernel
+constexpr int kMaxGroupTc = 15;  // ... on the tensor-core decode kernel (16 operand rows: the read heads + the write query)
 
 // Where the step vectors of one launch live and how to walk them.
 struct StepIO {
@@ -71,13 +72,13 @@ int launch_decode(const bct_cache* c, const StepIO& io, int len, int do_write, c
 // Whether launch_decode has a kernel for these parameters (shape limits of the library).
 bool decode_supported(const bct_params_t& p, int smem_optin, const char** why);
 
-// Tensor-core (tcgen05 + TMA) decode path: bfloat16, head_dim 128, group <= 7.
+// Tensor-core (tcgen05 + TMA) decode path: bfloat16, head_dim 128, group <= 15.
 bool tc_prepare(bct_cache* c);          // encode the planes' tensor maps; false if unavailable
 bool tc_eligible(const bct_cache* c);   // this cache's decode steps run on the tensor path
 int launch_decode_tc(const bct_cache* c, const StepIO& io, int len, int do_write, cudaStream_t stream,
                      cudaError_t* err);
 
-// Chunked tensor-core stream kernel (full cache, bfloat16, head_dim 128, G <= 7, C <= 2048):
+// Chunked tensor-core stream kernel (bfloat16, head_dim 128, G <= 7, C <= 16384):
 // tokens per chunk for this cache, or 0 when the kernel does not apply.
 int stream_chunk_tokens(const bct_cache* c);
 // n_chunks whole chunks starting at token t_begin of the [B][T][H][d] step arrays.  fill_len < 0:

@@ -1,4 +1,6 @@
 """GPU parity of bct_decode_step / bct_prefill_stream against the CPU oracle (through the C ABI)."""
+import ctypes
+
 import numpy as np
 import pytest
 import torch
@@ -46,7 +48,7 @@ def test_small_shapes_match_oracle(dtype, d, G, C, init_len, steps):
     assert state_err <= TOL[dtype], state_err
 
 
-# ---- the tensor-core kernel (bfloat16, head_dim 128, G <= 7, C >= 128) and the CUDA-core kernel
+# ---- the tensor-core kernel (bfloat16, head_dim 128, G <= 15, C >= 128) and the CUDA-core kernel
 # ---- on the same shapes: both must match the oracle ----------------------------------------------------
 @pytest.mark.parametrize("cores", [False, True])
 @pytest.mark.parametrize("B_,G,C,init_len,steps", [
@@ -63,9 +65,15 @@ def test_small_shapes_match_oracle(dtype, d, G, C, init_len, steps):
     (20, 1, 16384, 16384, 3),  # cluster of 2, 8192-slot slices in four sub-slices
     (20, 3, 5000, 4993, 12),   # sub-slices while the cache is still filling
     (80, 1, 128, 0, 5),        # starts empty with more units than SMs: several tile-less units per CTA
+    (3, 8, 600, 590, 24),      # 8 read heads: the 16-row query / weight operands; fill finishes mid-run
+    (2, 12, 2048, 2048, 5),    # 12 read heads, a full 16-tile slice
+    (2, 15, 2500, 2500, 5),    # 15 read heads + the write query = all 16 rows; cluster of 2
+    (6, 8, 5000, 5000, 4),     # 8 read heads, sub-slices
 ])
 def test_tensor_core_and_cuda_core_kernels_match_oracle(cores, B_, G, C, init_len, steps):
     d = 128
+    if cores and G > 8:
+        pytest.skip("the CUDA-core kernel serves at most 8 query heads per kv-head")
     w = W.Workload("t", B_, 2 * G, 2, d, C, "bf16", init_len, steps, 13, d ** -0.5, 1.0, 1.0, "decode")
     units = pick_units(w, 6)
     out_err, state_err = run_decode_parity(w, units, flags=B.FLAG_CUDA_CORES if cores else 0,
@@ -76,10 +84,10 @@ def test_tensor_core_and_cuda_core_kernels_match_oracle(cores, B_, G, C, init_le
 
 @pytest.mark.parametrize("flag,oflag", [(B.FLAG_WRITE_THEN_READ, O.WRITE_THEN_READ), (B.FLAG_DENSE_WRITE, 0),
                                         (B.FLAG_OUT_F32, 0)])
-@pytest.mark.parametrize("C,B_", [(400, 2), (5000, 2), (6000, 20)])
-def test_tensor_core_kernel_flags(flag, oflag, C, B_):
+@pytest.mark.parametrize("C,B_,G", [(400, 2, 3), (5000, 2, 3), (6000, 20, 3), (700, 2, 9)])
+def test_tensor_core_kernel_flags(flag, oflag, C, B_, G):
     d = 128
-    w = W.Workload("t", B_, 6, 2, d, C, "bf16", C, 6, 17, d ** -0.5, 1.0, 1.0, "decode", 1.0, 0.3)
+    w = W.Workload("t", B_, 2 * G, 2, d, C, "bf16", C, 6, 17, d ** -0.5, 1.0, 1.0, "decode", 1.0, 0.3)
     out_err, state_err = run_decode_parity(w, pick_units(w, 4), flags=flag, oracle_flags=oflag,
                                            expect_tensor_path=True)
     assert out_err <= TOL["bf16"] and state_err <= TOL["bf16"], (out_err, state_err)
@@ -227,3 +235,17 @@ def test_bad_arguments_on_device_launch_nothing():
     assert st == B.BCT_ERR_UNSUPPORTED and not h.value
     c.destroy()
     assert c.lib.bct_cache_destroy(None) == B.BCT_OK
+
+
+def test_groups_above_eight_need_the_tensor_core_path():
+    # 9..15 query heads per kv-head exist on the tensor-core kernel only: a float cache of that shape is refused
+    prm = B.make_params(2, 24, 2, 128, 256, torch.float32)
+    lib = B.load()
+    n, al = ctypes.c_size_t(0), ctypes.c_size_t(0)
+    assert lib.bct_cache_bytes(ctypes.byref(prm), ctypes.byref(n), ctypes.byref(al)) == B.BCT_OK
+    ws = torch.empty(n.value, dtype=torch.uint8, device="cuda")
+    h = ctypes.c_void_p(None)
+    st = lib.bct_cache_create(ctypes.byref(prm), ws.data_ptr(), n.value, None, None, None, ctypes.byref(h))
+    assert st == B.BCT_ERR_UNSUPPORTED and "tensor-core" in B.last_error()
+    prm = B.make_params(2, 34, 2, 128, 256, torch.bfloat16)      # 17 per kv-head: nowhere
+    assert lib.bct_cache_bytes(ctypes.byref(prm), ctypes.byref(n), ctypes.byref(al)) == B.BCT_ERR_UNSUPPORTED
