@@ -333,24 +333,44 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         const int r = tid;  // tensor-memory lane: slot row of a score tile, d of the output
         const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
 
-        // Q operand of a unit: rows 0..G-1 its read queries, row G its write query (128-byte swizzle)
-        auto write_q = [&](int u, int buf) {
+        // Q operand of a unit: rows 0..G-1 its read queries, row G its write query (128-byte swizzle).
+        // The words are fetched from global memory at the start of the previous unit's turn and put in
+        // place when that unit's score tiles have been consumed: their latency would otherwise sit in
+        // every unit's chain (about 1 us of the 6 us a unit of 256 slots takes).
+        constexpr int kQWords = (NR + 7) / 8;  // 16-byte words of the operand per thread
+        auto load_q = [&](int u, uint4* w) {
             const int b = u / a.Hkv;
             const int h_kv = u - b * a.Hkv;
             const int c = tid & 15;
 #pragma unroll
-            for (int h = tid >> 4; h <= G; h += kSThreads / 16) {  // 8 rows per sweep of the 128 threads
-                const char* src = (h < G) ? a.q + ((size_t)b * a.q_bs + (size_t)h_kv * G * D) * 2 + (size_t)h * ROW_BYTES
-                                          : a.k + ((size_t)b * a.kv_bs + (size_t)h_kv * D) * 2;
-                const uint4 w = *reinterpret_cast<const uint4*>(src + c * 16);
-                unsigned char* dst = qbuf + buf * kQBufBytes + (c >> 3) * kQHalf + h * 128 + (((c & 7) ^ (h & 7)) * 16);
-                *reinterpret_cast<uint4*>(dst) = w;
+            for (int i = 0; i < kQWords; ++i) {
+                const int h = (tid >> 4) + i * (kSThreads / 16);
+                if (h <= G) {
+                    const char* src = (h < G) ? a.q + ((size_t)b * a.q_bs + (size_t)h_kv * G * D) * 2 + (size_t)h * ROW_BYTES
+                                              : a.k + ((size_t)b * a.kv_bs + (size_t)h_kv * D) * 2;
+                    w[i] = *reinterpret_cast<const uint4*>(src + c * 16);
+                }
+            }
+        };
+        auto store_q = [&](int buf, const uint4* w) {
+            const int c = tid & 15;
+#pragma unroll
+            for (int i = 0; i < kQWords; ++i) {
+                const int h = (tid >> 4) + i * (kSThreads / 16);
+                if (h <= G) {
+                    unsigned char* dst = qbuf + buf * kQBufBytes + (c >> 3) * kQHalf + h * 128 + (((c & 7) ^ (h & 7)) * 16);
+                    *reinterpret_cast<uint4*>(dst) = w[i];
+                }
             }
             fence_proxy_async_smem();
             tc_fence_before();
             mbar_arrive(&qready[buf]);
         };
-        if (cid < a.U) write_q(cid, 0);
+        uint4 qnext[kQWords];
+        if (cid < a.U) {
+            load_q(cid, qnext);
+            store_q(0, qnext);
+        }
 
         int it = 0;
         uint32_t sp = 0;  // sub-slices processed so far (phase of the per-tile barriers)
@@ -367,11 +387,16 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             // step size of this token's write: MV_t = MV_{t-1} + eta_t ww_t^T wv_t
             const float eta_u = (a.eta != nullptr && a.do_write) ? a.eta[(size_t)b * a.eta_bs + h_kv] : 1.f;
             const size_t unit_off = (size_t)u * a.C * ROW_BYTES;
+            if (u + ncl < a.U) load_q(u + ncl, qnext);  // the next unit's operand words: used after this unit's pass 2
+            // this thread's 16 bytes of v_t for the update, asked for now so that they have arrived by then
+            const uint4 vt_raw = a.do_write ? *reinterpret_cast<const uint4*>(a.v + kv_off + (tid & 15) * 16) : make_uint4(0, 0, 0, 0);
 
-            // the appended slot (fill phase) is scored from the step vectors
+            // the appended slot (fill phase) is scored from the step vectors; v_t[d] is also what a read that
+            // follows its own write adds
             float vq[G];
-            const float kd = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(a.k + kv_off)[r]);
-            const float vd = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(a.v + kv_off)[r]);
+            const float kd = has_virtual ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(a.k + kv_off)[r]) : 0.f;
+            const float vd = (has_virtual || (a.wtr && a.do_write))
+                                 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(a.v + kv_off)[r]) : 0.f;
 #pragma unroll
             for (int g = 0; g < G; ++g) {
                 vq[g] = 0.f;
@@ -479,7 +504,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 }
                 if (last_sub) {
                     // the next unit's scores may start as soon as this unit's V tiles are through
-                    if (u + ncl < a.U) write_q(u + ncl, (it + 1) & 1);
+                    if (u + ncl < a.U) store_q((it + 1) & 1, qnext);
                 } else {
                     tc_fence_before();
                     mbar_arrive(subfree);  // this sub-slice's score tiles may be overwritten
@@ -684,7 +709,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             // ---- more rows than lww keeps (diffuse write weights): then it is applied here ----
             if (a.do_write && n_touched > 0) {
                 float vt[8];
-                Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(a.v + kv_off + c16 * 16), vt);
+                Chunk<__nv_bfloat16>::unpack(vt_raw, vt);
 #pragma unroll
                 for (int e = 0; e < 8; ++e) vt[e] *= eta_u;
                 if (n_touched <= kLwwCap) {
