@@ -121,7 +121,7 @@ def algorithmic_bytes_per_step(w: W.Workload) -> int:
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the committed ncu capture of
 # decode_tc_kernel (profiles/decode_tc_kernel_ncu_full.txt), taken at batch 37 and scaled by units:
 # 1.0949 MB per (sequence, kv-head) unit of the mha7b shape.  None for any other kernel / shape.
-TRAFFIC_PER_UNIT = {("mha7b", True): 1.2945e9 / 1184}
+TRAFFIC_PER_UNIT = {("mha7b", True): 1.2942e9 / 1184}
 
 
 def measured_traffic(w, tensor_path):
