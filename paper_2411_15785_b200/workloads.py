@@ -80,6 +80,9 @@ CONFIGS: Dict[str, Workload] = {
                            128 ** -0.5, 1.0),
     "stream_b8_c1024": _w("stream_b8_c1024", 8, 32, 32, 128, 1024, "bf16", 0, 131072, 3,
                           128 ** -0.5, 1.0, api="stream"),
+    # not one of the five named configurations: 64 query heads over 8 kv-heads (G = 8), the 16-row operand form
+    "gqa70b_b64_c2048": _w("gqa70b_b64_c2048", 64, 64, 8, 128, 2048, "bf16", 2048, 256, 5,
+                           128 ** -0.5, 1.0),
 }
 for _C in (256, 1024, 4096, 16384):
     CONFIGS["sweep_b256_c%d" % _C] = _w("sweep_b256_c%d" % _C, 256, 32, 8, 128, _C, "bf16", _C,
