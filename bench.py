@@ -132,7 +132,8 @@ def measured_traffic(w, tensor_path):
 def stream_roofline(w, tok_per_step, ms_step, precise=False, write_only=False):
     """Tensor-core roofline of stream_tc_kernel: the dense flops its MMAs execute per step (operand rows padded
     to M = 128 included) against the measured bf16 matmul peak."""
-    Tc = 64 if w.group == 1 else (32 if w.group <= 3 else 16)
+    Tc = {1: 64, 2: 40, 3: 32, 4: 24}.get(w.group, 16)
+    Tcp = (Tc + 15) // 16 * 16                    # the products run on the chunk padded to 16 tokens
     C, d = w.capacity, w.head_dim
     if write_only:                                 # bct_update_kv: chunks of 128 write rows, no outputs
         Tc = 128
@@ -140,9 +141,9 @@ def stream_roofline(w, tok_per_step, ms_step, precise=False, write_only=False):
     else:
         per_chunk = 2 * (2 * 128 * C * d)          # scores of the 128 operand rows, two passes over MK
         per_chunk += (3 if precise else 1) * (2 * 128 * C * d)   # outputs: P MV_hi (+ P_lo MV_hi + P MV_lo with PRECISE_READ)
-        per_chunk += 2 * 128 * C * Tc              # A = P WW^T
-        per_chunk += 2 * (2 * C * Tc * d)          # MV increment with value + residual weights
-        per_chunk += 2 * 128 * Tc * d              # strict_tril(A) Vc
+        per_chunk += 2 * 128 * C * Tcp             # A = P WW^T
+        per_chunk += 2 * (2 * C * Tcp * d)         # MV increment with value + residual weights
+        per_chunk += 2 * 128 * Tcp * d             # strict_tril(A) Vc
     flops = per_chunk * (tok_per_step // Tc) * w.units
     peak = FALLBACK_BF16_TFLOPS
     kind = "fallback"

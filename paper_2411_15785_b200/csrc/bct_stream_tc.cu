@@ -166,7 +166,8 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     auto chunk_len = [&](int ch) { return a.fill ? a.len0 + ch * a.Tc : a.C; };
     auto chunk_tiles = [&](int ch) { return a.fill ? (a.len0 + ch * a.Tc + kStTile - 1) / kStTile : nt_full; };
     const int n_read = Tc * G;         // rows [0, n_read): read queries (t, g); then Tc write rows
-    const int vc_half = Tc * 128;      // bytes between the two 64-column halves of Vc
+    const int Tcp = (Tc + 15) & ~15;   // the chunk padded to the 16-token step of the products (padding rows are zero)
+    const int vc_half = Tcp * 128;     // bytes between the two 64-column halves of Vc
     // Ring use.  Pass 1 streams the MK tiles round the stages.  In pass 2 stage 0 takes the MK tiles, the
     // last stage the residual tiles of MV, and the stages between them the value tiles of MV: two of
     // them with four stages, so that tile t + 1's values arrive while tile t is rebuilt and stored.
@@ -217,7 +218,8 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         *abort_flag = 0;
         fence_mbar_init_cluster();
     }
-    // rows of the query operand beyond the chunk's G*Tc + Tc stay zero for good
+    // rows of the query operand beyond the chunk's G*Tc + Tc, and rows of Vc beyond Tc, stay zero for good
+    for (int i = tid; i < (L.phi - L.vc) / 16; i += kStThreads) reinterpret_cast<uint4*>(vc)[i] = make_uint4(0, 0, 0, 0);
     for (int i = tid; i < kStTileBytes / 16; i += kStThreads) reinterpret_cast<uint4*>(qall)[i] = make_uint4(0, 0, 0, 0);
     if (warp == kStRowWarps + 1) tmem_alloc(tmem_slot, 512);
     fence_proxy_async_smem();
@@ -366,7 +368,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             constexpr uint32_t id_scores = instr_desc_mn(128, 128, false, false);  // Qall (K) x tile (K)
             constexpr uint32_t id_out = instr_desc_mn(128, 128, false, true);      // P (K) x V tile (MN)
             constexpr uint32_t id_delta = instr_desc_mn(128, 128, true, true);     // WW^T (MN) x Vc (MN)
-            const uint32_t id_a = instr_desc_mn(128, (uint32_t)(Tc < 16 ? 16 : (Tc > kStMaxTc ? kStMaxTc : Tc)), false, false);  // P (K) x WW (K)
+            const uint32_t id_a = instr_desc_mn(128, (uint32_t)(Tcp > kStMaxTc ? kStMaxTc : Tcp), false, false);  // P (K) x WW (K)
             uint32_t qn = 0, su0 = 0, su1 = 0, np = 0, nd = 0;
             uint32_t use[kStMaxStages] = {0, 0, 0, 0};
             const uint32_t plo_row0 = a.precise ? 0u : (uint32_t)n_read;  // first operand row the residual buffer holds
@@ -463,7 +465,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                             continue;
                         }
                         // increment of this tile's MV rows: (WW + WW_residual)^T x Vc, 16 tokens per step
-                        for (int kk = 0; kk < Tc / 16; ++kk) {
+                        for (int kk = 0; kk < Tcp / 16; ++kk) {
                             const uint64_t vd = desc_at(dvc0, vcaddr + kk * 2048);
                             umma_bf16(tmem_base + kColD, desc_at(dmn0, phiaddr + n_read * 128 + kk * 2048), vd,
                                       id_delta, kk > 0);
@@ -487,7 +489,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     // chunk's own slots, value + residual, times Vc)
                     ST_WAIT(aready, qn, 50);
                     tc_fence_after();
-                    for (int kk = 0; kk < (G > 0 ? Tc / 16 : 0); ++kk) {
+                    for (int kk = 0; kk < (G > 0 ? Tcp / 16 : 0); ++kk) {
                         const uint64_t vd = desc_at(dvc0, vcaddr + kk * 2048);
                         umma_bf16(tmem_base + kColO, desc_at(dk0, ploaddr + kk * 32), vd, id_out, (nt > 0) || (kk > 0));
                         if (a.fill && a.precise)
@@ -515,6 +517,8 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         const int poff = (cq >> 1) * kStHalf + r * 128;      // this thread's 64 bytes: chunks (cq & 1) * 4 + j
         const int pch = (cq & 1) * 4;
         const bool active = is_read || (is_write && !a.fill);  // rows that produce numerators
+        // rows whose residual the increment's product reads: the write rows and the zero rows that pad the chunk to 16 tokens
+        const bool lo_row = !is_read && r < n_read + Tcp;
         uint32_t qn = 0, su0 = 0, su1 = 0, np = 0, nd = 0;
         uint32_t use[kStMaxStages] = {0, 0, 0, 0};
         const int lo_off = (cq >> 1) * L.plo_half + (r - (a.precise ? 0 : n_read)) * 128;  // residual buffer: write rows only unless precise
@@ -652,7 +656,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 if (nt > 0) numerators(0);
                 for (int t = 0; t < nt; ++t) {
                     if (np > 0) ST_WAIT(pfree, np - 1, 63);  // the previous tile's MMAs have read the operand buffers
-                    if (is_write || a.precise) {  // write weights always keep the residual
+                    if (lo_row || a.precise) {  // write weights always keep the residual
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {  // 16-byte chunk = 8 slots
                             uint4 hi, lo;
@@ -864,7 +868,15 @@ int stream_chunk_tokens(const bct_cache* c) {
     if (p.flags & BCT_FLAG_CUDA_CORES) return 0;
     if (p.capacity < kStTile || p.capacity > kStMaxCapacity) return 0;
     if (c->plane_bytes < (size_t)1 << 18) return 0;
-    return c->G == 1 ? 64 : (c->G <= 3 ? 32 : 16);
+    // as many tokens as leave the chunk's G*Tc read rows + Tc write rows (padded to 16) within 128 operand rows,
+    // with the read rows a multiple of 8
+    switch (c->G) {
+        case 1: return 64;
+        case 2: return 40;
+        case 3: return 32;
+        case 4: return 24;
+        default: return 16;
+    }
 }
 
 int launch_stream_tc(const bct_cache* c, const void* q, const void* k, const void* v, void* out, int64_t T,
@@ -876,7 +888,7 @@ int launch_stream_tc(const bct_cache* c, const void* q, const void* k, const voi
     const int G = write_only ? 0 : c->G;
     StKernelFn fn = pick_stream(G);
     const int Tc = write_only ? write_only_tc : stream_chunk_tokens(c);
-    if (fn == nullptr || Tc == 0 || stream_chunk_tokens(c) == 0 || T > (int64_t)1 << 30 || Tc % 16 != 0 || Tc > 128 ||
+    if (fn == nullptr || Tc == 0 || stream_chunk_tokens(c) == 0 || T > (int64_t)1 << 30 || Tc % 8 != 0 || Tc > 128 ||
         (write_only && fill_len >= 0)) {
         *err = cudaErrorInvalidConfiguration;
         return -1;
