@@ -136,7 +136,7 @@ bct_status_t run_tokens(bct_cache_t* c, const void* q, const void* k, const void
         if (Tc > 0 && full && do_write && T - t >= Tc) {
             const int64_t n_chunks = (T - t) / Tc;
             cudaError_t e = cudaSuccess;
-            const int n = bct::launch_stream_tc(c, q, k, v, out, T, eta, t, n_chunks, -1, 0, stream, &e);
+            const int n = bct::launch_stream_tc(c, q, k, v, out, T, eta, t, n_chunks, -1, 0, 0, stream, &e);
             if (n < 0) return fail_cuda("stream launch", e);
             c->launches += n;
             c->n_full_tokens += n_chunks * Tc;
@@ -148,12 +148,39 @@ bct_status_t run_tokens(bct_cache_t* c, const void* q, const void* k, const void
             const int64_t by_tokens = (T - t) / Tc, by_slots = (p.capacity - c->len) / Tc;
             const int64_t n_chunks = by_tokens < by_slots ? by_tokens : by_slots;
             cudaError_t e = cudaSuccess;
-            const int n = bct::launch_stream_tc(c, q, k, v, out, T, eta, t, n_chunks, c->len, 0, stream, &e);
+            const int n = bct::launch_stream_tc(c, q, k, v, out, T, eta, t, n_chunks, c->len, 0, 0, stream, &e);
             if (n < 0) return fail_cuda("stream launch (fill)", e);
             c->launches += n;
             c->len += (int)(n_chunks * Tc);
             t += n_chunks * Tc;
             continue;
+        }
+        // the ragged end of the call: with a full cache one shorter chunk (rounded up to 8 tokens; the rows past
+        // the last token are zero-filled, add nothing and store nothing); while the cache fills, a chunk of
+        // exactly the largest multiple of 8 that fits, and single tokens for the rest
+        if (Tc > 0 && full && do_write) {
+            const int64_t r = T - t;  // < Tc here
+            const int tc = (int)((r + 7) / 8 * 8);
+            cudaError_t e = cudaSuccess;
+            const int n = bct::launch_stream_tc(c, q, k, v, out, T, eta, t, 1, -1, 0, tc, stream, &e);
+            if (n < 0) return fail_cuda("stream launch (last chunk)", e);
+            c->launches += n;
+            c->n_full_tokens += r;
+            t += r;
+            continue;
+        }
+        if (Tc > 0 && !full) {
+            const int64_t m = T - t < p.capacity - c->len ? T - t : p.capacity - c->len;  // < Tc here
+            const int tc = (int)(m / 8 * 8);
+            if (tc >= 8) {
+                cudaError_t e = cudaSuccess;
+                const int n = bct::launch_stream_tc(c, q, k, v, out, T, eta, t, 1, c->len, 0, tc, stream, &e);
+                if (n < 0) return fail_cuda("stream launch (fill, last chunk)", e);
+                c->launches += n;
+                c->len += tc;
+                t += tc;
+                continue;
+            }
         }
         bct::StepIO io;
         io.q = static_cast<const char*>(q) + (size_t)t * q_tok * eb;
@@ -341,13 +368,13 @@ bct_status_t bct_update_kv(bct_cache_t* c, const void* wq, const void* wv, const
     const int64_t whole = T / 128, rest = T - whole * 128;
     cudaError_t e = cudaSuccess;
     if (whole > 0) {
-        const int n = bct::launch_stream_tc(c, nullptr, wq, wv, nullptr, T, eta, 0, whole, -1, 128, stream, &e);
+        const int n = bct::launch_stream_tc(c, nullptr, wq, wv, nullptr, T, eta, 0, whole, -1, 1, 128, stream, &e);
         if (n < 0) return fail_cuda("write-only stream launch", e);
         c->launches += n;
     }
     if (rest > 0) {  // one shorter chunk; its rows past the last token read as zeros
         const int tc = (int)((rest + 15) / 16 * 16);
-        const int n = bct::launch_stream_tc(c, nullptr, wq, wv, nullptr, T, eta, whole * 128, 1, -1, tc, stream, &e);
+        const int n = bct::launch_stream_tc(c, nullptr, wq, wv, nullptr, T, eta, whole * 128, 1, -1, 1, tc, stream, &e);
         if (n < 0) return fail_cuda("write-only stream launch", e);
         c->launches += n;
     }

@@ -84,11 +84,12 @@ int stream_chunk_tokens(const bct_cache* c);
 // n_chunks whole chunks starting at token t_begin of the [B][T][H][d] step arrays.  fill_len < 0:
 // the cache is full and every token is a read plus a soft write; fill_len >= 0: the cache holds
 // fill_len slots, each chunk is appended (fill_len + n_chunks * Tc <= capacity) and read causally.
-// eta: step size of each token's write, [B][T][Hkv] floats, or NULL.  write_only_tc > 0: the form without
-// read queries and outputs (q and out unused), in chunks of write_only_tc tokens (a multiple of 16, at most
-// 128; tokens past T in the last chunk are zero-filled), full cache only.
+// eta: step size of each token's write, [B][T][Hkv] floats, or NULL.  write_only: the form without read
+// queries and outputs (q and out unused; chunks of up to 128 tokens), full cache only.  tc_tokens: tokens per
+// chunk, a multiple of 8 (16 for the write-only form) up to the cache's default, or 0 for that default; with a
+// full cache the tokens of the last chunk that lie past T are zero-filled and store nothing.
 int launch_stream_tc(const bct_cache* c, const void* q, const void* k, const void* v, void* out, int64_t T,
-                     const float* eta, int64_t t_begin, int64_t n_chunks, int fill_len, int write_only_tc,
+                     const float* eta, int64_t t_begin, int64_t n_chunks, int fill_len, int write_only, int tc_tokens,
                      cudaStream_t stream, cudaError_t* err);
 
 // The projections in front of the layer (bct_project.cu): q = x W_q^T, k = x W_wq^T, v = x W_wv^T for

@@ -786,7 +786,8 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     const size_t orow = (((size_t)b * a.T + t0 + my_t) * a.Hq + (size_t)h * G + my_g) * 128 + cq * 32;
                     float o[32];
                     tmem_ld32(lane_base + kColO, o);
-                    if (is_read && a.out != nullptr && !*abort_flag) {
+                    // (a ragged last chunk has rows past the last token: nothing is stored for them)
+                    if (is_read && a.out != nullptr && t0 + my_t < a.T && !*abort_flag) {
 #pragma unroll
                         for (int i = 0; i < 32; ++i) o[i] *= inv_l;
                         if (a.out_f32) {
@@ -880,16 +881,17 @@ int stream_chunk_tokens(const bct_cache* c) {
 }
 
 int launch_stream_tc(const bct_cache* c, const void* q, const void* k, const void* v, void* out, int64_t T,
-                     const float* eta, int64_t t_begin, int64_t n_chunks, int fill_len, int write_only_tc,
+                     const float* eta, int64_t t_begin, int64_t n_chunks, int fill_len, int write_only, int tc_tokens,
                      cudaStream_t stream, cudaError_t* err) {
     const bct_params_t& p = c->p;
-    // write_only_tc > 0: the form without read queries (Algorithm 1's UpdateKV), chunks of that many tokens
-    const bool write_only = write_only_tc > 0;
+    // write_only: the form without read queries (Algorithm 1's UpdateKV); tc_tokens: tokens per chunk
+    // (0: the cache's default; a shorter chunk serves the ragged end of a call)
     const int G = write_only ? 0 : c->G;
     StKernelFn fn = pick_stream(G);
-    const int Tc = write_only ? write_only_tc : stream_chunk_tokens(c);
-    if (fn == nullptr || Tc == 0 || stream_chunk_tokens(c) == 0 || T > (int64_t)1 << 30 || Tc % 8 != 0 || Tc > 128 ||
-        (write_only && fill_len >= 0)) {
+    const int Tc_max = write_only ? 128 : stream_chunk_tokens(c);
+    const int Tc = tc_tokens > 0 ? tc_tokens : Tc_max;
+    if (fn == nullptr || Tc_max == 0 || stream_chunk_tokens(c) == 0 || T > (int64_t)1 << 30 || Tc % 8 != 0 || Tc > Tc_max ||
+        (write_only && fill_len >= 0) || (write_only && Tc % 16 != 0)) {
         *err = cudaErrorInvalidConfiguration;
         return -1;
     }
