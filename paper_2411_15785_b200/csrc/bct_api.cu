@@ -158,7 +158,8 @@ bct_status_t run_tokens(bct_cache_t* c, const void* q, const void* k, const void
         // the ragged end of the call: with a full cache one shorter chunk (rounded up to 8 tokens; the rows past
         // the last token are zero-filled, add nothing and store nothing); while the cache fills, a chunk of
         // exactly the largest multiple of 8 that fits, and single tokens for the rest
-        if (Tc > 0 && full && do_write) {
+        // (a chunk streams the unit's planes about three times as often as a decode step does: not below 4 tokens)
+        if (Tc > 0 && full && do_write && T - t >= 4) {
             const int64_t r = T - t;  // < Tc here
             const int tc = (int)((r + 7) / 8 * 8);
             cudaError_t e = cudaSuccess;

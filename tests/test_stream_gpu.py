@@ -138,6 +138,7 @@ def test_fill_phase_chunks_equal_single_tokens_in_the_cache():
 @pytest.mark.parametrize("G,C,init_len,T,max_launches", [
     (1, 256, 256, 100, 2),       # one chunk of 64, one of 40 tokens of which 36 exist
     (1, 512, 512, 5, 1),         # fewer tokens than the smallest chunk: 8 rows, 5 of them real
+    (1, 512, 512, 3, 3),         # below 4 tokens the decode kernel is the cheaper one
     (4, 384, 384, 61, 3),        # chunks of 24: two whole ones and 13 tokens in a chunk of 16
     (2, 300, 130, 250, 12),      # fill: 4 chunks of 40, one of 8, 2 single tokens; then 40 + 40 of the full phase
     (1, 256, 251, 30, 7),        # 5 free slots: single tokens, then one ragged chunk of the full phase
