@@ -263,15 +263,17 @@ def run_project(args, w):
             for _ in range(2)]
     xs = [torch.randn((M, K), generator=g, device=dev).to(torch.bfloat16) for _ in range(4)]
     warm = max(args.warmup, 3)
+    outs = (torch.empty((M, n_q), dtype=torch.bfloat16, device=dev), torch.empty((M, n_kv), dtype=torch.bfloat16, device=dev),
+            torch.empty((M, n_kv), dtype=torch.bfloat16, device=dev))
     for i in range(warm):
-        B.project_qkv(xs[i % 4], *sets[i & 1])
+        B.project_qkv(xs[i % 4], *sets[i & 1], out=outs)
     torch.cuda.synchronize()
     sampler = ClockSampler(dev.index)
     sampler.start()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for i in range(args.steps):
-        B.project_qkv(xs[i % 4], *sets[i & 1])
+        B.project_qkv(xs[i % 4], *sets[i & 1], out=outs)
     e1.record()
     torch.cuda.synchronize()
     clocks = sampler.stop()

@@ -132,7 +132,7 @@ def _ptr(t: Optional[torch.Tensor]):
     return None if t is None else t.data_ptr()
 
 
-def project_qkv(x, w_q, w_wq, w_wv, stream=None):
+def project_qkv(x, w_q, w_wq, w_wv, stream=None, out=None):
     """q = x W_q^T, k = x W_wq^T, v = x W_wv^T: x ``[..., d_model]`` bfloat16 on the device, weights
     ``[features, d_model]``; returns q ``[..., n_q]``, k, v ``[..., n_kv]`` (bfloat16)."""
     lib = load()
@@ -142,9 +142,12 @@ def project_qkv(x, w_q, w_wq, w_wv, stream=None):
         if t.dtype != torch.bfloat16 or not t.is_cuda or not t.is_contiguous():
             raise ValueError("x and the weights must be contiguous bfloat16 device tensors")
     n_q, n_kv = w_q.shape[0], w_wq.shape[0]
-    q = torch.empty(x.shape[:-1] + (n_q,), dtype=torch.bfloat16, device=x.device)
-    k = torch.empty(x.shape[:-1] + (n_kv,), dtype=torch.bfloat16, device=x.device)
-    v = torch.empty_like(k)
+    if out is not None:   # (q, k, v) tensors to write into
+        q, k, v = out
+    else:
+        q = torch.empty(x.shape[:-1] + (n_q,), dtype=torch.bfloat16, device=x.device)
+        k = torch.empty(x.shape[:-1] + (n_kv,), dtype=torch.bfloat16, device=x.device)
+        v = torch.empty_like(k)
     _check(lib.bct_project_qkv(n_tokens, d_model, n_q, n_kv, x.data_ptr(), w_q.data_ptr(), w_wq.data_ptr(),
                                w_wv.data_ptr(), q.data_ptr(), k.data_ptr(), v.data_ptr(), _stream_ptr(stream)))
     return q, k, v

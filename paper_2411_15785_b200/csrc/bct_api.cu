@@ -3,6 +3,8 @@
 // memory is allocated here; everything lives in the caller's workspace.
 #include <cuda_runtime.h>
 
+#include <mutex>
+
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
@@ -408,14 +410,30 @@ bct_status_t check_project_args(int64_t n_tokens, int32_t d_model, int32_t n_q, 
 }
 
 // SM count and opt-in shared memory of the current device, which must offer the sm_100 tensor path.
-bct_status_t tensor_device(int* sm_count, int* smem_optin) {
-    int dev = 0, major = 0;
+// Looked up once per device: the projection of a decode step takes tens of microseconds, and four
+// attribute queries per call were a visible part of it.
+bct_status_t tensor_device(int* device, int* sm_count, int* smem_optin) {
+    constexpr int kMaxDev = 64;
+    static std::mutex mu;
+    static int known[kMaxDev] = {}, sms[kMaxDev] = {}, optin[kMaxDev] = {}, majors[kMaxDev] = {};
+    int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
-    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
-    if (e == cudaSuccess) e = cudaDeviceGetAttribute(sm_count, cudaDevAttrMultiProcessorCount, dev);
-    if (e == cudaSuccess) e = cudaDeviceGetAttribute(smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
     if (e != cudaSuccess) return fail_cuda("device query", e);
-    if (major != 10) return fail(BCT_ERR_UNSUPPORTED, "the projections need an sm_100 device");
+    if (dev < 0 || dev >= kMaxDev) return fail(BCT_ERR_UNSUPPORTED, "device index %d out of range", dev);
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        if (!known[dev]) {
+            e = cudaDeviceGetAttribute(&majors[dev], cudaDevAttrComputeCapabilityMajor, dev);
+            if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms[dev], cudaDevAttrMultiProcessorCount, dev);
+            if (e == cudaSuccess) e = cudaDeviceGetAttribute(&optin[dev], cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+            if (e != cudaSuccess) return fail_cuda("device query", e);
+            known[dev] = 1;
+        }
+        *device = dev;
+        *sm_count = sms[dev];
+        *smem_optin = optin[dev];
+        if (majors[dev] != 10) return fail(BCT_ERR_UNSUPPORTED, "the projections need an sm_100 device");
+    }
     return BCT_OK;
 }
 
@@ -428,10 +446,10 @@ bct_status_t bct_project_qkv(int64_t n_tokens, int32_t d_model, int32_t n_q, int
                              void* cuda_stream) {
     bct_status_t st = check_project_args(n_tokens, d_model, n_q, n_kv, x, w_q, w_wq, w_wv, q, k, v);
     if (st != BCT_OK) return st;
-    int sm_count = 0, smem_optin = 0;
-    st = tensor_device(&sm_count, &smem_optin);
+    int device = 0, sm_count = 0, smem_optin = 0;
+    st = tensor_device(&device, &sm_count, &smem_optin);
     if (st != BCT_OK) return st;
-    cudaError_t e = bct::launch_project(n_tokens, d_model, n_q, n_kv, x, w_q, w_wq, w_wv, q, k, v, nullptr, sm_count,
+    cudaError_t e = bct::launch_project(n_tokens, d_model, n_q, n_kv, x, w_q, w_wq, w_wv, q, k, v, nullptr, device, sm_count,
                                         smem_optin, static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) return fail_cuda("projection launch", e);
     return BCT_OK;
@@ -475,7 +493,7 @@ bct_status_t bct_layer_forward(bct_cache_t* c, const void* x, const void* w_q, c
     if (!c->tc_ready) return fail(BCT_ERR_UNSUPPORTED, "the projections need the driver's tensor-map encoder");
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     cudaError_t e = bct::launch_project(n_tokens, d_model, n_q, n_kv, x, w_q, w_wq, w_wv, q, k, v, c->status,
-                                        c->sm_count, c->smem_optin, stream);
+                                        c->device, c->sm_count, c->smem_optin, stream);
     if (e != cudaSuccess) return fail_cuda("projection launch", e);
     c->launches += 1;
     return run_tokens(c, q, k, v, eta, out, T, stream);

@@ -95,8 +95,8 @@ int launch_stream_tc(const bct_cache* c, const void* q, const void* k, const voi
 // The projections in front of the layer (bct_project.cu): q = x W_q^T, k = x W_wq^T, v = x W_wv^T for
 // n_tokens rows of x, bfloat16 throughout; status may be NULL.
 cudaError_t launch_project(long long n_tokens, int d_model, int n_q, int n_kv, const void* x, const void* w_q,
-                           const void* w_wq, const void* w_wv, void* q, void* k, void* v, int* status, int sm_count,
-                           int smem_optin, cudaStream_t stream);
+                           const void* w_wq, const void* w_wv, void* q, void* k, void* v, int* status, int device,
+                           int sm_count, int smem_optin, cudaStream_t stream);
 
 // Set the calling thread's bct_last_error() message (for entry points outside bct_api.cu).
 void set_last_error(const char* msg);

@@ -255,7 +255,7 @@ bool make_matrix_map(CUtensorMap* map, const void* base, long long rows, int K, 
 
 template <int BN, int KPER>
 cudaError_t launch_bn(const CUtensorMap& mx, const CUtensorMap& m0, const CUtensorMap& m1, const CUtensorMap& m2,
-                      PjArgs a, int sm_count, int smem_optin, cudaStream_t stream) {
+                      PjArgs a, int device, int sm_count, int smem_optin, cudaStream_t stream) {
     const int kStage = KPER * (a.a_bytes + BN * kPjBK * 2);
     const int pad = kPjABytes - a.a_bytes;  // the 128-row operand read of the last stage stays inside the allocation
     int stages = (smem_optin - 2048 - pad) / kStage;
@@ -264,8 +264,14 @@ cudaError_t launch_bn(const CUtensorMap& mx, const CUtensorMap& m0, const CUtens
     a.stages = stages;
     const int smem = stages * kStage + pad + (2 * kPjMaxStages + 8) * 8 + 1024;
     auto fn = project_kernel<BN, KPER>;
-    cudaError_t e = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e != cudaSuccess) return e;
+    // the shared-memory limit of this kernel on this device is raised only when it has to grow (a decode
+    // step's projection is short enough for one more runtime call per launch to show)
+    static int smem_set[64] = {};
+    if (device < 0 || device >= 64 || smem_set[device] < smem) {
+        cudaError_t e = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        if (device >= 0 && device < 64) smem_set[device] = smem;
+    }
     const long long m_tiles = (a.M + kPjBM - 1) / kPjBM;
     const long long tiles = m_tiles * ((a.n_seg[0] + a.n_seg[1] + a.n_seg[2]) / BN);
     const int grid = (int)(tiles < sm_count ? tiles : sm_count);
@@ -277,8 +283,8 @@ cudaError_t launch_bn(const CUtensorMap& mx, const CUtensorMap& m0, const CUtens
 
 // q = x W_q^T, k = x W_wq^T, v = x W_wv^T for n_tokens rows of x.  Returns the CUDA error of the launch.
 cudaError_t launch_project(long long n_tokens, int d_model, int n_q, int n_kv, const void* x, const void* w_q,
-                           const void* w_wq, const void* w_wv, void* q, void* k, void* v, int* status, int sm_count,
-                           int smem_optin, cudaStream_t stream) {
+                           const void* w_wq, const void* w_wv, void* q, void* k, void* v, int* status, int device,
+                           int sm_count, int smem_optin, cudaStream_t stream) {
     // feature tiles: 256 wide for long blocks of tokens (fewest operand bytes per product), 128 for
     // shorter ones, 64 (else 32) for a decode step (more tiles than SMs while the weights stream once)
     int BN = 32;
@@ -289,7 +295,9 @@ cudaError_t launch_project(long long n_tokens, int d_model, int n_q, int n_kv, c
     if (n_q % 128 == 0 && n_kv % 128 == 0 && (n_tokens > 256 || m_tiles * ((n_q + 2 * n_kv) / 128) * 8 >= 5LL * sm_count))
         BN = 128;
     if (n_tokens >= 1024 && n_q % 256 == 0 && n_kv % 256 == 0) BN = 256;
-    if (const char* e = getenv("BCT_PJ_BN")) {  // tuning knob: width of the feature tiles
+    static const char* env_bn = getenv("BCT_PJ_BN");      // tuning knobs, read once
+    static const char* env_kper = getenv("BCT_PJ_KPER");
+    if (const char* e = env_bn) {  // width of the feature tiles
         const int v = atoi(e);
         if ((v == 32 || v == 64 || v == 128 || v == 256) && n_q % v == 0 && n_kv % v == 0) BN = v;
     }
@@ -316,12 +324,12 @@ cudaError_t launch_project(long long n_tokens, int d_model, int n_q, int n_kv, c
     // 57.6 / 43.1 / 34.8 us with 1 / 2 / 4 blocks per stage; 128-wide: 33.0 / 28.1 us with 1 / 2).
     const int block = a.a_bytes + BN * kPjBK * 2;
     int kper = 12 * block <= 200 * 1024 ? 4 : (6 * block <= 200 * 1024 ? 2 : 1);
-    if (const char* e = getenv("BCT_PJ_KPER")) {  // tuning knob: 64-column blocks per stage (1, 2, 4)
+    if (const char* e = env_kper) {  // 64-column blocks per stage (1, 2, 4)
         const int v = atoi(e);
         if (v == 1 || v == 2 || v == 4) kper = v;
     }
 #define PJ_LAUNCH(bn, kp) \
-    if (BN == bn && kper == kp) return launch_bn<bn, kp>(mx, m0, m1, m2, a, sm_count, smem_optin, stream);
+    if (BN == bn && kper == kp) return launch_bn<bn, kp>(mx, m0, m1, m2, a, device, sm_count, smem_optin, stream);
     PJ_LAUNCH(256, 1)
     PJ_LAUNCH(256, 2)
     PJ_LAUNCH(128, 1)
