@@ -918,7 +918,8 @@ int launch_decode_tc(const bct_cache* c, const StepIO& io, int len, int do_write
     // (A deeper ring for short slices was measured: no gain, the softmax chain of a unit is the limit.)
     int lo_cap = 80;
     int stages = 4;
-    if (const char* e = getenv("BCT_TC_STAGES")) {  // tuning knob: depth of the tile ring (2..8)
+    static const char* env_stages = getenv("BCT_TC_STAGES");  // read once
+    if (const char* e = env_stages) {  // tuning knob: depth of the tile ring (2..8)
         const int v = atoi(e);
         if (v >= 2 && v <= 8) stages = v;
     }
@@ -963,8 +964,19 @@ int launch_decode_tc(const bct_cache* c, const StepIO& io, int len, int do_write
     a.write_scale = p.write_scale;
     a.write_eps = p.write_eps;
 
-    *err = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (*err != cudaSuccess) return -1;
+    // Per (device, group size): the shared-memory limit already set for the kernel, and the last cluster
+    // occupancy answer.  Both are runtime calls that a step of tens of microseconds would notice.
+    struct Seen {
+        int smem_set, occ_S, occ_smem, occ_active;
+    };
+    static Seen seen[64][16] = {};
+    Seen local = {};
+    Seen& sn = (c->device >= 0 && c->device < 64) ? seen[c->device][c->G] : local;
+    if (sn.smem_set < smem) {
+        *err = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (*err != cudaSuccess) return -1;
+        sn.smem_set = smem;
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.blockDim = dim3(kTcThreads, 1, 1);
     cfg.dynamicSmemBytes = (size_t)smem;
@@ -980,8 +992,15 @@ int launch_decode_tc(const bct_cache* c, const StepIO& io, int len, int do_write
     if (S > 1) {
         cfg.gridDim = dim3((unsigned)(S * (c->sm_count / S)), 1, 1);
         int active = 0;
-        *err = cudaOccupancyMaxActiveClusters(&active, reinterpret_cast<const void*>(fn), &cfg);
-        if (*err != cudaSuccess) return -1;
+        if (sn.occ_S == S && sn.occ_smem == smem) {
+            active = sn.occ_active;
+        } else {
+            *err = cudaOccupancyMaxActiveClusters(&active, reinterpret_cast<const void*>(fn), &cfg);
+            if (*err != cudaSuccess) return -1;
+            sn.occ_S = S;
+            sn.occ_smem = smem;
+            sn.occ_active = active;
+        }
         if (active < 1) {
             *err = cudaErrorInvalidConfiguration;
             return -1;
