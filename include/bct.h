@@ -148,7 +148,8 @@ bct_status_t bct_decode_step(bct_cache_t *cache, const void *q, const void *k, c
  *   q    DEVICE [B][T][Hq][d]
  *   k,v  DEVICE [B][T][Hkv][d]
  *   out  DEVICE [B][T][Hq][d] or NULL
- * May be called repeatedly; successive calls concatenate.  T >= 1.
+ * May be called repeatedly; successive calls concatenate.  T >= 1.  With out == NULL and a full cache
+ * the call takes the write-only route of bct_update_kv (q is then not read).
  */
 bct_status_t bct_prefill_stream(bct_cache_t *cache, const void *q, const void *k, const void *v,
                                 void *out, int64_t T, void *cuda_stream);

@@ -122,6 +122,27 @@ void release_host_objects(bct_cache_t* c) {
 }
 
 // T tokens, one decode launch each.  Pointers are device pointers in [B][T][H][d].
+// Tokens [t, T) of the call into a full cache with nothing read: the write-only chunks of the stream
+// kernel (128 tokens, then one shorter chunk rounded up to 16 whose rows past T are zero-filled).
+bct_status_t write_only_tokens(bct_cache_t* c, const void* k, const void* v, const float* eta, int64_t T, int64_t t,
+                               cudaStream_t stream) {
+    const int64_t whole = (T - t) / 128, rest = (T - t) - whole * 128;
+    cudaError_t e = cudaSuccess;
+    if (whole > 0) {
+        const int n = bct::launch_stream_tc(c, nullptr, k, v, nullptr, T, eta, t, whole, -1, 1, 128, stream, &e);
+        if (n < 0) return fail_cuda("write-only stream launch", e);
+        c->launches += n;
+    }
+    if (rest > 0) {
+        const int tc = (int)((rest + 15) / 16 * 16);
+        const int n = bct::launch_stream_tc(c, nullptr, k, v, nullptr, T, eta, t + whole * 128, 1, -1, 1, tc, stream, &e);
+        if (n < 0) return fail_cuda("write-only stream launch", e);
+        c->launches += n;
+    }
+    c->n_full_tokens += T - t;
+    return BCT_OK;
+}
+
 // eta: [B][T][Hkv] floats on the device, or NULL.
 bct_status_t run_tokens(bct_cache_t* c, const void* q, const void* k, const void* v, const float* eta, void* out,
                         int64_t T, cudaStream_t stream) {
@@ -134,6 +155,8 @@ bct_status_t run_tokens(bct_cache_t* c, const void* q, const void* k, const void
     while (t < T) {
         const bool full = (c->len == p.capacity);
         const int do_write = !((p.flags & BCT_FLAG_SKIP_FIRST_WRITE) && c->n_full_tokens == 0);
+        // no output asked for (UpdateKV): the rest of the call goes through the write-only chunks
+        if (out == nullptr && Tc > 0 && full && do_write && T - t >= 4) return write_only_tokens(c, k, v, eta, T, t, stream);
         // whole chunks against a full cache go through the chunked tensor-core kernel
         if (Tc > 0 && full && do_write && T - t >= Tc) {
             const int64_t n_chunks = (T - t) / Tc;
@@ -367,22 +390,7 @@ bct_status_t bct_update_kv(bct_cache_t* c, const void* wq, const void* wv, const
         return fail(BCT_ERR_UNSUPPORTED,
                     "the write-only form serves bfloat16 caches with head_dim 128 and 128..16384 slots, without "
                     "SKIP_FIRST_WRITE; use bct_prefill_stream with out = NULL");
-    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    const int64_t whole = T / 128, rest = T - whole * 128;
-    cudaError_t e = cudaSuccess;
-    if (whole > 0) {
-        const int n = bct::launch_stream_tc(c, nullptr, wq, wv, nullptr, T, eta, 0, whole, -1, 1, 128, stream, &e);
-        if (n < 0) return fail_cuda("write-only stream launch", e);
-        c->launches += n;
-    }
-    if (rest > 0) {  // one shorter chunk; its rows past the last token read as zeros
-        const int tc = (int)((rest + 15) / 16 * 16);
-        const int n = bct::launch_stream_tc(c, nullptr, wq, wv, nullptr, T, eta, whole * 128, 1, -1, 1, tc, stream, &e);
-        if (n < 0) return fail_cuda("write-only stream launch", e);
-        c->launches += n;
-    }
-    c->n_full_tokens += T;
-    return BCT_OK;
+    return write_only_tokens(c, wq, wv, eta, T, 0, static_cast<cudaStream_t>(cuda_stream));
 }
 
 bct_status_t bct_decode_step_eta(bct_cache_t* c, const void* q, const void* k, const void* v, const float* eta,
