@@ -246,6 +246,36 @@ def run_reference(args, w):
     print(json.dumps(line))
 
 
+def secondary_regime(B, w, wr, dev, pool, outs, peak, steps=200):
+    """The diffuse write regime (write_scale = 1/sqrt(d): every row of the value memory is rewritten each
+    token) on a second cache of the same shape: ms per step and the bytes it must move, five planes
+    (K and MV value read, MV residual read, MV value and residual written), against the copy peak."""
+    ws = w.head_dim ** -0.5
+    mk, mv = W.initial_cache(wr, dev)
+    cache = B.Cache(w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.capacity, w.torch_dtype, read_scale=w.read_scale,
+                    write_scale=ws, init_len=w.init_len, mk_init=mk, mv_init=mv, device=dev)
+    del mk, mv
+    for i in range(5):
+        cache.decode_step(*pool[i % len(pool)], out=outs[i & 1])
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(steps):
+        cache.decode_step(*pool[i % len(pool)], out=outs[i & 1])
+    e1.record()
+    torch.cuda.synchronize()
+    cache.check_status()
+    ms = e0.elapsed_time(e1) / steps
+    eb = 4 if w.dtype == "f32" else 2
+    planes = 3 if w.dtype == "f32" else 5
+    nbytes = planes * w.units * w.capacity * w.head_dim * eb
+    ach = nbytes / (ms * 1e-3) / 1e9
+    cache.destroy()
+    return {"write_scale": ws, "steps": steps, "ms_per_step": ms, "value": w.batch / (ms * 1e-3), "unit": UNIT,
+            "bytes_per_step": nbytes, "achieved": ach, "peak": peak, "frac": ach / peak,
+            "note": "every row rewritten: K, MV value and residual read, MV value and residual written"}
+
+
 def run_project(args, w):
     """Times bct_project_qkv alone (the projections in front of the layer) for --project-tokens rows of
     x with the workload's head counts: one step = one launch.  Two weight sets are used alternately so
@@ -322,6 +352,7 @@ def main():
     ap.add_argument("--flags", type=int, default=0, help="BCT_FLAG_* bits for the cache")
     ap.add_argument("--batch", type=int, default=None, help="override the batch (profiling on a smaller case)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-secondary", action="store_true", help="skip the short run of the diffuse write regime")
     ap.add_argument("--update-kv", action="store_true",
                     help="stream workloads: time bct_update_kv (Algorithm 1's UpdateKV, state only) instead of bct_prefill_stream")
     ap.add_argument("--project-tokens", type=int, default=0,
@@ -478,6 +509,8 @@ def main():
             "gpu_launches": launches,
             "roofline": roof,
         }
+        if world == 1 and not stream and args.write_scale is None and not args.no_secondary:
+            line["secondary_write_regime"] = secondary_regime(B, w, wr, dev, pool, outs, peak)
         if world == 1 and not args.no_cpu_baseline:
             cb = cpu_oracle_sample(w)
             line["cpu_baseline"] = {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")}

@@ -35,6 +35,8 @@ def test_default_workload_line_has_the_contract_keys():
     r = d["roofline"]
     assert r["bound"] == "hbm" and r["unit"] == "GB/s" and r["kernel"] == "decode_tc_kernel"
     assert abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9 and r["traffic"] > 0
+    sec = d["secondary_write_regime"]               # the diffuse write regime, timed on a second cache
+    assert sec["ms_per_step"] > d["ms_per_step"] and 0 < sec["frac"] < 1.2 and abs(sec["write_scale"] - 128 ** -0.5) < 1e-9
 
 
 def test_stream_workload_line_reports_the_tensor_roofline():
