@@ -12,8 +12,8 @@
  *   MV  [C][d]                key-value vector sequence; the state the rule rewrites
  *   wq_t (here k_t)           write query of token t
  *   wv_t (here v_t)           write key-value vector of token t
- *   score_t = wq_t . MK^T     (Algorithm 1, "Calculate similarity scores")
- *   ww_t    = softmax(score_t) (Algorithm 1, "Normalize scores to weights")
+ *   score_t = wq_t . MK^T     (Algorithm 1, the score statement)
+ *   ww_t    = softmax(score_t) (Algorithm 1, the softmax statement)
  *   MV_t    = MV_{t-1} + ww_t^T . wv_t   (Method step 4; Illustration step 3)
  *
  * The paper does not print the read path; the layer is an attention layer
@@ -33,6 +33,10 @@
  *     increment, MV_t = MV_{t-1} + eta_t * ww_t^T . wv_t.  eta_t = 1 is Method
  *     step 4 as printed.  How eta_t is produced is upstream of this layer: it is
  *     an input.  The fill phase has no soft write and ignores it.
+ *   - write threshold (not in the paper; a reading of the library under test): with
+ *     write_eps > 0 a slot whose write weight ww_j is below write_eps keeps its row,
+ *     i.e. its increment eta_t * ww_j * wv_t is dropped.  write_eps = 0 is the printed
+ *     rule, every slot updated.  The weights themselves stay normalised over all slots.
  *   - fill phase (not in the paper, whose MV_0 is full-size): while len < C the
  *     token's (k_t, v_t) is appended at slot len, the read then covers the
  *     len+1 resident slots (so the token sees itself), and no soft write happens.
@@ -77,18 +81,22 @@ static void read_head(const double *q, const double *MK, const double *MV, int64
         for (int e = 0; e < d; ++e) o[e] += p[j] * MV[j * d + e];
 }
 
-/* Write path: score = write_scale * wq . MK^T; ww = softmax(score); MV += eta * ww^T . wv.
+/* Write path: score = write_scale * wq . MK^T; ww = softmax(score); MV += eta * ww^T . wv
+ * on the slots with ww_j >= write_eps (all of them when write_eps = 0).
  * ww (length C) is left in `ww` for the caller. */
 static void write_update(const double *wq, const double *wv, const double *MK, double *MV,
-                         int64_t C, int d, double write_scale, double eta, double *s, double *ww) {
+                         int64_t C, int d, double write_scale, double eta, double write_eps,
+                         double *s, double *ww) {
     for (int64_t j = 0; j < C; ++j) {
         double dot = 0.0;
         for (int e = 0; e < d; ++e) dot += wq[e] * MK[j * d + e];
         s[j] = write_scale * dot;
     }
     softmax(s, C, ww);
-    for (int64_t j = 0; j < C; ++j)
+    for (int64_t j = 0; j < C; ++j) {
+        if (ww[j] < write_eps) continue;
         for (int e = 0; e < d; ++e) MV[j * d + e] += eta * (ww[j] * wv[e]);
+    }
 }
 
 /*
@@ -99,8 +107,8 @@ static void write_update(const double *wq, const double *wv, const double *MK, d
  */
 static int64_t unit_token(int G, int d, int64_t C, int64_t len, double *MK, double *MV,
                           const double *q, const double *k, const double *v, double *out,
-                          double read_scale, double write_scale, double eta, unsigned flags,
-                          int do_write, double *s, double *p) {
+                          double read_scale, double write_scale, double eta, double write_eps,
+                          unsigned flags, int do_write, double *s, double *p) {
     if (len < C) { /* fill phase: append, then read over len+1 slots, no soft write */
         memcpy(MK + len * d, k, sizeof(double) * (size_t)d);
         memcpy(MV + len * d, v, sizeof(double) * (size_t)d);
@@ -111,12 +119,12 @@ static int64_t unit_token(int G, int d, int64_t C, int64_t len, double *MK, doub
         return len;
     }
     if ((flags & BCT_ORACLE_WRITE_THEN_READ) && do_write)
-        write_update(k, v, MK, MV, C, d, write_scale, eta, s, p);
+        write_update(k, v, MK, MV, C, d, write_scale, eta, write_eps, s, p);
     if (out)
         for (int g = 0; g < G; ++g)
             read_head(q + (int64_t)g * d, MK, MV, C, d, read_scale, s, p, out + (int64_t)g * d);
     if (!(flags & BCT_ORACLE_WRITE_THEN_READ) && do_write)
-        write_update(k, v, MK, MV, C, d, write_scale, eta, s, p);
+        write_update(k, v, MK, MV, C, d, write_scale, eta, write_eps, s, p);
     return len;
 }
 
@@ -132,13 +140,15 @@ static int64_t unit_token(int G, int d, int64_t C, int64_t len, double *MK, doub
  * len_io        resident slots, the same for every unit (in/out)
  * n_written_io  soft writes applied so far per unit history (in/out); only its
  *               being zero matters (BCT_ORACLE_SKIP_FIRST_WRITE)
+ * write_eps     slots whose write weight is below it are not rewritten (0: the printed rule)
  * nthreads      OpenMP threads over units (<= 0: library default)
  * Returns the number of threads used, or -1 on bad arguments / allocation failure.
  */
-int bct_oracle_stream_eta(int64_t U, int64_t T, int G, int d, int64_t C, int64_t *len_io,
+int bct_oracle_stream_eps(int64_t U, int64_t T, int G, int d, int64_t C, int64_t *len_io,
                           int64_t *n_written_io, double *MK, double *MV, const double *q,
                           const double *k, const double *v, const double *eta, double *out,
-                          double read_scale, double write_scale, unsigned flags, int nthreads) {
+                          double read_scale, double write_scale, double write_eps, unsigned flags,
+                          int nthreads) {
     if (U < 0 || T < 0 || G < 1 || d < 1 || C < 1 || !len_io || !n_written_io) return -1;
     if (*len_io < 0 || *len_io > C) return -1;
     int used = 1;
@@ -169,7 +179,7 @@ int bct_oracle_stream_eta(int64_t U, int64_t T, int G, int d, int64_t C, int64_t
                 int full = (len == C);
                 int do_write = !((flags & BCT_ORACLE_SKIP_FIRST_WRITE) && nw == 0);
                 len = unit_token(G, d, C, len, mk, mv, qt, kt, vt, ot, read_scale, write_scale,
-                                 eta ? eta[u * T + t] : 1.0, flags, do_write, s, p);
+                                 eta ? eta[u * T + t] : 1.0, write_eps, flags, do_write, s, p);
                 if (full) nw += 1; /* counts full-phase tokens seen, written or skipped */
             }
         }
@@ -185,6 +195,15 @@ int bct_oracle_stream_eta(int64_t U, int64_t T, int G, int d, int64_t C, int64_t
     *len_io = len;
     *n_written_io = nw;
     return used;
+}
+
+/* The same without a write threshold: every slot is updated. */
+int bct_oracle_stream_eta(int64_t U, int64_t T, int G, int d, int64_t C, int64_t *len_io,
+                          int64_t *n_written_io, double *MK, double *MV, const double *q,
+                          const double *k, const double *v, const double *eta, double *out,
+                          double read_scale, double write_scale, unsigned flags, int nthreads) {
+    return bct_oracle_stream_eps(U, T, G, d, C, len_io, n_written_io, MK, MV, q, k, v, eta, out,
+                                 read_scale, write_scale, 0.0, flags, nthreads);
 }
 
 /* The same with every step size equal to one: Method step 4 as printed. */
@@ -230,9 +249,9 @@ int bct_oracle_read_weights(int64_t n, int d, const double *MK, const double *q,
 }
 
 /*
- * The projections in front of the layer (Algorithm 1, "Compute write query" and "Compute
- * write key-value vector": wq_t = W_wq x_t, wv_t = W_wv x_t; the read query of the
- * attention layer is projected the same way):
+ * The projections in front of the layer (Algorithm 1, first two statements of the loop body:
+ * wq_t = W_wq x_t, wv_t = W_wv x_t; the read query of the attention layer is projected the
+ * same way):
  *     y[m][n] = sum_k x[m][k] * W[n][k]
  * x [M][K] one row per token, W [N][K] one row per output feature, y [M][N].
  * Returns the number of threads used, or -1 on bad arguments.

@@ -66,6 +66,11 @@ def _load():
             ctypes.c_int64, ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.c_int64,
             ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64),
             dp, dp, dp, dp, dp, dp, dp, ctypes.c_double, ctypes.c_double, ctypes.c_uint, ctypes.c_int]
+        lib.bct_oracle_stream_eps.restype = ctypes.c_int
+        lib.bct_oracle_stream_eps.argtypes = [
+            ctypes.c_int64, ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.c_int64,
+            ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64),
+            dp, dp, dp, dp, dp, dp, dp, ctypes.c_double, ctypes.c_double, ctypes.c_double, ctypes.c_uint, ctypes.c_int]
         lib.bct_oracle_project.restype = ctypes.c_int
         lib.bct_oracle_project.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, dp, dp, dp, ctypes.c_int]
         lib.bct_oracle_write_weights.restype = ctypes.c_int
@@ -154,11 +159,12 @@ class OracleCache:
     MK and MV_0; ``mv_init=None`` with ``init_len > 0`` means zeros, one of the two
     initialisations the Method section allows).  ``read_scale=None`` means
     ``1/sqrt(head_dim)``; ``write_scale=None`` means 1.0 (Algorithm 1 prints no scale).
+    ``write_eps``: slots whose write weight is below it keep their row (0 = the printed rule).
     """
 
     def __init__(self, batch, n_q_heads, n_kv_heads, head_dim, capacity, *, read_scale=None,
                  write_scale=None, init_len=0, mk_init=None, mv_init=None, flags=0,
-                 nthreads=0):
+                 nthreads=0, write_eps=0.0):
         if n_q_heads % n_kv_heads:
             raise ValueError("n_q_heads must be a multiple of n_kv_heads")
         if not (0 <= init_len <= capacity):
@@ -169,6 +175,7 @@ class OracleCache:
         self.read_scale = float(1.0 / np.sqrt(head_dim) if read_scale is None else read_scale)
         self.write_scale = float(1.0 if write_scale is None else write_scale)
         self.flags = int(flags)
+        self.write_eps = float(write_eps)
         self.nthreads = int(nthreads)
         self.threads_used = 0
         self.len = int(init_len)
@@ -215,11 +222,11 @@ class OracleCache:
             eta = _f64(eta)
             assert eta.shape == (self.B, T, self.Hkv), eta.shape
             eu = np.ascontiguousarray(eta.transpose(0, 2, 1)).reshape(self.U, T)
-        rc = _load().bct_oracle_stream_eta(
+        rc = _load().bct_oracle_stream_eps(
             self.U, T, self.G, self.d, self.C, ctypes.byref(ln), ctypes.byref(nw),
             _dptr(self.MK), _dptr(self.MV), _dptr(qu), _dptr(ku), _dptr(vu),
             _dptr(eu) if eu is not None else None,
-            _dptr(ou) if want_out else None, self.read_scale, self.write_scale,
+            _dptr(ou) if want_out else None, self.read_scale, self.write_scale, self.write_eps,
             self.flags, self.nthreads)
         if rc < 0:
             raise RuntimeError("bct_oracle_stream failed")

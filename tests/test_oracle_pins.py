@@ -498,6 +498,41 @@ def test_layer_step_inputs_feed_the_layer():
     np.testing.assert_array_equal(a.prefill_stream(q, k, v), b.prefill_stream(f32[:, :, None], 2 * f32[:, :, None], -f32[:, :, None]))
 
 
+def test_layer_step_inputs_head_split_with_several_heads():
+    # Weights stacked from per-head scaled identities: head h of q must be (h + 1) x, head h of the write query
+    # -(h + 1) x and of the write value 10 (h + 1) x, token by token and sequence by sequence.  Hq != Hkv, B > 1 and
+    # T != H != d, so that a split along the wrong axis, a transposed (T, H) order or a swapped k / v cannot pass.
+    B, T, Hq, Hkv, d = 2, 5, 6, 3, 4
+    x = _rand(B, T, d)
+    I = np.eye(d)
+    Wq = np.concatenate([(h + 1.0) * I for h in range(Hq)], axis=0)            # [Hq * d, d]
+    Wwq = np.concatenate([-(h + 1.0) * I for h in range(Hkv)], axis=0)         # [Hkv * d, d]
+    Wwv = np.concatenate([10.0 * (h + 1.0) * I for h in range(Hkv)], axis=0)
+    q, k, v = O.layer_step_inputs(x, Wq, Wwq, Wwv, Hq, Hkv, d, bf16=False)
+    assert q.shape == (B, T, Hq, d) and k.shape == (B, T, Hkv, d) and v.shape == (B, T, Hkv, d)
+    f32 = lambda z: np.asarray(z, dtype=np.float32).astype(np.float64)
+    for b in range(B):
+        for t in range(T):
+            for h in range(Hq):
+                np.testing.assert_array_equal(q[b, t, h], f32((h + 1.0) * x[b, t]))
+            for h in range(Hkv):
+                np.testing.assert_array_equal(k[b, t, h], f32(-(h + 1.0) * x[b, t]))
+                np.testing.assert_array_equal(v[b, t, h], f32(10.0 * (h + 1.0) * x[b, t]))
+    # with bfloat16 storage every element is the nearest bfloat16 of the same product
+    qb, kb, vb = O.layer_step_inputs(x, Wq, Wwq, Wwv, Hq, Hkv, d, bf16=True)
+    ref = torch.tensor(3.0 * x[1, 2], dtype=torch.float32).to(torch.bfloat16).double().numpy()
+    np.testing.assert_array_equal(qb[1, 2, 2], ref)
+    # and the layer on those vectors is the layer fed head by head: kv-head h serves query heads h*G .. h*G+G-1
+    C, G = 3, Hq // Hkv
+    whole = O.OracleCache(B, Hq, Hkv, d, C)
+    out = whole.prefill_stream(q, k, v)
+    for h in range(Hkv):
+        one = O.OracleCache(B, G, 1, d, C)
+        qs = np.stack([f32((h * G + g + 1.0) * x) for g in range(G)], axis=2)
+        o1 = one.prefill_stream(qs, f32(-(h + 1.0) * x)[:, :, None], f32(10.0 * (h + 1.0) * x)[:, :, None])
+        np.testing.assert_array_equal(out[:, :, h * G:(h + 1) * G], o1)
+
+
 def test_update_kv_is_algorithm_1():
     # UpdateKV(x_1..x_N, MV_0, MK, ...) returns MV_N = MV_0 + sum_t ww_t^T wv_t, reads nothing, leaves MK alone
     B, Hq, Hkv, d, C, T = 2, 4, 2, 6, 5, 11
@@ -511,3 +546,54 @@ def test_update_kv_is_algorithm_1():
             np.testing.assert_allclose(c.values()[b, h], mv[b, h] + WW.T @ v[b, :, h], rtol=0, atol=1e-12)
     np.testing.assert_array_equal(c.keys(), mk)
     assert c.len == C and c.n_written == T
+
+
+# ---------------------------------------------------------------------------------------
+# Write threshold (a reading of the library, not of the paper): slots with ww_j < write_eps keep their row
+# ---------------------------------------------------------------------------------------
+@pytest.mark.parametrize("flags", [0, O.WRITE_THEN_READ])
+def test_write_threshold_masked_two_matmul_restatement(flags):
+    # MV_N = MV_0 + (WW * [WW >= eps])^T Vc ;  O = Pr MV_0 + tril(Pr (WW * mask)^T) Vc: the read of a token that
+    # follows its own write sees the rows actually rewritten.  eps = 0 is the printed rule, bit for bit.
+    d, C, T, G, eps = 6, 11, 9, 2, 0.08
+    mk, mv0 = _rand(1, 1, C, d), _rand(1, 1, C, d)
+    q, k, v = _rand(1, T, G, d), _rand(1, T, 1, d), _rand(1, T, 1, d)
+    eta = RNG.uniform(0.2, 1.5, size=(1, T, 1))
+    c = O.OracleCache(1, G, 1, d, C, init_len=C, mk_init=mk, mv_init=mv0, read_scale=0.5, write_scale=0.9, flags=flags,
+                      write_eps=eps)
+    out = c.prefill_stream(q, k, v, eta=eta)
+    MK, MV0, Kc, Vc = mk[0, 0], mv0[0, 0], k[0, :, 0], v[0, :, 0]
+    WW = _np_softmax(0.9 * Kc @ MK.T)
+    assert (WW < eps).any() and (WW >= eps).any()                      # the threshold bites, but not everywhere
+    WM = np.where(WW >= eps, WW, 0.0)
+    EV = eta[0, :, 0, None] * Vc
+    np.testing.assert_allclose(c.values()[0, 0], MV0 + WM.T @ EV, rtol=0, atol=1e-12)
+    for g in range(G):
+        Pr = _np_softmax(0.5 * q[0, :, g] @ MK.T)
+        A = np.tril(Pr @ WM.T, 0 if flags else -1)
+        np.testing.assert_allclose(out[0, :, g], Pr @ MV0 + A @ EV, rtol=0, atol=1e-12)
+    # mass added per token = (sum of the weights that pass) * eta_t * v_t
+    np.testing.assert_allclose(c.values()[0, 0].sum(axis=0) - MV0.sum(axis=0), (WM.sum(axis=1)[:, None] * EV).sum(axis=0),
+                               rtol=0, atol=1e-12)
+    a = O.OracleCache(1, G, 1, d, C, init_len=C, mk_init=mk, mv_init=mv0, flags=flags, write_eps=0.0)
+    b = O.OracleCache(1, G, 1, d, C, init_len=C, mk_init=mk, mv_init=mv0, flags=flags)
+    np.testing.assert_array_equal(a.prefill_stream(q, k, v), b.prefill_stream(q, k, v))
+    np.testing.assert_array_equal(a.values(), b.values())
+
+
+def test_write_threshold_against_uniform_weights():
+    # a zero write query gives ww_j = 1/C exactly: a threshold just above 1/C freezes the state, one at 1/C does not
+    B, Hq, Hkv, d, C, T = 1, 1, 1, 3, 8, 4
+    mk, mv = _rand(B, Hkv, C, d), _rand(B, Hkv, C, d)
+    q, v = _rand(B, T, Hq, d), _rand(B, T, Hkv, d)
+    k = np.zeros((B, T, Hkv, d))
+    frozen = O.OracleCache(B, Hq, Hkv, d, C, init_len=C, mk_init=mk, mv_init=mv, write_eps=0.126)
+    frozen.prefill_stream(q, k, v)
+    np.testing.assert_array_equal(frozen.values(), mv)
+    live = O.OracleCache(B, Hq, Hkv, d, C, init_len=C, mk_init=mk, mv_init=mv, write_eps=0.125)
+    live.prefill_stream(q, k, v)
+    np.testing.assert_allclose(live.values()[0, 0], mv[0, 0] + v[0, :, 0].sum(axis=0)[None, :] / C, rtol=0, atol=1e-13)
+    # the fill phase appends whatever the threshold
+    f = O.OracleCache(B, Hq, Hkv, d, C, write_eps=0.9)
+    f.prefill_stream(q, _rand(B, T, Hkv, d), v)
+    np.testing.assert_array_equal(f.values()[0, 0, :T], v[0, :, 0])
