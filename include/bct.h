@@ -26,12 +26,21 @@
  *  - The library never allocates or frees device memory: all device storage is the
  *    caller's workspace given to bct_cache_create.
  *  - Every call validates its arguments on the host before enqueuing anything and
- *    returns a bct_status_t; a failed call enqueues nothing and leaves the cache as
- *    it was.  bct_last_error() gives a thread-local message for the last failure.
+ *    returns a bct_status_t.  A call refused with BCT_ERR_INVALID_ARG, BCT_ERR_UNSUPPORTED
+ *    or BCT_ERR_STATE has enqueued nothing and leaves the cache as it was.  BCT_ERR_CUDA
+ *    means the CUDA runtime refused a launch or a copy: a call that covers several
+ *    launches (bct_prefill_stream and the calls built on it split T tokens into chunk
+ *    and single-token launches) may then have enqueued a prefix of its tokens; that
+ *    prefix is applied in full, bct_cache_len and the token counters describe exactly
+ *    the tokens enqueued, and the cache stays consistent and usable.
+ *    bct_last_error() gives a thread-local message for the last failure.
  *  - Work is enqueued on the `cuda_stream` argument (a cudaStream_t passed as void*;
  *    NULL is the default stream) and the call returns without synchronising, except
  *    where stated.
- *  - A handle is not thread-safe; different handles are independent.
+ *  - A handle is not thread-safe; different handles are independent.  The library keeps a
+ *    mutex-guarded list of its live handles, so that a handle passed in after
+ *    bct_cache_destroy is answered with BCT_ERR_STATE without being dereferenced.
+ *  - No environment variable is read.
  *  - `len` (resident slots) is the same for every sequence of the batch.
  */
 #ifndef BCT_H_
@@ -82,7 +91,8 @@ typedef enum bct_dtype {
 
 typedef struct bct_params {
     int32_t batch;      /* B  >= 1 sequences */
-    int32_t n_q_heads;  /* Hq >= 1, a multiple of n_kv_heads; G = Hq / Hkv <= 8 */
+    int32_t n_q_heads;  /* Hq >= 1, a multiple of n_kv_heads; G = Hq / Hkv <= 8 on the CUDA-core
+                           kernel, <= 15 on the tensor-core kernel */
     int32_t n_kv_heads; /* Hkv >= 1; one (MK, MV) memory per (sequence, kv-head) */
     int32_t head_dim;   /* d in {64, 128} */
     int32_t capacity;   /* C >= 1: the paper's predefined number of slots M */
@@ -92,8 +102,12 @@ typedef struct bct_params {
     int32_t init_len;   /* resident slots at create, 0..C; C is the paper's full-size MV_0 */
     uint32_t flags;     /* BCT_FLAG_* */
     float write_eps;    /* a slot whose write weight ww_j is below this is not rewritten
-                           (its increment ww_j * v_t is dropped); <= 0 selects 2^-24.
-                           Ignored with BCT_FLAG_DENSE_WRITE. */
+                           (its increment ww_j * v_t is dropped), in every entry point:
+                           decode steps, stream chunks and bct_update_kv alike;
+                           <= 0 selects 2^-24.  Ignored with BCT_FLAG_DENSE_WRITE.  With
+                           BCT_FLAG_WRITE_THEN_READ the token's own read sees the slots
+                           actually rewritten (the tensor-core decode kernel adds the
+                           dropped slots' share as well: at most write_eps * |eta_t v_t|). */
     int32_t max_stream; /* largest T a later bct_prefill_stream_host call may pass;
                            sizes the staging area of the host-buffer entry points.
                            <= 0 selects 1. */
@@ -123,7 +137,7 @@ bct_status_t bct_cache_bytes(const bct_params_t *params, size_t *bytes, size_t *
  *   mk_init    DEVICE [B][Hkv][init_len][d] in `dtype`: the paper's MK (rows beyond
  *              init_len do not exist yet).  NULL allowed iff init_len == 0.
  *   mv_init    DEVICE, same shape: the paper's MV_0.  NULL with init_len > 0 means
- *              zeros ("initialized to zero or random values").
+ *              zeros (one of the two initialisations Method, "Model Structure" allows).
  * The import is enqueued on cuda_stream.  On success *out receives the handle.
  */
 bct_status_t bct_cache_create(const bct_params_t *params, void *workspace, size_t bytes,
@@ -174,8 +188,8 @@ bct_status_t bct_prefill_stream_eta(bct_cache_t *cache, const void *q, const voi
  * Algorithm 1 itself, procedure UpdateKV: the write queries and write key-value vectors of T tokens
  * go into the state, MV_N = MV_0 + sum_t eta_t ww_t^T wv_t, and nothing is read.  The same state as
  * bct_prefill_stream_eta with out == NULL (within rounding), in chunks of up to 128 tokens whose
- * write weights are formed together ("token-level parallel training": MK is never assigned, so the
- * tokens' write weights do not depend on one another).
+ * write weights are formed together (Key Implementation Aspects, "Optimized for Parallelism": MK is
+ * never assigned, so the tokens' write weights do not depend on one another).
  *   wq   DEVICE [B][T][Hkv][d]  write queries     wv  DEVICE [B][T][Hkv][d]  write key-value vectors
  *   eta  DEVICE float [B][T][Hkv] or NULL (all ones)
  * Needs a full cache (the paper's full-size MV_0; BCT_ERR_STATE otherwise) of the shape the chunked
@@ -186,9 +200,9 @@ bct_status_t bct_update_kv(bct_cache_t *cache, const void *wq, const void *wv, c
                            void *cuda_stream);
 
 /*
- * The projections in front of the layer (Algorithm 1, "Compute write query" wq_t = W_wq x_t and
- * "Compute write key-value vector" wv_t = W_wv x_t; the read query q_t = W_q x_t of the attention
- * layer likewise), for a block of tokens, as one tensor-core contraction:
+ * The projections in front of the layer (Algorithm 1, first two statements of the loop body:
+ * wq_t = W_wq x_t and wv_t = W_wv x_t; the read query q_t = W_q x_t of the attention layer
+ * likewise), for a block of tokens, as one tensor-core contraction:
  *     q = x W_q^T   [n_tokens][n_q]      k = x W_wq^T, v = x W_wv^T   [n_tokens][n_kv]
  *   x      DEVICE bfloat16 [n_tokens][d_model]      one row per token (tokens of all sequences, [B][T] order)
  *   w_q    DEVICE bfloat16 [n_q][d_model]           one row per output feature, n_q = Hq * head_dim
@@ -267,8 +281,8 @@ bct_status_t bct_prefill_stream_host_static(bct_cache_t *cache, const void *q, c
 bct_status_t bct_cache_len(const bct_cache_t *cache, int32_t *len);
 
 /*
- * Copy the state out in the canonical layout (Method step 5, "stored back into the
- * cache", made visible): k_out DEVICE [B][Hkv][C][d] in the cache dtype, v_out DEVICE
+ * Copy the state out in the canonical layout (Method step 5, the store of the updated
+ * sequence, made visible): k_out DEVICE [B][Hkv][C][d] in the cache dtype, v_out DEVICE
  * [B][Hkv][C][d] in v_dtype (BCT_F32 gives the bfloat16 value plus its residual,
  * exactly; BCT_BF16 the rounded value; BCT_BF16_PAIR both planes bit for bit).  Rows
  * >= len are written as zeros.  Either pointer may be NULL to skip that plane.
@@ -293,6 +307,31 @@ bct_status_t bct_cache_import(bct_cache_t *cache, const void *k_in, const void *
  * results are then undefined; the context stays usable).  The only call that blocks.
  */
 bct_status_t bct_cache_status(bct_cache_t *cache, void *cuda_stream);
+
+/* Set the device-side status word back to BCT_OK (enqueued on cuda_stream, no synchronisation):
+ * after a reported BCT_ERR_TIMEOUT the cache can be re-imported and used again. */
+bct_status_t bct_cache_status_clear(bct_cache_t *cache, void *cuda_stream);
+
+/*
+ * Rows of MV that the kernels of this cache have stored back so far (Method step 5: the store of the
+ * updated sequence): decode steps count the slots whose write weight reached write_eps (every slot
+ * with BCT_FLAG_DENSE_WRITE), the chunked stream kernel rebuilds whole tiles and counts every slot
+ * of every chunk; appended fill-phase slots are not counted.  Synchronises cuda_stream like
+ * bct_cache_status.  The fraction w = rows / (units * full-phase tokens * capacity) is the share of
+ * MV the update rule rewrites per token, the term w*C*d*s of the bytes a decode step must move.
+ *   rows  HOST, receives the count (64 bits).
+ */
+bct_status_t bct_cache_rows_rewritten(bct_cache_t *cache, void *cuda_stream, uint64_t *rows);
+
+/*
+ * Self-test of the bounded device-side waits (no step of the method): launches one thread block on
+ * cuda_stream that waits, with a limit of about a thousand polls, on a barrier in its shared memory
+ * that nothing ever arrives on; the wait gives up, the block records BCT_ERR_TIMEOUT with site code
+ * 99 in the cache's status word and returns normally.  Nothing faults, hangs or traps, and the cache's
+ * planes are not touched.  bct_cache_status then reports BCT_ERR_TIMEOUT until
+ * bct_cache_status_clear.  Asynchronous.
+ */
+bct_status_t bct_selftest_timeout(bct_cache_t *cache, void *cuda_stream);
 
 /* *yes = 1 if this cache's decode steps run on the tensor-core kernel (tcgen05 + TMA tensor
  * copies: bfloat16, head_dim 128, G <= 15, 128 <= C <= 65536, no PRECISE_READ / CUDA_CORES

@@ -16,8 +16,7 @@ BCT_OK, BCT_ERR_INVALID_ARG, BCT_ERR_UNSUPPORTED, BCT_ERR_STATE, BCT_ERR_CUDA, B
 BCT_F32, BCT_BF16, BCT_BF16_PAIR = 0, 1, 2
 FLAG_SKIP_FIRST_WRITE, FLAG_WRITE_THEN_READ, FLAG_DENSE_WRITE, FLAG_OUT_F32, FLAG_PRECISE_READ, FLAG_CUDA_CORES = 1, 2, 4, 8, 16, 32
 
-# BCT_LIBRARY selects another build of the same ABI (e.g. one compiled with different tuning constants).
-LIB_PATH = os.environ.get("BCT_LIBRARY") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "libbct_b200.so")
+LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libbct_b200.so")
 
 EXPORTS = (
     "bct_version", "bct_last_error", "bct_cache_bytes", "bct_cache_create", "bct_decode_step",
@@ -25,6 +24,7 @@ EXPORTS = (
     "bct_cache_export", "bct_cache_import", "bct_cache_status", "bct_cache_launches", "bct_cache_destroy",
     "bct_cache_tensor_path", "bct_prefill_stream_host_static", "bct_decode_step_eta", "bct_prefill_stream_eta",
     "bct_project_qkv", "bct_layer_scratch_bytes", "bct_layer_forward", "bct_update_kv",
+    "bct_cache_status_clear", "bct_cache_rows_rewritten", "bct_selftest_timeout",
 )
 STATIC_STAGE_BYTES = 8 << 20
 
@@ -81,6 +81,9 @@ def load() -> ctypes.CDLL:
     lib.bct_cache_destroy.argtypes = [vp]
     lib.bct_cache_tensor_path.argtypes = [vp, ctypes.POINTER(i32)]
     lib.bct_prefill_stream_host_static.argtypes = [vp, vp, vp, vp, vp, i64, vp]
+    lib.bct_cache_status_clear.argtypes = [vp, vp]
+    lib.bct_cache_rows_rewritten.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint64)]
+    lib.bct_selftest_timeout.argtypes = [vp, vp]
     for name in EXPORTS[2:]:
         getattr(lib, name).restype = ctypes.c_int
     _lib = lib
@@ -288,6 +291,19 @@ class Cache:
 
     def check_status(self, stream=None) -> None:
         _check(self.status(stream))
+
+    def status_clear(self, stream=None) -> None:
+        _check(self.lib.bct_cache_status_clear(self._h, _stream_ptr(stream)))
+
+    def rows_rewritten(self, stream=None) -> int:
+        """MV rows stored back by this cache's kernels so far (synchronises the stream)."""
+        n = ctypes.c_uint64(0)
+        _check(self.lib.bct_cache_rows_rewritten(self._h, _stream_ptr(stream), ctypes.byref(n)))
+        return n.value
+
+    def selftest_timeout(self, stream=None) -> None:
+        """Launch the block whose bounded wait runs out (reports BCT_ERR_TIMEOUT, site 99)."""
+        _check(self.lib.bct_selftest_timeout(self._h, _stream_ptr(stream)))
 
     def destroy(self) -> None:
         if self._h:

@@ -10,6 +10,7 @@
 #include <cstdio>
 #include <cstring>
 #include <new>
+#include <unordered_set>
 
 #include "bct_internal.h"
 
@@ -97,9 +98,22 @@ Carve carve(const bct_params_t& p) {
     return c;
 }
 
+// The handles bct_cache_create has given out and bct_cache_destroy has not yet taken back.  A handle
+// is looked up here before it is dereferenced, so that a destroyed one is refused, not read.
+std::mutex g_live_mu;
+std::unordered_set<const bct_cache_t*>& live_handles() {
+    static std::unordered_set<const bct_cache_t*> set;
+    return set;
+}
+bool handle_is_live(const bct_cache_t* c) {
+    std::lock_guard<std::mutex> lock(g_live_mu);
+    return live_handles().count(c) != 0;
+}
+
 bct_status_t check_handle(const bct_cache_t* c) {
     if (c == nullptr) return fail(BCT_ERR_INVALID_ARG, "cache handle is NULL");
-    if (c->magic != bct::kMagic) return fail(BCT_ERR_STATE, "cache handle is destroyed or corrupted");
+    if (!handle_is_live(c) || c->magic != bct::kMagic)
+        return fail(BCT_ERR_STATE, "cache handle is destroyed or was never created");
     return BCT_OK;
 }
 
@@ -121,7 +135,6 @@ void release_host_objects(bct_cache_t* c) {
     c->copy_stream = nullptr;
 }
 
-// T tokens, one decode launch each.  Pointers are device pointers in [B][T][H][d].
 // Tokens [t, T) of the call into a full cache with nothing read: the write-only chunks of the stream
 // kernel (128 tokens, then one shorter chunk rounded up to 16 whose rows past T are zero-filled).
 bct_status_t write_only_tokens(bct_cache_t* c, const void* k, const void* v, const float* eta, int64_t T, int64_t t,
@@ -143,6 +156,10 @@ bct_status_t write_only_tokens(bct_cache_t* c, const void* k, const void* v, con
     return BCT_OK;
 }
 
+// T tokens of the [B][T][H][d] step arrays (device pointers) through the cache: whole chunks on the
+// chunked stream kernel where it applies, single tokens on the decode kernels otherwise.  Everything
+// that can be refused on the host has been refused by the callers; a failure here is the CUDA runtime
+// refusing a launch, and the counters then describe exactly the tokens already enqueued.
 // eta: [B][T][Hkv] floats on the device, or NULL.
 bct_status_t run_tokens(bct_cache_t* c, const void* q, const void* k, const void* v, const float* eta, void* out,
                         int64_t T, cudaStream_t stream) {
@@ -235,6 +252,7 @@ bct_status_t run_tokens(bct_cache_t* c, const void* q, const void* k, const void
 
 namespace bct {
 void set_last_error(const char* msg) { snprintf(g_err, sizeof(g_err), "%s", msg); }
+bct_status_t check_live_handle(const bct_cache* c) { return check_handle(c); }
 }  // namespace bct
 
 extern "C" {
@@ -341,6 +359,10 @@ bct_status_t bct_cache_create(const bct_params_t* params, void* workspace, size_
         return fail_cuda("state import", e);
     }
     c->launches += 1;
+    {
+        std::lock_guard<std::mutex> lock(g_live_mu);
+        live_handles().insert(c);
+    }
     *out = c;
     return BCT_OK;
 }
@@ -358,7 +380,8 @@ bct_status_t bct_prefill_stream(bct_cache_t* c, const void* q, const void* k, co
                                 void* cuda_stream) {
     bct_status_t st = check_handle(c);
     if (st != BCT_OK) return st;
-    if (T < 1) return fail(BCT_ERR_INVALID_ARG, "T must be >= 1 (got %lld)", (long long)T);
+    if (T < 1 || T > bct::kMaxCallTokens)
+        return fail(BCT_ERR_INVALID_ARG, "T must be in [1, 2^30] (got %lld)", (long long)T);
     st = check_step_ptrs(q, k, v, out, true);
     if (st != BCT_OK) return st;
     return run_tokens(c, q, k, v, nullptr, out, T, static_cast<cudaStream_t>(cuda_stream));
@@ -368,7 +391,8 @@ bct_status_t bct_prefill_stream_eta(bct_cache_t* c, const void* q, const void* k
                                     void* out, int64_t T, void* cuda_stream) {
     bct_status_t st = check_handle(c);
     if (st != BCT_OK) return st;
-    if (T < 1) return fail(BCT_ERR_INVALID_ARG, "T must be >= 1 (got %lld)", (long long)T);
+    if (T < 1 || T > bct::kMaxCallTokens)
+        return fail(BCT_ERR_INVALID_ARG, "T must be in [1, 2^30] (got %lld)", (long long)T);
     st = check_step_ptrs(q, k, v, out, true);
     if (st != BCT_OK) return st;
     if ((reinterpret_cast<uintptr_t>(eta) & 3u) != 0) return fail(BCT_ERR_INVALID_ARG, "eta must be 4-byte aligned");
@@ -379,7 +403,8 @@ bct_status_t bct_update_kv(bct_cache_t* c, const void* wq, const void* wv, const
                            void* cuda_stream) {
     bct_status_t st = check_handle(c);
     if (st != BCT_OK) return st;
-    if (T < 1) return fail(BCT_ERR_INVALID_ARG, "T must be >= 1 (got %lld)", (long long)T);
+    if (T < 1 || T > bct::kMaxCallTokens)
+        return fail(BCT_ERR_INVALID_ARG, "T must be in [1, 2^30] (got %lld)", (long long)T);
     if (wq == nullptr || wv == nullptr) return fail(BCT_ERR_INVALID_ARG, "wq and wv must not be NULL");
     if (!aligned16(wq) || !aligned16(wv)) return fail(BCT_ERR_INVALID_ARG, "wq and wv must be 16-byte aligned");
     if ((reinterpret_cast<uintptr_t>(eta) & 3u) != 0) return fail(BCT_ERR_INVALID_ARG, "eta must be 4-byte aligned");
@@ -466,7 +491,8 @@ bct_status_t bct_project_qkv(int64_t n_tokens, int32_t d_model, int32_t n_q, int
 bct_status_t bct_layer_scratch_bytes(const bct_cache_t* c, int64_t T, size_t* bytes) {
     bct_status_t st = check_handle(c);
     if (st != BCT_OK) return st;
-    if (T < 1 || bytes == nullptr) return fail(BCT_ERR_INVALID_ARG, "T must be >= 1 and bytes not NULL");
+    if (T < 1 || T > bct::kMaxCallTokens || bytes == nullptr)
+        return fail(BCT_ERR_INVALID_ARG, "T must be in [1, 2^30] and bytes not NULL");
     const size_t eb = (size_t)c->elem_bytes;
     const size_t qb = (size_t)c->p.batch * (size_t)T * c->p.n_q_heads * c->p.head_dim * eb;
     const size_t kb = (size_t)c->p.batch * (size_t)T * c->p.n_kv_heads * c->p.head_dim * eb;
@@ -480,7 +506,8 @@ bct_status_t bct_layer_forward(bct_cache_t* c, const void* x, const void* w_q, c
     bct_status_t st = check_handle(c);
     if (st != BCT_OK) return st;
     if (c->p.dtype != BCT_BF16) return fail(BCT_ERR_UNSUPPORTED, "the fused projections serve bfloat16 caches only");
-    if (T < 1) return fail(BCT_ERR_INVALID_ARG, "T must be >= 1 (got %lld)", (long long)T);
+    if (T < 1 || T > bct::kMaxCallTokens)
+        return fail(BCT_ERR_INVALID_ARG, "T must be in [1, 2^30] (got %lld)", (long long)T);
     size_t need = 0;
     st = bct_layer_scratch_bytes(c, T, &need);
     if (st != BCT_OK) return st;
@@ -605,6 +632,36 @@ bct_status_t bct_cache_status(bct_cache_t* c, void* cuda_stream) {
     return BCT_OK;
 }
 
+bct_status_t bct_cache_status_clear(bct_cache_t* c, void* cuda_stream) {
+    bct_status_t st = check_handle(c);
+    if (st != BCT_OK) return st;
+    cudaError_t e = cudaMemsetAsync(c->status, 0, 2 * sizeof(int), static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return fail_cuda("status clear", e);
+    return BCT_OK;
+}
+
+bct_status_t bct_cache_rows_rewritten(bct_cache_t* c, void* cuda_stream, uint64_t* rows) {
+    bct_status_t st = check_handle(c);
+    if (st != BCT_OK) return st;
+    if (rows == nullptr) return fail(BCT_ERR_INVALID_ARG, "rows is NULL");
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    unsigned long long host = 0;
+    cudaError_t e = cudaMemcpyAsync(&host, c->status + bct::kStatusRowsWord, sizeof(host), cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+    if (e != cudaSuccess) return fail_cuda("counter read", e);
+    *rows = (uint64_t)host;
+    return BCT_OK;
+}
+
+bct_status_t bct_selftest_timeout(bct_cache_t* c, void* cuda_stream) {
+    bct_status_t st = check_handle(c);
+    if (st != BCT_OK) return st;
+    cudaError_t e = bct::launch_wait_selftest(c, static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return fail_cuda("self-test launch", e);
+    c->launches += 1;
+    return BCT_OK;
+}
+
 bct_status_t bct_cache_tensor_path(const bct_cache_t* c, int32_t* yes) {
     bct_status_t st = check_handle(c);
     if (st != BCT_OK) return st;
@@ -623,7 +680,10 @@ bct_status_t bct_cache_launches(const bct_cache_t* c, int64_t* launches) {
 
 bct_status_t bct_cache_destroy(bct_cache_t* c) {
     if (c == nullptr) return BCT_OK;
-    if (c->magic != bct::kMagic) return fail(BCT_ERR_STATE, "cache handle is destroyed or corrupted");
+    {
+        std::lock_guard<std::mutex> lock(g_live_mu);
+        if (live_handles().erase(c) == 0) return fail(BCT_ERR_STATE, "cache handle is destroyed or was never created");
+    }
     release_host_objects(c);
     c->magic = 0;
     delete c;

@@ -370,6 +370,7 @@ __global__ void __launch_bounds__(kThreads, (G <= 4 ? 2 : 1)) decode_kernel(cons
         Ck::unpack(v_raw, vt);
 #pragma unroll
         for (int e = 0; e < EPL; ++e) vt[e] *= eta_u;
+        int rows_stored = 0;  // rows of MV this thread's row group rewrites (counted by the lane of chunk 0)
         for (int i = 0; i < nt; ++i) {
             const int item = precise ? nt + 2 * i : nt + i;
             const int stage = item % kStages;
@@ -416,9 +417,11 @@ __global__ void __launch_bounds__(kThreads, (G <= 4 ? 2 : 1)) decode_kernel(cons
                     }
                     if (a.do_write) {
                         const float ww = sc[G * stride + row] * wfac;
-#pragma unroll
-                        for (int g = 0; g < G; ++g) wd[g] = fmaf(p[g], ww, wd[g]);
                         if (a.dense || ww >= a.write_eps) {
+                            // (a read that follows its own write sees the rows actually rewritten)
+#pragma unroll
+                            for (int g = 0; g < G; ++g) wd[g] = fmaf(p[g], ww, wd[g]);
+                            if (chunk == 0) ++rows_stored;
                             const size_t off = (size_t)row * ROW_BYTES + chunk * 16;
                             float nv[EPL];
                             if constexpr (sizeof(T) == 2) {
@@ -452,6 +455,9 @@ __global__ void __launch_bounds__(kThreads, (G <= 4 ? 2 : 1)) decode_kernel(cons
                 if (precise) mbar_arrive(&empty[stage_lo]);
             }
         }
+        rows_stored = __reduce_add_sync(0xffffffffu, rows_stored);
+        if (lane == 0 && rows_stored > 0)
+            atomicAdd(reinterpret_cast<unsigned long long*>(a.status + kStatusRowsWord), (unsigned long long)rows_stored);
         if (has_virtual && warp == 0 && sub == 0) {  // the appended slot's own value row
 #pragma unroll
             for (int g = 0; g < G; ++g) {

@@ -22,7 +22,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
-#include <cstdlib>
+#include <mutex>
 
 #include "bct_internal.h"
 #include "bct_tc.cuh"
@@ -124,6 +124,24 @@ __device__ __forceinline__ void tmem_st_rows(uint32_t taddr, const float* x) {
 }
 
 __device__ __forceinline__ void s_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kSThreads) : "memory"); }
+
+// The update rule on 16 bytes (8 elements) of one row, MV_t = MV_{t-1} + ww * (eta_t wv_t): the staged value and
+// residual chunks give MV_{t-1}, the sum is split again into a bfloat16 value and a bfloat16 residual and
+// stored to the two planes.
+__device__ __forceinline__ void rewrite_chunk(const unsigned char* staged_hi, const unsigned char* staged_lo, char* dst_hi,
+                                              char* dst_lo, float ww, const float* vtv) {
+    float x[8], lo[8], nv[8], hf[8];
+    Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(staged_hi), x);
+    Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(staged_lo), lo);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) nv[e] = fmaf(ww, vtv[e], x[e] + lo[e]);
+    const uint4 hi_new = Chunk<__nv_bfloat16>::pack(nv);
+    Chunk<__nv_bfloat16>::unpack(hi_new, hf);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) nv[e] -= hf[e];
+    *reinterpret_cast<uint4*>(dst_hi) = hi_new;
+    *reinterpret_cast<uint4*>(dst_lo) = Chunk<__nv_bfloat16>::pack(nv);
+}
 
 template <int G>
 __global__ void __launch_bounds__(kTcThreads, 1)
@@ -372,6 +390,44 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             store_q(0, qnext);
         }
 
+        // Staging of the rows the update rule rewrites: copies of their value and residual rows arrive in shared
+        // memory by 16-byte asynchronous copies, so that no global-memory latency is left for the update.
+        const int c16 = tid & 15;  // 16-byte chunk of a 256-byte row
+        auto stage_rows = [&](size_t uoff, int base, int n, int sbase) {
+            for (int i = tid >> 4; i < n; i += kSThreads / 16) {
+                const size_t goff = uoff + (size_t)(slice_start + list[base + i]) * ROW_BYTES + c16 * 16;
+                cp_async16(histage + (sbase + i) * ROW_BYTES + c16 * 16, a.vhi + goff);
+                cp_async16(lostage + (sbase + i) * ROW_BYTES + c16 * 16, a.vlo + goff);
+            }
+            cp_async_commit();
+        };
+        // The update rule MV_t = MV_{t-1} + ww_t^T . wv_t on listed rows [base, base + n), staged from row sbase
+        // of the staging area on; their weights come from lww (kept across units) or from the scaled scores.
+        auto rewrite_rows = [&](size_t uoff, int base, int n, int sbase, const float* vtv, bool from_lww, float wmax, float wfac) {
+            for (int i = tid >> 4; i < n; i += kSThreads / 16) {
+                const int row = list[base + i];
+                const float ww = from_lww ? lww[base + i] : __expf(wsm[row] - wmax) * wfac;
+                const size_t goff = uoff + (size_t)(slice_start + row) * ROW_BYTES + c16 * 16;
+                rewrite_chunk(histage + (sbase + i) * ROW_BYTES + c16 * 16, lostage + (sbase + i) * ROW_BYTES + c16 * 16,
+                              a.vhi + goff, a.vlo + goff, ww, vtv);
+            }
+        };
+        // A unit's deferred update: rounds of kLoCap staged rows (weights kept in lww), whose first round has been
+        // in flight since that unit's epilogue.
+        auto apply_update = [&](int n_rows, size_t uoff, const float* vtv) {
+            for (int base = 0; base < n_rows; base += kLoCap) {
+                const int n = min(n_rows - base, kLoCap);
+                if (base > 0) {
+                    s_sync();  // the previous round's staged rows have been consumed
+                    stage_rows(uoff, base, n, 0);
+                }
+                cp_async_wait_all();
+                s_sync();  // every thread's staged chunks have landed
+                rewrite_rows(uoff, base, n, 0, vtv, true, 0.f, 0.f);
+            }
+        };
+        unsigned long long rows_stored = 0;  // thread 0: MV rows this CTA has rewritten
+
         int it = 0;
         uint32_t sp = 0;  // sub-slices processed so far (phase of the per-tile barriers)
         // update of the previous unit, applied during this unit's turn: rows listed, plane offset, v_t * eta_t
@@ -562,47 +618,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 }
             }
 
-            // ---- list the slots the rule rewrites and stage copies of their value and residual rows with
-            // ---- 16-byte asynchronous copies, so that no global-memory latency is left for the update ----
-            const int c16 = tid & 15;  // 16-byte chunk of a 256-byte row
-            auto stage_rows = [&](size_t uoff, int base, int n) {
-                for (int i = tid >> 4; i < n; i += kSThreads / 16) {
-                    const size_t goff = uoff + (size_t)(slice_start + list[base + i]) * ROW_BYTES + c16 * 16;
-                    cp_async16(histage + i * ROW_BYTES + c16 * 16, a.vhi + goff);
-                    cp_async16(lostage + i * ROW_BYTES + c16 * 16, a.vlo + goff);
-                }
-                cp_async_commit();
-            };
-            // The update rule MV_t = MV_{t-1} + ww_t^T . wv_t on the rows it changes: rounds of kLoCap staged
-            // rows of the previous unit (weights kept in lww), whose first round has been in flight since that
-            // unit's epilogue.
-            auto apply_update = [&](int n_rows, size_t uoff, const float* vtv) {
-                for (int base = 0; base < n_rows; base += kLoCap) {
-                    const int n = min(n_rows - base, kLoCap);
-                    if (base > 0) {
-                        s_sync();  // the previous round's staged rows have been consumed
-                        stage_rows(uoff, base, n);
-                    }
-                    cp_async_wait_all();
-                    s_sync();  // every thread's staged chunks have landed
-                    for (int i = tid >> 4; i < n; i += kSThreads / 16) {
-                        const int row = list[base + i];
-                        const float ww = lww[base + i];
-                        const size_t goff = uoff + (size_t)(slice_start + row) * ROW_BYTES + c16 * 16;
-                        float x[8], lo[8], nv[8], hf[8];
-                        Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(histage + i * ROW_BYTES + c16 * 16), x);
-                        Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(lostage + i * ROW_BYTES + c16 * 16), lo);
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) nv[e] = fmaf(ww, vtv[e], x[e] + lo[e]);
-                        const uint4 hi_new = Chunk<__nv_bfloat16>::pack(nv);
-                        Chunk<__nv_bfloat16>::unpack(hi_new, hf);
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) nv[e] -= hf[e];
-                        *reinterpret_cast<uint4*>(a.vhi + goff) = hi_new;
-                        *reinterpret_cast<uint4*>(a.vlo + goff) = Chunk<__nv_bfloat16>::pack(nv);
-                    }
-                }
-            };
+            // ---- list the slots the rule rewrites and stage copies of their value and residual rows (stage_rows),
+            // ---- so that no global-memory latency is left for the update ----
             // The previous unit's rows first: their staged copies had this unit's whole softmax to arrive,
             // and this unit's V tiles are being multiplied meanwhile.  (Units are independent memories.)
             if (pend_n > 0) {
@@ -626,7 +643,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 s_sync();
                 n_touched = *lo_count;
                 // (a unit that rewrites more rows than lww keeps goes in double-buffered half rounds, below)
-                stage_rows(unit_off, 0, min(n_touched, n_touched > kLwwCap ? kLoCap / 2 : kLoCap));
+                stage_rows(unit_off, 0, min(n_touched, n_touched > kLwwCap ? kLoCap / 2 : kLoCap), 0);
+                if (tid == 0) rows_stored += (unsigned long long)n_touched;
             }
 
             // ---- epilogue: O[d][g] from tensor memory once every V tile has been read ----
@@ -726,34 +744,14 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         const int base = rd * hcap, n = min(n_touched - base, hcap);
                         const int sbase = (rd & 1) * hcap;  // first staging row of this half round
                         if (rd + 1 < n_rounds) {  // ask for the next half round (its half was consumed a round ago)
-                            const int nb = base + hcap, nn = min(n_touched - nb, hcap), nsb = ((rd + 1) & 1) * hcap;
-                            for (int i = tid >> 4; i < nn; i += kSThreads / 16) {
-                                const size_t goff = unit_off + (size_t)(slice_start + list[nb + i]) * ROW_BYTES + c16 * 16;
-                                cp_async16(histage + (nsb + i) * ROW_BYTES + c16 * 16, a.vhi + goff);
-                                cp_async16(lostage + (nsb + i) * ROW_BYTES + c16 * 16, a.vlo + goff);
-                            }
-                            cp_async_commit();
+                            const int nb = base + hcap;
+                            stage_rows(unit_off, nb, min(n_touched - nb, hcap), ((rd + 1) & 1) * hcap);
                             cp_async_wait_but_one();
                         } else {
                             cp_async_wait_all();
                         }
                         s_sync();  // this half round's chunks have landed for every thread
-                        for (int i = tid >> 4; i < n; i += kSThreads / 16) {
-                            const int row = list[base + i];
-                            const float ww = __expf(wsm[row] - st_m[G]) * wfac;
-                            const size_t goff = unit_off + (size_t)(slice_start + row) * ROW_BYTES + c16 * 16;
-                            float x[8], lo[8], nv[8], hf[8];
-                            Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(histage + (sbase + i) * ROW_BYTES + c16 * 16), x);
-                            Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(lostage + (sbase + i) * ROW_BYTES + c16 * 16), lo);
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) nv[e] = fmaf(ww, vt[e], x[e] + lo[e]);
-                            const uint4 hi_new = Chunk<__nv_bfloat16>::pack(nv);
-                            Chunk<__nv_bfloat16>::unpack(hi_new, hf);
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) nv[e] -= hf[e];
-                            *reinterpret_cast<uint4*>(a.vhi + goff) = hi_new;
-                            *reinterpret_cast<uint4*>(a.vlo + goff) = Chunk<__nv_bfloat16>::pack(nv);
-                        }
+                        rewrite_rows(unit_off, base, n, sbase, vt, false, st_m[G], wfac);
                         s_sync();  // the half is free for the round after next
                     }
                 }
@@ -767,39 +765,9 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             s_sync();  // st_*, red and wsm are reused by the next unit (the list and the staging rows: after its deferred update)
             if (pend_n == 0 && tid == 0) *lo_count = 0;
         }
-        if (pend_n > 0) {  // the last unit's rows
-            const int c16 = tid & 15;
-            for (int base = 0; base < pend_n; base += kLoCap) {
-                const int n = min(pend_n - base, kLoCap);
-                if (base > 0) {
-                    s_sync();
-                    for (int i = tid >> 4; i < n; i += kSThreads / 16) {
-                        const size_t goff = pend_off + (size_t)(slice_start + list[base + i]) * ROW_BYTES + c16 * 16;
-                        cp_async16(histage + i * ROW_BYTES + c16 * 16, a.vhi + goff);
-                        cp_async16(lostage + i * ROW_BYTES + c16 * 16, a.vlo + goff);
-                    }
-                    cp_async_commit();
-                }
-                cp_async_wait_all();
-                s_sync();
-                for (int i = tid >> 4; i < n; i += kSThreads / 16) {
-                    const int row = list[base + i];
-                    const float ww = lww[base + i];
-                    const size_t goff = pend_off + (size_t)(slice_start + row) * ROW_BYTES + c16 * 16;
-                    float x[8], lo[8], nv[8], hf[8];
-                    Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(histage + i * ROW_BYTES + c16 * 16), x);
-                    Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(lostage + i * ROW_BYTES + c16 * 16), lo);
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) nv[e] = fmaf(ww, pend_vt[e], x[e] + lo[e]);
-                    const uint4 hi_new = Chunk<__nv_bfloat16>::pack(nv);
-                    Chunk<__nv_bfloat16>::unpack(hi_new, hf);
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) nv[e] -= hf[e];
-                    *reinterpret_cast<uint4*>(a.vhi + goff) = hi_new;
-                    *reinterpret_cast<uint4*>(a.vlo + goff) = Chunk<__nv_bfloat16>::pack(nv);
-                }
-            }
-        }
+        if (pend_n > 0) apply_update(pend_n, pend_off, pend_vt);  // the last unit's rows
+        if (tid == 0 && rows_stored > 0)
+            atomicAdd(reinterpret_cast<unsigned long long*>(a.status + kStatusRowsWord), rows_stored);
     }
 
     tc_fence_before();
@@ -918,11 +886,6 @@ int launch_decode_tc(const bct_cache* c, const StepIO& io, int len, int do_write
     // (A deeper ring for short slices was measured: no gain, the softmax chain of a unit is the limit.)
     int lo_cap = 80;
     int stages = 4;
-    static const char* env_stages = getenv("BCT_TC_STAGES");  // read once
-    if (const char* e = env_stages) {  // tuning knob: depth of the tile ring (2..8)
-        const int v = atoi(e);
-        if (v >= 2 && v <= 8) stages = v;
-    }
     while (tc_smem(stages, c->G, S, slice, lo_cap).total > c->smem_optin && (stages > 3 || lo_cap > 32)) {
         if (stages > 4 || (stages > 3 && lo_cap <= 48))
             --stages;
@@ -969,7 +932,11 @@ int launch_decode_tc(const bct_cache* c, const StepIO& io, int len, int do_write
     struct Seen {
         int smem_set, occ_S, occ_smem, occ_active;
     };
+    // (The table is the only state shared between handles: guarded, and held for the launch itself so that
+    // two threads cannot interleave the attribute update and the launches that rely on it.)
+    static std::mutex seen_mu;
     static Seen seen[64][16] = {};
+    std::lock_guard<std::mutex> seen_lock(seen_mu);
     Seen local = {};
     Seen& sn = (c->device >= 0 && c->device < 64) ? seen[c->device][c->G] : local;
     if (sn.smem_set < smem) {

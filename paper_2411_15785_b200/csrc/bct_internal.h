@@ -10,6 +10,7 @@ namespace bct {
 constexpr uint64_t kMagic = 0x4243545f43414348ull;  // "BCT_CACH"
 constexpr size_t kAlign = 256;                      // alignment of every workspace section
 constexpr int kMaxGroup = 8;     // query heads per kv-head on the CUDA-core kernel
+constexpr int64_t kMaxCallTokens = (int64_t)1 << 30;  // tokens per sequence one call may pass
 constexpr int kMaxGroupTc = 15;  // ... on the tensor-core decode kernel (16 operand rows: the read heads + the write query)
 
 // Where the step vectors of one launch live and how to walk them.
@@ -100,10 +101,19 @@ cudaError_t launch_project(long long n_tokens, int d_model, int n_q, int n_kv, c
 
 // Set the calling thread's bct_last_error() message (for entry points outside bct_api.cu).
 void set_last_error(const char* msg);
+// BCT_OK if `c` is a handle bct_cache_create gave out and bct_cache_destroy has not taken back (looked up
+// in the list of live handles, not dereferenced); otherwise the status to return, with the message set.
+bct_status_t check_live_handle(const bct_cache* c);
 
 // State import / export.
 cudaError_t launch_import(const bct_cache* c, const void* k_in, const void* v_in, int v_dtype, int len,
                           cudaStream_t stream);
 cudaError_t launch_export(const bct_cache* c, void* k_out, void* v_out, int v_dtype, cudaStream_t stream);
+// One block whose bounded wait runs out and reports BCT_ERR_TIMEOUT (site 99) to the status words.
+cudaError_t launch_wait_selftest(const bct_cache* c, cudaStream_t stream);
+
+// Status area of the workspace (kAlign bytes of ints): word 0 = status code, word 1 = site of the
+// first timeout, words 2-3 = 64-bit count of MV rows stored back by the kernels.
+constexpr int kStatusRowsWord = 2;
 
 }  // namespace bct

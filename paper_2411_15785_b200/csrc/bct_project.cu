@@ -24,7 +24,7 @@
 
 #include <cstdint>
 #include <cstdio>
-#include <cstdlib>
+#include <mutex>
 
 #include "bct_internal.h"
 #include "bct_tc.cuh"
@@ -266,7 +266,9 @@ cudaError_t launch_bn(const CUtensorMap& mx, const CUtensorMap& m0, const CUtens
     auto fn = project_kernel<BN, KPER>;
     // the shared-memory limit of this kernel on this device is raised only when it has to grow (a decode
     // step's projection is short enough for one more runtime call per launch to show)
+    static std::mutex smem_mu;
     static int smem_set[64] = {};
+    std::lock_guard<std::mutex> smem_lock(smem_mu);
     if (device < 0 || device >= 64 || smem_set[device] < smem) {
         cudaError_t e = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
@@ -295,12 +297,6 @@ cudaError_t launch_project(long long n_tokens, int d_model, int n_q, int n_kv, c
     if (n_q % 128 == 0 && n_kv % 128 == 0 && (n_tokens > 256 || m_tiles * ((n_q + 2 * n_kv) / 128) * 8 >= 5LL * sm_count))
         BN = 128;
     if (n_tokens >= 1024 && n_q % 256 == 0 && n_kv % 256 == 0) BN = 256;
-    static const char* env_bn = getenv("BCT_PJ_BN");      // tuning knobs, read once
-    static const char* env_kper = getenv("BCT_PJ_KPER");
-    if (const char* e = env_bn) {  // width of the feature tiles
-        const int v = atoi(e);
-        if ((v == 32 || v == 64 || v == 128 || v == 256) && n_q % v == 0 && n_kv % v == 0) BN = v;
-    }
     const int a_rows = n_tokens >= kPjBM ? kPjBM : (int)((n_tokens + 7) / 8 * 8);
     alignas(64) CUtensorMap mx, m0, m1, m2;
     if (!make_matrix_map(&mx, x, n_tokens, d_model, a_rows) || !make_matrix_map(&m0, w_q, n_q, d_model, BN) ||
@@ -324,10 +320,6 @@ cudaError_t launch_project(long long n_tokens, int d_model, int n_q, int n_kv, c
     // 57.6 / 43.1 / 34.8 us with 1 / 2 / 4 blocks per stage; 128-wide: 33.0 / 28.1 us with 1 / 2).
     const int block = a.a_bytes + BN * kPjBK * 2;
     int kper = 12 * block <= 200 * 1024 ? 4 : (6 * block <= 200 * 1024 ? 2 : 1);
-    if (const char* e = env_kper) {  // 64-column blocks per stage (1, 2, 4)
-        const int v = atoi(e);
-        if (v == 1 || v == 2 || v == 4) kper = v;
-    }
 #define PJ_LAUNCH(bn, kp) \
     if (BN == bn && kper == kp) return launch_bn<bn, kp>(mx, m0, m1, m2, a, device, sm_count, smem_optin, stream);
     PJ_LAUNCH(256, 1)

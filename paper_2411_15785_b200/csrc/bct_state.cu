@@ -4,6 +4,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include "bct_device.cuh"
 #include "bct_internal.h"
 
 namespace bct {
@@ -77,6 +78,18 @@ __global__ void export_kernel(const CacheT* kplane, const CacheT* vhi, const __n
     }
 }
 
+// Self-test of the bounded waits: a barrier that expects one arrival and never gets it.  The wait
+// runs out after `limit` polls, the failure goes to the status words like any other, and the block
+// returns normally.
+__global__ void wait_selftest_kernel(int* status, uint32_t limit, int site) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        fence_mbar_init_cluster();
+        if (!mbar_wait(&bar, 0, limit)) report_timeout(status, site);
+    }
+}
+
 inline unsigned grid_for(size_t n, int sm_count) {
     size_t blocks = (n + 255) / 256;
     size_t cap = (size_t)sm_count * 16;
@@ -100,6 +113,11 @@ cudaError_t launch_import(const bct_cache* c, const void* k_in, const void* v_in
             reinterpret_cast<__nv_bfloat16*>(c->vlo), static_cast<const __nv_bfloat16*>(k_in), v_in, v_mode,
             (size_t)c->U, c->p.capacity, c->p.head_dim, len);
     }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_wait_selftest(const bct_cache* c, cudaStream_t stream) {
+    wait_selftest_kernel<<<1, 32, 0, stream>>>(c->status, 1000u, 99);
     return cudaGetLastError();
 }
 

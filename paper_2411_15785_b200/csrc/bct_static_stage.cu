@@ -50,10 +50,8 @@ extern "C" {
 bct_status_t bct_prefill_stream_host_static(bct_cache_t* c, const void* q, const void* k, const void* v, void* out,
                                             int64_t T, void* cuda_stream) {
     char msg[256] = "";
-    if (c == nullptr || c->magic != bct::kMagic) {
-        bct::set_last_error("cache handle is NULL, destroyed or corrupted");
-        return c == nullptr ? BCT_ERR_INVALID_ARG : BCT_ERR_STATE;
-    }
+    bct_status_t hs = bct::check_live_handle(c);
+    if (hs != BCT_OK) return hs;
     if (q == nullptr || k == nullptr || v == nullptr || out == nullptr) {
         bct::set_last_error("q, k, v and out must not be NULL");
         return BCT_ERR_INVALID_ARG;
@@ -66,11 +64,17 @@ bct_status_t bct_prefill_stream_host_static(bct_cache_t* c, const void* q, const
     const bct_params_t& p = c->p;
     const size_t eb = (size_t)c->elem_bytes;
     const size_t ob = (p.flags & BCT_FLAG_OUT_F32) ? 4 : eb;
-    const size_t q_elems = (size_t)p.batch * (size_t)T * p.n_q_heads * p.head_dim;
-    const size_t kv_elems = (size_t)p.batch * (size_t)T * p.n_kv_heads * p.head_dim;
+    // T is bounded before any product with it: the bytes one token of every sequence needs, then the
+    // largest T that could fit at all (a huge T must not wrap the sizes below)
+    const size_t q_tok = (size_t)p.batch * p.n_q_heads * p.head_dim, kv_tok = (size_t)p.batch * p.n_kv_heads * p.head_dim;
+    const size_t per_token = q_tok * (eb + ob) + 2 * kv_tok * eb;
+    const bool t_fits = (uint64_t)T <= kStaticStageBytes / per_token;
+    const size_t q_elems = t_fits ? q_tok * (size_t)T : 0;
+    const size_t kv_elems = t_fits ? kv_tok * (size_t)T : 0;
     const size_t q_bytes = q_elems * eb, kv_bytes = kv_elems * eb, out_bytes = q_elems * ob;
-    const size_t need = round256(q_bytes) + 2 * round256(kv_bytes) + round256(out_bytes);
-    if (need > kStaticStageBytes) {
+    const size_t need = t_fits ? round256(q_bytes) + 2 * round256(kv_bytes) + round256(out_bytes)
+                               : (T > (1 << 20) ? ~(size_t)0 : per_token * (size_t)T);
+    if (!t_fits || need > kStaticStageBytes) {
         snprintf(msg, sizeof(msg),
                  "T = %lld needs %zu bytes of staging; the static staging area holds %zu (use fewer tokens per call)",
                  (long long)T, need, kStaticStageBytes);

@@ -57,6 +57,7 @@ struct StArgs {
     int fill, len0;  // fill = 1: the cache holds len0 slots and each chunk is appended (no soft write)
     int wtr, out_f32, precise;  // precise: the read uses value + residual of both the numerators and MV
     float read_scale, write_scale;
+    float write_eps;  // write weights below it are dropped (0 with BCT_FLAG_DENSE_WRITE)
 };
 
 struct StSmem {
@@ -238,6 +239,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         // =========================== producer ===========================
         if (lane == 0) {
             uint32_t qn = 0, nw = 0;
+            unsigned long long rows_stored = 0;  // MV rows this CTA has stored back
             uint32_t use[kStMaxStages] = {0, 0, 0, 0};
             auto load_tile = [&](const CUtensorMap* map, int u, int t, int stage) {
                 const uint32_t n = use_at(use, stage)++;
@@ -358,8 +360,10 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         }
                     }
                     bulk_wait_all();  // the next chunk reads these rows again
+                    if (!a.fill) rows_stored += (unsigned long long)a.C;  // every tile of the unit was rebuilt and stored
                 }
             }
+            if (rows_stored > 0) atomicAdd(reinterpret_cast<unsigned long long*>(a.status + kStatusRowsWord), rows_stored);
         }
         __syncwarp();
     } else if (warp == kStRowWarps + 1) {
@@ -610,11 +614,11 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 float lr = 0.f;  // read rows: sum of this thread's numerators
                 // write weights are stored normalised and carry the token's step size:
                 // MV += sum_t eta_t ww_t^T wv_t, and A = Pr WW^T then holds eta_t as well
-                float wmul = 1.f;
+                float winv = 1.f, weta = 1.f;
                 if (is_write && !a.fill) {
-                    wmul = 1.f / l;
+                    winv = 1.f / l;
                     // (a ragged last chunk of the write-only form has rows past the last token: their Vc rows are zero)
-                    if (a.eta != nullptr && !a.fill && t0 + my_t < a.T) wmul *= a.eta[((size_t)b * a.T + t0 + my_t) * a.Hkv + h];
+                    if (a.eta != nullptr && !a.fill && t0 + my_t < a.T) weta = a.eta[((size_t)b * a.T + t0 + my_t) * a.Hkv + h];
                 }
 
                 // ---- pass 2: numerators of each tile, then the write-back of its MV rows.  The numerators of
@@ -639,8 +643,12 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         for (int i = 0; i < 32; ++i) e[i] = (i < n_valid) ? ex2(fmaf(e[i], c2, -m)) : 0.f;
                     }
                     if (is_write) {
+                        // ww_j below write_eps: the slot keeps its row (and a read that follows the write sees none of it)
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) e[i] *= wmul;
+                        for (int i = 0; i < 32; ++i) {
+                            const float ww = e[i] * winv;
+                            e[i] = ww >= a.write_eps ? ww * weta : 0.f;
+                        }
                     } else {
                         float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
@@ -927,6 +935,7 @@ int launch_stream_tc(const bct_cache* c, const void* q, const void* k, const voi
     a.precise = (p.flags & BCT_FLAG_PRECISE_READ) ? 1 : 0;
     a.read_scale = p.read_scale;
     a.write_scale = p.write_scale;
+    a.write_eps = (p.flags & BCT_FLAG_DENSE_WRITE) ? 0.f : p.write_eps;
     const int smem = st_smem(a.precise, Tc > kStMaxTc).total;
     *err = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (*err != cudaSuccess) return -1;

@@ -36,8 +36,11 @@ def _unit_slices(w, units, q, k, v):
     return qs, ks, vs
 
 
-def make_pair(w: W.Workload, units, device="cuda", flags=0, oracle_flags=0, write_eps=0.0, max_stream=1):
-    """(gpu cache, oracle cache over `units`) from the workload's seeded initial state."""
+def make_pair(w: W.Workload, units, device="cuda", flags=0, oracle_flags=0, write_eps=0.0, max_stream=1,
+              oracle_write_eps=0.0):
+    """(gpu cache, oracle cache over `units`) from the workload's seeded initial state.  write_eps = 0 leaves
+    the library at its default threshold of 2^-24, which the oracle's exact rule (oracle_write_eps = 0) is
+    compared with; a test of the threshold itself passes the same value to both."""
     mk = mv = None
     ok = ov = None
     if w.init_len:
@@ -51,7 +54,7 @@ def make_pair(w: W.Workload, units, device="cuda", flags=0, oracle_flags=0, writ
     del mk, mv
     ora = O.OracleCache(len(units), w.group, 1, w.head_dim, w.capacity, read_scale=w.read_scale,
                         write_scale=w.write_scale, init_len=w.init_len, mk_init=ok, mv_init=ov,
-                        flags=oracle_flags)
+                        flags=oracle_flags, write_eps=oracle_write_eps)
     return gpu, ora
 
 

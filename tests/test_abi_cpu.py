@@ -90,3 +90,26 @@ def test_null_arguments_rejected(lib):
     assert lib.bct_cache_create(ctypes.byref(p), 256, 16, None, None, None, ctypes.byref(h)) == B.BCT_ERR_INVALID_ARG
     assert lib.bct_cache_create(ctypes.byref(p), 264, 1 << 20, None, None, None, ctypes.byref(h)) == B.BCT_ERR_INVALID_ARG
     assert not h.value
+
+
+def test_a_pointer_that_is_no_live_handle_is_refused_without_being_read(lib):
+    # the library looks a handle up in its list of live handles before touching it: an address that was never a
+    # handle (here: not even mapped) is answered with BCT_ERR_STATE
+    bogus = ctypes.c_void_p(0x1000)
+    n = ctypes.c_int32(0)
+    assert lib.bct_cache_len(bogus, ctypes.byref(n)) == B.BCT_ERR_STATE
+    assert lib.bct_cache_destroy(bogus) == B.BCT_ERR_STATE
+    assert lib.bct_decode_step(bogus, 256, 256, 256, 256, None) == B.BCT_ERR_STATE
+    assert lib.bct_prefill_stream_host_static(bogus, 256, 256, 256, 256, 1, None) == B.BCT_ERR_STATE
+    assert lib.bct_selftest_timeout(bogus, None) == B.BCT_ERR_STATE
+    r = ctypes.c_uint64(0)
+    assert lib.bct_cache_rows_rewritten(bogus, None, ctypes.byref(r)) == B.BCT_ERR_STATE
+    assert "destroyed" in B.last_error()
+
+
+def test_no_environment_variable_is_read():
+    # the library and its binding take every setting through arguments
+    assert "environ" not in open(os.path.join(ROOT, "paper_2411_15785_b200", "binding.py")).read()
+    csrc = os.path.join(ROOT, "paper_2411_15785_b200", "csrc")
+    for name in os.listdir(csrc):
+        assert "getenv" not in open(os.path.join(csrc, name)).read(), name

@@ -34,7 +34,17 @@ def test_default_workload_line_has_the_contract_keys():
     assert e["value"] > 0 and e["h2d_bytes_per_step"] > 0 and e["d2h_bytes_per_step"] > 0 and e["value"] < d["value"] * 1.05
     r = d["roofline"]
     assert r["bound"] == "hbm" and r["unit"] == "GB/s" and r["kernel"] == "decode_tc_kernel"
-    assert abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9 and r["traffic"] > 0
+    assert abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9 and "traffic" in r
+    # the rows the update rule rewrote, counted by the kernel, are part of the algorithmic bytes
+    assert 0 < r["rows_rewritten_fraction"] < 0.2
+    planes = 4 * 32 * 2048 * 128 * 2
+    assert r["algorithmic_bytes_per_launch"] > 2 * planes
+    p = d["parity"]                                 # the timed launch configuration replayed beside the oracle
+    assert p["pass"] and p["max_abs_out_per_step"] <= p["tol"] == 2e-2 and p["max_abs_state_final"] <= p["tol"]
+    assert p["units_checked"] >= 8 and p["steps"] >= 20
+    rep = d["repeats"]
+    assert rep["blocks"] == 5 and rep["min_ms_per_step"] <= rep["median_ms_per_step"] <= rep["max_ms_per_step"]
+    assert d["paper_context"]["hardware"] == "not stated"
     sec = d["secondary_write_regime"]               # the diffuse write regime, timed on a second cache
     assert sec["ms_per_step"] > d["ms_per_step"] and 0 < sec["frac"] < 1.2 and abs(sec["write_scale"] - 128 ** -0.5) < 1e-9
 
@@ -44,3 +54,6 @@ def test_stream_workload_line_reports_the_tensor_roofline():
     r = d["roofline"]
     assert r["bound"] == "tensor" and r["unit"] == "TFLOP/s" and r["kernel"] == "stream_tc_kernel"
     assert d["config"]["tokens_per_step"] == 256 and d["gpu_launches"] == 20
+    assert d["config"]["flags"] == 24               # the flags at which the full-length stream holds 2e-2
+    assert 0 < r["frac"] < r["frac_executed"] < 1.2  # on the method's flops, and on the flops the MMAs execute
+    assert d["parity"]["pass"] and d["parity"]["steps"] == 1024 + 512

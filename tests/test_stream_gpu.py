@@ -20,9 +20,9 @@ def _built():
     B.load()
 
 
-def _stream_parity(w, T, pieces, flags=0, oracle_flags=0, want_out=True):
+def _stream_parity(w, T, pieces, flags=0, oracle_flags=0, want_out=True, write_eps=0.0):
     units = pick_units(w, 8)
-    gpu, ora = make_pair(w, units, flags=flags, oracle_flags=oracle_flags)
+    gpu, ora = make_pair(w, units, flags=flags, oracle_flags=oracle_flags, write_eps=write_eps, oracle_write_eps=write_eps)
     q, k, v = W.stream_inputs(w, 0, T, "cuda")
     launches0 = gpu.launches
     outs, t = [], 0
@@ -149,3 +149,33 @@ def test_ragged_ends_go_in_short_chunks(G, C, init_len, T, max_launches):
     err, state, n_launch = _stream_parity(w, T, [T])
     assert err <= TOL["bf16"] and state <= TOL["bf16"], (err, state)
     assert n_launch <= max_launches + 1, n_launch   # + the export launch of the state comparison
+
+
+@pytest.mark.parametrize("flags,oflags", [(0, 0), (B.FLAG_WRITE_THEN_READ, O.WRITE_THEN_READ)])
+def test_write_threshold_is_the_same_in_chunks_and_in_decode_steps(flags, oflags):
+    # a caller-chosen write_eps drops the same slots whether the tokens go through the chunked kernel, the
+    # write-only chunks or one decode step each; all three against the oracle with the same threshold
+    d, eps, T = 128, 1e-3, 150
+    w = W.Workload("t", 3, 4, 2, d, 384, "bf16", 384, T, 71, d ** -0.5, 1.0, 1.0, "stream", 1.0, 0.35)
+    err, state, _ = _stream_parity(w, T, [T], flags=flags, oracle_flags=oflags, write_eps=eps)
+    assert err <= TOL["bf16"] and state <= TOL["bf16"], (err, state)
+    units = pick_units(w, 8)
+    chunks, ora = make_pair(w, units, flags=flags, oracle_flags=oflags, write_eps=eps, oracle_write_eps=eps)
+    steps, exact = make_pair(w, units, flags=flags, oracle_flags=oflags, write_eps=eps, oracle_write_eps=0.0)
+    wonly, _ = make_pair(w, units, flags=flags, write_eps=eps)
+    q, k, v = W.stream_inputs(w, 0, T, "cuda")
+    chunks.prefill_stream(q, k, v)
+    for t in range(T):
+        steps.decode_step(q[:, t].contiguous(), k[:, t].contiguous(), v[:, t].contiguous())
+    wonly.update_kv(k, v)
+    qs, ks, vs = _unit_slices(w, units, q, k, v)
+    ora.prefill_stream(qs, ks, vs)
+    exact.prefill_stream(qs, ks, vs)
+    # the threshold matters at this write scale: the exact rule's state is measurably different
+    assert float(np.abs(ora.MV - exact.MV).max()) > 8e-3
+    for gpu in (chunks, steps, wonly):
+        gpu.check_status()
+        # (a weight within rounding of the threshold may fall either way in fp32: one such slot moves an element by
+        # about eps * |v|, so the bar sits between that and the distance to the exact rule)
+        assert compare_state(w, units, gpu, ora) <= 6e-3
+        gpu.destroy()

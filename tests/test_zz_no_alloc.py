@@ -49,11 +49,14 @@ def test_static_staging_matches_workspace_staging_on_two_calls_in_a_row():
         assert torch.isfinite(out_sta.float()).all()
         err = (out_sta.float() - out_ref.float()).abs().max().item()
         assert err <= TOL_BF16, (call, err)
+        # the same kernels on the same inputs, only staged elsewhere: the results agree bit for bit
+        assert torch.equal(out_sta, out_ref), call
     ref.check_status()
     sta.check_status()
     assert ref.len == sta.len == w.capacity
     for a, b in zip(ref.export(torch.float32), sta.export(torch.float32)):
         assert (a.float() - b.float()).abs().max().item() <= TOL_BF16
+        assert torch.equal(a, b)
 
     # a request that cannot fit the built-in array is refused before anything is enqueued
     n0 = sta.launches
@@ -62,5 +65,9 @@ def test_static_staging_matches_workspace_staging_on_two_calls_in_a_row():
                                                 out_sta.data_ptr(), too_many, None)
     assert st == B.BCT_ERR_INVALID_ARG and "static staging area" in B.last_error()
     assert sta.launches == n0 and sta.len == w.capacity
+    # a token count so large that its byte sizes would wrap is refused the same way
+    st = sta.lib.bct_prefill_stream_host_static(sta._h, hq.data_ptr(), hk.data_ptr(), hv.data_ptr(),
+                                                out_sta.data_ptr(), 1 << 56, None)
+    assert st == B.BCT_ERR_INVALID_ARG and sta.launches == n0
     ref.destroy()
     sta.destroy()
