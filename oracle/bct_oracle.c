@@ -273,3 +273,95 @@ int bct_oracle_project(int64_t M, int64_t K, int64_t N, const double *x, const d
         }
     return used;
 }
+
+/*
+ * Backward of Algorithm 1's procedure UpdateKV in its token-parallel form (Key
+ * Implementation Aspects, "Optimized for Parallelism": MK is never assigned, so every
+ * ww_t depends on MK and wq_t alone and the final state is a plain sum over the tokens):
+ *
+ *     MV_N = MV_0 + sum_t eta_t * ww_t^T . wv_t,   ww_t = softmax(write_scale * wq_t . MK^T)
+ *
+ * Given G = dL/dMV_N for a scalar L, the chain rule through that sum and through the
+ * softmax, token by token (nothing is blocked or reordered):
+ *     r_t      = sum_j ww_tj * G_j                        (what the token's write sees of G)
+ *     dwv_t    = eta_t * r_t
+ *     deta_t   = <wv_t, r_t>
+ *     dww_tj   = eta_t * <wv_t, G_j>
+ *     ds_tj    = ww_tj * (dww_tj - sum_k ww_tk dww_tk)    (softmax Jacobian; the sum is eta_t * deta_t)
+ *     dwq_t    = write_scale * sum_j ds_tj * MK_j
+ *     dMK_j   += write_scale * ds_tj * wq_t               (summed over the tokens)
+ *     dL/dMV_0 = G                                        (the state enters the sum as it is)
+ * With a write threshold (write_eps > 0) the forward drops the slots with ww_tj < write_eps;
+ * the mask is piecewise constant, so it multiplies ww_tj in r_t and dww_tj and nothing else.
+ *
+ * Layouts (row-major, double): MK [U][C][d] (full cache), wq, wv [U][T][d], eta [U][T] or NULL
+ * (ones), G [U][C][d]; outputs dwq, dwv [U][T][d], dMK [U][C][d], deta [U][T] (any may be NULL).
+ * Returns the number of threads used, or -1 on bad arguments / allocation failure.
+ */
+int bct_oracle_update_kv_backward(int64_t U, int64_t T, int d, int64_t C, const double *MK,
+                                  const double *wq, const double *wv, const double *eta,
+                                  const double *G, double write_scale, double write_eps,
+                                  double *dwq, double *dwv, double *dMK, double *deta,
+                                  int nthreads) {
+    if (U < 0 || T < 0 || d < 1 || C < 1 || !MK || !wq || !wv || !G) return -1;
+    int used = 1;
+#ifdef _OPENMP
+    if (nthreads > 0) omp_set_num_threads(nthreads);
+    used = omp_get_max_threads();
+    if (used > U && U > 0) used = (int)U;
+#endif
+    int failed = 0;
+#ifdef _OPENMP
+#pragma omp parallel for schedule(dynamic, 1)
+#endif
+    for (int64_t u = 0; u < U; ++u) {
+        double *s = (double *)malloc(sizeof(double) * (size_t)C);
+        double *ww = (double *)malloc(sizeof(double) * (size_t)C);
+        double *r = (double *)malloc(sizeof(double) * (size_t)d);
+        if (!s || !ww || !r) {
+            failed = 1;
+        } else {
+            const double *mk = MK + u * C * d, *g = G + u * C * d;
+            if (dMK)
+                for (int64_t i = 0; i < C * d; ++i) dMK[u * C * d + i] = 0.0;
+            for (int64_t t = 0; t < T; ++t) {
+                const double *qt = wq + (u * T + t) * d, *vt = wv + (u * T + t) * d;
+                const double et = eta ? eta[u * T + t] : 1.0;
+                for (int64_t j = 0; j < C; ++j) {
+                    double dot = 0.0;
+                    for (int e = 0; e < d; ++e) dot += qt[e] * mk[j * d + e];
+                    s[j] = write_scale * dot;
+                }
+                softmax(s, C, ww);
+                for (int e = 0; e < d; ++e) r[e] = 0.0;
+                for (int64_t j = 0; j < C; ++j) {
+                    if (ww[j] < write_eps) continue;
+                    for (int e = 0; e < d; ++e) r[e] += ww[j] * g[j * d + e];
+                }
+                double de = 0.0;
+                for (int e = 0; e < d; ++e) de += vt[e] * r[e];
+                if (dwv)
+                    for (int e = 0; e < d; ++e) dwv[(u * T + t) * d + e] = et * r[e];
+                if (deta) deta[u * T + t] = de;
+                if (dwq)
+                    for (int e = 0; e < d; ++e) dwq[(u * T + t) * d + e] = 0.0;
+                for (int64_t j = 0; j < C; ++j) {
+                    double dww = 0.0;
+                    if (ww[j] >= write_eps) {
+                        for (int e = 0; e < d; ++e) dww += vt[e] * g[j * d + e];
+                        dww *= et;
+                    }
+                    const double ds = ww[j] * (dww - et * de);
+                    if (dwq)
+                        for (int e = 0; e < d; ++e) dwq[(u * T + t) * d + e] += write_scale * ds * mk[j * d + e];
+                    if (dMK)
+                        for (int e = 0; e < d; ++e) dMK[(u * C + j) * d + e] += write_scale * ds * qt[e];
+                }
+            }
+        }
+        free(s);
+        free(ww);
+        free(r);
+    }
+    return failed ? -1 : used;
+}

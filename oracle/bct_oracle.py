@@ -71,6 +71,10 @@ def _load():
             ctypes.c_int64, ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.c_int64,
             ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64),
             dp, dp, dp, dp, dp, dp, dp, ctypes.c_double, ctypes.c_double, ctypes.c_double, ctypes.c_uint, ctypes.c_int]
+        lib.bct_oracle_update_kv_backward.restype = ctypes.c_int
+        lib.bct_oracle_update_kv_backward.argtypes = [
+            ctypes.c_int64, ctypes.c_int64, ctypes.c_int, ctypes.c_int64, dp, dp, dp, dp, dp, ctypes.c_double,
+            ctypes.c_double, dp, dp, dp, dp, ctypes.c_int]
         lib.bct_oracle_project.restype = ctypes.c_int
         lib.bct_oracle_project.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, dp, dp, dp, ctypes.c_int]
         lib.bct_oracle_write_weights.restype = ctypes.c_int
@@ -150,6 +154,34 @@ def layer_step_inputs(x, Wq, Wwq, Wwv, n_q_heads, n_kv_heads, head_dim, bf16: bo
     k = rnd(project(x, Wwq)).reshape(B, T, n_kv_heads, head_dim)
     v = rnd(project(x, Wwv)).reshape(B, T, n_kv_heads, head_dim)
     return q, k, v
+
+
+def update_kv_backward(MK, wq, wv, dMV, eta=None, write_scale: float = 1.0, write_eps: float = 0.0, nthreads: int = 0):
+    """Backward of Algorithm 1's UpdateKV (token-parallel form): MK ``[B, Hkv, C, d]`` (full cache), wq, wv
+    ``[B, T, Hkv, d]``, eta ``[B, T, Hkv]`` or None, dMV = dL/dMV_N ``[B, Hkv, C, d]``.  Returns
+    (dwq, dwv ``[B, T, Hkv, d]``, dMK ``[B, Hkv, C, d]``, deta ``[B, T, Hkv]``); dL/dMV_0 is dMV itself."""
+    MK, wq, wv, dMV = _f64(MK), _f64(wq), _f64(wv), _f64(dMV)
+    B, Hkv, C, d = MK.shape
+    T = wq.shape[1]
+    assert wq.shape == (B, T, Hkv, d) and wv.shape == (B, T, Hkv, d) and dMV.shape == (B, Hkv, C, d)
+    U = B * Hkv
+    qu = np.ascontiguousarray(wq.transpose(0, 2, 1, 3)).reshape(U, T, d)
+    vu = np.ascontiguousarray(wv.transpose(0, 2, 1, 3)).reshape(U, T, d)
+    eu = None
+    if eta is not None:
+        eta = _f64(eta)
+        assert eta.shape == (B, T, Hkv), eta.shape
+        eu = np.ascontiguousarray(eta.transpose(0, 2, 1)).reshape(U, T)
+    dq, dv = np.empty((U, T, d)), np.empty((U, T, d))
+    dmk, de = np.empty((U, C, d)), np.empty((U, T))
+    rc = _load().bct_oracle_update_kv_backward(
+        U, T, d, C, _dptr(MK.reshape(U, C, d)), _dptr(qu), _dptr(vu), _dptr(eu) if eu is not None else None,
+        _dptr(dMV.reshape(U, C, d)), float(write_scale), float(write_eps), _dptr(dq), _dptr(dv), _dptr(dmk), _dptr(de),
+        int(nthreads))
+    if rc < 0:
+        raise RuntimeError("bct_oracle_update_kv_backward failed")
+    back = lambda a: np.ascontiguousarray(a.reshape(B, Hkv, T, d).transpose(0, 2, 1, 3))
+    return back(dq), back(dv), dmk.reshape(B, Hkv, C, d), np.ascontiguousarray(de.reshape(B, Hkv, T).transpose(0, 2, 1))
 
 
 class OracleCache:

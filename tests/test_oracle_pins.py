@@ -597,3 +597,114 @@ def test_write_threshold_against_uniform_weights():
     f = O.OracleCache(B, Hq, Hkv, d, C, write_eps=0.9)
     f.prefill_stream(q, _rand(B, T, Hkv, d), v)
     np.testing.assert_array_equal(f.values()[0, 0, :T], v[0, :, 0])
+
+
+# ---------------------------------------------------------------------------------------
+# Backward of UpdateKV in its token-parallel form ("Optimized for Parallelism"): pinned by central
+# finite differences of the forward oracle, by automatic differentiation of the two-matmul form,
+# and by closed forms
+# ---------------------------------------------------------------------------------------
+def _loss_through_forward(mk, mv0, k, v, eta, G, ws, eps=0.0):
+    """L = <G, MV_N> with MV_N from the forward oracle's sequential loop."""
+    B, Hkv, C, d = mk.shape
+    c = O.OracleCache(B, Hkv, Hkv, d, C, init_len=C, mk_init=mk, mv_init=mv0, write_scale=ws, write_eps=eps)
+    c.update_kv(k, v, eta=eta)
+    return float((G * c.values()).sum())
+
+
+def test_update_kv_backward_against_finite_differences_of_the_forward_oracle():
+    B, Hkv, C, d, T, ws = 2, 2, 5, 3, 4, 0.8
+    mk, mv0 = _rand(B, Hkv, C, d), _rand(B, Hkv, C, d)
+    k, v = _rand(B, T, Hkv, d), _rand(B, T, Hkv, d)
+    eta = RNG.uniform(0.3, 1.7, size=(B, T, Hkv))
+    G = _rand(B, Hkv, C, d)
+    dk, dv, dmk, deta = O.update_kv_backward(mk, k, v, G, eta=eta, write_scale=ws)
+    h = 1e-6
+
+    def fd(arr, idx, which):
+        out = []
+        for sgn in (+1, -1):
+            a = arr.copy()
+            a[idx] += sgn * h
+            args = dict(mk=mk, mv0=mv0, k=k, v=v, eta=eta)
+            args[which] = a
+            out.append(_loss_through_forward(args["mk"], args["mv0"], args["k"], args["v"], args["eta"], G, ws))
+        return (out[0] - out[1]) / (2 * h)
+
+    for which, arr, grad in (("k", k, dk), ("v", v, dv), ("mk", mk, dmk), ("eta", eta, deta), ("mv0", mv0, G)):
+        for _ in range(12):
+            idx = tuple(int(RNG.integers(0, n)) for n in arr.shape)
+            assert abs(fd(arr, idx, which) - grad[idx]) <= 2e-8 * (1 + abs(grad[idx])), (which, idx)
+
+
+def test_update_kv_backward_against_autograd_of_the_two_matmul_form():
+    B, Hkv, C, d, T, ws = 1, 3, 7, 4, 6, 1.3
+    mk, k, v, G = _rand(B, Hkv, C, d), _rand(B, T, Hkv, d), _rand(B, T, Hkv, d), _rand(B, Hkv, C, d)
+    eta = RNG.uniform(0.0, 2.0, size=(B, T, Hkv))
+    dk, dv, dmk, deta = O.update_kv_backward(mk, k, v, G, eta=eta, write_scale=ws)
+    tmk, tk, tv, te = (torch.tensor(a, requires_grad=True) for a in (mk, k, v, eta))
+    loss = 0.0
+    for h in range(Hkv):   # MV_N - MV_0 = softmax(ws Kc MK^T)^T diag(eta) Vc, head by head
+        WW = torch.softmax(ws * tk[0, :, h] @ tmk[0, h].T, dim=-1)
+        loss = loss + (torch.tensor(G[0, h]) * (WW.T @ (te[0, :, h, None] * tv[0, :, h]))).sum()
+    loss.backward()
+    for got, ref in ((dk, tk.grad), (dv, tv.grad), (dmk, tmk.grad), (deta, te.grad)):
+        np.testing.assert_allclose(got, ref.numpy(), rtol=0, atol=1e-12)
+
+
+def test_update_kv_backward_closed_forms():
+    B, Hkv, C, d, T = 1, 1, 6, 3, 5
+    mk, v, G = _rand(B, Hkv, C, d), _rand(B, T, Hkv, d), _rand(B, Hkv, C, d)
+    eta = RNG.uniform(0.5, 1.5, size=(B, T, Hkv))
+    # a zero write query writes uniformly: dwv_t = eta_t * mean_j G_j, and dwq_t is the covariance, under the
+    # uniform weights, of <wv_t, G_j> with MK_j
+    k0 = np.zeros((B, T, Hkv, d))
+    dk, dv, dmk, deta = O.update_kv_backward(mk, k0, v, G, eta=eta, write_scale=0.7)
+    gbar = G[0, 0].mean(axis=0)
+    np.testing.assert_allclose(dv[0, :, 0], eta[0, :, 0, None] * gbar[None, :], rtol=0, atol=1e-13)
+    np.testing.assert_allclose(deta[0, :, 0], v[0, :, 0] @ gbar, rtol=0, atol=1e-13)
+    a = v[0, :, 0] @ G[0, 0].T                                  # [T, C]: <wv_t, G_j>
+    cov = ((a - a.mean(axis=1, keepdims=True))[:, :, None] * mk[0, 0][None]).mean(axis=1)
+    np.testing.assert_allclose(dk[0, :, 0], 0.7 * eta[0, :, 0, None] * cov, rtol=0, atol=1e-13)
+    np.testing.assert_allclose(dmk, 0.0, atol=1e-13)           # dMK_j is proportional to the write queries: zero here
+    # a G whose rows are all equal tells the softmax nothing: dwq = 0, dMK = 0, dwv_t = eta_t * that row
+    k = _rand(B, T, Hkv, d)
+    Gc = np.broadcast_to(_rand(d), (B, Hkv, C, d)).copy()
+    dk, dv, dmk, deta = O.update_kv_backward(mk, k, v, Gc, eta=eta, write_scale=1.0)
+    np.testing.assert_allclose(dk, 0.0, atol=1e-13)
+    np.testing.assert_allclose(dmk, 0.0, atol=1e-13)
+    np.testing.assert_allclose(dv[0, :, 0], eta[0, :, 0, None] * Gc[0, 0, 0][None, :], rtol=0, atol=1e-13)
+    # eta = 0 leaves the state alone: only deta survives
+    dk, dv, dmk, deta = O.update_kv_backward(mk, k, v, G, eta=np.zeros((B, T, Hkv)))
+    assert not dk.any() and not dv.any() and not dmk.any() and np.abs(deta).max() > 0
+    # units do not mix, and the gradient is linear in G
+    mk2, k2, v2, G2 = _rand(2, 2, C, d), _rand(2, T, 2, d), _rand(2, T, 2, d), _rand(2, 2, C, d)
+    full = O.update_kv_backward(mk2, k2, v2, G2)
+    one = O.update_kv_backward(mk2[1:, 1:], k2[1:, :, 1:], v2[1:, :, 1:], G2[1:, 1:])
+    np.testing.assert_array_equal(full[0][1:, :, 1:], one[0])
+    np.testing.assert_array_equal(full[2][1:, 1:], one[2])
+    twice = O.update_kv_backward(mk2, k2, v2, 2.0 * G2)
+    for a, b in zip(full, twice):
+        np.testing.assert_allclose(2.0 * a, b, rtol=0, atol=1e-13)
+
+
+def test_update_kv_backward_with_the_write_threshold():
+    # the mask of dropped slots is piecewise constant: away from the threshold the gradient is that of the masked sum
+    B, Hkv, C, d, T, ws, eps = 1, 1, 8, 3, 3, 1.1, 0.07
+    mk, mv0 = _rand(B, Hkv, C, d), _rand(B, Hkv, C, d)
+    k, v, G = _rand(B, T, Hkv, d), _rand(B, T, Hkv, d), _rand(B, Hkv, C, d)
+    WW = _np_softmax(ws * k[0, :, 0] @ mk[0, 0].T)
+    assert (WW < eps).any() and (WW >= eps).any() and np.abs(WW - eps).min() > 1e-3
+    dk, dv, dmk, deta = O.update_kv_backward(mk, k, v, G, write_scale=ws, write_eps=eps)
+    h = 1e-6
+    for which, arr, grad in (("k", k, dk), ("v", v, dv), ("mk", mk, dmk)):
+        for _ in range(10):
+            idx = tuple(int(RNG.integers(0, n)) for n in arr.shape)
+            vals = []
+            for sgn in (+1, -1):
+                a = arr.copy()
+                a[idx] += sgn * h
+                args = dict(mk=mk, k=k, v=v)
+                args[which] = a
+                vals.append(_loss_through_forward(args["mk"], mv0, args["k"], args["v"], None, G, ws, eps))
+            assert abs((vals[0] - vals[1]) / (2 * h) - grad[idx]) <= 2e-8 * (1 + abs(grad[idx])), (which, idx)
