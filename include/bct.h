@@ -200,6 +200,30 @@ bct_status_t bct_update_kv(bct_cache_t *cache, const void *wq, const void *wv, c
                            void *cuda_stream);
 
 /*
+ * Backward of bct_update_kv (Key Implementation Aspects, "Optimized for Parallelism": token-level
+ * parallel training; Algorithm 1 as the forward).  For a scalar loss L and G = dL/dMV_N, with
+ * ww_t = softmax(write_scale * wq_t . MK^T) of the cache's resident MK:
+ *     r_t = sum_j ww_tj G_j      d_wv_t = eta_t r_t      d_eta_t = <wv_t, r_t>
+ *     ds_tj = write_scale * ww_tj * (eta_t <wv_t, G_j> - eta_t d_eta_t)
+ *     d_wq_t = sum_j ds_tj MK_j      d_mk_j = sum_t ds_tj wq_t      dL/dMV_0 = G (not written: it is d_mv)
+ * Slots whose write weight is below write_eps are left out of r_t and of <wv_t, G_j>, as the forward
+ * leaves their increments out.  The cache is read (MK only), not modified, and need not hold the MV_0
+ * of the forward call: the state does not enter the gradients.
+ *   wq, wv  DEVICE bfloat16 [B][T][Hkv][d]   the forward call's inputs
+ *   eta     DEVICE float [B][T][Hkv] or NULL (all ones)
+ *   d_mv    DEVICE bfloat16 [B][Hkv][C][d]   G
+ *   d_wq, d_wv  DEVICE float [B][T][Hkv][d], written
+ *   d_mk    DEVICE float [B][Hkv][C][d], written (zeroed, then summed with atomic adds: the order of the
+ *           additions, hence the last bits, may differ from run to run when T > 128), or NULL
+ *   d_eta   DEVICE float [B][T][Hkv], written, or NULL
+ * bfloat16 operands, fp32 accumulation.  Needs a full cache of the shape the chunked kernels serve
+ * (bfloat16, head_dim 128, 128..16384 slots): BCT_ERR_STATE / BCT_ERR_UNSUPPORTED otherwise.
+ */
+bct_status_t bct_update_kv_backward(bct_cache_t *cache, const void *wq, const void *wv, const float *eta,
+                                    const void *d_mv, int64_t T, float *d_wq, float *d_wv, float *d_mk,
+                                    float *d_eta, void *cuda_stream);
+
+/*
  * The projections in front of the layer (Algorithm 1, first two statements of the loop body:
  * wq_t = W_wq x_t and wv_t = W_wv x_t; the read query q_t = W_q x_t of the attention layer
  * likewise), for a block of tokens, as one tensor-core contraction:
@@ -230,6 +254,24 @@ bct_status_t bct_layer_scratch_bytes(const bct_cache_t *cache, int64_t T, size_t
 bct_status_t bct_layer_forward(bct_cache_t *cache, const void *x, const void *w_q, const void *w_wq,
                                const void *w_wv, int32_t d_model, const float *eta, void *scratch,
                                size_t scratch_bytes, void *out, int64_t T, void *cuda_stream);
+
+/*
+ * A stack of layers (Method, "Model Structure": the mechanism sits in every attention layer of the
+ * decoder): layer 0 reads x, layer l > 0 reads the outputs of layer l - 1 taken as its tokens,
+ * [B][T][Hq * d] of layer l - 1 = [B][T][d_model] of layer l; each layer is one bct_layer_forward on its own
+ * cache.  No residual path, normalisation or feed-forward block is applied between the layers: those are
+ * outside this library.
+ *   caches   HOST array of n_layers handles (bfloat16, the same batch, without BCT_FLAG_OUT_F32)
+ *   w_q, w_wq, w_wv   HOST arrays of n_layers DEVICE pointers: layer l's weights, [Hq_l * d][d_model_l] etc.,
+ *            d_model_0 = d_model, d_model_l = Hq_(l-1) * head_dim
+ *   scratch  DEVICE, 256-byte aligned, at least bct_stack_scratch_bytes bytes
+ *   out      DEVICE [B][T][Hq][d] of the last layer
+ * BCT_ERR_CUDA after the first layers have been enqueued leaves those layers' caches advanced by T tokens.
+ */
+bct_status_t bct_stack_scratch_bytes(bct_cache_t *const *caches, int32_t n_layers, int64_t T, size_t *bytes);
+bct_status_t bct_stack_forward(bct_cache_t *const *caches, int32_t n_layers, const void *x, int32_t d_model,
+                               const void *const *w_q, const void *const *w_wq, const void *const *w_wv,
+                               void *scratch, size_t scratch_bytes, void *out, int64_t T, void *cuda_stream);
 
 /*
  * Host-buffer forms of bct_decode_step and bct_prefill_stream: the same shapes, but q, k, v and out are

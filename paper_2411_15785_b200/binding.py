@@ -25,6 +25,7 @@ EXPORTS = (
     "bct_cache_tensor_path", "bct_prefill_stream_host_static", "bct_decode_step_eta", "bct_prefill_stream_eta",
     "bct_project_qkv", "bct_layer_scratch_bytes", "bct_layer_forward", "bct_update_kv",
     "bct_cache_status_clear", "bct_cache_rows_rewritten", "bct_selftest_timeout",
+    "bct_update_kv_backward", "bct_stack_scratch_bytes", "bct_stack_forward",
 )
 STATIC_STAGE_BYTES = 8 << 20
 
@@ -84,6 +85,10 @@ def load() -> ctypes.CDLL:
     lib.bct_cache_status_clear.argtypes = [vp, vp]
     lib.bct_cache_rows_rewritten.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint64)]
     lib.bct_selftest_timeout.argtypes = [vp, vp]
+    lib.bct_update_kv_backward.argtypes = [vp, vp, vp, vp, vp, i64, vp, vp, vp, vp, vp]
+    lib.bct_stack_scratch_bytes.argtypes = [ctypes.POINTER(vp), i32, i64, ctypes.POINTER(ctypes.c_size_t)]
+    lib.bct_stack_forward.argtypes = [ctypes.POINTER(vp), i32, vp, i32, ctypes.POINTER(vp), ctypes.POINTER(vp),
+                                      ctypes.POINTER(vp), vp, ctypes.c_size_t, vp, i64, vp]
     for name in EXPORTS[2:]:
         getattr(lib, name).restype = ctypes.c_int
     _lib = lib
@@ -156,6 +161,28 @@ def project_qkv(x, w_q, w_wq, w_wv, stream=None, out=None):
     return q, k, v
 
 
+def stack_forward(caches, x, w_q, w_wq, w_wv, out=None, scratch=None, stream=None):
+    """A stack of layers: layer 0 reads x ``[B, T, d_model]``, layer l > 0 the outputs of layer l - 1 as its
+    tokens.  caches: list of Cache; w_q, w_wq, w_wv: lists of that layer's weights.  Returns the last layer's
+    outputs ``[B, T, Hq, d]``."""
+    lib = load()
+    n = len(caches)
+    T = x.shape[1]
+    arr = lambda ptrs: (ctypes.c_void_p * n)(*ptrs)
+    hs = arr([c._h.value for c in caches])
+    need = ctypes.c_size_t(0)
+    _check(lib.bct_stack_scratch_bytes(hs, n, T, ctypes.byref(need)))
+    if scratch is None:
+        scratch = torch.empty(max(need.value, 256), dtype=torch.uint8, device=x.device)
+    last = caches[-1]
+    if out is None:
+        out = torch.empty((last.B, T, last.Hq, last.d), dtype=torch.bfloat16, device=x.device)
+    _check(lib.bct_stack_forward(hs, n, x.data_ptr(), x.shape[2], arr([w.data_ptr() for w in w_q]),
+                                 arr([w.data_ptr() for w in w_wq]), arr([w.data_ptr() for w in w_wv]), scratch.data_ptr(),
+                                 scratch.numel(), out.data_ptr(), T, _stream_ptr(stream)))
+    return out
+
+
 class Cache:
     """A bounded cache over a torch-allocated workspace.  Methods map 1:1 to the C calls."""
 
@@ -219,6 +246,21 @@ class Cache:
         if eta is not None:
             _check_eta(eta, (self.B, T, self.Hkv))
         _check(self.lib.bct_update_kv(self._h, wq.data_ptr(), wv.data_ptr(), _ptr(eta), T, _stream_ptr(stream)))
+
+    def update_kv_backward(self, wq, wv, d_mv, eta=None, want_d_mk=True, want_d_eta=True, stream=None):
+        """Backward of update_kv: d_mv = dL/dMV_N ``[B, Hkv, C, d]`` bfloat16 -> (d_wq, d_wv ``[B, T, Hkv, d]``,
+        d_mk ``[B, Hkv, C, d]`` or None, d_eta ``[B, T, Hkv]`` or None), float32."""
+        T = wq.shape[1]
+        if eta is not None:
+            _check_eta(eta, (self.B, T, self.Hkv))
+        f32 = dict(dtype=torch.float32, device=self.device)
+        d_wq, d_wv = torch.empty(tuple(wq.shape), **f32), torch.empty(tuple(wv.shape), **f32)
+        d_mk = torch.empty((self.B, self.Hkv, self.C, self.d), **f32) if want_d_mk else None
+        d_eta = torch.empty((self.B, T, self.Hkv), **f32) if want_d_eta else None
+        _check(self.lib.bct_update_kv_backward(self._h, wq.data_ptr(), wv.data_ptr(), _ptr(eta), d_mv.data_ptr(), T,
+                                               d_wq.data_ptr(), d_wv.data_ptr(), _ptr(d_mk), _ptr(d_eta),
+                                               _stream_ptr(stream)))
+        return d_wq, d_wv, d_mk, d_eta
 
     def layer_scratch_bytes(self, T: int) -> int:
         n = ctypes.c_size_t(0)

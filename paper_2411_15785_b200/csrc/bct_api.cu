@@ -418,6 +418,30 @@ bct_status_t bct_update_kv(bct_cache_t* c, const void* wq, const void* wv, const
     return write_only_tokens(c, wq, wv, eta, T, 0, static_cast<cudaStream_t>(cuda_stream));
 }
 
+bct_status_t bct_update_kv_backward(bct_cache_t* c, const void* wq, const void* wv, const float* eta, const void* d_mv,
+                                    int64_t T, float* d_wq, float* d_wv, float* d_mk, float* d_eta, void* cuda_stream) {
+    bct_status_t st = check_handle(c);
+    if (st != BCT_OK) return st;
+    if (T < 1 || T > bct::kMaxCallTokens)
+        return fail(BCT_ERR_INVALID_ARG, "T must be in [1, 2^30] (got %lld)", (long long)T);
+    if (!wq || !wv || !d_mv || !d_wq || !d_wv) return fail(BCT_ERR_INVALID_ARG, "wq, wv, d_mv, d_wq and d_wv must not be NULL");
+    if (!aligned16(wq) || !aligned16(wv) || !aligned16(d_mv) || !aligned16(d_wq) || !aligned16(d_wv) || !aligned16(d_mk))
+        return fail(BCT_ERR_INVALID_ARG, "wq, wv, d_mv, d_wq, d_wv and d_mk must be 16-byte aligned");
+    if ((reinterpret_cast<uintptr_t>(eta) & 3u) != 0 || (reinterpret_cast<uintptr_t>(d_eta) & 3u) != 0)
+        return fail(BCT_ERR_INVALID_ARG, "eta and d_eta must be 4-byte aligned");
+    if (c->len != c->p.capacity)
+        return fail(BCT_ERR_STATE, "UpdateKV works on a full-size cache: this one holds %d of %d slots", c->len,
+                    c->p.capacity);
+    if (!bct::update_bwd_supported(c))
+        return fail(BCT_ERR_UNSUPPORTED, "the backward serves bfloat16 caches with head_dim 128 and 128..16384 slots");
+    cudaError_t e = cudaSuccess;
+    const int n = bct::launch_update_bwd(c, wq, wv, eta, d_mv, T, d_wq, d_wv, d_mk, d_eta,
+                                         static_cast<cudaStream_t>(cuda_stream), &e);
+    if (n < 0) return fail_cuda("UpdateKV backward launch", e);
+    c->launches += n;
+    return BCT_OK;
+}
+
 bct_status_t bct_decode_step_eta(bct_cache_t* c, const void* q, const void* k, const void* v, const float* eta,
                                  void* out, void* cuda_stream) {
     if (out == nullptr) return fail(BCT_ERR_INVALID_ARG, "out must not be NULL");
@@ -532,6 +556,81 @@ bct_status_t bct_layer_forward(bct_cache_t* c, const void* x, const void* w_q, c
     if (e != cudaSuccess) return fail_cuda("projection launch", e);
     c->launches += 1;
     return run_tokens(c, q, k, v, eta, out, T, stream);
+}
+
+namespace {
+
+// Validation shared by the two stack calls; fills the per-layer scratch need and the activation size.
+bct_status_t stack_plan(bct_cache_t* const* caches, int32_t n_layers, int64_t T, size_t* layer_scratch, size_t* act_bytes) {
+    if (caches == nullptr || n_layers < 1 || n_layers > 1024)
+        return fail(BCT_ERR_INVALID_ARG, "caches must not be NULL and n_layers must be in [1, 1024]");
+    if (T < 1 || T > bct::kMaxCallTokens) return fail(BCT_ERR_INVALID_ARG, "T must be in [1, 2^30] (got %lld)", (long long)T);
+    *layer_scratch = 0;
+    *act_bytes = 0;
+    for (int l = 0; l < n_layers; ++l) {
+        bct_status_t st = check_handle(caches[l]);
+        if (st != BCT_OK) return st;
+        const bct_params_t& p = caches[l]->p;
+        if (p.dtype != BCT_BF16 || (p.flags & BCT_FLAG_OUT_F32))
+            return fail(BCT_ERR_UNSUPPORTED, "layer %d: a stack needs bfloat16 caches with bfloat16 outputs", l);
+        if (p.batch != caches[0]->p.batch) return fail(BCT_ERR_INVALID_ARG, "layer %d: batch differs from layer 0", l);
+        for (int k = 0; k < l; ++k)
+            if (caches[k] == caches[l]) return fail(BCT_ERR_INVALID_ARG, "layer %d: the same cache twice", l);
+        size_t need = 0;
+        st = bct_layer_scratch_bytes(caches[l], T, &need);
+        if (st != BCT_OK) return st;
+        if (need > *layer_scratch) *layer_scratch = need;
+        const size_t act = round256((size_t)p.batch * (size_t)T * p.n_q_heads * p.head_dim * 2);
+        if (l + 1 < n_layers && act > *act_bytes) *act_bytes = act;
+    }
+    return BCT_OK;
+}
+
+}  // namespace
+
+bct_status_t bct_stack_scratch_bytes(bct_cache_t* const* caches, int32_t n_layers, int64_t T, size_t* bytes) {
+    if (bytes == nullptr) return fail(BCT_ERR_INVALID_ARG, "bytes is NULL");
+    size_t layer_scratch = 0, act = 0;
+    bct_status_t st = stack_plan(caches, n_layers, T, &layer_scratch, &act);
+    if (st != BCT_OK) return st;
+    *bytes = layer_scratch + 2 * act;
+    return BCT_OK;
+}
+
+bct_status_t bct_stack_forward(bct_cache_t* const* caches, int32_t n_layers, const void* x, int32_t d_model,
+                               const void* const* w_q, const void* const* w_wq, const void* const* w_wv, void* scratch,
+                               size_t scratch_bytes, void* out, int64_t T, void* cuda_stream) {
+    size_t layer_scratch = 0, act = 0;
+    bct_status_t st = stack_plan(caches, n_layers, T, &layer_scratch, &act);
+    if (st != BCT_OK) return st;
+    if (x == nullptr || out == nullptr || w_q == nullptr || w_wq == nullptr || w_wv == nullptr)
+        return fail(BCT_ERR_INVALID_ARG, "x, out and the weight arrays must not be NULL");
+    if (scratch == nullptr || (reinterpret_cast<uintptr_t>(scratch) & 255u) != 0 || scratch_bytes < layer_scratch + 2 * act)
+        return fail(BCT_ERR_INVALID_ARG, "scratch must be 256-byte aligned and hold %zu bytes (got %zu)",
+                    layer_scratch + 2 * act, scratch_bytes);
+    // everything the layers would refuse is refused here, before the first of them is enqueued
+    int dm = d_model;
+    for (int l = 0; l < n_layers; ++l) {
+        const bct_params_t& p = caches[l]->p;
+        const int n_q = p.n_q_heads * p.head_dim, n_kv = p.n_kv_heads * p.head_dim;
+        st = check_project_args((int64_t)p.batch * T, dm, n_q, n_kv, x, w_q[l], w_wq[l], w_wv[l], scratch, scratch, scratch);
+        if (st != BCT_OK) return st;
+        if (!caches[l]->tc_ready) return fail(BCT_ERR_UNSUPPORTED, "layer %d: the projections need the driver's tensor-map encoder", l);
+        dm = n_q;
+    }
+    if (!aligned16(out)) return fail(BCT_ERR_INVALID_ARG, "out must be 16-byte aligned");
+    char* base = static_cast<char*>(scratch);
+    char* acts[2] = {base + layer_scratch, base + layer_scratch + act};
+    const void* in = x;
+    dm = d_model;
+    for (int l = 0; l < n_layers; ++l) {
+        void* o = (l + 1 == n_layers) ? out : static_cast<void*>(acts[l & 1]);
+        st = bct_layer_forward(caches[l], in, w_q[l], w_wq[l], w_wv[l], dm, nullptr, base, layer_scratch, o, T, cuda_stream);
+        if (st != BCT_OK) return st;
+        in = o;
+        dm = caches[l]->p.n_q_heads * caches[l]->p.head_dim;
+    }
+    return BCT_OK;
 }
 
 bct_status_t bct_prefill_stream_host(bct_cache_t* c, const void* q, const void* k, const void* v, void* out,

@@ -93,6 +93,13 @@ int launch_stream_tc(const bct_cache* c, const void* q, const void* k, const voi
                      const float* eta, int64_t t_begin, int64_t n_chunks, int fill_len, int write_only, int tc_tokens,
                      cudaStream_t stream, cudaError_t* err);
 
+// Backward of UpdateKV in its token-parallel form (bct_update_bwd.cu): bfloat16 caches, head_dim 128,
+// 128..16384 slots.  wq, wv [B][T][Hkv][128] bfloat16, d_mv = dL/dMV_N [B][Hkv][C][128] bfloat16; outputs float:
+// d_wq, d_wv [B][T][Hkv][128], d_mk [B][Hkv][C][128] (zeroed here, may be NULL), d_eta [B][T][Hkv] (may be NULL).
+bool update_bwd_supported(const bct_cache* c);
+int launch_update_bwd(const bct_cache* c, const void* wq, const void* wv, const float* eta, const void* d_mv, int64_t T,
+                      float* d_wq, float* d_wv, float* d_mk, float* d_eta, cudaStream_t stream, cudaError_t* err);
+
 // The projections in front of the layer (bct_project.cu): q = x W_q^T, k = x W_wq^T, v = x W_wv^T for
 // n_tokens rows of x, bfloat16 throughout; status may be NULL.
 cudaError_t launch_project(long long n_tokens, int d_model, int n_q, int n_kv, const void* x, const void* w_q,
