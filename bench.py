@@ -139,6 +139,15 @@ def stream_chunk_tokens(group: int) -> int:
     return {1: 64, 2: 40, 3: 32, 4: 24}.get(group, 16)
 
 
+def backward_flops(w, tok_per_step):
+    """(executed, algorithmic) flops of one bct_update_kv_backward step: five contractions of 2 T C d per unit
+    (scores, R = WW G, A = Wv G^T, dWq = dS MK, dMK = dS^T Wq); the kernel forms the scores three times and pads
+    the tokens to blocks of 128."""
+    C, d = w.capacity, w.head_dim
+    Tp = (tok_per_step + 127) // 128 * 128
+    return 7 * 2 * Tp * C * d * w.units, 5 * 2 * tok_per_step * C * d * w.units
+
+
 def stream_flops(w, tok_per_step, precise=False, write_only=False):
     """(executed, algorithmic) dense flops of one stream step.  Executed: what stream_tc_kernel's MMAs run
     (operand rows padded to M = 128, two score passes, value + residual products).  Algorithmic: the method's
@@ -163,15 +172,15 @@ def stream_flops(w, tok_per_step, precise=False, write_only=False):
     return executed * n, algorithmic * n
 
 
-def stream_roofline(w, tok_per_step, ms_step, precise=False, write_only=False):
-    """Tensor-core roofline of stream_tc_kernel against the measured sustained bf16 matmul rate: `frac` on the
-    method's own flops, `frac_executed` on the flops the kernel's MMAs run."""
-    executed, algorithmic = stream_flops(w, tok_per_step, precise, write_only)
+def stream_roofline(w, tok_per_step, ms_step, precise=False, write_only=False, backward=False):
+    """Tensor-core roofline of stream_tc_kernel (update_bwd_kernel for the backward) against the measured
+    sustained bf16 matmul rate: `frac` on the method's own flops, `frac_executed` on the flops the kernel's MMAs run."""
+    executed, algorithmic = backward_flops(w, tok_per_step) if backward else stream_flops(w, tok_per_step, precise, write_only)
     pk = _peaks()
     ach = algorithmic / (ms_step * 1e-3) / 1e12
     ach_x = executed / (ms_step * 1e-3) / 1e12
     return {"bound": "tensor", "achieved": ach, "peak": pk["tf"], "unit": "TFLOP/s", "frac": ach / pk["tf"],
-            "traffic": None, "peak_kind": "of " + pk["kind"], "kernel": "stream_tc_kernel",
+            "traffic": None, "peak_kind": "of " + pk["kind"], "kernel": "update_bwd_kernel" if backward else "stream_tc_kernel",
             "flops_per_launch": algorithmic, "executed_flops_per_launch": executed, "achieved_executed": ach_x,
             "frac_executed": ach_x / pk["tf"]}
 
@@ -315,7 +324,9 @@ def secondary_regime(B, w, wr, dev, pool, outs, steps=200):
     token) on a second cache of the same shape: ms per step and the bytes it must move (K and MV value read,
     MV residual read, MV value and residual written), against the copy peak."""
     ws = w.head_dim ** -0.5
-    cache = make_cache(B, w, wr, dev, write_scale=ws)
+    # BCT_FLAG_DENSE_WRITE states what this regime does anyway (no weight is below the threshold at this scale) and
+    # lets the tensor-core kernel rebuild whole tiles in its ring instead of listing and staging single rows
+    cache = make_cache(B, w, wr, dev, write_scale=ws, flags=4)
     rows0 = cache.rows_rewritten()
     ms = timed(lambda i: cache.decode_step(*pool[i % len(pool)], out=outs[i & 1]), steps, 5) / steps
     cache.check_status()
@@ -324,7 +335,7 @@ def secondary_regime(B, w, wr, dev, pool, outs, steps=200):
     return {"write_scale": ws, "steps": steps, "ms_per_step": ms, "value": w.batch / (ms * 1e-3), "unit": UNIT,
             "bytes_per_step": roof["algorithmic_bytes_per_launch"], "achieved": roof["achieved"], "peak": roof["peak"],
             "frac": roof["frac"], "rows_rewritten_fraction": roof["rows_rewritten_fraction"], "kernel": roof["kernel"],
-            "note": "every row rewritten: K, MV value and residual read, MV value and residual written"}
+            "flags": 4, "note": "every row rewritten: K, MV value and residual read, MV value and residual written"}
 
 
 def parity_check(B, w, wr, dev, flags, n_steps, n_units=8, stream_tokens=0):
@@ -541,6 +552,8 @@ def main():
     ap.add_argument("--repeats", type=int, default=5, help="timed blocks of --steps steps (median and spread are reported)")
     ap.add_argument("--update-kv", action="store_true",
                     help="stream workloads: time bct_update_kv (Algorithm 1's UpdateKV, state only) instead of bct_prefill_stream")
+    ap.add_argument("--update-kv-backward", action="store_true",
+                    help="stream workloads: time bct_update_kv_backward (gradients of UpdateKV's token-parallel form)")
     ap.add_argument("--project-tokens", type=int, default=0,
                     help="time bct_project_qkv alone on this many tokens (the workload gives the head counts)")
     ap.add_argument("--d-model", type=int, default=4096, help="model width of the projections")
@@ -549,7 +562,7 @@ def main():
     default_run = (args.workload == "mha7b_b64_c2048" and args.write_scale is None and args.batch is None and
                    args.flags is None and args.write_eps == 0.0)
     if args.flags is None:
-        args.flags = 24 if (w.api == "stream" and not args.update_kv) else 0
+        args.flags = 24 if (w.api == "stream" and not args.update_kv and not args.update_kv_backward) else 0
     if args.write_scale is not None:
         w = w.scaled(write_scale=args.write_scale)
     if args.batch is not None:
@@ -594,10 +607,19 @@ def main():
         pool = [W.step_inputs(wr, t, dev) for t in range(min(args.steps + args.warmup, 64))]
     outs = [torch.empty_like(pool[0][0], dtype=cache.out_dtype) for _ in range(2)]
 
-    update_only = stream and args.update_kv
+    update_only = stream and (args.update_kv or args.update_kv_backward)
+    backward = stream and args.update_kv_backward
+    if backward:   # G = dL/dMV_N and the gradient tensors, allocated once
+        gen = torch.Generator(device=dev).manual_seed(wr.seed + 77)
+        d_mv = torch.randn((w.batch, w.n_kv_heads, w.capacity, w.head_dim), generator=gen, device=dev).to(torch.bfloat16)
+        f32 = dict(dtype=torch.float32, device=dev)
+        grads = (torch.empty(tuple(pool[0][1].shape), **f32), torch.empty(tuple(pool[0][2].shape), **f32),
+                 torch.empty(tuple(d_mv.shape), **f32), torch.empty((w.batch, tok_per_step, w.n_kv_heads), **f32))
 
     def step_dev(i):
-        if update_only:
+        if backward:
+            cache.update_kv_backward(pool[i % len(pool)][1], pool[i % len(pool)][2], d_mv, out=grads)
+        elif update_only:
             cache.update_kv(pool[i % len(pool)][1], pool[i % len(pool)][2])
         elif stream:
             cache.prefill_stream(*pool[i % len(pool)], out=outs[i & 1])
@@ -645,9 +667,14 @@ def main():
     # ---------- end to end through the host-buffer entry point ----------
     hpool = [tuple(x.cpu().pin_memory() for x in pool[i]) for i in range(min(len(pool), 16))]
     hout = [torch.empty_like(hpool[0][0], dtype=cache.out_dtype).pin_memory() for _ in range(2)]
+    hgrad = torch.empty(tuple(grads[0].shape), dtype=torch.float32).pin_memory() if backward else None
 
     def step_host(i):
-        if update_only:   # no host-buffer form of UpdateKV: the stream call without outputs
+        if backward:      # no host-buffer form: inputs up, the call, one gradient tensor down
+            xs = [x.to(dev, non_blocking=True) for x in hpool[i % len(hpool)][1:]]
+            cache.update_kv_backward(xs[0], xs[1], d_mv, out=grads)
+            hgrad.copy_(grads[0], non_blocking=True)
+        elif update_only:   # no host-buffer form of UpdateKV: the stream call without outputs
             cache.prefill_stream_host(*hpool[i % len(hpool)], None)
         elif stream:
             cache.prefill_stream_host(*hpool[i % len(hpool)], hout[i & 1])
@@ -666,7 +693,7 @@ def main():
     ms_e2e = e2.elapsed_time(e3)
     cache.check_status()
     h2d = sum(x.numel() * x.element_size() for x in hpool[0])
-    d2h = 0 if update_only else hout[0].numel() * hout[0].element_size()
+    d2h = hgrad.numel() * 4 if backward else (0 if update_only else hout[0].numel() * hout[0].element_size())
 
     if world > 1:
         ms_total, ms_e2e = max_over_ranks([ms_total, ms_e2e], dev)
@@ -677,7 +704,8 @@ def main():
         ms_step = ms_total / args.steps
         tokens = w.batch * world * args.steps * tok_per_step
         if stream:
-            roof = stream_roofline(w, tok_per_step, ms_step, precise=bool(args.flags & 16), write_only=update_only)
+            roof = stream_roofline(w, tok_per_step, ms_step, precise=bool(args.flags & 16), write_only=update_only,
+                                   backward=backward)
             moved = 3 * w.units * w.capacity * w.head_dim * w.elem_bytes
             l2_note = "cache planes of all units (%.2f GB) exceed L2" % (moved / 1e9)
         else:
@@ -695,7 +723,7 @@ def main():
             l2_note = "cache planes streamed per step (%.2f GB) exceed L2" % (alg / 1e9)
         srt = sorted(rep_ms)
         cfg = config_of(w, tok_per_step)
-        cfg.update({"call": "bct_update_kv" if update_only else ("bct_prefill_stream" if stream else "bct_decode_step"),
+        cfg.update({"call": "bct_update_kv_backward" if backward else "bct_update_kv" if update_only else ("bct_prefill_stream" if stream else "bct_decode_step"),
                     "flags": args.flags, "l2": l2_note,
                     "parallelism": "independent units; replicas per GPU" if world > 1 else "1 GPU"})
         line = {

@@ -247,16 +247,19 @@ class Cache:
             _check_eta(eta, (self.B, T, self.Hkv))
         _check(self.lib.bct_update_kv(self._h, wq.data_ptr(), wv.data_ptr(), _ptr(eta), T, _stream_ptr(stream)))
 
-    def update_kv_backward(self, wq, wv, d_mv, eta=None, want_d_mk=True, want_d_eta=True, stream=None):
+    def update_kv_backward(self, wq, wv, d_mv, eta=None, want_d_mk=True, want_d_eta=True, out=None, stream=None):
         """Backward of update_kv: d_mv = dL/dMV_N ``[B, Hkv, C, d]`` bfloat16 -> (d_wq, d_wv ``[B, T, Hkv, d]``,
-        d_mk ``[B, Hkv, C, d]`` or None, d_eta ``[B, T, Hkv]`` or None), float32."""
+        d_mk ``[B, Hkv, C, d]`` or None, d_eta ``[B, T, Hkv]`` or None), float32.  out: that tuple, to write into."""
         T = wq.shape[1]
         if eta is not None:
             _check_eta(eta, (self.B, T, self.Hkv))
         f32 = dict(dtype=torch.float32, device=self.device)
-        d_wq, d_wv = torch.empty(tuple(wq.shape), **f32), torch.empty(tuple(wv.shape), **f32)
-        d_mk = torch.empty((self.B, self.Hkv, self.C, self.d), **f32) if want_d_mk else None
-        d_eta = torch.empty((self.B, T, self.Hkv), **f32) if want_d_eta else None
+        if out is not None:
+            d_wq, d_wv, d_mk, d_eta = out
+        else:
+            d_wq, d_wv = torch.empty(tuple(wq.shape), **f32), torch.empty(tuple(wv.shape), **f32)
+            d_mk = torch.empty((self.B, self.Hkv, self.C, self.d), **f32) if want_d_mk else None
+            d_eta = torch.empty((self.B, T, self.Hkv), **f32) if want_d_eta else None
         _check(self.lib.bct_update_kv_backward(self._h, wq.data_ptr(), wv.data_ptr(), _ptr(eta), d_mv.data_ptr(), T,
                                                d_wq.data_ptr(), d_wv.data_ptr(), _ptr(d_mk), _ptr(d_eta),
                                                _stream_ptr(stream)))

@@ -71,7 +71,7 @@ struct TcArgs {
 };
 
 struct TcSmem {
-    int ring, pbuf, qbuf, wsm, list, lww, lostage, red, stat, wstat, merge, bars, total;
+    int ring, pbuf, qbuf, wsm, list, lww, lostage, red, stat, vtb, wstat, merge, bars, total;
 };
 __host__ __device__ inline TcSmem tc_smem(int stages, int G, int S, int slice_rows, int lo_cap) {
     const int rows = (slice_rows + kTileRows - 1) / kTileRows * kTileRows;
@@ -97,13 +97,15 @@ __host__ __device__ inline TcSmem tc_smem(int stages, int G, int S, int slice_ro
     off += 4 * 32 * 4;  // per softmax warp: 16 partial maxima / sums, 16 partial appended-slot scores / overlaps
     L.stat = off;  // m[16], l[16], wd[16], ev[16], alpha[16], abort, tmem address, list count
     off += 512;
+    L.vtb = off;   // eta_t * wv_t as floats: the in-ring rewrite of whole tiles reads it as a broadcast
+    off += 128 * 4;
     L.wstat = off;
     off += 2 * kMaxClusterTc * 2 * 4;
     L.merge = off;
     off += (S > 1) ? 2 * (S - 1) * G * (128 + 3) * 4 : 0;
     off = (off + 15) & ~15;
     L.bars = off;
-    off += (2 * stages + 2 * kMaxTiles + 2 + 1 + 2 + 2 + 1) * 8;
+    off += (2 * stages + 3 * kMaxTiles + 2 + 1 + 2 + 2 + 1) * 8;
     L.total = ((off + 127) & ~127) + 1024;  // + slack to align the ring to 1024 bytes
     return L;
 }
@@ -145,7 +147,8 @@ __device__ __forceinline__ void rewrite_chunk(const unsigned char* staged_hi, co
 
 template <int G>
 __global__ void __launch_bounds__(kTcThreads, 1)
-decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const TcArgs a) {
+decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                 const __grid_constant__ CUtensorMap tmLo, const TcArgs a) {
     constexpr int D = 128;
     constexpr int ROW_BYTES = 256;
     constexpr int NR = tc_rows(G);                 // operand rows kept: read heads, write query, zero rows
@@ -185,6 +188,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     uint64_t* xbar = oready + 1;            // [2]
     uint64_t* mbar = xbar + 2;              // [2]
     uint64_t* subfree = mbar + 2;           // the score tiles of a sub-slice have been consumed (128 arrivals)
+    uint64_t* vdone = subfree + 1;          // [kMaxTiles]: the MMAs that read MV tile t are complete (in-ring rewrite only)
+    float* vtb = reinterpret_cast<float*>(smem + L.vtb);
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
@@ -199,6 +204,10 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     const bool has_virtual = (a.len < a.C) && (a.len >= slice_start) && (a.len < slice_start + n_slice);
     const int nt = (n_stream + kTileRows - 1) / kTileRows;   // tiles of the slice
     const int n_sub = (nt + kMaxTiles - 1) / kMaxTiles;       // sub-slices of up to kMaxTiles tiles
+    // Every slot rewritten (BCT_FLAG_DENSE_WRITE) and the slice scored in one go: the residual tiles travel through
+    // the ring behind their value tiles, the softmax warps rebuild both in place once the tile's products are
+    // complete, and the stages go home as TMA stores (no row is read twice, nothing is staged).
+    const bool ring_rewrite = a.dense && a.do_write && n_sub == 1;
 
     if (tid == 0) {
         for (int i = 0; i < NST; ++i) {
@@ -213,6 +222,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         mbar_init(&qready[1], kSThreads);
         mbar_init(oready, 1);
         mbar_init(subfree, kSThreads);
+        for (int i = 0; i < kMaxTiles; ++i) mbar_init(&vdone[i], 1);
         mbar_init(&xbar[0], S);
         mbar_init(&xbar[1], S);
         mbar_init(&mbar[0], kSThreads * (S > 1 ? S - 1 : 1));
@@ -248,7 +258,11 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 for (int ph = 0; ph < 2 * n_sub && ok; ++ph) {  // per sub-slice: its MK tiles, then its MV tiles
                     const CUtensorMap* map = (ph & 1) == 0 ? &tmK : &tmV;
                     const int t_begin = (ph >> 1) * kMaxTiles, t_end = min(nt, t_begin + kMaxTiles);
-                    for (int t = t_begin; t < t_end; ++t) {
+                    // (with the in-ring rewrite every MV tile is followed by its residual tile)
+                    const int per_tile = ((ph & 1) && ring_rewrite) ? 2 : 1;
+                    for (int item = t_begin * per_tile; item < t_end * per_tile && ok; ++item) {
+                        const int t = item / per_tile;
+                        const CUtensorMap* m = (per_tile == 2 && (item & 1)) ? &tmLo : map;
                         if (!first_pass && !mbar_wait_abortable(&empty[stage], rph ^ 1u, abort_flag)) {
                             report_timeout(a.status, 11);
                             *abort_flag = 1;
@@ -257,8 +271,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         }
                         unsigned char* dst = ring + (size_t)stage * kTcTileBytes;
                         mbar_arrive_expect_tx(&full[stage], kTcTileBytes);
-                        tma_load_3d(dst, map, 0, slice_start + t * kTileRows, u, &full[stage]);
-                        tma_load_3d(dst + kHalfBytes, map, 64, slice_start + t * kTileRows, u, &full[stage]);
+                        tma_load_3d(dst, m, 0, slice_start + t * kTileRows, u, &full[stage]);
+                        tma_load_3d(dst + kHalfBytes, m, 64, slice_start + t * kTileRows, u, &full[stage]);
                         if (++stage == NST) {
                             stage = 0;
                             rph ^= 1u;
@@ -335,7 +349,17 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                             const uint64_t bd = desc_at(dk0, paddr + (kk >> 2) * kPHalf + (kk & 3) * 32);
                             umma_bf16(tmem_base + kOCol, ad, bd, idesc_o, (t > 0) || (kk > 0));
                         }
-                        umma_commit(&empty[stage]);
+                        if (ring_rewrite) {
+                            // the softmax warps rebuild the tile in its stage and release it; the residual tile's
+                            // stage is theirs alone
+                            umma_commit(&vdone[t - t_begin]);
+                            if (++stage == NST) {
+                                stage = 0;
+                                rph ^= 1u;
+                            }
+                        } else {
+                            umma_commit(&empty[stage]);
+                        }
                         if (++stage == NST) {
                             stage = 0;
                             rph ^= 1u;
@@ -453,6 +477,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             const float kd = has_virtual ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(a.k + kv_off)[r]) : 0.f;
             const float vd = (has_virtual || (a.wtr && a.do_write))
                                  ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(a.v + kv_off)[r]) : 0.f;
+            const float vd_w = ring_rewrite ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(a.v + kv_off)[r]) : 0.f;
 #pragma unroll
             for (int g = 0; g < G; ++g) {
                 vq[g] = 0.f;
@@ -629,8 +654,59 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 if (tid == 0) *lo_count = 0;
                 s_sync();
             }
+            if (ring_rewrite) {
+                // Every slot is rewritten: tile by tile in the ring stages the value and residual tiles arrived in,
+                // as soon as the products that read the value tile are complete; the stages go home as TMA stores.
+                // Thread r holds row r of the tile; eta_t * wv_t is read from shared memory as a broadcast.
+                vtb[r] = vd_w * eta_u;
+                s_sync();
+                const uint32_t item0 = (uint32_t)it * (3u * (uint32_t)nt) + (uint32_t)nt;  // ring items so far: 3 nt per unit
+                const int sw7 = r & 7;
+                for (int t = 0; t < nt; ++t) {
+                    const uint32_t ih = item0 + 2u * t, il = ih + 1u;
+                    const int sh = (int)(ih % (uint32_t)NST), sl = (int)(il % (uint32_t)NST);
+                    if (!mbar_wait_abortable(&vdone[t], (sp - 1) & 1, abort_flag) ||
+                        !mbar_wait_abortable(&full[sh], (ih / (uint32_t)NST) & 1u, abort_flag) ||
+                        !mbar_wait_abortable(&full[sl], (il / (uint32_t)NST) & 1u, abort_flag)) {
+                        report_timeout(a.status, 24);
+                        *abort_flag = 1;
+                    }
+                    const int row = t * kTileRows + r;
+                    const float ww = (row < n_stream) ? __expf(wsm[row] - st_m[G]) * wfac : 0.f;
+                    unsigned char* th = ring + (size_t)sh * kTcTileBytes + r * 128;
+                    unsigned char* tl = ring + (size_t)sl * kTcTileBytes + r * 128;
+#pragma unroll
+                    for (int hh = 0; hh < 2; ++hh) {
+#pragma unroll 2
+                        for (int c = 0; c < 8; ++c) {
+                            const int off = hh * kHalfBytes + ((c ^ sw7) * 16);
+                            const float4 va = *reinterpret_cast<const float4*>(vtb + hh * 64 + c * 8);
+                            const float4 vb = *reinterpret_cast<const float4*>(vtb + hh * 64 + c * 8 + 4);
+                            const float v8[8] = {va.x, va.y, va.z, va.w, vb.x, vb.y, vb.z, vb.w};
+                            rewrite_chunk(th + off, tl + off, reinterpret_cast<char*>(th + off), reinterpret_cast<char*>(tl + off),
+                                          ww, v8);
+                        }
+                    }
+                    fence_proxy_async_smem();
+                    s_sync();  // the whole tile has been rebuilt
+                    if (tid == 0) {
+                        const int y = slice_start + t * kTileRows;  // rows past C are clipped by the store
+                        unsigned char* bh = ring + (size_t)sh * kTcTileBytes;
+                        unsigned char* bl = ring + (size_t)sl * kTcTileBytes;
+                        tma_store_3d(&tmV, 0, y, u, bh);
+                        tma_store_3d(&tmV, 64, y, u, bh + kHalfBytes);
+                        tma_store_3d(&tmLo, 0, y, u, bl);
+                        tma_store_3d(&tmLo, 64, y, u, bl + kHalfBytes);
+                        bulk_commit();
+                        bulk_wait_read();  // the stages have been read out: they may be refilled
+                        mbar_arrive(&empty[sh]);
+                        mbar_arrive(&empty[sl]);
+                    }
+                }
+                if (tid == 0) rows_stored += (unsigned long long)n_stream;
+            }
             int n_touched = 0;
-            if (a.do_write) {
+            if (a.do_write && !ring_rewrite) {
                 for (int t = 0; t < nt; ++t) {
                     const int row = t * kTileRows + r;
                     const float ww = (row < n_stream) ? __expf(wsm[row] - st_m[G]) * wfac : 0.f;
@@ -766,6 +842,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             if (pend_n == 0 && tid == 0) *lo_count = 0;
         }
         if (pend_n > 0) apply_update(pend_n, pend_off, pend_vt);  // the last unit's rows
+        if (ring_rewrite && tid == 0) bulk_wait_all();              // the last tiles' stores have landed
         if (tid == 0 && rows_stored > 0)
             atomicAdd(reinterpret_cast<unsigned long long*>(a.status + kStatusRowsWord), rows_stored);
     }
@@ -782,7 +859,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     }
 }
 
-using TcKernelFn = void (*)(const CUtensorMap, const CUtensorMap, const TcArgs);
+using TcKernelFn = void (*)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const TcArgs);
 
 TcKernelFn pick_tc(int G) {
     switch (G) {
@@ -977,7 +1054,8 @@ int launch_decode_tc(const bct_cache* c, const StepIO& io, int len, int do_write
     if (n_clusters > c->U) n_clusters = c->U;
     cfg.gridDim = dim3((unsigned)(n_clusters * S), 1, 1);
     *err = cudaLaunchKernelEx(&cfg, fn, *reinterpret_cast<const CUtensorMap*>(c->tmap_k),
-                              *reinterpret_cast<const CUtensorMap*>(c->tmap_v), a);
+                              *reinterpret_cast<const CUtensorMap*>(c->tmap_v),
+                              *reinterpret_cast<const CUtensorMap*>(c->tmap_lo), a);
     if (*err != cudaSuccess) return -1;
     return 1;
 }

@@ -341,3 +341,35 @@ def test_every_unit_tensor_core_kernel_against_cuda_core_kernel(name, steps):
     a.destroy()
     b.destroy()
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("B_,G,C,steps,write_scale,flags,oflags", [
+    (3, 1, 333, 6, 1.0, 0, 0),                                   # ragged last tile: its rows past C are clipped by the store
+    (5, 2, 2048, 5, 128 ** -0.5, 0, 0),                         # 16 tiles: a full slice, diffuse weights
+    (2, 3, 2500, 5, 128 ** -0.5, 0, 0),                         # cluster of 2, ragged
+    (40, 4, 384, 8, 0.3, 0, 0),                                  # more units than one pass of the persistent grid
+    (2, 4, 640, 6, 128 ** -0.5, B.FLAG_WRITE_THEN_READ, O.WRITE_THEN_READ),
+    (2, 1, 4096, 4, 128 ** -0.5, 0, 0),                          # two CTAs of 2048 slots each
+    (1, 2, 8192, 3, 128 ** -0.5, 0, 0),                          # slices beyond one sub-slice: the staged path serves them
+])
+def test_dense_write_rebuilds_whole_tiles(B_, G, C, steps, write_scale, flags, oflags):
+    # BCT_FLAG_DENSE_WRITE on the tensor-core kernel: value and residual tiles are rebuilt in their ring stages and
+    # stored whole; against the oracle's exact rule (every slot updated), with step sizes
+    w = W.Workload("t", B_, 2 * G, 2, 128, C, "bf16", C, steps, 83, 128 ** -0.5, 1.0, 1.0, "decode", 1.0, write_scale)
+    units = pick_units(w, 6)
+    gpu, ora = make_pair(w, units, flags=flags | B.FLAG_DENSE_WRITE, oracle_flags=oflags)
+    assert gpu.tensor_path
+    g = torch.Generator(device="cpu").manual_seed(3)
+    worst = 0.0
+    for t in range(steps):
+        q, k, v = W.step_inputs(w, t, "cuda")
+        eta = (torch.rand((w.batch, w.n_kv_heads), generator=g) * 1.5 + 0.25).cuda()
+        out = gpu.decode_step(q, k, v, eta=eta)
+        qs, ks, vs = _unit_slices(w, units, q, k, v)
+        es = torch.stack([eta[b, h] for b, h in units])[:, None, None].double().cpu().numpy()
+        worst = max(worst, compare_out(w, units, out, ora.prefill_stream(qs, ks, vs, eta=es)))
+    gpu.check_status()
+    assert gpu.rows_rewritten() == w.units * steps * C
+    state = compare_state(w, units, gpu, ora)
+    assert worst <= TOL["bf16"] and state <= TOL["bf16"], (worst, state)
+    gpu.destroy()
