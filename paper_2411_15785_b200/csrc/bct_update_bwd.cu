@@ -17,10 +17,14 @@
 //   pass 1  S = Wq MK_t^T                      -> row maxima and sums
 //   pass 2  S again -> WW_t (bfloat16), R += WW_t G_t
 //   pass 3  S and A_t = Wv G_t^T -> dS_t (bfloat16), dWq += dS_t MK_t, dMK_t = dS_t^T Wq -> atomics
-//   warps 0-3  one thread per token row (= tensor-memory lane): statistics, WW / dS operand, outputs
-//   warp 4     one thread issues the TMA loads (ring of four tile buffers, loaded ahead) and every MMA
-// The roles meet at block-wide barriers; the issuing thread's waits on the TMA and MMA barriers are
-// bounded, a timeout sets the status word and the kernel runs to its end.
+//   warps 0-15  four threads per token row (= tensor-memory lane), 32 accumulator columns each: statistics, the
+//               WW / dS operand, outputs
+//   warp 16     one thread issues the TMA loads (four tile buffers, loaded one tile ahead) and every MMA
+// Software pipeline: the row threads hold the operand of tile t in registers while the products of tile t-1 read
+// the operand buffer, and the scores of the tile after are issued before the products of the current one, so
+// that exponentials and tensor work overlap.  The roles meet at block-wide barriers plus one mbarrier (scores
+// consumed); the issuing thread's waits on the TMA and MMA barriers are bounded, a timeout sets the status word
+// and the kernel runs to its end.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -32,15 +36,16 @@ namespace bct {
 namespace {
 
 constexpr int kBwRows = 128;                 // tokens per block = operand rows = tensor-memory lanes
-constexpr int kBwThreads = kBwRows + 32;     // + the issuing warp
+constexpr int kBwRowThreads = 4 * kBwRows;   // four threads per row
+constexpr int kBwThreads = kBwRowThreads + 32;  // + the issuing warp
 constexpr int kBwTile = 128;                 // slots per tile
 constexpr int kBwHalf = 128 * 128;           // 64 columns (128 bytes) x 128 rows
 constexpr int kBwTileBytes = 2 * kBwHalf;
 constexpr int kBwRing = 4;                   // tile buffers
 constexpr float kBwNegBig = -3.0e38f;
 // tensor-memory columns
-constexpr int kColS = 0;      // scores            [token] x [slot]
-constexpr int kColA = 128;    // A = Wv G_t^T      [token] x [slot]
+constexpr int kColS = 0;      // scores [token] x [slot]; buffer 0 of the scores in passes 1 and 2
+constexpr int kColA = 128;    // A = Wv G_t^T [token] x [slot] in pass 3; buffer 1 of the scores in passes 1 and 2
 constexpr int kColR = 256;    // R (pass 2), then dWq (pass 3)   [token] x [d]
 constexpr int kColM = 384;    // dMK of one tile   [slot] x [d]
 
@@ -66,7 +71,7 @@ __host__ __device__ inline BwSmem bw_smem() {
     off += kBwTileBytes;
     L.wv = off;       // ... and write key-value vectors
     off += kBwTileBytes;
-    L.op = off;       // WW_t (pass 2) / dS_t (pass 3) of one tile, bfloat16, rows = tokens
+    L.op = off;       // WW_t (pass 2) / dS_t (pass 3) of one tile, bfloat16, rows = tokens; between the passes: row statistics
     off += kBwTileBytes;
     L.ring = off;     // MK and G tiles
     off += kBwRing * kBwTileBytes;
@@ -94,10 +99,12 @@ update_bwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     unsigned char* wvb = smem + L.wv;
     unsigned char* opb = smem + L.op;
     unsigned char* ring = smem + L.ring;
-    uint64_t* full = reinterpret_cast<uint64_t*>(smem + L.bars);   // [4] tile landed; [4] the block's operands landed
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + L.bars);   // [4] tile landed; [4]: the block's operands landed
     uint64_t* mma_done = full + 5;                                   // every MMA issued so far is complete
+    uint64_t* sa_free = full + 6;                                    // pass 3: the scores and A of a tile are in registers (512 arrivals)
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L.misc);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L.misc + 8);
+    float* xch = reinterpret_cast<float*>(opb);                      // [4 quarters][128 rows][2]: exchange between the four threads of a row
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
@@ -106,15 +113,17 @@ update_bwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     const int b = u / a.Hkv, h = u - b * a.Hkv;
     const int t0 = blk * kBwRows;
     const int nt = (a.C + kBwTile - 1) / kBwTile;
-    const bool issuer = (tid == kBwRows);
+    const bool issuer = (tid == kBwRowThreads);
+    constexpr int kIssuerWarp = kBwRowThreads / 32;
 
     if (tid == 0) {
         for (int i = 0; i < 5; ++i) mbar_init(&full[i], 1);
         mbar_init(mma_done, 1);
+        mbar_init(sa_free, kBwRowThreads);
         *abort_flag = 0;
         fence_mbar_init_cluster();
     }
-    if (warp == 4) tmem_alloc(tmem_slot, 512);
+    if (warp == kIssuerWarp) tmem_alloc(tmem_slot, 512);
     fence_proxy_async_smem();
     tc_fence_before();
     __syncthreads();
@@ -127,25 +136,17 @@ update_bwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         *abort_flag = 1;                                           \
     }
 
-    // ---- the issuing thread's bookkeeping: items are the tile loads in the order they are used
-    // ---- (pass 1: MK_0 .. MK_nt-1; passes 2 and 3: MK_0, G_0, MK_1, G_1, ...) ----
-    const int n_items = 5 * nt;
-    int issued = 0;      // items whose load has been issued
-    int released = 0;    // items whose buffer is free again (every MMA that reads them is complete)
-    uint32_t n_mma = 0;  // commits waited for so far
-    auto item_load = [&](int item) {
-        const bool is_g = item >= nt && ((item - nt) & 1);
-        const int t = item < nt ? item : ((item - nt) >> 1) % nt;
-        unsigned char* dst = ring + (size_t)(item % kBwRing) * kBwTileBytes;
-        uint64_t* bar = &full[item % kBwRing];
-        mbar_arrive_expect_tx(bar, kBwTileBytes);
-        tma_load_3d(dst, is_g ? &tmG : &tmK, 0, t * kBwTile, u, bar);
-        tma_load_3d(dst + kBwHalf, is_g ? &tmG : &tmK, 64, t * kBwTile, u, bar);
+    // ---- the issuing thread's tools: tile buffers with a use count each (the phase of their barriers) ----
+    uint32_t use[kBwRing] = {0, 0, 0, 0};  // loads issued into each buffer
+    uint32_t n_mma = 0, n_sa = 0;          // commits waited for, score hand-overs waited for
+    auto buf_ptr = [&](int bf) { return ring + (size_t)bf * kBwTileBytes; };
+    auto load_tile = [&](int bf, bool is_g, int t) {   // tile t of MK (or of G) into buffer bf
+        mbar_arrive_expect_tx(&full[bf], kBwTileBytes);
+        tma_load_3d(buf_ptr(bf), is_g ? &tmG : &tmK, 0, t * kBwTile, u, &full[bf]);
+        tma_load_3d(buf_ptr(bf) + kBwHalf, is_g ? &tmG : &tmK, 64, t * kBwTile, u, &full[bf]);
+        ++use[bf];
     };
-    auto top_up = [&]() {  // keep the ring full: an item may be loaded once the item four before it is released
-        while (issued < n_items && issued < released + kBwRing) item_load(issued++);
-    };
-    auto wait_item = [&](int item) { BW_WAIT(&full[item % kBwRing], item / kBwRing, 81); };
+    auto wait_tile = [&](int bf) { BW_WAIT(&full[bf], use[bf] - 1, 81); };  // the buffer's latest load has landed
     auto commit_and_wait = [&]() {
         umma_commit(mma_done);
         BW_WAIT(mma_done, n_mma, 82);
@@ -188,194 +189,285 @@ update_bwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         tma_load_4d(wqb + kBwHalf, &tmWq, 64, h, t0, b, &full[4]);
         tma_load_4d(wvb, &tmWv, 0, h, t0, b, &full[4]);
         tma_load_4d(wvb + kBwHalf, &tmWv, 64, h, t0, b, &full[4]);
-        top_up();
+        for (int t = 0; t < nt && t < kBwRing; ++t) load_tile(t, false, t);  // pass 1: MK_t in buffer t mod 4
         BW_WAIT(&full[4], 0, 80);
     }
 
-    // ---- row threads: this thread's token ----
+    // ---- row threads: thread (r, cq) holds columns [32 cq, 32 cq + 32) of row r of every 128-column accumulator ----
     const int r = tid & 127;
-    const bool is_row = tid < kBwRows;
+    const int cq = (tid >> 7) & 3;
+    const bool is_row = tid < kBwRowThreads;
     const bool row_valid = is_row && (t0 + r < a.T);
-    const uint32_t lane_base = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+    const uint32_t lane_base = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + cq * 32;
     const float c2 = a.write_scale * 1.4426950408889634f;  // exponentials are taken in base 2
     const size_t tok = ((size_t)b * a.T + (size_t)(t0 + r)) * a.Hkv + h;  // this token's row in [B][T][Hkv]
     const float eta = (row_valid && a.eta != nullptr) ? a.eta[tok] : 1.f;
     const int sw = r & 7;  // swizzle phase of this row in the operand buffer
-    // 32 consecutive slots of this row, as bfloat16, into the operand buffer (K-major, 128-byte swizzle)
-    auto store_op32 = [&](int c32, const float* x) {
-        unsigned char* row = opb + (c32 >> 1) * kBwHalf + r * 128;
+    // this thread's 32 slots of its row, as bfloat16, into the operand buffer (K-major, 128-byte swizzle)
+    auto store_op = [&](const float* x) {
+        unsigned char* row = opb + (cq >> 1) * kBwHalf + r * 128;
 #pragma unroll
         for (int j = 0; j < 4; ++j)
-            *reinterpret_cast<uint4*>(row + ((((c32 & 1) * 4 + j) ^ sw) * 16)) = Chunk<__nv_bfloat16>::pack(x + 8 * j);
+            *reinterpret_cast<uint4*>(row + ((((cq & 1) * 4 + j) ^ sw) * 16)) = Chunk<__nv_bfloat16>::pack(x + 8 * j);
     };
 
-    // ---------------- pass 1: maximum and sum of every row's scaled scores ----------------
+    // ---------------- pass 1: maximum and sum of every row's scaled scores (this thread: its 32 columns of every tile) ----
+    // The scores of tile t + 1 are issued while the row threads work on tile t (two score buffers).
     float m = kBwNegBig, l = 0.f;
+    if (issuer && nt > 0) {
+        wait_tile(0);
+        tc_fence_after();
+        mma_kk(kColS, wqb, buf_ptr(0), false);
+        commit_and_wait();
+        if (4 < nt) load_tile(0, false, 4);
+    }
     for (int t = 0; t < nt; ++t) {
-        if (issuer) {
-            wait_item(t);
+        __syncthreads();  // the scores of tile t are complete, and tile t - 1's have been read
+        if (issuer && t + 1 < nt) {
+            const int bf = (t + 1) % kBwRing;
+            wait_tile(bf);
             tc_fence_after();
-            mma_kk(kColS, wqb, ring + (size_t)(t % kBwRing) * kBwTileBytes, false);
+            mma_kk(((t + 1) & 1) ? kColA : kColS, wqb, buf_ptr(bf), false);
             commit_and_wait();
-            released = t + 1;
-            top_up();
+            if (t + 5 < nt) load_tile(bf, false, t + 5);
         }
-        __syncthreads();
         if (is_row) {
             tc_fence_after();
-            const int n_valid = min(kBwTile, a.C - t * kBwTile);
-            float mt = kBwNegBig;
+            const int n_valid = min(kBwTile, a.C - t * kBwTile) - cq * 32;
             float x[32];
-#pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-                tmem_ld32(lane_base + kColS + c * 32, x);
+            tmem_ld32(lane_base + ((t & 1) ? kColA : kColS), x);
+            float mt = kBwNegBig;
 #pragma unroll
-                for (int i = 0; i < 32; ++i) mt = fmaxf(mt, (c * 32 + i < n_valid) ? x[i] * c2 : kBwNegBig);
+            for (int i = 0; i < 32; ++i) {
+                x[i] = (i < n_valid) ? x[i] * c2 : kBwNegBig;
+                mt = fmaxf(mt, x[i]);
             }
             const float mn = fmaxf(m, mt);
-            float s = 0.f;
-#pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-                tmem_ld32(lane_base + kColS + c * 32, x);
+            float s0 = 0.f, s1 = 0.f;
 #pragma unroll
-                for (int i = 0; i < 32; ++i) s += (c * 32 + i < n_valid) ? bw_ex2(fmaf(x[i], c2, -mn)) : 0.f;
+            for (int i = 0; i < 32; i += 2) {
+                s0 += (i < n_valid) ? bw_ex2(x[i] - mn) : 0.f;
+                s1 += (i + 1 < n_valid) ? bw_ex2(x[i + 1] - mn) : 0.f;
             }
-            l = l * bw_ex2(m - mn) + s;
+            l = l * bw_ex2(m - mn) + (s0 + s1);
             m = mn;
             tc_fence_before();
         }
-        __syncthreads();
+    }
+    __syncthreads();
+    // combine the four quarters of every row (through the operand buffer, idle here)
+    if (is_row) {
+        xch[(cq * 128 + r) * 2] = m;
+        xch[(cq * 128 + r) * 2 + 1] = l;
+    }
+    __syncthreads();
+    if (is_row) {
+        float mn = m;
+#pragma unroll
+        for (int o = 1; o < 4; ++o) mn = fmaxf(mn, xch[(((cq + o) & 3) * 128 + r) * 2]);
+        l *= bw_ex2(m - mn);
+#pragma unroll
+        for (int o = 1; o < 4; ++o) {
+            const int idx = (((cq + o) & 3) * 128 + r) * 2;
+            l += xch[idx + 1] * bw_ex2(xch[idx] - mn);
+        }
+        m = mn;
     }
     const float inv_l = 1.f / l;
 
     // ---------------- pass 2: WW_t as an operand, R += WW_t G_t ----------------
-    for (int t = 0; t < nt; ++t) {
-        const int it_k = nt + 2 * t, it_g = it_k + 1;
-        if (issuer) {
-            wait_item(it_k);
-            tc_fence_after();
-            mma_kk(kColS, wqb, ring + (size_t)(it_k % kBwRing) * kBwTileBytes, false);
-            commit_and_wait();       // also: the previous tile's R product has read the operand buffer and its G tile
-            released = it_k + 1;     // every item up to this MK tile has been consumed
-            top_up();
-        }
-        __syncthreads();
-        if (is_row) {
-            tc_fence_after();
-            const int n_valid = min(kBwTile, a.C - t * kBwTile);
-            float x[32];
-#pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-                tmem_ld32(lane_base + kColS + c * 32, x);
+    // MK_t sits in buffer t & 1, G_t in buffer 2 + (t & 1).  Iteration t stores the weights of tile t (held in
+    // registers since the iteration before) and, while R += WW_t G_t and the scores of tile t + 2 run, takes the
+    // weights of tile t + 1 from its scores.
+    float p[32];
+    auto weights_of = [&](int t) {   // normalised, thresholded write weights of tile t, this thread's 32 slots
+        const int n_valid = min(kBwTile, a.C - t * kBwTile) - cq * 32;
+        tmem_ld32(lane_base + ((t & 1) ? kColA : kColS), p);
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    const float ww = (c * 32 + i < n_valid) ? bw_ex2(fmaf(x[i], c2, -m)) * inv_l : 0.f;
-                    x[i] = ww >= a.write_eps ? ww : 0.f;   // a dropped slot's increment does not depend on anything
-                }
-                store_op32(c, x);
-            }
+        for (int i = 0; i < 32; ++i) {
+            const float ww = (i < n_valid) ? bw_ex2(fmaf(p[i], c2, -m)) * inv_l : 0.f;
+            p[i] = ww >= a.write_eps ? ww : 0.f;   // a dropped slot's increment does not depend on anything
+        }
+    };
+    __syncthreads();  // the statistics have been read out of the operand buffer
+    if (issuer && nt > 0) {
+        load_tile(0, false, 0);
+        load_tile(2, true, 0);
+        if (nt > 1) {
+            load_tile(1, false, 1);
+            load_tile(3, true, 1);
+        }
+        wait_tile(0);
+        tc_fence_after();
+        mma_kk(kColS, wqb, buf_ptr(0), false);
+        commit_and_wait();
+        if (nt > 2) load_tile(0, false, 2);
+        if (nt > 1) {
+            wait_tile(1);
+            tc_fence_after();
+            mma_kk(kColA, wqb, buf_ptr(1), false);
+        }
+    }
+    __syncthreads();
+    if (is_row && nt > 0) {
+        tc_fence_after();
+        weights_of(0);
+        tc_fence_before();
+    }
+    for (int t = 0; t < nt; ++t) {
+        if (issuer) {
+            commit_and_wait();  // R of tile t - 1 and the scores of tile t + 1 are complete
+            if (t + 3 < nt) load_tile((t + 1) & 1, false, t + 3);
+            if (t >= 1 && t + 1 < nt) load_tile(2 + ((t + 1) & 1), true, t + 1);
+        }
+        __syncthreads();  // the operand buffer is free
+        if (is_row) {
+            store_op(p);
             fence_proxy_async_smem();
+        }
+        __syncthreads();  // WW_t is in the operand buffer
+        if (issuer) {
+            wait_tile(2 + (t & 1));
+            tc_fence_after();
+            mma_kn(kColR, opb, buf_ptr(2 + (t & 1)), t > 0);
+            if (t + 2 < nt) {
+                wait_tile(t & 1);
+                mma_kk((t & 1) ? kColA : kColS, wqb, buf_ptr(t & 1), false);
+            }
+        }
+        if (is_row && t + 1 < nt) {
+            tc_fence_after();
+            weights_of(t + 1);
             tc_fence_before();
         }
-        __syncthreads();
-        if (issuer) {
-            wait_item(it_g);
-            tc_fence_after();
-            mma_kn(kColR, opb, ring + (size_t)(it_g % kBwRing) * kBwTileBytes, t > 0);
-        }
     }
-    if (issuer) {
-        commit_and_wait();
-        released = 3 * nt;
-        top_up();
-    }
+    if (issuer) commit_and_wait();
     __syncthreads();
     // R_t is complete: dwv_t = eta_t R_t, deta_t = <wv_t, R_t>, delta_t = eta_t deta_t
     float delta = 0.f;
-    if (is_row) {
-        tc_fence_after();
+    {
         float de = 0.f;
-        const __nv_bfloat16* vrow = reinterpret_cast<const __nv_bfloat16*>(a.wv) + tok * 128;
-        float x[32];
-#pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
-            tmem_ld32(lane_base + kColR + c * 32, x);
+        if (is_row) {
+            tc_fence_after();
+            float x[32];
+            tmem_ld32(lane_base + kColR, x);
             if (row_valid) {
+                const __nv_bfloat16* vrow = reinterpret_cast<const __nv_bfloat16*>(a.wv) + tok * 128 + cq * 32;
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     float v8[8];
-                    Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(vrow + c * 32 + j * 8), v8);
+                    Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(vrow + j * 8), v8);
 #pragma unroll
                     for (int i = 0; i < 8; ++i) de = fmaf(v8[i], x[8 * j + i], de);
                 }
-                float4* dst = reinterpret_cast<float4*>(a.d_wv + tok * 128 + c * 32);
+                float4* dst = reinterpret_cast<float4*>(a.d_wv + tok * 128 + cq * 32);
 #pragma unroll
                 for (int j = 0; j < 8; ++j)
                     dst[j] = make_float4(eta * x[4 * j], eta * x[4 * j + 1], eta * x[4 * j + 2], eta * x[4 * j + 3]);
             }
-        }
-        if (row_valid && a.d_eta != nullptr) a.d_eta[tok] = de;
-        delta = eta * de;
-        tc_fence_before();
-    }
-    __syncthreads();
-
-    // ---------------- pass 3: dS_t as an operand, dWq += dS_t MK_t, dMK_t = dS_t^T Wq ----------------
-    // The slot rows of dMK_t leave tensor memory one tile late, while the next tile's products are prepared.
-    auto flush_dmk = [&](int t) {
-        const int slot = t * kBwTile + r;  // this thread's tensor-memory lane is a slot of the tile here
-        float x[32];
-#pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
-            tmem_ld32(lane_base + kColM + c * 32, x);
-            if (slot < a.C && a.d_mk != nullptr) {
-                float4* dst = reinterpret_cast<float4*>(a.d_mk + ((size_t)u * a.C + slot) * 128 + c * 32);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) atomicAdd(dst + j, make_float4(x[4 * j], x[4 * j + 1], x[4 * j + 2], x[4 * j + 3]));
-            }
-        }
-    };
-    for (int t = 0; t < nt; ++t) {
-        const int it_k = 3 * nt + 2 * t, it_g = it_k + 1;
-        if (issuer) {
-            wait_item(it_k);
-            wait_item(it_g);
-            tc_fence_after();
-            mma_kk(kColS, wqb, ring + (size_t)(it_k % kBwRing) * kBwTileBytes, false);
-            mma_kk(kColA, wvb, ring + (size_t)(it_g % kBwRing) * kBwTileBytes, false);
-            commit_and_wait();   // also: the previous tile's dWq and dMK products are complete
-            released = it_k;     // this tile's MK is still to be read by the dWq product; everything before it is free
-            top_up();
+            tc_fence_before();
+            xch[cq * 128 + r] = de;
         }
         __syncthreads();
         if (is_row) {
+            de = (xch[r] + xch[128 + r]) + (xch[256 + r] + xch[384 + r]);
+            if (row_valid && cq == 0 && a.d_eta != nullptr) a.d_eta[tok] = de;
+            delta = eta * de;
+        }
+        __syncthreads();  // the sums have been read out of the operand buffer
+    }
+
+    // ---------------- pass 3: dS_t as an operand, dWq += dS_t MK_t, dMK_t = dS_t^T Wq ----------------
+    // MK_t sits in buffer t mod 3 (it is read twice: by the scores and, a tile later, by the dWq product), G_t in
+    // buffer 3.  Iteration t stores dS_t (held in registers) and flushes dMK of tile t - 1; dS of tile t + 1 is taken
+    // from its scores while the products of tile t run.
+    auto ds_of = [&](int t) {   // dS of tile t, this thread's 32 slots, into p
+        const int n_valid = min(kBwTile, a.C - t * kBwTile) - cq * 32;
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+            float x[16], g[16];
+            tmem_ld16(lane_base + kColS + hh * 16, x);
+            tmem_ld16(lane_base + kColA + hh * 16, g);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const float ww = (hh * 16 + i < n_valid) ? bw_ex2(fmaf(x[i], c2, -m)) * inv_l : 0.f;
+                const float dww = ww >= a.write_eps ? eta * g[i] : 0.f;
+                // the weight as pass 2 rounded it: delta was formed with those, and dww - delta cancels to
+                // the last bits for the slot that holds most of the weight
+                const float wr = __bfloat162float(__float2bfloat16_rn(ww));
+                p[hh * 16 + i] = row_valid ? a.write_scale * wr * (dww - delta) : 0.f;   // rows past the last token add nothing
+            }
+        }
+    };
+    // the slot rows of dMK_t leave tensor memory one tile late (lanes are slots there), as atomic adds: the token
+    // blocks of a unit run on different SMs
+    auto flush_dmk = [&](int t) {
+        const int slot = t * kBwTile + r;
+        float x[32];
+        tmem_ld32(lane_base + kColM, x);
+        if (slot < a.C && a.d_mk != nullptr) {
+            float4* dst = reinterpret_cast<float4*>(a.d_mk + ((size_t)u * a.C + slot) * 128 + cq * 32);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) atomicAdd(dst + j, make_float4(x[4 * j], x[4 * j + 1], x[4 * j + 2], x[4 * j + 3]));
+        }
+    };
+    if (issuer && nt > 0) {
+        load_tile(0, false, 0);
+        load_tile(3, true, 0);
+        if (nt > 1) load_tile(1, false, 1);
+        wait_tile(0);
+        wait_tile(3);
+        tc_fence_after();
+        mma_kk(kColS, wqb, buf_ptr(0), false);
+        mma_kk(kColA, wvb, buf_ptr(3), false);
+        commit_and_wait();
+        if (nt > 1) load_tile(3, true, 1);
+    }
+    __syncthreads();
+    if (is_row && nt > 0) {
+        tc_fence_after();
+        ds_of(0);
+        tc_fence_before();
+        mbar_arrive(sa_free);
+    }
+    for (int t = 0; t < nt; ++t) {
+        if (issuer) {
+            BW_WAIT(sa_free, n_sa, 83);  // the scores and A of tile t are in registers
+            ++n_sa;
+            tc_fence_after();
+            if (t + 1 < nt) {
+                const int bf = (t + 1) % 3;
+                wait_tile(bf);
+                wait_tile(3);
+                tc_fence_after();
+                mma_kk(kColS, wqb, buf_ptr(bf), false);
+                mma_kk(kColA, wvb, buf_ptr(3), false);
+            }
+            commit_and_wait();  // the products of tile t - 1 and the scores and A of tile t + 1 are complete
+            if (t + 2 < nt) {
+                load_tile((t + 2) % 3, false, t + 2);
+                load_tile(3, true, t + 2);
+            }
+        }
+        __syncthreads();  // the operand buffer is free, dMK of tile t - 1 is complete
+        if (is_row) {
             tc_fence_after();
             if (t > 0) flush_dmk(t - 1);
-            const int n_valid = min(kBwTile, a.C - t * kBwTile);
-            float x[32], g[32];
-#pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-                tmem_ld32(lane_base + kColS + c * 32, x);
-                tmem_ld32(lane_base + kColA + c * 32, g);
-#pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    const float ww = (c * 32 + i < n_valid) ? bw_ex2(fmaf(x[i], c2, -m)) * inv_l : 0.f;
-                    const float dww = ww >= a.write_eps ? eta * g[i] : 0.f;
-                    // the weight as pass 2 rounded it: delta was formed with those, and dww - delta cancels to
-                    // the last bits for the slot that holds most of the weight
-                    const float wr = __bfloat162float(__float2bfloat16_rn(ww));
-                    x[i] = row_valid ? a.write_scale * wr * (dww - delta) : 0.f;   // rows past the last token add nothing
-                }
-                store_op32(c, x);
-            }
+            store_op(p);
             fence_proxy_async_smem();
             tc_fence_before();
         }
-        __syncthreads();
+        __syncthreads();  // dS_t is in the operand buffer, dMK of tile t - 1 has left tensor memory
         if (issuer) {
             tc_fence_after();
-            mma_kn(kColR, opb, ring + (size_t)(it_k % kBwRing) * kBwTileBytes, t > 0);
+            mma_kn(kColR, opb, buf_ptr(t % 3), t > 0);
             mma_nn(kColM, opb, wqb);
+        }
+        if (is_row && t + 1 < nt) {
+            tc_fence_after();
+            ds_of(t + 1);
+            tc_fence_before();
+            mbar_arrive(sa_free);
         }
     }
     if (issuer) commit_and_wait();
@@ -385,20 +477,17 @@ update_bwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         if (nt > 0) flush_dmk(nt - 1);
         const bool store = row_valid && !*abort_flag;
         float x[32];
-#pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
-            tmem_ld32(lane_base + kColR + c * 32, x);  // (the whole warp takes part in the load, whatever it stores)
-            if (store) {
-                float4* dst = reinterpret_cast<float4*>(a.d_wq + tok * 128 + c * 32);
+        tmem_ld32(lane_base + kColR, x);  // (the whole warp takes part in the load, whatever it stores)
+        if (store) {
+            float4* dst = reinterpret_cast<float4*>(a.d_wq + tok * 128 + cq * 32);
 #pragma unroll
-                for (int j = 0; j < 8; ++j) dst[j] = make_float4(x[4 * j], x[4 * j + 1], x[4 * j + 2], x[4 * j + 3]);
-            }
+            for (int j = 0; j < 8; ++j) dst[j] = make_float4(x[4 * j], x[4 * j + 1], x[4 * j + 2], x[4 * j + 3]);
         }
         tc_fence_before();
     }
 #undef BW_WAIT
     __syncthreads();
-    if (warp == 4) {
+    if (warp == kIssuerWarp) {
         tc_fence_after();
         tmem_dealloc(tmem_base, 512);
     }
