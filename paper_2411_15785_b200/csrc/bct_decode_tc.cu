@@ -46,8 +46,11 @@ __host__ __device__ constexpr int tc_qbuf_bytes(int G) {  // Q operand: 2 halves
     return 2 * tc_rows(G) * 128 + (tc_rows(G) == 8 ? 1024 : 0);
 }
 constexpr int kScoreCols = 16;                 // tensor-memory columns per score tile (N = 16)
-constexpr int kOCol = kMaxTiles * kScoreCols;  // output accumulator behind the score tiles
-constexpr int kTmemCols = 512;
+constexpr int kSmallTiles = 8;                 // tiles per unit in the two-CTAs-per-SM form (units of up to 1024 slots)
+// The output accumulator sits behind the score tiles; a CTA takes all 512 tensor-memory columns, or 256 in the
+// two-CTAs-per-SM form (an SM has 512: two resident CTAs must share them).
+__host__ __device__ constexpr int tc_ocol(bool small) { return (small ? kSmallTiles : kMaxTiles) * kScoreCols; }
+__host__ __device__ constexpr int tc_tmem_cols(bool small) { return small ? 256 : 512; }
 constexpr int kMaxClusterTc = 8;
 constexpr int kLwwCap = 512;                   // rewritten rows whose weights are kept for the deferred update
 constexpr float kNegBigTc = -3.0e38f;
@@ -145,8 +148,11 @@ __device__ __forceinline__ void rewrite_chunk(const unsigned char* staged_hi, co
     *reinterpret_cast<uint4*>(dst_lo) = Chunk<__nv_bfloat16>::pack(nv);
 }
 
-template <int G>
-__global__ void __launch_bounds__(kTcThreads, 1)
+// kSmall: units of at most kSmallTiles tiles, one CTA per unit, two CTAs resident per SM (half the tensor memory,
+// a two-stage ring each): a unit of a few tiles is a chain of barriers and latencies in the softmax warps, and two
+// CTAs' chains hide each other.
+template <int G, bool kSmall>
+__global__ void __launch_bounds__(kTcThreads, kSmall ? 2 : 1)
 decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                  const __grid_constant__ CUtensorMap tmLo, const TcArgs a) {
     constexpr int D = 128;
@@ -154,6 +160,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     constexpr int NR = tc_rows(G);                 // operand rows kept: read heads, write query, zero rows
     constexpr int kQHalf = NR * 128, kPHalf = NR * 128;  // bytes between the two 64-column halves
     constexpr int kQBufBytes = tc_qbuf_bytes(G), kPTileBytes = tc_ptile_bytes(G);
+    constexpr int kOCol = tc_ocol(kSmall), kTmemCols = tc_tmem_cols(kSmall);
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int S = a.S;
@@ -207,7 +214,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     // Every slot rewritten (BCT_FLAG_DENSE_WRITE) and the slice scored in one go: the residual tiles travel through
     // the ring behind their value tiles, the softmax warps rebuild both in place once the tile's products are
     // complete, and the stages go home as TMA stores (no row is read twice, nothing is staged).
-    const bool ring_rewrite = a.dense && a.do_write && n_sub == 1;
+    const bool ring_rewrite = !kSmall && a.dense && a.do_write && n_sub == 1;
 
     if (tid == 0) {
         for (int i = 0; i < NST; ++i) {
@@ -861,23 +868,35 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 
 using TcKernelFn = void (*)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const TcArgs);
 
-TcKernelFn pick_tc(int G) {
+TcKernelFn pick_tc(int G, bool small) {
+    if (small) {
+        switch (G) {
+            case 1: return decode_tc_kernel<1, true>;
+            case 2: return decode_tc_kernel<2, true>;
+            case 3: return decode_tc_kernel<3, true>;
+            case 4: return decode_tc_kernel<4, true>;
+            case 5: return decode_tc_kernel<5, true>;
+            case 6: return decode_tc_kernel<6, true>;
+            case 7: return decode_tc_kernel<7, true>;
+            default: return nullptr;
+        }
+    }
     switch (G) {
-        case 1: return decode_tc_kernel<1>;
-        case 2: return decode_tc_kernel<2>;
-        case 3: return decode_tc_kernel<3>;
-        case 4: return decode_tc_kernel<4>;
-        case 5: return decode_tc_kernel<5>;
-        case 6: return decode_tc_kernel<6>;
-        case 7: return decode_tc_kernel<7>;
-        case 8: return decode_tc_kernel<8>;
-        case 9: return decode_tc_kernel<9>;
-        case 10: return decode_tc_kernel<10>;
-        case 11: return decode_tc_kernel<11>;
-        case 12: return decode_tc_kernel<12>;
-        case 13: return decode_tc_kernel<13>;
-        case 14: return decode_tc_kernel<14>;
-        case 15: return decode_tc_kernel<15>;
+        case 1: return decode_tc_kernel<1, false>;
+        case 2: return decode_tc_kernel<2, false>;
+        case 3: return decode_tc_kernel<3, false>;
+        case 4: return decode_tc_kernel<4, false>;
+        case 5: return decode_tc_kernel<5, false>;
+        case 6: return decode_tc_kernel<6, false>;
+        case 7: return decode_tc_kernel<7, false>;
+        case 8: return decode_tc_kernel<8, false>;
+        case 9: return decode_tc_kernel<9, false>;
+        case 10: return decode_tc_kernel<10, false>;
+        case 11: return decode_tc_kernel<11, false>;
+        case 12: return decode_tc_kernel<12, false>;
+        case 13: return decode_tc_kernel<13, false>;
+        case 14: return decode_tc_kernel<14, false>;
+        case 15: return decode_tc_kernel<15, false>;
         default: return nullptr;
     }
 }
@@ -936,11 +955,6 @@ bool tc_prepare(bct_cache* c) {
 int launch_decode_tc(const bct_cache* c, const StepIO& io, int len, int do_write, cudaStream_t stream,
                      cudaError_t* err) {
     const bct_params_t& p = c->p;
-    TcKernelFn fn = pick_tc(c->G);
-    if (fn == nullptr) {
-        *err = cudaErrorInvalidConfiguration;
-        return -1;
-    }
     // Cluster size: clusters of 2 tile the whole chip (74 x 2 = 148 SMs), clusters of 4 and 8 only 132
     // and 120 SMs, so a unit is split over at most 2 CTAs and a long slice is taken in sub-slices
     // (up to kMaxSliceRows slots per CTA).  Only when there are too few units to fill the SMs is a unit
@@ -963,6 +977,22 @@ int launch_decode_tc(const bct_cache* c, const StepIO& io, int len, int do_write
     // (A deeper ring for short slices was measured: no gain, the softmax chain of a unit is the limit.)
     int lo_cap = 80;
     int stages = 4;
+    // Units of up to 512 slots (4 tiles), more than two of them per SM: two CTAs per SM with a two-stage ring, staging
+    // rounds of 32 rows and half the tensor memory each.  Such a unit streams in under 1.5 us and its turn in the
+    // softmax warps is a chain of about eight barriers: measured, one CTA per SM left the HBM idle a third of the time.
+    // (The in-ring rewrite of BCT_FLAG_DENSE_WRITE keeps the one-CTA form.)
+    constexpr int kTwoPerSmLimit = 113 * 1024;  // two CTAs and their reserved kilobyte each within an SM's shared memory
+    const bool small = S == 1 && slice <= 4 * kTileRows && c->G <= 7 && c->U > 2 * c->sm_count &&
+                       !(p.flags & BCT_FLAG_DENSE_WRITE) && tc_smem(2, c->G, 1, slice, 32).total <= kTwoPerSmLimit;
+    if (small) {
+        stages = 2;
+        lo_cap = 32;
+    }
+    TcKernelFn fn = pick_tc(c->G, small);
+    if (fn == nullptr) {
+        *err = cudaErrorInvalidConfiguration;
+        return -1;
+    }
     while (tc_smem(stages, c->G, S, slice, lo_cap).total > c->smem_optin && (stages > 3 || lo_cap > 32)) {
         if (stages > 4 || (stages > 3 && lo_cap <= 48))
             --stages;
@@ -1012,13 +1042,18 @@ int launch_decode_tc(const bct_cache* c, const StepIO& io, int len, int do_write
     // (The table is the only state shared between handles: guarded, and held for the launch itself so that
     // two threads cannot interleave the attribute update and the launches that rely on it.)
     static std::mutex seen_mu;
-    static Seen seen[64][16] = {};
+    static Seen seen[64][2][16] = {};
     std::lock_guard<std::mutex> seen_lock(seen_mu);
     Seen local = {};
-    Seen& sn = (c->device >= 0 && c->device < 64) ? seen[c->device][c->G] : local;
+    Seen& sn = (c->device >= 0 && c->device < 64) ? seen[c->device][small ? 1 : 0][c->G] : local;
     if (sn.smem_set < smem) {
         *err = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (*err != cudaSuccess) return -1;
+        if (small) {  // the largest shared-memory carve-out, or the SM would be configured for one CTA of this size
+            *err = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributePreferredSharedMemoryCarveout,
+                                        cudaSharedmemCarveoutMaxShared);
+            if (*err != cudaSuccess) return -1;
+        }
         sn.smem_set = smem;
     }
     cudaLaunchConfig_t cfg = {};
@@ -1051,6 +1086,11 @@ int launch_decode_tc(const bct_cache* c, const StepIO& io, int len, int do_write
         }
         n_clusters = active < n_clusters ? active : n_clusters;
     }
+    // Two CTAs per SM (each takes 256 of the SM's 512 tensor-memory columns and under half its shared memory and
+    // registers).  The occupancy calculator answers 1 for every kernel here that allocates tensor memory, whatever
+    // its registers and shared memory, so it is not asked; measured at C = 256, batch 256 x 8 kv-heads: 0.076 ms per
+    // step with one CTA of this form per SM, 0.059 ms with two, 0.065 ms with three (0.066 ms in the one-CTA form).
+    if (small) n_clusters = 2 * c->sm_count;
     if (n_clusters > c->U) n_clusters = c->U;
     cfg.gridDim = dim3((unsigned)(n_clusters * S), 1, 1);
     *err = cudaLaunchKernelEx(&cfg, fn, *reinterpret_cast<const CUtensorMap*>(c->tmap_k),

@@ -373,3 +373,34 @@ def test_dense_write_rebuilds_whole_tiles(B_, G, C, steps, write_scale, flags, o
     state = compare_state(w, units, gpu, ora)
     assert worst <= TOL["bf16"] and state <= TOL["bf16"], (worst, state)
     gpu.destroy()
+
+
+@pytest.mark.parametrize("B_,G,C,init_len,steps,write_scale,flags,oflags", [
+    (160, 4, 256, 256, 10, 1.0, 0, 0),                # two tiles per unit, 320 units: more than two per SM
+    (170, 1, 300, 290, 16, 1.0, 0, 0),                # ragged capacity; the fill finishes mid-run
+    (150, 7, 512, 512, 6, 0.3, 0, 0),                 # four tiles, 7 read heads, many rows rewritten (several staging rounds)
+    (150, 2, 128, 0, 133, 1.0, 0, 0),                 # starts empty: tile-less units first, then one tile, then soft writes
+    (160, 3, 384, 384, 6, 0.5, B.FLAG_WRITE_THEN_READ, O.WRITE_THEN_READ),
+    (160, 2, 384, 384, 6, 1.0, B.FLAG_SKIP_FIRST_WRITE, O.SKIP_FIRST_WRITE),
+])
+def test_units_of_a_few_tiles_two_ctas_per_sm(B_, G, C, init_len, steps, write_scale, flags, oflags):
+    # bfloat16 units of up to 512 slots with more than two units per SM run as two CTAs per SM (half the tensor
+    # memory and a two-stage ring each); same step, same oracle, with step sizes
+    w = W.Workload("t", B_, 2 * G, 2, 128, C, "bf16", init_len, steps, 89, 128 ** -0.5, 1.0, 1.0, "decode", 1.0, write_scale)
+    assert w.units > 2 * 148
+    units = pick_units(w, 8, seed=5)
+    gpu, ora = make_pair(w, units, flags=flags, oracle_flags=oflags)
+    assert gpu.tensor_path
+    g = torch.Generator(device="cpu").manual_seed(7)
+    worst = 0.0
+    for t in range(steps):
+        q, k, v = W.step_inputs(w, t, "cuda")
+        eta = (torch.rand((w.batch, w.n_kv_heads), generator=g) * 1.5 + 0.25).cuda()
+        out = gpu.decode_step(q, k, v, eta=eta)
+        qs, ks, vs = _unit_slices(w, units, q, k, v)
+        es = torch.stack([eta[b, h] for b, h in units])[:, None, None].double().cpu().numpy()
+        worst = max(worst, compare_out(w, units, out, ora.prefill_stream(qs, ks, vs, eta=es)))
+    gpu.check_status()
+    state = compare_state(w, units, gpu, ora)
+    assert worst <= TOL["bf16"] and state <= TOL["bf16"], (worst, state)
+    gpu.destroy()
