@@ -404,3 +404,51 @@ def test_units_of_a_few_tiles_two_ctas_per_sm(B_, G, C, init_len, steps, write_s
     state = compare_state(w, units, gpu, ora)
     assert worst <= TOL["bf16"] and state <= TOL["bf16"], (worst, state)
     gpu.destroy()
+
+
+def test_largest_capacity_the_tensor_core_kernel_takes():
+    # 65536 slots: a cluster of 8 CTAs with 8192 slots each, four sub-slices per CTA; beyond it the CUDA-core kernel's limits
+    # apply and the create call refuses the shape
+    w = W.Workload("t", 1, 2, 1, 128, 65536, "bf16", 65536, 3, 97, 128 ** -0.5, 1.0, 1.0, "decode")
+    out_err, state_err = run_decode_parity(w, [(0, 0)], expect_tensor_path=True)
+    assert out_err <= TOL["bf16"] and state_err <= TOL["bf16"], (out_err, state_err)
+    prm = B.make_params(1, 2, 1, 128, 65537, torch.bfloat16)
+    need, align = B.cache_bytes(prm)
+    ws = torch.empty(need + align, dtype=torch.uint8, device="cuda")
+    h = ctypes.c_void_p(None)
+    base = (ws.data_ptr() + align - 1) // align * align
+    st = B.load().bct_cache_create(ctypes.byref(prm), base, need, None, None, None, ctypes.byref(h))
+    if st == B.BCT_OK:       # served by the CUDA-core kernel when its score array still fits: then it must be usable
+        assert h.value
+        B.load().bct_cache_destroy(h)
+    else:
+        assert st == B.BCT_ERR_UNSUPPORTED and not h.value
+
+
+def test_two_handles_on_two_streams_are_independent():
+    # different handles share nothing but read-only tables: steps enqueued alternately on two streams give each cache
+    # the results it gives alone
+    w = W.Workload("t", 4, 8, 2, 128, 640, "bf16", 640, 12, 101, 128 ** -0.5, 1.0, 1.0, "decode")
+    units = pick_units(w, 4)
+    solo, _ = make_pair(w, units)
+    a, _ = make_pair(w, units)
+    b, _ = make_pair(w.scaled(seed=202), units)
+    sa, sb = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    outs_solo, outs_a = [], []
+    for t in range(w.steps):
+        q, k, v = W.step_inputs(w, t, "cuda")
+        q2, k2, v2 = W.step_inputs(w.scaled(seed=202), t, "cuda")
+        torch.cuda.synchronize()
+        outs_solo.append(solo.decode_step(q, k, v))
+        with torch.cuda.stream(sa):
+            outs_a.append(a.decode_step(q, k, v, stream=sa))
+        with torch.cuda.stream(sb):
+            b.decode_step(q2, k2, v2, stream=sb)
+    torch.cuda.synchronize()
+    for x, y in zip(outs_solo, outs_a):
+        assert torch.equal(x, y)
+    assert all(torch.equal(x, y) for x, y in zip(solo.export(v_dtype=torch.int32), a.export(v_dtype=torch.int32)))
+    for c in (solo, a, b):
+        c.check_status()
+        c.destroy()
