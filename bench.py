@@ -253,7 +253,7 @@ def run_reference(args, w):
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * w.batch / val, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": config_of(w, 1),
+            "config": config_of(w, args.stream_tokens if w.api == "stream" else 1),
             "cpu_baseline": {"value": val, "unit": UNIT, "cores": smp.cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -261,10 +261,17 @@ def run_reference(args, w):
 
 
 def config_of(w: W.Workload, tok_per_step: int):
-    """The workload's description, the same keys on both arms."""
+    """The workload's description, the same keys and values on both arms (`l2` says why no L2 flush is needed
+    between the GPU arm's timed steps)."""
+    planes = (3 if w.dtype == "bf16" else 2) * w.units * w.capacity * w.head_dim * w.elem_bytes
+    if w.api == "stream":
+        l2 = "cache planes of all units (%.2f GB) exceed L2" % (planes / 1e9)
+    else:
+        l2 = "cache planes streamed per step (%.2f GB of %.2f GB resident) exceed L2" % (
+            2 * w.units * w.capacity * w.head_dim * w.elem_bytes / 1e9, planes / 1e9)
     return {"workload": w.name, "batch_per_gpu": w.batch, "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads,
             "head_dim": w.head_dim, "capacity": w.capacity, "write_scale": w.write_scale, "read_scale": w.read_scale,
-            "tokens_per_step": tok_per_step}
+            "tokens_per_step": tok_per_step, "l2": l2}
 
 
 def make_cache(B, w, wr, dev, flags=0, write_eps=0.0, max_stream=1, write_scale=None):
@@ -706,8 +713,6 @@ def main():
         if stream:
             roof = stream_roofline(w, tok_per_step, ms_step, precise=bool(args.flags & 16), write_only=update_only,
                                    backward=backward)
-            moved = 3 * w.units * w.capacity * w.head_dim * w.elem_bytes
-            l2_note = "cache planes of all units (%.2f GB) exceed L2" % (moved / 1e9)
         else:
             rows = max(0, rows1 - rows0)
             w_frac = rows / float(max(1, w.units * args.steps * w.capacity))
@@ -720,17 +725,16 @@ def main():
                     "algorithmic_bytes_per_launch": alg, "rows_rewritten_fraction": w_frac,
                     "rows_rewritten_per_unit_step": rows / float(max(1, w.units * args.steps)),
                     "frac_of_8TBps_nominal": achieved / 8000.0}
-            l2_note = "cache planes streamed per step (%.2f GB) exceed L2" % (alg / 1e9)
         srt = sorted(rep_ms)
         cfg = config_of(w, tok_per_step)
-        cfg.update({"call": "bct_update_kv_backward" if backward else "bct_update_kv" if update_only else ("bct_prefill_stream" if stream else "bct_decode_step"),
-                    "flags": args.flags, "l2": l2_note,
-                    "parallelism": "independent units; replicas per GPU" if world > 1 else "1 GPU"})
+        run = {"call": "bct_update_kv_backward" if backward else "bct_update_kv" if update_only else (
+                   "bct_prefill_stream" if stream else "bct_decode_step"),
+               "flags": args.flags, "parallelism": "independent units; replicas per GPU" if world > 1 else "1 GPU"}
         line = {
             "metric": METRIC, "value": tokens / (ms_total * 1e-3), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32" if w.dtype == "f32" else "bf16 cache, f32 accumulate",
-            "data": "synthetic", "config": cfg, "clocks": clocks,
+            "data": "synthetic", "config": cfg, "run": run, "clocks": clocks,
             "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.steps},
             "gpu_launches": launches,

@@ -249,6 +249,16 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 tma_load_3d(dst, map, 0, t * kStTile, u, &full[stage]);
                 tma_load_3d(dst + kStHalf, map, 64, t * kStTile, u, &full[stage]);
             };
+            // A cache of a single tile (C <= 128 slots) stays resident in shared memory for all chunks of the launch:
+            // MK keeps stage 0, MV's value and residual tiles keep their stages, where the row threads rebuild them
+            // chunk after chunk.  The loads after the first chunk and the stores before the last one are left out;
+            // the barriers are handed over as if they had happened, so the other roles do not change.
+            const bool resident = !a.fill && nt_full == 1 && a.n_chunks > 1;
+            auto keep_tile = [&](int stage) {   // the stage already holds the tile: complete the barrier's phase without a copy
+                const uint32_t n = use_at(use, stage)++;
+                if (n > 0) ST_WAIT(&empty[stage], n - 1, 37);
+                mbar_arrive(&full[stage]);
+            };
             // read and write queries of chunk ch of unit u into the query operand
             auto load_queries = [&](int u, int ch) {
                 const int b = u / a.Hkv, h = u - b * a.Hkv;
@@ -283,7 +293,10 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     const int n_early = nt < ns - 1 ? nt : ns - 1;
                     int st1 = 0;  // pass-1 stage of the next tile, t mod ns without the division
                     for (int t = 0; t < n_early; ++t) {
-                        load_tile(&tmK, u, t, st1);
+                        if (resident && ch > 0)
+                            keep_tile(st1);
+                        else
+                            load_tile(&tmK, u, t, st1);
                         if (++st1 == ns) st1 = 0;
                     }
                     if (qn == 0) load_queries(u, ch);
@@ -314,7 +327,16 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     // there are two value stages.  The residual stage is stored and refilled first: the next
                     // tile's write-back waits for it.
                     const bool two_vh = ns == kStMaxStages;
-                    if (nt > 0) {
+                    if (nt > 0 && resident) {
+                        keep_tile(0);  // pass 1 left the MK tile in stage 0
+                        if (ch == 0) {
+                            load_tile(&tmVhi, u, 0, st_vh(0));
+                            load_tile(&tmVlo, u, 0, st_vl);
+                        } else {
+                            keep_tile(st_vh(0));
+                            keep_tile(st_vl);
+                        }
+                    } else if (nt > 0) {
                         load_tile(&tmK, u, 0, 0);
                         load_tile(&tmVhi, u, 0, st_vh(0));
                         if (load_vl) load_tile(&tmVlo, u, 0, st_vl);
@@ -326,6 +348,14 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         if (t + 2 < nt) load_tile(&tmK, u, t + 2, 0);
                         if (t == nt - 1) next_queries(u, ch);
                         const int pvh = st_vh(t);
+                        if (resident && ch + 1 < a.n_chunks) {
+                            // the rebuilt tile is the next chunk's MV: nothing goes to HBM yet
+                            ST_WAIT(wready, nw, 33);
+                            ++nw;
+                            mbar_arrive(&empty[st_vl]);
+                            mbar_arrive(&empty[pvh]);
+                            continue;
+                        }
                         if (!a.fill) {
                             ST_WAIT(wready, nw, 33);
                             ++nw;
@@ -360,7 +390,8 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         }
                     }
                     bulk_wait_all();  // the next chunk reads these rows again
-                    if (!a.fill) rows_stored += (unsigned long long)a.C;  // every tile of the unit was rebuilt and stored
+                    // every tile of the unit was rebuilt and stored (a resident tile goes home after the last chunk only)
+                    if (!a.fill && (!resident || ch + 1 == a.n_chunks)) rows_stored += (unsigned long long)a.C;
                 }
             }
             if (rows_stored > 0) atomicAdd(reinterpret_cast<unsigned long long*>(a.status + kStatusRowsWord), rows_stored);

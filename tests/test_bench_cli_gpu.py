@@ -54,6 +54,6 @@ def test_stream_workload_line_reports_the_tensor_roofline():
     r = d["roofline"]
     assert r["bound"] == "tensor" and r["unit"] == "TFLOP/s" and r["kernel"] == "stream_tc_kernel"
     assert d["config"]["tokens_per_step"] == 256 and d["gpu_launches"] == 20
-    assert d["config"]["flags"] == 24               # the flags at which the full-length stream holds 2e-2
+    assert d["run"]["flags"] == 24 and d["run"]["call"] == "bct_prefill_stream"               # the flags at which the full-length stream holds 2e-2
     assert 0 < r["frac"] < r["frac_executed"] < 1.2  # on the method's flops, and on the flops the MMAs execute
     assert d["parity"]["pass"] and d["parity"]["steps"] == 1024 + 512

@@ -179,3 +179,35 @@ def test_write_threshold_is_the_same_in_chunks_and_in_decode_steps(flags, oflags
         # about eps * |v|, so the bar sits between that and the distance to the exact rule)
         assert compare_state(w, units, gpu, ora) <= 6e-3
         gpu.destroy()
+
+
+@pytest.mark.parametrize("B_,G,T,pieces,flags,oflags", [
+    (4, 1, 256, [256], 0, 0),                                         # four chunks of 64 on a resident tile
+    (80, 1, 200, [200], 0, 0),                                        # 160 units on 148 CTAs: a CTA takes a second unit after a resident one
+    (4, 2, 250, [120, 130], B.FLAG_PRECISE_READ | B.FLAG_OUT_F32, 0),  # two calls, chunks of 40, value + residual read
+    (4, 4, 100, [100], B.FLAG_WRITE_THEN_READ, O.WRITE_THEN_READ),
+])
+def test_single_tile_cache_stays_resident_across_chunks(B_, G, T, pieces, flags, oflags):
+    # C = 128: the unit's one tile of MK and of MV (value + residual) stays in shared memory for all chunks of a call;
+    # only the first chunk loads it and only the last one stores it
+    d = 128
+    w = W.Workload("t", B_, 2 * G, 2, d, 128, "bf16", 128, T, 73, d ** -0.5, 1.0, 1.0, "stream", 1.0, 0.5)
+    err, state, n_launch = _stream_parity(w, T, pieces, flags=flags, oracle_flags=oflags)
+    tol = 2e-3 if flags & B.FLAG_PRECISE_READ else TOL["bf16"]
+    assert err <= tol and state <= TOL["bf16"], (err, state)
+    assert n_launch <= 3 * len(pieces) + 1
+
+
+def test_single_tile_cache_resident_in_update_kv_and_counts_its_stores():
+    d, T = 128, 384
+    w = W.Workload("t", 8, 2, 2, d, 128, "bf16", 128, T, 79, d ** -0.5, 1.0, 1.0, "stream", 1.0, 0.5)
+    units = pick_units(w, 6)
+    gpu, ora = make_pair(w, units)
+    q, k, v = W.stream_inputs(w, 0, T, "cuda")
+    gpu.update_kv(k, v)            # three chunks of 128 write rows
+    gpu.check_status()
+    _, ks, vs = _unit_slices(w, units, q, k, v)
+    ora.update_kv(ks, vs)
+    assert compare_state(w, units, gpu, ora) <= TOL["bf16"]
+    assert gpu.rows_rewritten() == w.units * 128      # one store of the tile per unit, after the last chunk
+    gpu.destroy()
