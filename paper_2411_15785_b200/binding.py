@@ -189,7 +189,7 @@ class Cache:
     def __init__(self, batch, n_q_heads, n_kv_heads, head_dim, capacity, dtype=torch.bfloat16, *,
                  read_scale=0.0, write_scale=0.0, init_len=0, flags=0, write_eps=0.0, max_stream=1,
                  mk_init: Optional[torch.Tensor] = None, mv_init: Optional[torch.Tensor] = None,
-                 device="cuda", stream=None):
+                 device="cuda", stream=None, guard_bytes: int = 0):
         self.lib = load()
         self.params = make_params(batch, n_q_heads, n_kv_heads, head_dim, capacity, dtype,
                                   read_scale=read_scale, write_scale=write_scale, init_len=init_len,
@@ -199,10 +199,14 @@ class Cache:
         self.device = torch.device(device)
         self.B, self.Hq, self.Hkv, self.d, self.C = batch, n_q_heads, n_kv_heads, head_dim, capacity
         nbytes, align = cache_bytes(self.params)
-        self.workspace = torch.empty(nbytes + align, dtype=torch.uint8, device=self.device)
+        # guard_bytes > 0 (tests): a band of 0xA5 bytes on either side of the workspace, checked by check_guards()
+        self._guard = (int(guard_bytes) + align - 1) // align * align
+        self.workspace = torch.empty(nbytes + align + 2 * self._guard, dtype=torch.uint8, device=self.device)
         base = self.workspace.data_ptr()
-        self._ws_ptr = (base + align - 1) // align * align
+        self._ws_ptr = (base + align - 1) // align * align + self._guard
         self.workspace_bytes = nbytes
+        if self._guard:
+            self.workspace.fill_(0xA5)
         for t, name in ((mk_init, "mk_init"), (mv_init, "mv_init")):
             if t is not None:
                 assert t.is_cuda and t.is_contiguous() and t.dtype == dtype, name
@@ -330,6 +334,17 @@ class Cache:
     def import_state(self, k, v, length, stream=None):
         vd = _dtype_code(v.dtype) if v is not None else _dtype_code(self.dtype)
         _check(self.lib.bct_cache_import(self._h, _ptr(k), _ptr(v), vd, length, _stream_ptr(stream)))
+
+    def check_guards(self) -> None:
+        """Raise if anything wrote outside the workspace (needs guard_bytes > 0 at construction)."""
+        if not self._guard:
+            return
+        torch.cuda.synchronize(self.device)
+        lo = self._ws_ptr - self.workspace.data_ptr()
+        hi = lo + self.workspace_bytes
+        for name, band in (("below", self.workspace[lo - self._guard:lo]), ("above", self.workspace[hi:hi + self._guard])):
+            if not bool((band == 0xA5).all()):
+                raise AssertionError("guard band %s the workspace was overwritten" % name)
 
     def status(self, stream=None) -> int:
         return self.lib.bct_cache_status(self._h, _stream_ptr(stream))

@@ -1,8 +1,7 @@
 // The projections in front of the bounded-cache layer on the sm_100a tensor path.
 //
-// Algorithm 1 starts every token with two products, wq_t = W_wq x_t ("Compute write query") and
-// wv_t = W_wv x_t ("Compute write key-value vector"); the read query of the attention layer is a
-// third product of the same token.  For a block of tokens they are one contraction
+// Algorithm 1 starts every token with two products, wq_t = W_wq x_t and wv_t = W_wv x_t (the first two
+// statements of its loop body); the read query of the attention layer is a third product of the same token.  For a block of tokens they are one contraction
 //     [q | k | v][m][n] = sum_c x[m][c] * W[n][c]        W = W_q, W_wq, W_wv stacked over n
 // with bfloat16 operands, fp32 accumulation in tensor memory and bfloat16 results, written straight
 // into the three step-vector arrays the layer reads.

@@ -49,7 +49,7 @@ def make_pair(w: W.Workload, units, device="cuda", flags=0, oracle_flags=0, writ
         ov = torch.stack([mv[b, h] for b, h in units])[:, None].double().cpu().numpy()
     gpu = B.Cache(w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.capacity, w.torch_dtype,
                   read_scale=w.read_scale, write_scale=w.write_scale, init_len=w.init_len, flags=flags,
-                  write_eps=write_eps, max_stream=max_stream, mk_init=mk, mv_init=mv, device=device)
+                  write_eps=write_eps, max_stream=max_stream, mk_init=mk, mv_init=mv, device=device, guard_bytes=4096)
     torch.cuda.synchronize()
     del mk, mv
     ora = O.OracleCache(len(units), w.group, 1, w.head_dim, w.capacity, read_scale=w.read_scale,
@@ -72,6 +72,7 @@ def compare_state(w, units, gpu, ora):
     """Max-abs error of the exported MV (and exact equality of MK) on the checked units."""
     k, v = gpu.export(torch.float32)
     torch.cuda.synchronize()
+    gpu.check_guards()   # nothing wrote outside the workspace (0xA5 bands on either side of it)
     n = ora.len
     assert gpu.len == n
     err = 0.0
