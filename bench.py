@@ -162,7 +162,7 @@ def stream_flops(w, tok_per_step, precise=False, write_only=False):
         algorithmic = 2 * Tc * C * d + 2 * C * Tc * d
     else:
         executed = 2 * (2 * 128 * C * d)          # scores of the 128 operand rows, two passes over MK
-        executed += (3 if precise else 1) * (2 * 128 * C * d)   # outputs: P MV_hi (+ P_lo MV_hi + P MV_lo with PRECISE_READ)
+        executed += (2 if precise else 1) * (2 * 128 * C * d)   # outputs: P MV_hi (+ P MV_lo with PRECISE_READ)
         executed += 2 * 128 * C * Tcp             # A = P WW^T
         executed += 2 * (2 * C * Tcp * d)         # MV increment with value + residual weights
         executed += 2 * 128 * Tcp * d             # strict_tril(A) Vc

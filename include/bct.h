@@ -80,9 +80,8 @@ typedef enum bct_dtype {
 #define BCT_FLAG_DENSE_WRITE 4u      /* rewrite every slot, whatever its write weight */
 #define BCT_FLAG_PRECISE_READ 16u     /* bfloat16 cache: the read uses MV's value plus its
                                         residual (one more plane streamed per token; in the
-                                        chunked stream kernel, value + residual numerators
-                                        as well); for states whose magnitude makes a
-                                        bfloat16 ulp matter */
+                                        chunked stream kernel one more product per tile); for
+                                        states whose magnitude makes a bfloat16 ulp matter */
 #define BCT_FLAG_CUDA_CORES 32u       /* keep every decode step on the CUDA-core kernel (the
                                         tensor-core kernel serves bfloat16, head_dim 128,
                                         G <= 15, C >= 128 by default) */

@@ -16,9 +16,11 @@
 // streams through shared memory twice for MK (row statistics, then numerators) and once for MV
 // (value and residual planes), instead of twice per token, and every product runs as tcgen05.mma
 // with fp32 accumulators in tensor memory.  The write weights are always kept as bfloat16
-// value + residual pairs (the state must not drift); with BCT_FLAG_PRECISE_READ the read numerators
-// and MV are too, so that a long stream whose state grows large keeps the output precision.
-//   warp 16 producer : TMA loads (chunk operands, MK / MV tiles through a 3-stage ring)
+// value + residual pairs (the state must not drift); with BCT_FLAG_PRECISE_READ the read uses MV's residual
+// tile as well (one more product per tile), so that a long stream whose state grows large keeps the output
+// precision.  (Measured over a 131072-token stream whose |MV| reaches 75: 0.040 max-abs with the value plane
+// alone, 0.0075 with the residual tile, 0.0014 with residual numerators on top, which are therefore not kept.)
+//   warp 16 producer : TMA loads (chunk operands, MK / MV tiles through a ring of stages)
 //   warp 17 MMA      : issues all tensor-core work, commits to mbarriers
 //   warps 0-15       : four threads per operand row (32 accumulator columns each): online row statistics, numerators, the write-back
 //                      of MV rows, the intra-chunk term and the epilogue
@@ -55,7 +57,7 @@ struct StArgs {
     const float* eta;  // step size of each token's write, [B][T][Hkv], or NULL (all ones)
     int C, Hq, Hkv, U, T, t_begin, n_chunks, Tc;
     int fill, len0;  // fill = 1: the cache holds len0 slots and each chunk is appended (no soft write)
-    int wtr, out_f32, precise;  // precise: the read uses value + residual of both the numerators and MV
+    int wtr, out_f32, precise;  // precise: the read uses MV's value + residual (one more product per tile)
     float read_scale, write_scale;
     float write_eps;  // write weights below it are dropped (0 with BCT_FLAG_DENSE_WRITE)
 };
@@ -65,14 +67,13 @@ struct StSmem {
     int stages;    // ring stages of one tile each
     int plo_half;  // bytes between the two 64-column halves of the residual operand
 };
-// Shared-memory carve-up, the same on host and device.  With PRECISE_READ every operand row keeps
-// its residual (a full second operand buffer) and the ring has three stages; otherwise only the
-// write rows do (at most 64 rows), and the 16 KiB saved buy a fourth stage.  `wide`: chunks of more
-// than 64 tokens (the write-only form, up to 128 write rows): a full residual buffer and twice the Vc.
-__host__ __device__ inline StSmem st_smem(int precise, int wide) {
+// Shared-memory carve-up, the same on host and device.  Only the write rows keep a residual operand (at
+// most 64 rows), which leaves room for four ring stages.  `wide`: chunks of more than 64 tokens (the
+// write-only form, up to 128 write rows): a full residual buffer, twice the Vc and three stages.
+__host__ __device__ inline StSmem st_smem(int wide) {
     StSmem L;
-    L.stages = (precise || wide) ? 3 : kStMaxStages;
-    L.plo_half = (precise || wide) ? kStHalf : kStMaxTc * 128;
+    L.stages = wide ? 3 : kStMaxStages;
+    L.plo_half = wide ? kStHalf : kStMaxTc * 128;
     int off = 0;
     L.qall = off;
     off += kStTileBytes;        // [2 halves][128 rows][128 B]: G*Tc read queries, Tc write queries, zero rows
@@ -130,7 +131,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                  const StArgs a) {
     extern __shared__ unsigned char st_smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(st_smem_raw) + 1023) & ~uintptr_t(1023));
-    const StSmem L = st_smem(a.precise, a.Tc > kStMaxTc);
+    const StSmem L = st_smem(a.Tc > kStMaxTc);
     const int ns = L.stages;
     unsigned char* qall = smem + L.qall;
     unsigned char* vc = smem + L.vc;
@@ -406,7 +407,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             const uint32_t id_a = instr_desc_mn(128, (uint32_t)(Tcp > kStMaxTc ? kStMaxTc : Tcp), false, false);  // P (K) x WW (K)
             uint32_t qn = 0, su0 = 0, su1 = 0, np = 0, nd = 0;
             uint32_t use[kStMaxStages] = {0, 0, 0, 0};
-            const uint32_t plo_row0 = a.precise ? 0u : (uint32_t)n_read;  // first operand row the residual buffer holds
+            const uint32_t plo_row0 = (uint32_t)n_read;  // first operand row the residual buffer holds
             // descriptors at shared address 0 (K-major; MN-major with the half strides of the tiles, of Vc and of
             // the residual operand): the address field is added per use, addresses stay below 256 KiB
             const uint64_t dk0 = smem_desc(0, 16, 1024), dmn0 = smem_desc(0, kStHalf, 1024);
@@ -474,31 +475,39 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         ST_WAIT(pready, np, 46);
                         ++np;
                         ST_WAIT(&full[vh], vh_use(use, t), 47);
-                        if (a.precise) ST_WAIT(&full[vl], use_at(use, vl) + (uint32_t)t, 48);
-                        if (nd > 0 && !a.fill) ST_WAIT(dfree, nd - 1, 49);
                         tc_fence_after();
                         const uint32_t vhaddr = smem_u32(ring + (size_t)vh * kStTileBytes);
                         const uint32_t vladdr = smem_u32(ring + (size_t)vl * kStTileBytes);
-                        // outputs: (P + P_residual) x MV_value + P x MV_residual, accumulated over the tiles
-                        // (none in the write-only form, G = 0)
+                        // outputs: P x MV_value, accumulated over the tiles (none in the write-only form, G = 0).  Issued
+                        // first: they need nothing the rebuild of the previous tile's rows still holds.
 #pragma unroll
                         for (int kk = 0; kk < (G > 0 ? 8 : 0); ++kk) {
                             const uint32_t po = (kk >> 2) * kStHalf + (kk & 3) * 32;
-                            const uint64_t vhd = desc_at(dmn0, vhaddr + kk * 2048);
-                            umma_bf16(tmem_base + kColO, desc_at(dk0, phiaddr + po), vhd, id_out, (t > 0) || (kk > 0));
-                            if (a.precise) {
-                                umma_bf16(tmem_base + kColO, desc_at(dk0, ploaddr + po), vhd, id_out, true);
-                                umma_bf16(tmem_base + kColO, desc_at(dk0, phiaddr + po),
-                                          desc_at(dmn0, vladdr + kk * 2048), id_out, true);
-                            }
+                            umma_bf16(tmem_base + kColO, desc_at(dk0, phiaddr + po), desc_at(dmn0, vhaddr + kk * 2048), id_out,
+                                      (t > 0) || (kk > 0));
                         }
+                        // ... + P x MV_residual with PRECISE_READ: the residual tile arrives once the previous tile's
+                        // rows have been stored out of its stage
+                        auto residual_outputs = [&]() {
+                            ST_WAIT(&full[vl], use_at(use, vl) + (uint32_t)t, 48);
+                            tc_fence_after();
+#pragma unroll
+                            for (int kk = 0; kk < (G > 0 ? 8 : 0); ++kk) {
+                                const uint32_t po = (kk >> 2) * kStHalf + (kk & 3) * 32;
+                                umma_bf16(tmem_base + kColO, desc_at(dk0, phiaddr + po), desc_at(dmn0, vladdr + kk * 2048), id_out,
+                                          true);
+                            }
+                        };
                         if (a.fill) {
                             // no soft write while the cache fills: the stages are free once the outputs are done
+                            if (a.precise) residual_outputs();
                             umma_commit(pfree);
                             umma_commit(&empty[vh]);
                             if (load_vl) umma_commit(&empty[vl]);
                             continue;
                         }
+                        if (nd > 0) ST_WAIT(dfree, nd - 1, 49);  // the previous tile's increment has been read
+                        tc_fence_after();
                         // increment of this tile's MV rows: (WW + WW_residual)^T x Vc, 16 tokens per step
                         for (int kk = 0; kk < Tcp / 16; ++kk) {
                             const uint64_t vd = desc_at(dvc0, vcaddr + kk * 2048);
@@ -508,6 +517,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                                       desc_at(dpl0, ploaddr + ((uint32_t)n_read - plo_row0) * 128 + kk * 2048), vd,
                                       id_delta, true);
                         }
+                        if (a.precise) residual_outputs();
                         umma_commit(dready);  // the write-back may start: outputs and increment are complete
                         // A += P x WW^T over this tile's slots (write rows start at n_read)
 #pragma unroll
@@ -527,8 +537,6 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     for (int kk = 0; kk < (G > 0 ? Tcp / 16 : 0); ++kk) {
                         const uint64_t vd = desc_at(dvc0, vcaddr + kk * 2048);
                         umma_bf16(tmem_base + kColO, desc_at(dk0, ploaddr + kk * 32), vd, id_out, (nt > 0) || (kk > 0));
-                        if (a.fill && a.precise)
-                            umma_bf16(tmem_base + kColO, desc_at(dk0, ploaddr + kStHalf + kk * 32), vd, id_out, true);
                     }
                     umma_commit(oready);
                 }
@@ -556,7 +564,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         const bool lo_row = !is_read && r < n_read + Tcp;
         uint32_t qn = 0, su0 = 0, su1 = 0, np = 0, nd = 0;
         uint32_t use[kStMaxStages] = {0, 0, 0, 0};
-        const int lo_off = (cq >> 1) * L.plo_half + (r - (a.precise ? 0 : n_read)) * 128;  // residual buffer: write rows only unless precise
+        const int lo_off = (cq >> 1) * L.plo_half + (r - n_read) * 128;  // the residual buffer holds the write rows only
         for (int u = blockIdx.x; u < a.U; u += gridDim.x) {
             const int b = u / a.Hkv, h = u - b * a.Hkv;
             for (int ch = 0; ch < a.n_chunks; ++ch, ++qn) {
@@ -692,10 +700,11 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         lr += (s0 + s1) + (s2 + s3);
                     }
                 };
-                if (nt > 0) numerators(0);
-                for (int t = 0; t < nt; ++t) {
-                    if (np > 0) ST_WAIT(pfree, np - 1, 63);  // the previous tile's MMAs have read the operand buffers
-                    if (lo_row || a.precise) {  // write weights always keep the residual
+                // the numerators / write weights held in e, into the operand buffers, once the products that read the
+                // previous ones are complete
+                auto store_operand = [&]() {
+                    if (np > 0) ST_WAIT(pfree, np - 1, 63);
+                    if (lo_row) {  // write weights always keep the residual
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {  // 16-byte chunk = 8 slots
                             uint4 hi, lo;
@@ -713,8 +722,24 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     fence_proxy_async_smem();
                     mbar_arrive(pready);
                     ++np;
-                    if (t + 1 < nt) numerators(t + 1);  // overlaps the tensor-core work on tile t
-                    if (a.fill) continue;  // no soft write while the cache fills
+                };
+                // Order of a tile's turn: the operand of tile t + 1 goes out as soon as the products of tile t are
+                // complete, BEFORE tile t's rows are rebuilt, so that the tensor pipe works on tile t + 1 (its value
+                // tile sits in the other value stage, its increment waits for dfree) while the rows of tile t are
+                // rebuilt and the numerators of tile t + 2 are taken.
+                if (nt > 0) {
+                    numerators(0);
+                    store_operand();
+                    if (nt > 1) numerators(1);
+                }
+                for (int t = 0; t < nt; ++t) {
+                    if (a.fill) {  // no soft write while the cache fills: operands only
+                        if (t + 1 < nt) {
+                            store_operand();
+                            if (t + 2 < nt) numerators(t + 2);
+                        }
+                        continue;
+                    }
 
                     // the tile's MV rows: value + residual + increment, split again, stored (this thread: 32 of the 128 d)
                     const int vh = st_vh(t), vl = st_vl;
@@ -722,13 +747,14 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     ST_WAIT(&full[vl], use_at(use, vl) + (uint32_t)t, 65);
                     ST_WAIT(dready, nd, 66);
                     ++nd;
+                    if (t + 1 < nt) store_operand();  // tile t + 1's products may start
                     tc_fence_after();
                     {
                         unsigned char* th = ring + (size_t)vh * kStTileBytes + poff;
                         unsigned char* tl = ring + (size_t)vl * kStTileBytes + poff;
                         // rows past C of a ragged last tile are clipped by the store
 #pragma unroll
-                        for (int hh = 0; hh < 2; ++hh) {  // 16 columns at a time: the next tile's numerators stay in registers
+                        for (int hh = 0; hh < 2; ++hh) {  // 16 columns at a time
                             float dx[16];
                             tmem_ld16(lane_base + kColD + hh * 16, dx);
                             if (hh == 1) {
@@ -752,6 +778,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     }
                     fence_proxy_async_smem();
                     mbar_arrive(wready);
+                    if (t + 2 < nt) numerators(t + 2);  // overlaps the tensor-core work on tile t + 1
                 }
                 pass2_advance(use, nt);
 
@@ -774,10 +801,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                                 z[e] = (is_read && s <= my_t) ? ex2(fmaf(cc[8 * j + e], c2, -m)) : 0.f;
                                 lr += z[e];
                             }
-                            uint4 hi, lo;
-                            split8(z, &hi, &lo);
-                            *reinterpret_cast<uint4*>(plo + r * 128 + ((c ^ sw) * 16)) = hi;
-                            if (a.precise) *reinterpret_cast<uint4*>(plo + kStHalf + r * 128 + ((c ^ sw) * 16)) = lo;
+                            *reinterpret_cast<uint4*>(plo + r * 128 + ((c ^ sw) * 16)) = Chunk<__nv_bfloat16>::pack(z);
                         }
                     }
                     tc_fence_before();
@@ -967,7 +991,7 @@ int launch_stream_tc(const bct_cache* c, const void* q, const void* k, const voi
     a.read_scale = p.read_scale;
     a.write_scale = p.write_scale;
     a.write_eps = (p.flags & BCT_FLAG_DENSE_WRITE) ? 0.f : p.write_eps;
-    const int smem = st_smem(a.precise, Tc > kStMaxTc).total;
+    const int smem = st_smem(Tc > kStMaxTc).total;
     *err = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (*err != cudaSuccess) return -1;
     const int grid = c->U < c->sm_count ? c->U : c->sm_count;

@@ -110,7 +110,7 @@ def test_fill_phase_chunks_match_oracle(G, C, init_len, T, pieces, flags):
     w = W.Workload("t", 2, 2 * G, 2, d, C, "bf16", init_len, T, 59, d ** -0.5, 1.0, 1.0, "stream")
     w = w.scaled(batch=3 if C <= 512 else 2)
     err, state, n_launch = _stream_parity(w, T, pieces, flags=flags)
-    tol = 2e-3 if flags & B.FLAG_PRECISE_READ else TOL["bf16"]
+    tol = 5e-3 if flags & B.FLAG_PRECISE_READ else TOL["bf16"]   # float out; the numerators are bfloat16 (2^-9 relative)
     assert err <= tol and state <= TOL["bf16"], (err, state)
     Tc = 64 if G == 1 else (32 if G <= 3 else 16)
     assert n_launch <= len(pieces) * (2 + 2 * Tc)  # the fill phase went in chunks, not one launch per token
@@ -193,7 +193,7 @@ def test_single_tile_cache_stays_resident_across_chunks(B_, G, T, pieces, flags,
     d = 128
     w = W.Workload("t", B_, 2 * G, 2, d, 128, "bf16", 128, T, 73, d ** -0.5, 1.0, 1.0, "stream", 1.0, 0.5)
     err, state, n_launch = _stream_parity(w, T, pieces, flags=flags, oracle_flags=oflags)
-    tol = 2e-3 if flags & B.FLAG_PRECISE_READ else TOL["bf16"]
+    tol = 5e-3 if flags & B.FLAG_PRECISE_READ else TOL["bf16"]   # float out; the numerators are bfloat16 (2^-9 relative)
     assert err <= tol and state <= TOL["bf16"], (err, state)
     assert n_launch <= 3 * len(pieces) + 1
 
