@@ -410,15 +410,19 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             const uint32_t plo_row0 = (uint32_t)n_read;  // first operand row the residual buffer holds
             // descriptors at shared address 0 (K-major; MN-major with the half strides of the tiles, of Vc and of
             // the residual operand): the address field is added per use, addresses stay below 256 KiB
-            const uint64_t dk0 = smem_desc(0, 16, 1024), dmn0 = smem_desc(0, kStHalf, 1024);
-            const uint64_t dvc0 = smem_desc(0, (uint32_t)vc_half, 1024), dpl0 = smem_desc(0, (uint32_t)L.plo_half, 1024);
-            const uint32_t qaddr = smem_u32(qall), vcaddr = smem_u32(vc), phiaddr = smem_u32(phi), ploaddr = smem_u32(plo);
-            auto scores = [&](uint32_t col, uint32_t taddr) {
+            const DescKind dk(smem_desc(0, 16, 1024)), dmn(smem_desc(0, kStHalf, 1024));
+            const DescKind dvc(smem_desc(0, (uint32_t)vc_half, 1024)), dpl(smem_desc(0, (uint32_t)L.plo_half, 1024));
+            // the operand buffers in the 16-byte units of the address field
+            const uint32_t q16 = desc_addr16(smem_u32(qall)), vc16 = desc_addr16(smem_u32(vc)), phi16 = desc_addr16(smem_u32(phi));
+            const uint32_t plo16 = desc_addr16(smem_u32(plo)), ring16 = desc_addr16(smem_u32(ring));
+            const uint32_t qw16 = q16 + n_read * 8, pw16 = phi16 + n_read * 8;  // the write rows of the two operand buffers
+            const uint32_t plw16 = plo16 + ((uint32_t)n_read - plo_row0) * 8;
+            auto scores = [&](uint32_t col, int stage) {
+                const uint32_t t16 = ring16 + stage * (kStTileBytes / 16);
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk) {
-                    const uint32_t o = (kk >> 2) * kStHalf + (kk & 3) * 32;
-                    umma_bf16(tmem_base + col, desc_at(dk0, qaddr + o), desc_at(dk0, taddr + o), id_scores,
-                              kk > 0);
+                    const uint32_t o = ((kk >> 2) * kStHalf + (kk & 3) * 32) / 16;
+                    umma_bf16(tmem_base + col, dk.at(q16 + o), dk.at(t16 + o), id_scores, kk > 0);
                 }
             };
             for (int u = blockIdx.x; u < a.U; u += gridDim.x) {
@@ -431,9 +435,8 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         // operand buffer), into the columns the full phase uses for A
 #pragma unroll
                         for (int kk = 0; kk < 8; ++kk) {
-                            const uint32_t o = (kk >> 2) * kStHalf + (kk & 3) * 32;
-                            umma_bf16(tmem_base + kColA, desc_at(dk0, qaddr + o),
-                                      desc_at(dk0, qaddr + n_read * 128 + o), id_a, kk > 0);
+                            const uint32_t o = ((kk >> 2) * kStHalf + (kk & 3) * 32) / 16;
+                            umma_bf16(tmem_base + kColA, dk.at(q16 + o), dk.at(qw16 + o), id_a, kk > 0);
                         }
                         umma_commit(ccready);
                         if (nt == 0) umma_commit(qfree_q);  // nothing else reads the query operand
@@ -447,7 +450,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         if (su > 0) ST_WAIT(&sfree[buf], su - 1, 43);
                         if (buf == 1 && nd > 0) ST_WAIT(dfree, nd - 1, 51);  // buffer 1 is the increment's columns
                         tc_fence_after();
-                        scores(buf ? kColD : kColS0, smem_u32(ring + (size_t)stage * kStTileBytes));
+                        scores(buf ? kColD : kColS0, stage);
                         umma_commit(&sready[buf]);
                         umma_commit(&empty[stage]);
                         ++su;
@@ -458,7 +461,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         ST_WAIT(&full[0], use[0] + (uint32_t)t, 44);
                         if (su0 > 0) ST_WAIT(&sfree[0], su0 - 1, 45);
                         tc_fence_after();
-                        scores(kColS0, smem_u32(ring));
+                        scores(kColS0, 0);
                         umma_commit(&sready[0]);
                         umma_commit(&empty[0]);
                         if (t == nt - 1) umma_commit(qfree_q);  // the last product that reads the query operand
@@ -476,15 +479,13 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         ++np;
                         ST_WAIT(&full[vh], vh_use(use, t), 47);
                         tc_fence_after();
-                        const uint32_t vhaddr = smem_u32(ring + (size_t)vh * kStTileBytes);
-                        const uint32_t vladdr = smem_u32(ring + (size_t)vl * kStTileBytes);
+                        const uint32_t vh16 = ring16 + vh * (kStTileBytes / 16), vl16 = ring16 + vl * (kStTileBytes / 16);
                         // outputs: P x MV_value, accumulated over the tiles (none in the write-only form, G = 0).  Issued
                         // first: they need nothing the rebuild of the previous tile's rows still holds.
 #pragma unroll
                         for (int kk = 0; kk < (G > 0 ? 8 : 0); ++kk) {
-                            const uint32_t po = (kk >> 2) * kStHalf + (kk & 3) * 32;
-                            umma_bf16(tmem_base + kColO, desc_at(dk0, phiaddr + po), desc_at(dmn0, vhaddr + kk * 2048), id_out,
-                                      (t > 0) || (kk > 0));
+                            const uint32_t po = ((kk >> 2) * kStHalf + (kk & 3) * 32) / 16;
+                            umma_bf16(tmem_base + kColO, dk.at(phi16 + po), dmn.at(vh16 + kk * 128), id_out, (t > 0) || (kk > 0));
                         }
                         // ... + P x MV_residual with PRECISE_READ: the residual tile arrives once the previous tile's
                         // rows have been stored out of its stage
@@ -493,9 +494,8 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                             tc_fence_after();
 #pragma unroll
                             for (int kk = 0; kk < (G > 0 ? 8 : 0); ++kk) {
-                                const uint32_t po = (kk >> 2) * kStHalf + (kk & 3) * 32;
-                                umma_bf16(tmem_base + kColO, desc_at(dk0, phiaddr + po), desc_at(dmn0, vladdr + kk * 2048), id_out,
-                                          true);
+                                const uint32_t po = ((kk >> 2) * kStHalf + (kk & 3) * 32) / 16;
+                                umma_bf16(tmem_base + kColO, dk.at(phi16 + po), dmn.at(vl16 + kk * 128), id_out, true);
                             }
                         };
                         if (a.fill) {
@@ -510,21 +510,17 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         tc_fence_after();
                         // increment of this tile's MV rows: (WW + WW_residual)^T x Vc, 16 tokens per step
                         for (int kk = 0; kk < Tcp / 16; ++kk) {
-                            const uint64_t vd = desc_at(dvc0, vcaddr + kk * 2048);
-                            umma_bf16(tmem_base + kColD, desc_at(dmn0, phiaddr + n_read * 128 + kk * 2048), vd,
-                                      id_delta, kk > 0);
-                            umma_bf16(tmem_base + kColD,
-                                      desc_at(dpl0, ploaddr + ((uint32_t)n_read - plo_row0) * 128 + kk * 2048), vd,
-                                      id_delta, true);
+                            const uint64_t vd = dvc.at(vc16 + kk * 128);
+                            umma_bf16(tmem_base + kColD, dmn.at(pw16 + kk * 128), vd, id_delta, kk > 0);
+                            umma_bf16(tmem_base + kColD, dpl.at(plw16 + kk * 128), vd, id_delta, true);
                         }
                         if (a.precise) residual_outputs();
                         umma_commit(dready);  // the write-back may start: outputs and increment are complete
                         // A += P x WW^T over this tile's slots (write rows start at n_read)
 #pragma unroll
                         for (int kk = 0; kk < (G > 0 ? 8 : 0); ++kk) {
-                            const uint32_t po = (kk >> 2) * kStHalf + (kk & 3) * 32;
-                            umma_bf16(tmem_base + kColA, desc_at(dk0, phiaddr + po),
-                                      desc_at(dk0, phiaddr + n_read * 128 + po), id_a, (t > 0) || (kk > 0));
+                            const uint32_t po = ((kk >> 2) * kStHalf + (kk & 3) * 32) / 16;
+                            umma_bf16(tmem_base + kColA, dk.at(phi16 + po), dk.at(pw16 + po), id_a, (t > 0) || (kk > 0));
                         }
                         umma_commit(pfree);
                         ++nd;
@@ -535,8 +531,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     ST_WAIT(aready, qn, 50);
                     tc_fence_after();
                     for (int kk = 0; kk < (G > 0 ? Tcp / 16 : 0); ++kk) {
-                        const uint64_t vd = desc_at(dvc0, vcaddr + kk * 2048);
-                        umma_bf16(tmem_base + kColO, desc_at(dk0, ploaddr + kk * 32), vd, id_out, (nt > 0) || (kk > 0));
+                        umma_bf16(tmem_base + kColO, dk.at(plo16 + kk * 2), dvc.at(vc16 + kk * 128), id_out, (nt > 0) || (kk > 0));
                     }
                     umma_commit(oready);
                 }

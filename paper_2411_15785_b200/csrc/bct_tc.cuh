@@ -84,6 +84,16 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes
 // instead of the whole construction, for the single-thread MMA loops.  (The mask matters: in a cluster
 // launch the shared address of a CTA carries its rank above the 18 address bits.)
 __device__ __forceinline__ uint64_t desc_at(uint64_t d0, uint32_t saddr) { return d0 + (uint64_t)((saddr & 0x3FFFFu) >> 4); }
+// The same for the single-thread MMA loops that issue dozens of products per tile: the descriptor kept as its two
+// 32-bit words, placed by ONE 32-bit add on an address given in 16-byte units (the address field is the low 14 bits
+// of the low word and addresses stay below 256 KiB, so nothing carries into the offset fields above it).
+struct DescKind {
+    uint32_t lo, hi;
+    __device__ __forceinline__ explicit DescKind(uint64_t d0) : lo((uint32_t)d0), hi((uint32_t)(d0 >> 32)) {}
+    __device__ __forceinline__ uint64_t at(uint32_t addr16) const { return ((uint64_t)hi << 32) | (uint64_t)(lo + addr16); }
+};
+// a shared address in the 16-byte units of the descriptors' address field
+__device__ __forceinline__ uint32_t desc_addr16(uint32_t saddr) { return (saddr & 0x3FFFFu) >> 4; }
 // Instruction descriptor: bf16 x bf16 -> f32, M = 128, N = 16; A K-major or MN-major, B K-major.
 __host__ __device__ constexpr uint32_t instr_desc(bool a_mn_major) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn_major ? 1u : 0u) << 15) | ((16u >> 3) << 17) |
