@@ -156,31 +156,30 @@ update_bwd_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     constexpr uint32_t id_kk = instr_desc_mn(128, 128, false, false);  // A (K-major) x B (K-major): scores, A
     constexpr uint32_t id_kn = instr_desc_mn(128, 128, false, true);   // A (K-major) x B (MN-major): R, dWq
     constexpr uint32_t id_nn = instr_desc_mn(128, 128, true, true);    // A (MN-major) x B (MN-major): dMK
-    const uint64_t dk0 = smem_desc(0, 16, 1024), dmn0 = smem_desc(0, kBwHalf, 1024);
+    const DescKind dk(smem_desc(0, 16, 1024)), dmn(smem_desc(0, kBwHalf, 1024));
     // D[token][n] (+)= X[token][k] * Y[n][k], both operands K-major, k = 0..127 in eight steps
     auto mma_kk = [&](int col, const unsigned char* x, const unsigned char* y, bool accum) {
-        const uint32_t xa = smem_u32(x), ya = smem_u32(y);
+        const uint32_t xa = desc_addr16(smem_u32(x)), ya = desc_addr16(smem_u32(y));
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {
-            const uint32_t o = (kk >> 2) * kBwHalf + (kk & 3) * 32;
-            umma_bf16(tmem_base + col, desc_at(dk0, xa + o), desc_at(dk0, ya + o), id_kk, accum || kk > 0);
+            const uint32_t o = ((kk >> 2) * kBwHalf + (kk & 3) * 32) / 16;
+            umma_bf16(tmem_base + col, dk.at(xa + o), dk.at(ya + o), id_kk, accum || kk > 0);
         }
     };
     // D[token][n] (+)= X[token][k] * Y[k][n]: X K-major, Y stored as rows k (MN-major operand)
     auto mma_kn = [&](int col, const unsigned char* x, const unsigned char* y, bool accum) {
-        const uint32_t xa = smem_u32(x), ya = smem_u32(y);
+        const uint32_t xa = desc_addr16(smem_u32(x)), ya = desc_addr16(smem_u32(y));
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {
-            const uint32_t o = (kk >> 2) * kBwHalf + (kk & 3) * 32;
-            umma_bf16(tmem_base + col, desc_at(dk0, xa + o), desc_at(dmn0, ya + kk * 2048), id_kn, accum || kk > 0);
+            const uint32_t o = ((kk >> 2) * kBwHalf + (kk & 3) * 32) / 16;
+            umma_bf16(tmem_base + col, dk.at(xa + o), dmn.at(ya + kk * 128), id_kn, accum || kk > 0);
         }
     };
     // D[m][n] = sum_k X[k][m] * Y[k][n]: both stored as rows k (MN-major operands)
     auto mma_nn = [&](int col, const unsigned char* x, const unsigned char* y) {
-        const uint32_t xa = smem_u32(x), ya = smem_u32(y);
+        const uint32_t xa = desc_addr16(smem_u32(x)), ya = desc_addr16(smem_u32(y));
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk)
-            umma_bf16(tmem_base + col, desc_at(dmn0, xa + kk * 2048), desc_at(dmn0, ya + kk * 2048), id_nn, kk > 0);
+        for (int kk = 0; kk < 8; ++kk) umma_bf16(tmem_base + col, dmn.at(xa + kk * 128), dmn.at(ya + kk * 128), id_nn, kk > 0);
     };
 
     if (issuer) {
