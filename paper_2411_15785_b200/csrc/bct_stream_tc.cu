@@ -362,16 +362,26 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                             ++nw;
                             unsigned char* sh = ring + (size_t)pvh * kStTileBytes;
                             unsigned char* sl = ring + (size_t)st_vl * kStTileBytes;
-                            // the residual stage first and alone: the next tile's rebuild waits for its refill
                             tma_store_3d(&tmVlo, 0, t * kStTile, u, sl);
                             tma_store_3d(&tmVlo, 64, t * kStTile, u, sl + kStHalf);
                             bulk_commit();
-                            bulk_wait_read();  // the residual stage has been read out: it may be refilled
-                            mbar_arrive(&empty[st_vl]);
-                            if (t + 1 < nt) load_tile(&tmVlo, u, t + 1, st_vl);
-                            tma_store_3d(&tmVhi, 0, t * kStTile, u, sh);
-                            tma_store_3d(&tmVhi, 64, t * kStTile, u, sh + kStHalf);
-                            bulk_commit();
+                            if (two_vh) {
+                                // The residual stage first and alone: the next tile's rebuild waits for its refill, while
+                                // the next value tile is in its other stage already (0.381 -> 0.370 ms per 256-token step).
+                                bulk_wait_read();  // the residual stage has been read out: it may be refilled
+                                mbar_arrive(&empty[st_vl]);
+                                if (t + 1 < nt) load_tile(&tmVlo, u, t + 1, st_vl);
+                                tma_store_3d(&tmVhi, 0, t * kStTile, u, sh);
+                                tma_store_3d(&tmVhi, 64, t * kStTile, u, sh + kStHalf);
+                                bulk_commit();
+                            } else {  // one value stage: the next tile waits for both refills
+                                tma_store_3d(&tmVhi, 0, t * kStTile, u, sh);
+                                tma_store_3d(&tmVhi, 64, t * kStTile, u, sh + kStHalf);
+                                bulk_commit();
+                                bulk_wait_read_but_one();
+                                mbar_arrive(&empty[st_vl]);
+                                if (t + 1 < nt) load_tile(&tmVlo, u, t + 1, st_vl);
+                            }
                         } else if (t + 1 < nt && load_vl) {
                             load_tile(&tmVlo, u, t + 1, st_vl);
                         }
