@@ -83,7 +83,7 @@ Carve carve(const bct_params_t& p) {
     c.vlo = off;
     off += (p.dtype == BCT_BF16) ? round_up(c.plane_bytes, bct::kAlign) : 0;
     c.status = off;
-    off += bct::kAlign;
+    off += bct::kAlign + round_up(U * sizeof(unsigned long long), bct::kAlign);  // status words, then one progress word per unit
     for (int i = 0; i < 2; ++i) {  // two staging sets: one call's copies overlap the previous call's kernel
         c.stage_q[i] = off;
         off += round_up(c.q_bytes, bct::kAlign);
@@ -310,6 +310,8 @@ bct_status_t bct_cache_create(const bct_params_t* params, void* workspace, size_
     c->vhi = c->ws + cv.vhi;
     c->vlo = p.dtype == BCT_BF16 ? c->ws + cv.vlo : nullptr;
     c->status = reinterpret_cast<int*>(c->ws + cv.status);
+    c->progress = reinterpret_cast<unsigned long long*>(c->ws + cv.status + bct::kAlign);
+    c->stream_launches = 0;
     for (int i = 0; i < 2; ++i) {
         c->stage_q[i] = c->ws + cv.stage_q[i];
         c->stage_k[i] = c->ws + cv.stage_k[i];
@@ -350,7 +352,7 @@ bct_status_t bct_cache_create(const bct_params_t* params, void* workspace, size_
     }
 
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    e = cudaMemsetAsync(c->status, 0, bct::kAlign, stream);
+    e = cudaMemsetAsync(c->status, 0, cv.stage_q[0] - cv.status, stream);  // status and progress words
     if (e == cudaSuccess) e = bct::launch_import(c, mk_init, mv_init, p.dtype, p.init_len, stream);
     if (e != cudaSuccess) {
         release_host_objects(c);

@@ -41,6 +41,8 @@ struct bct_cache {
     char* vhi;      // MV  [U][C][d] (value, or its bfloat16 head)
     char* vlo;      // MV residual plane (bfloat16 only), else NULL
     int* status;    // device status words
+    unsigned long long* progress;  // [U] (launch number << 32 | chunks done) of the chunked stream kernel, behind the status words
+    mutable uint32_t stream_launches;  // launches of the chunked stream kernel so far (the launch number in `progress`)
     char* stage_q[2];  // staging of the host-buffer entry points, two sets used alternately
     char* stage_k[2];
     char* stage_v[2];

@@ -12,7 +12,8 @@
 // While the cache still has Tc free slots the same kernel runs in fill mode: the chunk's keys and
 // values are appended (TMA stores from the operand buffers), token t reads the resident slots plus
 // the chunk's own slots s <= t (scores Q Kc^T, masked causally), and nothing is soft-written.
-// One persistent CTA per (sequence, kv-head) unit at a time (C <= 16384 slots); per chunk the cache
+// One persistent CTA per (sequence, kv-head) unit and chunk at a time (C <= 16384 slots; see task_at for how the
+// chunks are dealt round the CTAs); per chunk the cache
 // streams through shared memory twice for MK (row statistics, then numerators) and once for MV
 // (value and residual planes), instead of twice per token, and every product runs as tcgen05.mma
 // with fp32 accumulators in tensor memory.  The write weights are always kept as bfloat16
@@ -53,6 +54,9 @@ constexpr int kColA = 384;    // A = Pr WW^T  [row (t,g)] x [write token]
 
 struct StArgs {
     char* out;
+    unsigned long long* progress;  // [U]: (launch << 32 | chunks of this launch done) per unit, for the chunk-major schedule
+    unsigned int launch;           // this launch's number
+    int chunk_major;               // 1: the (unit, chunk) pairs are dealt round the CTAs chunk by chunk (see task_at)
     int* status;
     const float* eta;  // step size of each token's write, [B][T][Hkv], or NULL (all ones)
     int C, Hq, Hkv, U, T, t_begin, n_chunks, Tc;
@@ -167,6 +171,25 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     // resident slots and tiles seen by chunk ch: everything once the cache is full, len0 + ch*Tc while it fills
     auto chunk_len = [&](int ch) { return a.fill ? a.len0 + ch * a.Tc : a.C; };
     auto chunk_tiles = [&](int ch) { return a.fill ? (a.len0 + ch * a.Tc + kStTile - 1) / kStTile : nt_full; };
+    // The k-th (unit, chunk) pair of this CTA.  Unit-major: a CTA takes whole units, chunk after chunk.  Chunk-major:
+    // pair i = chunk (i / U) of unit (i mod U) goes to CTA i mod gridDim, so that U units that do not divide by the
+    // number of CTAs leave no CTA idle for a whole unit (256 units x 4 chunks on 148 CTAs: 7 turns instead of 8).  A
+    // unit's chunks then run on different CTAs: chunk c waits until the unit's progress word says that chunk c - 1 of
+    // this launch is in global memory (it was dealt a whole turn earlier, so the wait is over before it starts).
+    const int n_pairs = a.U * a.n_chunks;
+    auto task_at = [&](int k, int& u, int& ch) {
+        if (a.chunk_major) {
+            const int i = (int)blockIdx.x + k * (int)gridDim.x;
+            if (i >= n_pairs) return false;
+            ch = i / a.U;
+            u = i - ch * a.U;
+            return true;
+        }
+        const int j = k / a.n_chunks;
+        u = (int)blockIdx.x + j * (int)gridDim.x;
+        ch = k - j * a.n_chunks;
+        return u < a.U;
+    };
     const int n_read = Tc * G;         // rows [0, n_read): read queries (t, g); then Tc write rows
     const int Tcp = (Tc + 15) & ~15;   // the chunk padded to the 16-token step of the products (padding rows are zero)
     const int vc_half = Tcp * 128;     // bytes between the two 64-column halves of Vc
@@ -254,7 +277,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             // MK keeps stage 0, MV's value and residual tiles keep their stages, where the row threads rebuild them
             // chunk after chunk.  The loads after the first chunk and the stores before the last one are left out;
             // the barriers are handed over as if they had happened, so the other roles do not change.
-            const bool resident = !a.fill && nt_full == 1 && a.n_chunks > 1;
+            const bool resident = !a.fill && nt_full == 1 && a.n_chunks > 1 && !a.chunk_major;
             auto keep_tile = [&](int stage) {   // the stage already holds the tile: complete the barrier's phase without a copy
                 const uint32_t n = use_at(use, stage)++;
                 if (n > 0) ST_WAIT(&empty[stage], n - 1, 37);
@@ -274,22 +297,34 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             };
             // The query operand is free once the last scores of a chunk are complete, well before the
             // chunk's last tile is stored: the next chunk's queries are asked for at that point.
-            auto next_queries = [&](int u, int ch) {
-                int u2 = u, ch2 = ch + 1;
-                if (ch2 == a.n_chunks) {
-                    u2 = u + gridDim.x;
-                    ch2 = 0;
-                }
-                if (u2 >= a.U) return;
+            auto next_queries = [&](int kt) {
+                int u2, ch2;
+                if (!task_at(kt + 1, u2, ch2)) return;
                 ST_WAIT(qfree_q, qn, 32);
                 if (a.fill) bulk_wait_read();  // the appended keys have been read out of the operand
                 load_queries(u2, ch2);
             };
-            for (int u = blockIdx.x; u < a.U; u += gridDim.x) {
+            for (int kt = 0, u = 0, ch = 0; task_at(kt, u, ch); ++kt, ++qn) {
                 const int b = u / a.Hkv, h = u - b * a.Hkv;
-                for (int ch = 0; ch < a.n_chunks; ++ch, ++qn) {
+                {
                     const int t0 = a.t_begin + ch * Tc;
                     const int nt = chunk_tiles(ch);
+                    if (a.chunk_major && ch > 0) {
+                        // the unit's previous chunk ran on another CTA: its rows (and appended keys) must be in global memory
+                        const unsigned long long want = ((unsigned long long)a.launch << 32) | (unsigned int)ch;
+                        bool seen = false;
+                        for (uint32_t i = 0; i < (*abort_flag ? 1024u : kWaitLimit) && !seen; ++i) {
+                            unsigned long long got;
+                            asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(got) : "l"(a.progress + u) : "memory");
+                            seen = got == want;
+                            if (!seen && i > 64) __nanosleep(i > 4096 ? 256 : 32);
+                        }
+                        if (!seen) {
+                            report_timeout(a.status, 30);
+                            *abort_flag = 1;
+                        }
+                        fence_proxy_async_global();  // ... before this chunk's copies read them
+                    }
                     // the first MK tiles of pass 1 do not depend on the chunk's operands: ask for them first
                     const int n_early = nt < ns - 1 ? nt : ns - 1;
                     int st1 = 0;  // pass-1 stage of the next tile, t mod ns without the division
@@ -344,10 +379,10 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         if (nt > 1) load_tile(&tmK, u, 1, 0);
                         if (nt > 1 && two_vh) load_tile(&tmVhi, u, 1, st_vh(1));
                     }
-                    if (nt == 0) next_queries(u, ch);
+                    if (nt == 0) next_queries(kt);
                     for (int t = 0; t < nt; ++t) {
                         if (t + 2 < nt) load_tile(&tmK, u, t + 2, 0);
-                        if (t == nt - 1) next_queries(u, ch);
+                        if (t == nt - 1) next_queries(kt);
                         const int pvh = st_vh(t);
                         if (resident && ch + 1 < a.n_chunks) {
                             // the rebuilt tile is the next chunk's MV: nothing goes to HBM yet
@@ -415,6 +450,11 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         }
                     }
                     bulk_wait_all();  // the next chunk reads these rows again
+                    if (a.chunk_major && ch + 1 < a.n_chunks) {  // ... on another CTA: hand the unit over
+                        fence_proxy_async_global();
+                        const unsigned long long done = ((unsigned long long)a.launch << 32) | (unsigned int)(ch + 1);
+                        asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(a.progress + u), "l"(done) : "memory");
+                    }
                     // every tile of the unit was rebuilt and stored (a resident tile goes home after the last chunk only)
                     if (!a.fill && (!resident || ch + 1 == a.n_chunks)) rows_stored += (unsigned long long)a.C;
                 }
@@ -449,8 +489,8 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     umma_bf16(tmem_base + col, dk.at(q16 + o), dk.at(t16 + o), id_scores, kk > 0);
                 }
             };
-            for (int u = blockIdx.x; u < a.U; u += gridDim.x) {
-                for (int ch = 0; ch < a.n_chunks; ++ch, ++qn) {
+            for (int kt = 0, u = 0, ch = 0; task_at(kt, u, ch); ++kt, ++qn) {
+                {
                     ST_WAIT(qfull, qn, 41);
                     tc_fence_after();
                     const int nt = chunk_tiles(ch);
@@ -584,9 +624,9 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         uint32_t qn = 0, su0 = 0, su1 = 0, np = 0, nd = 0;
         uint32_t use[kStMaxStages] = {0, 0, 0, 0};
         const int lo_off = (cq >> 1) * L.plo_half + (r - n_read) * 128;  // the residual buffer holds the write rows only
-        for (int u = blockIdx.x; u < a.U; u += gridDim.x) {
+        for (int kt = 0, u = 0, ch = 0; task_at(kt, u, ch); ++kt, ++qn) {
             const int b = u / a.Hkv, h = u - b * a.Hkv;
-            for (int ch = 0; ch < a.n_chunks; ++ch, ++qn) {
+            {
                 const int t0 = a.t_begin + ch * Tc;
                 const int nt = chunk_tiles(ch);
                 const int clen = chunk_len(ch);
@@ -1004,6 +1044,14 @@ int launch_stream_tc(const bct_cache* c, const void* q, const void* k, const voi
     *err = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (*err != cudaSuccess) return -1;
     const int grid = c->U < c->sm_count ? c->U : c->sm_count;
+    // Chunk-major dealing of the (unit, chunk) pairs where it saves a turn: units that do not divide by the CTAs, more
+    // than one chunk, and no single-tile cache (which stays in one CTA's shared memory from chunk to chunk).
+    const bool resident = fill_len < 0 && p.capacity <= kStTile && n_chunks > 1;
+    const int64_t turns_unit_major = ((c->U + grid - 1) / grid) * n_chunks;
+    const int64_t turns_chunk_major = ((int64_t)c->U * n_chunks + grid - 1) / grid;
+    a.chunk_major = (!resident && c->U >= grid && n_chunks > 1 && turns_chunk_major < turns_unit_major) ? 1 : 0;
+    a.progress = c->progress;
+    a.launch = ++c->stream_launches;
     fn<<<grid, kStThreads, smem, stream>>>(*reinterpret_cast<const CUtensorMap*>(c->tmap_k),
                                            *reinterpret_cast<const CUtensorMap*>(c->tmap_v),
                                            *reinterpret_cast<const CUtensorMap*>(c->tmap_lo), mq, mk, mv, mka, mva, a);

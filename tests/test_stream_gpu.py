@@ -20,8 +20,8 @@ def _built():
     B.load()
 
 
-def _stream_parity(w, T, pieces, flags=0, oracle_flags=0, want_out=True, write_eps=0.0):
-    units = pick_units(w, 8)
+def _stream_parity(w, T, pieces, flags=0, oracle_flags=0, want_out=True, write_eps=0.0, n_units=8):
+    units = pick_units(w, n_units)
     gpu, ora = make_pair(w, units, flags=flags, oracle_flags=oracle_flags, write_eps=write_eps, oracle_write_eps=write_eps)
     q, k, v = W.stream_inputs(w, 0, T, "cuda")
     launches0 = gpu.launches
@@ -211,3 +211,19 @@ def test_single_tile_cache_resident_in_update_kv_and_counts_its_stores():
     assert compare_state(w, units, gpu, ora) <= TOL["bf16"]
     assert gpu.rows_rewritten() == w.units * 128      # one store of the tile per unit, after the last chunk
     gpu.destroy()
+
+
+@pytest.mark.parametrize("G,C,init_len,T,pieces,flags,oflags", [
+    (1, 256, 256, 192, [192], 0, 0),               # 160 units x 3 chunks on 148 CTAs: 4 turns instead of 6
+    (1, 384, 0, 512, [512], 0, 0),                 # from empty: 6 fill chunks dealt round the CTAs (appended keys handed over), then 2
+    (2, 256, 256, 200, [120, 80], B.FLAG_WRITE_THEN_READ, O.WRITE_THEN_READ),   # chunks of 40, two calls (two launch numbers)
+    (1, 512, 512, 256, [256], B.FLAG_PRECISE_READ | B.FLAG_OUT_F32, 0),
+])
+def test_chunks_of_a_unit_go_round_the_ctas(G, C, init_len, T, pieces, flags, oflags):
+    # more units than CTAs and several chunks per call: the (unit, chunk) pairs are dealt chunk-major, so a unit's
+    # consecutive chunks run on different CTAs and are handed over through global memory and the unit's progress word
+    d = 128
+    w = W.Workload("t", 80, 2 * G, 2, d, C, "bf16", init_len, T, 57, d ** -0.5, 1.0, 1.0, "stream", 1.0, 0.5)
+    err, state, n_launch = _stream_parity(w, T, pieces, flags=flags, oracle_flags=oflags, n_units=16)
+    tol = 5e-3 if flags & B.FLAG_PRECISE_READ else TOL["bf16"]
+    assert err <= tol and state <= TOL["bf16"], (err, state)
