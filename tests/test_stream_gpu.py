@@ -227,3 +227,35 @@ def test_chunks_of_a_unit_go_round_the_ctas(G, C, init_len, T, pieces, flags, of
     err, state, n_launch = _stream_parity(w, T, pieces, flags=flags, oracle_flags=oflags, n_units=16)
     tol = 5e-3 if flags & B.FLAG_PRECISE_READ else TOL["bf16"]
     assert err <= tol and state <= TOL["bf16"], (err, state)
+
+
+@pytest.mark.parametrize("init_len,flags", [(256, 0), (0, 0), (256, B.FLAG_PRECISE_READ | B.FLAG_OUT_F32)])
+def test_chunk_major_launch_is_bit_equal_to_chunk_by_chunk_calls(init_len, flags):
+    # One call of 12 chunks on 170 units (chunks dealt round the CTAs, units handed from CTA to CTA) against the
+    # same tokens fed one chunk per call (every launch a single chunk: no hand-over).  The arithmetic of a chunk
+    # is the same in both, so outputs and the exported state agree bit for bit on every unit; three rounds.
+    d, C, G, Tc = 128, 256, 1, 64
+    T = 12 * Tc
+    w = W.Workload("t", 85, 2 * G, 2, d, C, "bf16", init_len, T, 61, d ** -0.5, 1.0, 1.0, "stream", 1.0, 0.5)
+    mk = mv = None
+    if init_len:
+        mk, mv = W.initial_cache(w, "cuda")
+    mk_cache = lambda: B.Cache(w.batch, w.n_q_heads, w.n_kv_heads, d, C, torch.bfloat16, read_scale=w.read_scale,
+                               write_scale=w.write_scale, init_len=init_len, flags=flags, mk_init=mk, mv_init=mv,
+                               guard_bytes=4096)
+    one, many = mk_cache(), mk_cache()
+    for rnd in range(3):
+        q, k, v = W.stream_inputs(w, rnd * T, T, "cuda")
+        o1 = one.prefill_stream(q, k, v)
+        parts = [many.prefill_stream(q[:, i:i + Tc].contiguous(), k[:, i:i + Tc].contiguous(), v[:, i:i + Tc].contiguous())
+                 for i in range(0, T, Tc)]
+        o2 = torch.cat(parts, dim=1)
+        one.check_status()
+        many.check_status()
+        assert torch.equal(o1, o2)
+        (k1, v1), (k2, v2) = one.export(), many.export()
+        assert torch.equal(k1, k2) and torch.equal(v1, v2)
+    one.check_guards()
+    many.check_guards()
+    one.destroy()
+    many.destroy()

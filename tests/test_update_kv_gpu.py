@@ -48,6 +48,22 @@ def test_update_kv_matches_oracle(G, C, T, with_eta, write_scale):
     gpu.destroy()
 
 
+def test_update_kv_with_more_units_than_ctas_deals_the_chunks_round_the_ctas():
+    # 160 units, three chunks of 128 tokens: the (unit, chunk) pairs go chunk-major (4 turns on 148 CTAs instead of 6),
+    # so a unit's state is handed from CTA to CTA between its chunks
+    d, C, T = 128, 256, 384
+    w = W.Workload("t", 80, 2, 2, d, C, "bf16", C, T, 103, d ** -0.5, 1.0, 1.0, "stream", 1.0, 0.5)
+    units = pick_units(w, 16)
+    gpu, ora = make_pair(w, units)
+    q, k, v = W.stream_inputs(w, 0, T, "cuda")
+    gpu.update_kv(k, v)
+    gpu.check_status()
+    _, uk, uv = _unit_slices(w, units, q, k, v)
+    ora.update_kv(uk, uv)
+    assert compare_state(w, units, gpu, ora) <= TOL["bf16"]
+    gpu.destroy()
+
+
 def test_update_kv_tracks_the_stream_call_and_continues_it():
     d, C, T = 128, 512, 200
     w = W.Workload("t", 2, 2, 2, d, C, "bf16", C, 2 * T, 101, d ** -0.5, 1.0, 1.0, "stream")
