@@ -49,7 +49,8 @@ def test_cache_bytes_accounts_for_planes_and_staging(lib):
     plane = 64 * 32 * 2048 * 128 * 2
     assert align == 256
     step = 64 * 32 * 128 * 2                                          # q, k, v or out of one token
-    assert 3 * plane + 2 * 4 * step <= nbytes <= 3 * plane + 2 * 4 * step + 32 * 256   # two staging sets
+    progress = 64 * 32 * 8                                            # one 64-bit progress word per (sequence, kv-head) unit
+    assert 3 * plane + 2 * 4 * step + progress <= nbytes <= 3 * plane + 2 * 4 * step + progress + 32 * 256   # two staging sets
     p32 = B.make_params(1, 1, 1, 64, 128, torch.float32)
     n32, _ = B.cache_bytes(p32)
     assert 2 * 128 * 64 * 4 <= n32 < 2 * 128 * 64 * 4 + 8192       # no residual plane in float
