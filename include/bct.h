@@ -123,7 +123,8 @@ const char *bct_last_error(void);
 /*
  * Size and alignment of the device workspace a cache with these parameters needs
  * (Method, "Model Structure": MK and MV of M slots each, per unit; plus the bfloat16
- * residual plane, the status words and the staging area of the *_host entry points).
+ * residual plane, the status words, one progress word per (sequence, kv-head) unit and the staging
+ * area of the *_host entry points).
  * The size depends on the parameters only and never grows afterwards, which is the
  * bounded-memory property of the method ("Fixed-Length Cache").
  */
