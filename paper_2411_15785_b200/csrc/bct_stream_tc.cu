@@ -12,7 +12,7 @@
 // While the cache still has Tc free slots the same kernel runs in fill mode: the chunk's keys and
 // values are appended (TMA stores from the operand buffers), token t reads the resident slots plus
 // the chunk's own slots s <= t (scores Q Kc^T, masked causally), and nothing is soft-written.
-// One persistent CTA per (sequence, kv-head) unit and chunk at a time (C <= 16384 slots; see task_at for how the
+// One persistent CTA per (sequence, kv-head) unit and chunk at a time (C <= 16384 slots; see task_next for how the
 // chunks are dealt round the CTAs); per chunk the cache
 // streams through shared memory twice for MK (row statistics, then numerators) and once for MV
 // (value and residual planes), instead of twice per token, and every product runs as tcgen05.mma
@@ -56,7 +56,7 @@ struct StArgs {
     char* out;
     unsigned long long* progress;  // [U]: (launch << 32 | chunks of this launch done) per unit, for the chunk-major schedule
     unsigned int launch;           // this launch's number
-    int chunk_major;               // 1: the (unit, chunk) pairs are dealt round the CTAs chunk by chunk (see task_at)
+    int chunk_major;               // 1: the (unit, chunk) pairs are dealt round the CTAs chunk by chunk (see task_next)
     int* status;
     const float* eta;  // step size of each token's write, [B][T][Hkv], or NULL (all ones)
     int C, Hq, Hkv, U, T, t_begin, n_chunks, Tc;
@@ -176,18 +176,24 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     // number of CTAs leave no CTA idle for a whole unit (256 units x 4 chunks on 148 CTAs: 7 turns instead of 8).  A
     // unit's chunks then run on different CTAs: chunk c waits until the unit's progress word says that chunk c - 1 of
     // this launch is in global memory (it was dealt a whole turn earlier, so the wait is over before it starts).
-    const int n_pairs = a.U * a.n_chunks;
-    auto task_at = [&](int k, int& u, int& ch) {
+    // (Walked without divisions: the single-thread roles have nothing to hide them behind.  gridDim <= U.)
+    auto task_first = [&](int& u, int& ch) {
+        u = (int)blockIdx.x;
+        ch = 0;
+        return u < a.U;
+    };
+    auto task_next = [&](int& u, int& ch) {  // the pair after (u, ch) on this CTA; false when there is none
         if (a.chunk_major) {
-            const int i = (int)blockIdx.x + k * (int)gridDim.x;
-            if (i >= n_pairs) return false;
-            ch = i / a.U;
-            u = i - ch * a.U;
-            return true;
+            u += (int)gridDim.x;
+            if (u >= a.U) {
+                u -= a.U;
+                ++ch;
+            }
+            return ch < a.n_chunks;
         }
-        const int j = k / a.n_chunks;
-        u = (int)blockIdx.x + j * (int)gridDim.x;
-        ch = k - j * a.n_chunks;
+        if (++ch < a.n_chunks) return true;
+        ch = 0;
+        u += (int)gridDim.x;
         return u < a.U;
     };
     const int n_read = Tc * G;         // rows [0, n_read): read queries (t, g); then Tc write rows
@@ -263,6 +269,19 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         // =========================== producer ===========================
         if (lane == 0) {
             uint32_t qn = 0, nw = 0;
+            int pre = 0;  // tiles of the next pair's pass 1 that have been asked for already
+            int handed_u = -1, handed_ch = 0;  // a finished chunk whose progress word has not been written yet
+            // The pair before is complete in global memory (its stores were waited for): say so in its unit's progress
+            // word.  The release takes about half a microsecond and only a CTA a whole turn behind waits for it, so it
+            // is written after the next pair's first copies have been asked for, and in any case before this CTA waits
+            // for anything another CTA has to hand over.
+            auto hand_over = [&]() {
+                if (handed_u < 0) return;
+                fence_proxy_async_global();
+                const unsigned long long done = ((unsigned long long)a.launch << 32) | (unsigned int)handed_ch;
+                asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(a.progress + handed_u), "l"(done) : "memory");
+                handed_u = -1;
+            };
             unsigned long long rows_stored = 0;  // MV rows this CTA has stored back
             uint32_t use[kStMaxStages] = {0, 0, 0, 0};
             auto load_tile = [&](const CUtensorMap* map, int u, int t, int stage) {
@@ -297,20 +316,24 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             };
             // The query operand is free once the last scores of a chunk are complete, well before the
             // chunk's last tile is stored: the next chunk's queries are asked for at that point.
-            auto next_queries = [&](int kt) {
-                int u2, ch2;
-                if (!task_at(kt + 1, u2, ch2)) return;
+            auto next_queries = [&](int u, int ch) {
+                int u2 = u, ch2 = ch;
+                if (!task_next(u2, ch2)) return;
                 ST_WAIT(qfree_q, qn, 32);
                 if (a.fill) bulk_wait_read();  // the appended keys have been read out of the operand
                 load_queries(u2, ch2);
             };
-            for (int kt = 0, u = 0, ch = 0; task_at(kt, u, ch); ++kt, ++qn) {
+            for (int u = 0, ch = 0, more = task_first(u, ch); more; more = task_next(u, ch), ++qn) {
                 const int b = u / a.Hkv, h = u - b * a.Hkv;
                 {
                     const int t0 = a.t_begin + ch * Tc;
                     const int nt = chunk_tiles(ch);
-                    if (a.chunk_major && ch > 0) {
-                        // the unit's previous chunk ran on another CTA: its rows (and appended keys) must be in global memory
+                    // The unit's previous chunk ran on another CTA: its rows (and appended keys) must be in global memory
+                    // before this chunk's copies read them.  While the cache fills that is every tile copy; with a full
+                    // cache MK is constant and only the MV tiles of pass 2 depend on it, so the check comes after pass 1's
+                    // copies have been issued, off the start of the pair.
+                    auto wait_for_previous_chunk = [&]() {
+                        if (!a.chunk_major || ch == 0) return;
                         const unsigned long long want = ((unsigned long long)a.launch << 32) | (unsigned int)ch;
                         bool seen = false;
                         for (uint32_t i = 0; i < (*abort_flag ? 1024u : kWaitLimit) && !seen; ++i) {
@@ -323,18 +346,23 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                             report_timeout(a.status, 30);
                             *abort_flag = 1;
                         }
-                        fence_proxy_async_global();  // ... before this chunk's copies read them
+                        fence_proxy_async_global();
+                    };
+                    if (a.fill) {
+                        hand_over();
+                        wait_for_previous_chunk();
                     }
                     // the first MK tiles of pass 1 do not depend on the chunk's operands: ask for them first
                     const int n_early = nt < ns - 1 ? nt : ns - 1;
-                    int st1 = 0;  // pass-1 stage of the next tile, t mod ns without the division
-                    for (int t = 0; t < n_early; ++t) {
+                    int st1 = pre;  // pass-1 stage of the next tile, t mod ns without the division
+                    for (int t = pre; t < n_early; ++t) {  // (the first `pre` tiles were asked for during the pair before)
                         if (resident && ch > 0)
                             keep_tile(st1);
                         else
                             load_tile(&tmK, u, t, st1);
                         if (++st1 == ns) st1 = 0;
                     }
+                    pre = 0;
                     if (qn == 0) load_queries(u, ch);
                     if (qn > 0) ST_WAIT(oready, qn - 1, 35);  // the previous chunk's last product has read Vc
                     mbar_arrive_expect_tx(vfull, (uint32_t)(Tc * 256));
@@ -363,6 +391,10 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     // there are two value stages.  The residual stage is stored and refilled first: the next
                     // tile's write-back waits for it.
                     const bool two_vh = ns == kStMaxStages;
+                    if (!a.fill) {
+                        hand_over();
+                        wait_for_previous_chunk();
+                    }
                     if (nt > 0 && resident) {
                         keep_tile(0);  // pass 1 left the MK tile in stage 0
                         if (ch == 0) {
@@ -379,10 +411,26 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         if (nt > 1) load_tile(&tmK, u, 1, 0);
                         if (nt > 1 && two_vh) load_tile(&tmVhi, u, 1, st_vh(1));
                     }
-                    if (nt == 0) next_queries(kt);
+                    if (nt == 0) next_queries(u, ch);
                     for (int t = 0; t < nt; ++t) {
                         if (t + 2 < nt) load_tile(&tmK, u, t + 2, 0);
-                        if (t == nt - 1) next_queries(kt);
+                        if (t == nt - 1) {
+                            next_queries(u, ch);
+                            // With a full cache MK never changes, so the first tiles of the next pair's pass 1 depend on
+                            // nothing that is still in flight: they are asked for now, into the stages that are already
+                            // free (the MK stage after the last scores; stage 1 when the tile before the last one had its
+                            // values there), instead of after this pair's last stores.  Without this the tensor pipe and the
+                            // row threads wait 4-5 us for MK tiles at the start of every pair.
+                            int u2 = u, ch2 = ch;
+                            if (!a.fill && !resident && task_next(u2, ch2)) {
+                                load_tile(&tmK, u2, 0, 0);
+                                pre = 1;
+                                if (nt >= 2 && ns > 2 && st_vh(nt - 2) == 1 && st_vh(nt - 1) != 1) {
+                                    load_tile(&tmK, u2, 1, 1);
+                                    pre = 2;
+                                }
+                            }
+                        }
                         const int pvh = st_vh(t);
                         if (resident && ch + 1 < a.n_chunks) {
                             // the rebuilt tile is the next chunk's MV: nothing goes to HBM yet
@@ -450,15 +498,16 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                         }
                     }
                     bulk_wait_all();  // the next chunk reads these rows again
-                    if (a.chunk_major && ch + 1 < a.n_chunks) {  // ... on another CTA: hand the unit over
-                        fence_proxy_async_global();
-                        const unsigned long long done = ((unsigned long long)a.launch << 32) | (unsigned int)(ch + 1);
-                        asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(a.progress + u), "l"(done) : "memory");
+                    if (a.chunk_major && ch + 1 < a.n_chunks) {
+                        // ... on another CTA: the unit is handed over (hand_over) once the next pair's first copies are out
+                        handed_u = u;
+                        handed_ch = ch + 1;
                     }
                     // every tile of the unit was rebuilt and stored (a resident tile goes home after the last chunk only)
                     if (!a.fill && (!resident || ch + 1 == a.n_chunks)) rows_stored += (unsigned long long)a.C;
                 }
             }
+            hand_over();
             if (rows_stored > 0) atomicAdd(reinterpret_cast<unsigned long long*>(a.status + kStatusRowsWord), rows_stored);
         }
         __syncwarp();
@@ -489,7 +538,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                     umma_bf16(tmem_base + col, dk.at(q16 + o), dk.at(t16 + o), id_scores, kk > 0);
                 }
             };
-            for (int kt = 0, u = 0, ch = 0; task_at(kt, u, ch); ++kt, ++qn) {
+            for (int u = 0, ch = 0, more = task_first(u, ch); more; more = task_next(u, ch), ++qn) {
                 {
                     ST_WAIT(qfull, qn, 41);
                     tc_fence_after();
@@ -624,7 +673,7 @@ stream_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         uint32_t qn = 0, su0 = 0, su1 = 0, np = 0, nd = 0;
         uint32_t use[kStMaxStages] = {0, 0, 0, 0};
         const int lo_off = (cq >> 1) * L.plo_half + (r - n_read) * 128;  // the residual buffer holds the write rows only
-        for (int kt = 0, u = 0, ch = 0; task_at(kt, u, ch); ++kt, ++qn) {
+        for (int u = 0, ch = 0, more = task_first(u, ch); more; more = task_next(u, ch), ++qn) {
             const int b = u / a.Hkv, h = u - b * a.Hkv;
             {
                 const int t0 = a.t_begin + ch * Tc;
