@@ -125,9 +125,9 @@ def algorithmic_bytes_per_step(w: W.Workload, w_frac: float = 0.0) -> int:
 
 
 # DRAM bytes per launch and unit (dram__bytes_read.sum + dram__bytes_write.sum) from the committed ncu capture of
-# decode_tc_kernel on the mha7b shape (profiles/decode_tc_kernel_ncu_full.txt: 1.2629 GB read + 0.0320 GB written at
+# decode_tc_kernel on the mha7b shape (profiles/decode_tc_kernel_ncu_full.txt: 1.2630 GB read + 0.0318 GB written at
 # batch 37 = 1184 units; the traffic grows in proportion to the units).  None for any other kernel / shape.
-NCU_TRAFFIC_PER_UNIT = {("mha7b", True): 1.2949e9 / 1184}
+NCU_TRAFFIC_PER_UNIT = {("mha7b", True): 1.2948e9 / 1184}
 
 
 def measured_traffic(w, tensor_path):
