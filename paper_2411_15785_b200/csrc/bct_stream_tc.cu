@@ -1101,6 +1101,18 @@ int launch_stream_tc(const bct_cache* c, const void* q, const void* k, const voi
     a.chunk_major = (!resident && c->U >= grid && n_chunks > 1 && turns_chunk_major < turns_unit_major) ? 1 : 0;
     a.progress = c->progress;
     a.launch = ++c->stream_launches;
+    if (a.chunk_major) {
+        // CTAs wait for one another here (a chunk for the unit's chunk before it, on another CTA), so every CTA of the
+        // grid must be resident: a cooperative launch, which the runtime refuses when the grid does not fit the device
+        // as it is (SMs held by other work, a partitioned device).  Refused: the unit-major walk, which waits for nobody.
+        CUtensorMap tk = *reinterpret_cast<const CUtensorMap*>(c->tmap_k), tv = *reinterpret_cast<const CUtensorMap*>(c->tmap_v),
+                    tl = *reinterpret_cast<const CUtensorMap*>(c->tmap_lo);
+        void* args[] = {&tk, &tv, &tl, &mq, &mk, &mv, &mka, &mva, &a};
+        *err = cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(fn), dim3(grid), dim3(kStThreads), args, (size_t)smem, stream);
+        if (*err == cudaSuccess) return 1;
+        (void)cudaGetLastError();
+        a.chunk_major = 0;
+    }
     fn<<<grid, kStThreads, smem, stream>>>(*reinterpret_cast<const CUtensorMap*>(c->tmap_k),
                                            *reinterpret_cast<const CUtensorMap*>(c->tmap_v),
                                            *reinterpret_cast<const CUtensorMap*>(c->tmap_lo), mq, mk, mv, mka, mva, a);
