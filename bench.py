@@ -241,7 +241,7 @@ def run_reference(args, w):
         return
     smp = OracleSample(w)
     total = args.steps + args.warmup
-    T = int(max(1, min(4096, (100.0 / total) / smp.per_token)))
+    T = int(max(1, min(4096, (args.ref_seconds / total) / smp.per_token)))
     elapsed = 0.0
     for i in range(total):
         dt = smp.run(T)
@@ -555,6 +555,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default="mha7b_b64_c2048", choices=sorted(W.CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--ref-seconds", type=float, default=100.0,
+                    help="--impl reference: CPU seconds the whole run (warm-up and timed steps) is sized for")
     ap.add_argument("--write-scale", type=float, default=None, help="override the write score scale")
     ap.add_argument("--stream-tokens", type=int, default=256,
                     help="tokens per sequence pushed by one step of a stream workload")
